@@ -1,0 +1,125 @@
+"""Seeded synthetic inputs for the BDLM attention layer.
+
+This module only makes inputs and picks sample rows; it holds none of the attention
+arithmetic, so both the CUDA path's callers and the CPU oracle's tests may use it.
+
+The paper's throughput runs use sequences that all have exactly the stated context length
+(section 5.1) and give no head counts or activation statistics; the workloads below use
+Llama-3-8B-like head shapes with q/k/v ~ 0.5 * N(0,1) rounded to bf16 and upstream
+gradients dO ~ N(0,1) rounded to bf16.  They stand in for the paper's long-context
+workloads.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, replace
+
+import numpy as np
+import torch
+
+
+@dataclass(frozen=True)
+class Workload:
+    name: str
+    batch: int
+    H: int
+    H_kv: int
+    d: int
+    L: int            # clean length; the noisy stream has the same length
+    block_size: int
+    rope_theta: float = 0.0   # > 0: rotate q and k before rounding to bf16
+    kv_shards: int = 1        # > 1: forward is also run as that many clean-K/V shard partials
+    seed: int = 0
+
+    def pairs_per_head(self):
+        """Unmasked (query, key) pairs per (batch, query head): clean L(L+1)/2 and noisy
+        L(L+M)/2 (appendix B, Eq. aligned-rank-work with P = 1)."""
+        L, M = self.L, self.block_size
+        return L * (L + 1) // 2, L * (L + M) // 2
+
+    def flops(self):
+        """(forward, backward) FLOPs over unmasked pairs only: 4d and 10d per pair."""
+        c, n = self.pairs_per_head()
+        pairs = (c + n) * self.batch * self.H
+        return 4 * self.d * pairs, 10 * self.d * pairs
+
+
+WORKLOADS = {
+    "tiny": Workload("tiny", 1, 2, 2, 64, 256, 16),
+    "8k": Workload("8k", 2, 16, 4, 128, 8192, 32),
+    "32k": Workload("32k", 1, 32, 8, 128, 32768, 64, rope_theta=5e5),
+    "csbp128k": Workload("csbp128k", 1, 32, 8, 128, 131072, 32, kv_shards=8),
+    "256k": Workload("256k", 1, 32, 8, 128, 262144, 16),
+    # paper-shaped block size (appendix J uses 128..1024, default 256); not a BASELINE config
+    "32k_m256": Workload("32k_m256", 1, 32, 8, 128, 32768, 256, rope_theta=5e5),
+}
+
+
+def small(w: Workload, **kw) -> Workload:
+    return replace(w, **kw)
+
+
+def _rope(x: torch.Tensor, theta: float) -> torch.Tensor:
+    """Rotary embedding in fp32, half-split pairing (x_k, x_{k+d/2}); token i of either
+    stream uses position i.  x is [batch, L, heads, d]."""
+    _, L, _, d = x.shape
+    half = d // 2
+    inv = theta ** (-torch.arange(half, device=x.device, dtype=torch.float32) / half)
+    ang = torch.arange(L, device=x.device, dtype=torch.float32)[:, None] * inv[None, :]
+    cos = ang.cos()[None, :, None, :]
+    sin = ang.sin()[None, :, None, :]
+    a, b = x[..., :half], x[..., half:]
+    return torch.cat([a * cos - b * sin, a * sin + b * cos], dim=-1)
+
+
+def make_inputs(w: Workload, device="cpu", with_grad=True):
+    """Dict of bf16 tensors: q_clean,k_clean,v_clean,q_noisy,k_noisy,v_noisy and (optionally)
+    do_clean, do_noisy.  The same seed on the same device type gives the same bits; callers
+    that compare two implementations hand both the SAME tensors."""
+    g = torch.Generator(device=device)
+    g.manual_seed(w.seed)
+    out = {}
+
+    def draw(heads, sigma):
+        return torch.randn(w.batch, w.L, heads, w.d, generator=g, device=device,
+                           dtype=torch.float32) * sigma
+
+    for stream in ("clean", "noisy"):
+        q, k, v = draw(w.H, 0.5), draw(w.H_kv, 0.5), draw(w.H_kv, 0.5)
+        if w.rope_theta > 0:
+            q, k = _rope(q, w.rope_theta), _rope(k, w.rope_theta)
+        out[f"q_{stream}"] = q.to(torch.bfloat16)
+        out[f"k_{stream}"] = k.to(torch.bfloat16)
+        out[f"v_{stream}"] = v.to(torch.bfloat16)
+        del q, k, v
+    if with_grad:
+        for stream in ("clean", "noisy"):
+            out[f"do_{stream}"] = draw(w.H, 1.0).to(torch.bfloat16)
+    return out
+
+
+def to_f64(t: torch.Tensor) -> np.ndarray:
+    """Exact widening of a (bf16/fp32) tensor to a float64 numpy array on the host."""
+    return t.detach().to("cpu").to(torch.float64).numpy()
+
+
+def sample_rows(w: Workload, n: int, seed: int, extra=()):
+    """Stratified query rows for the sampled-row checks: the rows where masks change
+    (sequence ends, block and 128-tile boundaries, K/V-shard boundaries) plus a uniform
+    random remainder.  Returns a sorted int64 array of n distinct rows in [0, L)."""
+    L, M = w.L, w.block_size
+    rng = np.random.default_rng(seed)
+    fixed = [0, 1, M - 1, M, 127, 128, L - M - 1, L - M, L - 1, L // 2 - 1, L // 2]
+    for blk in rng.integers(0, L // M, size=4):
+        fixed += [int(blk) * M, int(blk) * M + M - 1]
+    if w.kv_shards > 1:
+        step = L // w.kv_shards
+        for s in range(1, w.kv_shards):
+            fixed += [s * step - 1, s * step, s * step + M]
+    fixed += list(extra)
+    rows = sorted({r for r in fixed if 0 <= r < L})
+    rows = rows[:n]
+    if len(rows) < min(n, L):
+        pool = np.setdiff1d(np.arange(L), np.asarray(rows, dtype=np.int64))
+        more = rng.choice(pool, size=min(n, L) - len(rows), replace=False)
+        rows = sorted(set(rows) | set(int(x) for x in more))
+    return np.asarray(rows, dtype=np.int64)
