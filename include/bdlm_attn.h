@@ -1,0 +1,127 @@
+/*
+ * bdlm_attn.h -- C ABI of the block-diffusion (BDLM) attention layer for B200 (sm_100a).
+ *
+ * The layer (paper section 3.2; appendix A, Eqs. correctness-clean-attention and
+ * correctness-corrupted-attention): a length-L clean stream and a length-L corrupted
+ * ("noisy") stream, cut into blocks of `block_size` tokens.
+ *   - clean query i      sees clean keys 0..i                     (clean_mask_mode 0)
+ *   - noisy query i      sees noisy keys of its own block (bidirectional) and the clean
+ *                        keys of all earlier blocks: j < floor(i/block_size)*block_size
+ * Scores are q.k * scale (scale = 1/sqrt(d), Eq. context-parallel-attention), softmax is
+ * taken over the visible keys, LSE is the natural-log row log-sum-exp of the scaled scores.
+ * Partials over disjoint key sets are combined exactly by Eq. csbp-lse-merge.
+ *
+ * Conventions for every entry point
+ *   - All tensor pointers are DEVICE pointers, contiguous, 16-byte aligned, owned by the
+ *     caller.  The library allocates and frees nothing; work is enqueued on `cuda_stream`
+ *     (a cudaStream_t passed as void*, NULL = default stream) and the call returns without
+ *     synchronising.  Outputs are overwritten.
+ *   - Layouts: q, o, do, dq  [batch, L, H, d]      bf16
+ *              k, v, dk, dv  [batch, L, H_kv, d]   bf16   (query head h reads KV head h/(H/H_kv))
+ *              lse           [batch, H, L]         fp32
+ *   - Return value: 0 on success, a negative bdlm_status otherwise.  Arguments are
+ *     checked before anything is launched; a failed check launches nothing.  The library
+ *     never aborts, traps or prints.
+ */
+#ifndef BDLM_ATTN_H_
+#define BDLM_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  BDLM_OK = 0,
+  BDLM_ERR_INVALID_ARG = -1,        /* null/misaligned pointer, bad size, H % H_kv, L % block_size, bad shard range */
+  BDLM_ERR_UNSUPPORTED = -2,        /* d not in {64,128}; device is not sm_100; sharded backward */
+  BDLM_ERR_WORKSPACE_TOO_SMALL = -3,
+  BDLM_ERR_CUDA = -4,               /* a CUDA runtime/driver call or a launch failed */
+  BDLM_ERR_DEVICE_TIMEOUT = -5      /* a bounded device-side wait expired (see bdlm_get_device_status) */
+} bdlm_status;
+
+typedef struct {
+  int32_t batch, L, block_size, H, H_kv, d;
+  float   scale;               /* 0 => 1/sqrt(d) */
+  int32_t clean_mask_mode;     /* 0: clean query i sees clean keys <= i (the paper's block-causal mask);
+                                  1: clean query sees its whole own clean block as well */
+  int32_t kv_begin, kv_end;    /* clean key positions [kv_begin, kv_end) present in this call (one context
+                                  shard C_r, Eq. correctness-clean-partition).  kv_end == 0 with kv_begin == 0
+                                  means 0..L unless kv_range_set != 0.  k_clean/v_clean still point at
+                                  position 0 of the full [batch, L, H_kv, d] tensors. */
+  int32_t kv_range_set;        /* 0: ignore kv_begin/kv_end (full range); 1: use them (may be empty) */
+  int32_t include_noisy_diag;  /* 1: noisy queries also attend their own noisy block; 0: clean-shard partial only */
+  int32_t impl;                /* 0: automatic; 1: force the portable mma.sync kernels; 2: force the tcgen05 kernels */
+  int32_t reserved[5];
+} bdlm_params;
+
+enum { BDLM_WS_FWD = 0, BDLM_WS_BWD = 1 };
+
+/* Scratch bytes a call needs for these parameters (`which` = BDLM_WS_FWD or BDLM_WS_BWD).
+ * Returns 0 when none is needed or the parameters are invalid. */
+size_t bdlm_workspace_bytes(const bdlm_params* p, int32_t which);
+
+/*
+ * Forward (Algorithm 1 without the all-gather; Eq. csbp-block-attention).  For every clean
+ * and noisy query row writes the normalised output and its LSE.  A stream is skipped when
+ * its q pointer is NULL (its o/lse may then be NULL too).  A row whose visible key set is
+ * empty in this call (possible only with a shard range or include_noisy_diag = 0) gets
+ * O = 0 and LSE = -inf.
+ */
+int bdlm_attn_fwd(const bdlm_params* p,
+                  const void* q_clean, const void* k_clean, const void* v_clean,
+                  const void* q_noisy, const void* k_noisy, const void* v_noisy,
+                  void* o_clean, void* o_noisy,
+                  float* lse_clean, float* lse_noisy,
+                  void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Backward (Algorithm 2 without the reduce-scatter; Eqs. correctness-corrupted-gradient,
+ * correctness-clean-gradient, correctness-query-gradient).  Inputs are the forward's inputs,
+ * its saved O and LSE, and the upstream gradient dO of both streams.  dK/dV of a KV head are
+ * summed over the query heads of its group; clean dK/dV are summed over clean and noisy
+ * queries; noisy dK/dV only over the queries of the same block.  The summation order is
+ * fixed, so results are bitwise reproducible.  Requires the full clean key range.
+ * The workspace (bdlm_workspace_bytes(p, BDLM_WS_BWD)) holds D_i = sum_d dO_i,d * O_i,d.
+ */
+int bdlm_attn_bwd(const bdlm_params* p,
+                  const void* q_clean, const void* k_clean, const void* v_clean,
+                  const void* q_noisy, const void* k_noisy, const void* v_noisy,
+                  const void* o_clean, const void* o_noisy,
+                  const float* lse_clean, const float* lse_noisy,
+                  const void* do_clean, const void* do_noisy,
+                  void* dq_clean, void* dk_clean, void* dv_clean,
+                  void* dq_noisy, void* dk_noisy, void* dv_noisy,
+                  void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * LSE merge (Eq. csbp-lse-merge folded left to right; the final division and LSE write of
+ * Implementation 1 are part of the same kernel).  Combines n_partials (1..16) normalised
+ * partial outputs over disjoint key sets.  `o_partials` / `lse_partials` are HOST arrays of
+ * device pointers: o_partials[j] is [rows, H, d] (bf16 if partial_dtype == 0, fp32 if 1),
+ * lse_partials[j] is [batch, H, L] fp32 with rows = batch * L.  A partial row with a
+ * non-finite LSE has weight 0; if all are empty the row gets O = 0, LSE = -inf.
+ * o_out is bf16 [rows, H, d]; lse_out fp32 [batch, H, L].  o_out may be one of the bf16 partials;
+ * lse_out must not be any of the partial LSE buffers (rejected with BDLM_ERR_INVALID_ARG).
+ */
+int bdlm_lse_merge(int32_t n_partials, int32_t batch, int32_t L, int32_t H, int32_t d,
+                   const void* const* o_partials, const float* const* lse_partials,
+                   int32_t partial_dtype,
+                   void* o_out, float* lse_out, void* cuda_stream);
+
+/* Human-readable name of a status code (static storage). */
+const char* bdlm_status_string(int status);
+
+/*
+ * Synchronises `cuda_stream` and returns the device-side status word of the current
+ * device: BDLM_OK, or BDLM_ERR_DEVICE_TIMEOUT if a kernel gave up a bounded wait since the
+ * last call (the word is cleared).  BDLM_ERR_CUDA if the synchronise itself failed.
+ */
+int bdlm_get_device_status(void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* BDLM_ATTN_H_ */

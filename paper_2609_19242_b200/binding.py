@@ -1,0 +1,175 @@
+"""ctypes binding of `libbdlm_attn.so` (declarations in include/bdlm_attn.h).
+
+Argument marshalling only: PyTorch supplies device memory and the current stream; every
+step of the computation runs in the library's kernels.  There is no fallback: if the
+shared library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libbdlm_attn.so")
+
+BDLM_WS_FWD, BDLM_WS_BWD = 0, 1
+IMPL_AUTO, IMPL_PORTABLE, IMPL_TCGEN05 = 0, 1, 2
+
+EXPORTS = ("bdlm_workspace_bytes", "bdlm_attn_fwd", "bdlm_attn_bwd", "bdlm_lse_merge",
+           "bdlm_status_string", "bdlm_get_device_status")
+
+
+class BdlmError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+class BdlmParams(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("L", ctypes.c_int32), ("block_size", ctypes.c_int32),
+                ("H", ctypes.c_int32), ("H_kv", ctypes.c_int32), ("d", ctypes.c_int32),
+                ("scale", ctypes.c_float), ("clean_mask_mode", ctypes.c_int32),
+                ("kv_begin", ctypes.c_int32), ("kv_end", ctypes.c_int32),
+                ("kv_range_set", ctypes.c_int32), ("include_noisy_diag", ctypes.c_int32),
+                ("impl", ctypes.c_int32), ("reserved", ctypes.c_int32 * 5)]
+
+
+_lib = None
+
+
+def lib():
+    """The loaded shared library (loads it on first use; raises if it is not built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} is not built; run `python -m paper_2609_19242_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, pp = ctypes.c_void_p, ctypes.POINTER(BdlmParams)
+        L.bdlm_workspace_bytes.restype = ctypes.c_size_t
+        L.bdlm_workspace_bytes.argtypes = [pp, ctypes.c_int32]
+        L.bdlm_attn_fwd.restype = ctypes.c_int
+        L.bdlm_attn_fwd.argtypes = [pp] + [vp] * 10 + [vp, ctypes.c_size_t, vp]
+        L.bdlm_attn_bwd.restype = ctypes.c_int
+        L.bdlm_attn_bwd.argtypes = [pp] + [vp] * 18 + [vp, ctypes.c_size_t, vp]
+        L.bdlm_lse_merge.restype = ctypes.c_int
+        L.bdlm_lse_merge.argtypes = [ctypes.c_int32] * 5 + [ctypes.POINTER(vp), ctypes.POINTER(vp),
+                                                             ctypes.c_int32, vp, vp, vp]
+        L.bdlm_status_string.restype = ctypes.c_char_p
+        L.bdlm_status_string.argtypes = [ctypes.c_int]
+        L.bdlm_get_device_status.restype = ctypes.c_int
+        L.bdlm_get_device_status.argtypes = [vp]
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().bdlm_status_string(int(status)).decode()
+
+
+bdlm_status_string = status_string
+
+
+def make_params(batch, L, block_size, H, H_kv, d, scale=0.0, clean_mask_mode=0, kv_range=None,
+                include_noisy_diag=True, impl=IMPL_AUTO) -> BdlmParams:
+    p = BdlmParams()
+    p.batch, p.L, p.block_size, p.H, p.H_kv, p.d = batch, L, block_size, H, H_kv, d
+    p.scale = float(scale)
+    p.clean_mask_mode = clean_mask_mode
+    if kv_range is None:
+        p.kv_begin, p.kv_end, p.kv_range_set = 0, 0, 0
+    else:
+        p.kv_begin, p.kv_end, p.kv_range_set = int(kv_range[0]), int(kv_range[1]), 1
+    p.include_noisy_diag = 1 if include_noisy_diag else 0
+    p.impl = impl
+    return p
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "tensors must be contiguous CUDA tensors"
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _shape_params(q, k, block_size, **kw):
+    batch, L, H, d = q.shape
+    return make_params(batch, L, block_size, H, k.shape[2], d, **kw)
+
+
+def bdlm_workspace_bytes(params: BdlmParams, which: int) -> int:
+    return int(lib().bdlm_workspace_bytes(ctypes.byref(params), which))
+
+
+def bdlm_attn_fwd(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, block_size, *,
+                  out=None, scale=0.0, clean_mask_mode=0, kv_range=None, include_noisy_diag=True,
+                  impl=IMPL_AUTO):
+    """Forward of the layer.  Tensors: q [batch,L,H,d], k/v [batch,L,H_kv,d], bf16, on one CUDA
+    device.  Either q may be None (that stream is skipped).  Returns
+    (o_clean, lse_clean, o_noisy, lse_noisy); `out` may supply those four tensors."""
+    qref = q_clean if q_clean is not None else q_noisy
+    p = _shape_params(qref, k_clean, block_size, scale=scale, clean_mask_mode=clean_mask_mode,
+                      kv_range=kv_range, include_noisy_diag=include_noisy_diag, impl=impl)
+    dev = qref.device
+    if out is None:
+        mk_o = lambda q: None if q is None else torch.empty_like(q)
+        mk_l = lambda q: None if q is None else torch.empty(p.batch, p.H, p.L, dtype=torch.float32, device=dev)
+        out = (mk_o(q_clean), mk_l(q_clean), mk_o(q_noisy), mk_l(q_noisy))
+    o_c, l_c, o_n, l_n = out
+    rc = lib().bdlm_attn_fwd(ctypes.byref(p), _ptr(q_clean), _ptr(k_clean), _ptr(v_clean),
+                             _ptr(q_noisy), _ptr(k_noisy), _ptr(v_noisy),
+                             _ptr(o_c), _ptr(o_n), _ptr(l_c), _ptr(l_n), None, 0, _stream())
+    if rc != 0:
+        raise BdlmError(rc, "bdlm_attn_fwd")
+    return o_c, l_c, o_n, l_n
+
+
+def bdlm_attn_bwd(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, o_clean, lse_clean,
+                  o_noisy, lse_noisy, do_clean, do_noisy, block_size, *, out=None, workspace=None,
+                  scale=0.0, clean_mask_mode=0, impl=IMPL_AUTO):
+    """Backward of the layer.  Returns (dq_clean, dk_clean, dv_clean, dq_noisy, dk_noisy, dv_noisy)."""
+    p = _shape_params(q_clean, k_clean, block_size, scale=scale, clean_mask_mode=clean_mask_mode, impl=impl)
+    if out is None:
+        out = tuple(torch.empty_like(t) for t in (q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy))
+    need = bdlm_workspace_bytes(p, BDLM_WS_BWD)
+    if workspace is None:
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=q_clean.device)
+    dq_c, dk_c, dv_c, dq_n, dk_n, dv_n = out
+    rc = lib().bdlm_attn_bwd(ctypes.byref(p), _ptr(q_clean), _ptr(k_clean), _ptr(v_clean),
+                             _ptr(q_noisy), _ptr(k_noisy), _ptr(v_noisy), _ptr(o_clean), _ptr(o_noisy),
+                             _ptr(lse_clean), _ptr(lse_noisy), _ptr(do_clean), _ptr(do_noisy),
+                             _ptr(dq_c), _ptr(dk_c), _ptr(dv_c), _ptr(dq_n), _ptr(dk_n), _ptr(dv_n),
+                             _ptr(workspace), workspace.numel(), _stream())
+    if rc != 0:
+        raise BdlmError(rc, "bdlm_attn_bwd")
+    return out
+
+
+def bdlm_lse_merge(o_partials, lse_partials, *, out=None):
+    """Merge normalised partial outputs [batch,L,H,d] (all bf16 or all fp32) with row LSEs
+    [batch,H,L] over disjoint key sets.  Returns (o bf16, lse fp32)."""
+    n = len(o_partials)
+    batch, L, H, d = o_partials[0].shape
+    dtype = 1 if o_partials[0].dtype == torch.float32 else 0
+    if out is None:
+        out = (torch.empty(batch, L, H, d, dtype=torch.bfloat16, device=o_partials[0].device),
+               torch.empty(batch, H, L, dtype=torch.float32, device=o_partials[0].device))
+    arr_t = ctypes.c_void_p * n
+    o_arr = arr_t(*[t.data_ptr() for t in o_partials])
+    l_arr = arr_t(*[t.data_ptr() for t in lse_partials])
+    for t in list(o_partials) + list(lse_partials):
+        assert t.is_cuda and t.is_contiguous()
+    rc = lib().bdlm_lse_merge(n, batch, L, H, d, o_arr, l_arr, dtype, _ptr(out[0]), _ptr(out[1]), _stream())
+    if rc != 0:
+        raise BdlmError(rc, "bdlm_lse_merge")
+    return out
+
+
+def bdlm_get_device_status() -> int:
+    return int(lib().bdlm_get_device_status(_stream()))

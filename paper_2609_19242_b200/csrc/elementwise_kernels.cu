@@ -1,0 +1,144 @@
+// Bandwidth-bound kernels of the BDLM attention path: the LSE merge of partial outputs
+// (Eq. csbp-lse-merge, with the final division of Implementation 1 fused in) and the
+// backward preprocess D_i = sum_d dO_i,d * O_i,d.
+#include "bdlm_common.cuh"
+
+namespace bdlm {
+namespace {
+
+using bf16 = __nv_bfloat16;
+constexpr int MAX_PARTIALS = 16;
+
+struct MergeArgs {
+  const void* o[MAX_PARTIALS];
+  const float* lse[MAX_PARTIALS];
+  int n;
+};
+
+// One thread owns 8 consecutive head-dim elements of one (row, head).  The running state
+// (numerator, m, normaliser) stays in fp32 registers until the final division, so no thread
+// reads state another thread has already overwritten.
+template <bool F32IN>
+__global__ void __launch_bounds__(256) merge_kernel(MergeArgs ma, int64_t total_chunks, int L, int H, int d,
+                                                    bf16* __restrict__ o_out, float* __restrict__ lse_out) {
+  const int cpr = d / 8;   // chunks per (row, head)
+  for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total_chunks;
+       idx += (int64_t)gridDim.x * blockDim.x) {
+    const int c = (int)(idx % cpr);
+    const int64_t rh = idx / cpr;
+    const int h = (int)(rh % H);
+    const int64_t row = rh / H;
+    const int64_t bidx = row / L;
+    const int i = (int)(row % L);
+    const int64_t lidx = (bidx * H + h) * L + i;
+    float num[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) num[e] = 0.f;
+    float m = -INFINITY, norm = 0.f;
+    for (int j = 0; j < ma.n; ++j) {
+      const float z = ma.lse[j][lidx];
+      const float m_new = fmaxf(m, z);
+      const float w_acc = isfinite(m) ? expf(m - m_new) : 0.f;
+      const float w_j = isfinite(z) ? expf(z - m_new) : 0.f;
+      float x[8];
+      if (F32IN) {
+        const float4* p = reinterpret_cast<const float4*>(static_cast<const float*>(ma.o[j]) + idx * 8);
+        float4 u = p[0], v = p[1];
+        x[0] = u.x; x[1] = u.y; x[2] = u.z; x[3] = u.w; x[4] = v.x; x[5] = v.y; x[6] = v.z; x[7] = v.w;
+      } else {
+        uint4 u = *reinterpret_cast<const uint4*>(static_cast<const bf16*>(ma.o[j]) + idx * 8);
+        const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          float2 f = __bfloat1622float2(p2[e]);
+          x[2 * e] = f.x; x[2 * e + 1] = f.y;
+        }
+      }
+#pragma unroll
+      for (int e = 0; e < 8; ++e) num[e] = w_acc * num[e] + w_j * x[e];
+      norm = w_acc * norm + w_j;
+      m = m_new;
+    }
+    const float inv = norm > 0.f ? 1.f / norm : 0.f;
+    uint4 outv;
+    uint32_t* ow = reinterpret_cast<uint32_t*>(&outv);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) ow[e] = pack_bf16(num[2 * e] * inv, num[2 * e + 1] * inv);
+    *reinterpret_cast<uint4*>(o_out + idx * 8) = outv;
+    if (c == 0) lse_out[lidx] = norm > 0.f ? m + logf(norm) : -INFINITY;
+  }
+}
+
+// One warp per (batch, row, head): D = sum over d of dO * O, fp32.
+template <int D>
+__global__ void __launch_bounds__(256) dsum_kernel(const bf16* __restrict__ dout, const bf16* __restrict__ o,
+                                                   float* __restrict__ dsum, int64_t nrows, int L, int H) {
+  const int lane = threadIdx.x & 31;
+  const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  if (w >= nrows) return;   // whole warp leaves together
+  constexpr int EPL = D / 32;   // elements per lane: 4 (d=128) or 2 (d=64)
+  const bf16* pa = dout + w * D + lane * EPL;
+  const bf16* pb = o + w * D + lane * EPL;
+  float acc = 0.f;
+  if (EPL == 4) {
+    uint2 ua = *reinterpret_cast<const uint2*>(pa), ub = *reinterpret_cast<const uint2*>(pb);
+    float2 a0 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&ua.x));
+    float2 a1 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&ua.y));
+    float2 b0 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&ub.x));
+    float2 b1 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&ub.y));
+    acc = a0.x * b0.x + a0.y * b0.y + a1.x * b1.x + a1.y * b1.y;
+  } else {
+    uint32_t ua = *reinterpret_cast<const uint32_t*>(pa), ub = *reinterpret_cast<const uint32_t*>(pb);
+    float2 a0 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&ua));
+    float2 b0 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&ub));
+    acc = a0.x * b0.x + a0.y * b0.y;
+  }
+#pragma unroll
+  for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
+  if (lane == 0) {
+    // w indexes [batch, L, H]; D is stored [batch, H, L]
+    const int h = (int)(w % H);
+    const int64_t row = w / H;
+    const int64_t bidx = row / L;
+    const int i = (int)(row % L);
+    dsum[(bidx * H + h) * L + i] = acc;
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_merge(int n, int batch, int L, int H, int d, const void* const* o_parts,
+                         const float* const* lse_parts, int dtype, void* o_out, float* lse_out,
+                         cudaStream_t st) {
+  MergeArgs ma;
+  ma.n = n;
+  for (int j = 0; j < MAX_PARTIALS; ++j) {
+    ma.o[j] = j < n ? o_parts[j] : nullptr;
+    ma.lse[j] = j < n ? lse_parts[j] : nullptr;
+  }
+  const int64_t total = (int64_t)batch * L * H * (d / 8);
+  int64_t want = (total + 255) / 256;
+  int blocks = (int)(want < 148 * 16 ? (want > 0 ? want : 1) : 148 * 16);
+  if (dtype == 1)
+    merge_kernel<true><<<blocks, 256, 0, st>>>(ma, total, L, H, d, static_cast<bf16*>(o_out), lse_out);
+  else
+    merge_kernel<false><<<blocks, 256, 0, st>>>(ma, total, L, H, d, static_cast<bf16*>(o_out), lse_out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_dsum(const KArgs& a, float* dsum_clean, float* dsum_noisy, cudaStream_t st) {
+  const int64_t nrows = (int64_t)a.batch * a.L * a.H;
+  const int blocks = (int)((nrows * 32 + 255) / 256);
+  float* out[2] = {dsum_clean, dsum_noisy};
+  for (int s = 0; s < 2; ++s) {
+    if (a.d == 128)
+      dsum_kernel<128><<<blocks, 256, 0, st>>>(a.dout[s], a.o[s], out[s], nrows, a.L, a.H);
+    else
+      dsum_kernel<64><<<blocks, 256, 0, st>>>(a.dout[s], a.o[s], out[s], nrows, a.L, a.H);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+}  // namespace bdlm

@@ -1,0 +1,142 @@
+"""Helpers for the GPU-vs-oracle parity tests: run the CUDA path through the binding, run the
+fp64 oracle on the same bf16 bits, compare within the stated tolerances."""
+import numpy as np
+import torch
+
+from oracle import bdlm_oracle as orc
+from paper_2609_19242_b200 import binding, synth
+
+# Tolerances of the parity bar (bf16 inputs, fp32 accumulation, bf16 P and dS operands).
+TOL_O = 1e-2          # max |dO| elementwise on outputs
+TOL_LSE = 1e-3        # max |dLSE|
+TOL_GRAD = 2e-2       # relative L2 error of each of dQ, dK, dV per stream
+
+NAMES6 = ["q_clean", "k_clean", "v_clean", "q_noisy", "k_noisy", "v_noisy"]
+
+
+def rel_l2(got, ref):
+    ref = np.asarray(ref, dtype=np.float64)
+    got = np.asarray(got, dtype=np.float64)
+    den = np.linalg.norm(ref.ravel())
+    if den == 0:
+        return float(np.linalg.norm(got.ravel()))
+    return float(np.linalg.norm((got - ref).ravel()) / den)
+
+
+def to_cuda(inp):
+    return {k: v.cuda().contiguous() for k, v in inp.items()}
+
+
+def f64(inp):
+    return {k: synth.to_f64(v) for k, v in inp.items()}
+
+
+def gpu_fwd(g, M, **kw):
+    return binding.bdlm_attn_fwd(*[g[n] for n in NAMES6], M, **kw)
+
+
+def gpu_bwd(g, fwd_out, M, do_clean=None, do_noisy=None, **kw):
+    o_c, l_c, o_n, l_n = fwd_out
+    return binding.bdlm_attn_bwd(*[g[n] for n in NAMES6], o_c, l_c, o_n, l_n,
+                                 g["do_clean"] if do_clean is None else do_clean,
+                                 g["do_noisy"] if do_noisy is None else do_noisy, M, **kw)
+
+
+def check_full(w, impl, mode=0, check_bwd=True, inp=None):
+    """Whole-tensor parity against the full oracle (small shapes)."""
+    inp = synth.make_inputs(w, "cpu") if inp is None else inp
+    g = to_cuda(inp)
+    x = f64(inp)
+    M = w.block_size
+    out = gpu_fwd(g, M, clean_mask_mode=mode, impl=impl)
+    torch.cuda.synchronize()
+    ref = orc.attn_forward(*[x[n] for n in NAMES6], M, clean_mask_mode=mode)
+    for got, want, name in zip(out, ref, ["o_clean", "lse_clean", "o_noisy", "lse_noisy"]):
+        gotn = synth.to_f64(got)
+        assert np.isfinite(gotn).all(), name
+        err = np.abs(gotn - want).max()
+        assert err <= (TOL_LSE if "lse" in name else TOL_O), (name, err)
+    if not check_bwd:
+        return
+    grads = gpu_bwd(g, out, M, clean_mask_mode=mode, impl=impl)
+    torch.cuda.synchronize()
+    gref = orc.attn_backward(*[x[n] for n in NAMES6], x["do_clean"], x["do_noisy"], M, clean_mask_mode=mode)
+    for got, want, name in zip(grads, gref, ["dq_clean", "dk_clean", "dv_clean", "dq_noisy", "dk_noisy", "dv_noisy"]):
+        gotn = synth.to_f64(got)
+        assert np.isfinite(gotn).all(), name
+        err = rel_l2(gotn, want)
+        assert err <= TOL_GRAD, (name, err)
+    assert binding.bdlm_get_device_status() == 0
+
+
+def check_sampled(w, impl, n_rows=256, g=None, fwd_out=None, check_bwd=True, report=None):
+    """Sampled-row parity for sizes the full oracle cannot do: per (batch, head, stream)
+    `n_rows` stratified query rows are recomputed by the oracle.  O and LSE come from the
+    full forward.  dQ at the sampled rows comes from the full backward (a row's dQ depends on
+    that row's dO only).  dK/dV are linear in dO, so a second backward with dO zeroed outside
+    the sampled rows is compared, for every key, with the oracle's sum over those rows."""
+    M = w.block_size
+    if g is None:
+        g = synth.make_inputs(w, "cuda")
+    if fwd_out is None:
+        fwd_out = gpu_fwd(g, M, impl=impl)
+    torch.cuda.synchronize()
+    G = w.H // w.H_kv
+    rows_of = {}
+    for b in range(w.batch):
+        for h in range(w.H):
+            for s in (0, 1):
+                rows_of[(b, h, s)] = synth.sample_rows(w, n_rows, seed=1000 * b + 10 * h + s)
+    grads = grads_sp = None
+    if check_bwd:
+        grads = gpu_bwd(g, fwd_out, M, impl=impl)
+        do_sp = [torch.zeros_like(g["do_clean"]), torch.zeros_like(g["do_noisy"])]
+        for (b, h, s), rows in rows_of.items():
+            r = torch.from_numpy(rows).cuda()
+            src = g["do_clean"] if s == 0 else g["do_noisy"]
+            do_sp[s][b, r, h] = src[b, r, h]
+        grads_sp = gpu_bwd(g, fwd_out, M, do_clean=do_sp[0], do_noisy=do_sp[1], impl=impl)
+        torch.cuda.synchronize()
+        assert binding.bdlm_get_device_status() == 0
+    worst = {"o": 0.0, "lse": 0.0, "dq": 0.0, "dk": 0.0, "dv": 0.0}
+    qn = ["q_clean", "q_noisy"]
+    don = ["do_clean", "do_noisy"]
+    for b in range(w.batch):
+        for hk in range(w.H_kv):
+            kv = {n: synth.to_f64(g[n][b, :, hk]) for n in ("k_clean", "v_clean", "k_noisy", "v_noisy")}
+            acc = {n: np.zeros((w.L, w.d)) for n in ("dk_clean", "dv_clean", "dk_noisy", "dv_noisy")}
+            dq_num = [0.0, 0.0]
+            dq_den = [0.0, 0.0]
+            for h in range(hk * G, (hk + 1) * G):
+                for s in (0, 1):
+                    rows = rows_of[(b, h, s)]
+                    rt = torch.from_numpy(rows).cuda()
+                    q_rows = synth.to_f64(g[qn[s]][b, rt, h])
+                    do_rows = synth.to_f64(g[don[s]][b, rt, h]) if check_bwd else None
+                    ref = orc.attn_rows(s, rows, q_rows, kv["k_clean"], kv["v_clean"], kv["k_noisy"],
+                                        kv["v_noisy"], M, do_rows=do_rows)
+                    o_got = synth.to_f64(fwd_out[2 * s][b, rt, h])
+                    l_got = synth.to_f64(fwd_out[2 * s + 1][b, h, rt])
+                    worst["o"] = max(worst["o"], float(np.abs(o_got - ref["o"]).max()))
+                    worst["lse"] = max(worst["lse"], float(np.abs(l_got - ref["lse"]).max()))
+                    if check_bwd:
+                        dq_got = synth.to_f64(grads[3 * s][b, rt, h])
+                        dq_num[s] += float(((dq_got - ref["dq"]) ** 2).sum())
+                        dq_den[s] += float((ref["dq"] ** 2).sum())
+                        for n in acc:
+                            acc[n] += ref[n]
+            if check_bwd:
+                for s in (0, 1):
+                    worst["dq"] = max(worst["dq"], (dq_num[s] / max(dq_den[s], 1e-300)) ** 0.5)
+                idx = {"dk_clean": 1, "dv_clean": 2, "dk_noisy": 4, "dv_noisy": 5}
+                for n, want in acc.items():
+                    got = synth.to_f64(grads_sp[idx[n]][b, :, hk])
+                    assert np.isfinite(got).all(), n
+                    worst[n[:2]] = max(worst[n[:2]], rel_l2(got, want))
+    if report is not None:
+        report.update(worst)
+    assert worst["o"] <= TOL_O, worst
+    assert worst["lse"] <= TOL_LSE, worst
+    if check_bwd:
+        assert worst["dq"] <= TOL_GRAD and worst["dk"] <= TOL_GRAD and worst["dv"] <= TOL_GRAD, worst
+    return worst

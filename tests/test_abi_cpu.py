@@ -1,0 +1,81 @@
+"""CPU-only checks of the boundary: the shared library loads, exports every function the
+header declares, and rejects bad arguments before touching a device."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2609_19242_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_functions():
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for f in os.listdir(inc):
+        if f.endswith(".h"):
+            src = open(os.path.join(inc, f)).read()
+            src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+            names |= set(re.findall(r"\b(bdlm_[a-z0-9_]+)\s*\(", src))
+    return names
+
+
+def test_library_exports_every_declared_symbol():
+    L = binding.lib()
+    declared = _declared_functions()
+    assert {"bdlm_attn_fwd", "bdlm_attn_bwd", "bdlm_lse_merge"} <= declared
+    for name in declared:
+        assert hasattr(L, name), name
+    assert declared >= set(binding.EXPORTS)
+
+
+def test_status_strings():
+    assert binding.status_string(0) == "BDLM_OK"
+    assert binding.status_string(-1) == "BDLM_ERR_INVALID_ARG"
+    assert binding.status_string(-5) == "BDLM_ERR_DEVICE_TIMEOUT"
+    assert binding.status_string(-99) == "BDLM_ERR_UNKNOWN"
+
+
+@pytest.mark.parametrize("kw,code", [
+    (dict(batch=0), -1), (dict(L=100, block_size=16), -1), (dict(H=6, H_kv=4), -1),
+    (dict(d=96), -2), (dict(clean_mask_mode=3), -1), (dict(kv_range=(8, 4)), -1),
+    (dict(kv_range=(0, 4096)), -1), (dict(scale=-1.0), -1), (dict(impl=7), -1),
+])
+def test_bad_parameters_are_rejected_without_a_device(kw, code):
+    base = dict(batch=1, L=256, block_size=16, H=4, H_kv=2, d=64)
+    base.update(kw)
+    p = binding.make_params(**base)
+    fake = ctypes.c_void_p(0x1000)   # never dereferenced: parameter checks come first
+    rc = binding.lib().bdlm_attn_fwd(ctypes.byref(p), *([fake] * 10), None, 0, None)
+    assert rc == code
+    assert binding.bdlm_workspace_bytes(p, binding.BDLM_WS_BWD) == 0
+
+
+def test_null_and_misaligned_pointers_are_rejected():
+    p = binding.make_params(1, 256, 16, 4, 2, 64)
+    ok = ctypes.c_void_p(0x1000)
+    bad = ctypes.c_void_p(0x1004)
+    L = binding.lib()
+    assert L.bdlm_attn_fwd(ctypes.byref(p), None, ok, ok, None, ok, ok, ok, ok, ok, ok, None, 0, None) == -1
+    assert L.bdlm_attn_fwd(ctypes.byref(p), ok, None, ok, ok, ok, ok, ok, ok, ok, ok, None, 0, None) == -1
+    assert L.bdlm_attn_fwd(ctypes.byref(p), bad, ok, ok, ok, ok, ok, ok, ok, ok, ok, None, 0, None) == -1
+    assert L.bdlm_attn_fwd(None, *([ok] * 10), None, 0, None) == -1
+    args = [ok] * 18
+    assert L.bdlm_attn_bwd(ctypes.byref(p), *args, None, 0, None) == -1           # null workspace
+    assert L.bdlm_attn_bwd(ctypes.byref(p), *args, ok, 16, None) == -3            # workspace too small
+    ps = binding.make_params(1, 256, 16, 4, 2, 64, kv_range=(0, 128))
+    assert L.bdlm_attn_bwd(ctypes.byref(ps), *args, ok, 1 << 30, None) == -2       # sharded backward
+    arr = (ctypes.c_void_p * 2)(0x1000, 0x2000)
+    assert L.bdlm_lse_merge(0, 1, 8, 1, 64, arr, arr, 0, ok, ok, None) == -1
+    assert L.bdlm_lse_merge(17, 1, 8, 1, 64, arr, arr, 0, ok, ok, None) == -1
+    assert L.bdlm_lse_merge(2, 1, 8, 1, 60, arr, arr, 0, ok, ok, None) == -1
+    assert L.bdlm_lse_merge(2, 1, 8, 1, 64, arr, arr, 0, ok, ctypes.c_void_p(0x2000), None) == -1  # lse aliasing
+
+
+def test_workspace_size_formula():
+    p = binding.make_params(2, 512, 32, 8, 2, 128, impl=binding.IMPL_PORTABLE)
+    need = binding.bdlm_workspace_bytes(p, binding.BDLM_WS_BWD)
+    assert need >= 2 * 2 * 8 * 512 * 4
+    assert binding.bdlm_workspace_bytes(p, binding.BDLM_WS_FWD) == 0

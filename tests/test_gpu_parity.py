@@ -1,0 +1,116 @@
+"""GPU-vs-oracle parity, whole tensors, at sizes the full oracle finishes in seconds: several
+tiles and ragged tails, the block-size extremes, both mask modes, GQA, K/V shards + merge."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import bdlm_oracle as orc
+from paper_2609_19242_b200 import binding, synth
+from paper_2609_19242_b200.synth import Workload, WORKLOADS
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+IMPLS = [binding.IMPL_PORTABLE, binding.IMPL_AUTO]
+
+SMALL = [
+    WORKLOADS["tiny"],
+    Workload("d128_3tiles", 2, 4, 2, 128, 384, 32),
+    Workload("ragged_tail", 1, 2, 1, 64, 200, 8),
+    Workload("m1", 1, 2, 2, 64, 96, 1),
+    Workload("m_eq_L", 1, 2, 1, 128, 128, 128),
+    Workload("m256", 1, 4, 1, 128, 512, 256),
+    Workload("m48_odd", 1, 2, 2, 128, 336, 48),
+    Workload("gqa8", 1, 8, 1, 128, 256, 64, rope_theta=5e5),
+    Workload("m128", 1, 2, 1, 128, 640, 128),
+    Workload("m16_d128", 1, 2, 2, 128, 512, 16),
+]
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("w", SMALL, ids=lambda w: w.name)
+def test_forward_backward_match_oracle(w, impl):
+    pu.check_full(w, impl)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_clean_mask_mode_1(impl):
+    pu.check_full(Workload("mode1", 1, 2, 1, 128, 384, 32), impl, mode=1)
+    pu.check_full(Workload("mode1_big_block", 1, 2, 1, 64, 512, 256), impl, mode=1)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("cuts", [[0, 128, 256, 384], [0, 40, 200, 384], [0, 0, 384]])
+def test_shard_partials_and_merge(impl, cuts):
+    """Clean-K/V shard partials plus the noisy-diagonal partial, merged on the GPU, equal the
+    unsharded kernel and the oracle; each partial equals the oracle's partial."""
+    w = Workload("shards", 2, 4, 2, 128, 384, 32)
+    inp = synth.make_inputs(w, "cpu", with_grad=False)
+    g = pu.to_cuda(inp)
+    x = pu.f64(inp)
+    M = w.block_size
+    parts = []
+    for a, b in zip(cuts[:-1], cuts[1:]):
+        out = pu.gpu_fwd(g, M, kv_range=(a, b), include_noisy_diag=False, impl=impl)
+        ref = orc.attn_forward(*[x[n] for n in pu.NAMES6], M, kv_begin=a, kv_end=b, include_noisy_diag=False)
+        for got, want in zip(out, ref):
+            gotn = synth.to_f64(got)
+            assert not np.isnan(gotn).any()
+            assert (np.isneginf(gotn) == np.isneginf(want)).all()
+            fin = np.isfinite(want)
+            assert np.abs(gotn[fin] - want[fin]).max() <= pu.TOL_O if fin.any() else True
+        parts.append(out)
+    diag = binding.bdlm_attn_fwd(None, g["k_clean"], g["v_clean"], g["q_noisy"], g["k_noisy"], g["v_noisy"], M,
+                                 kv_range=(0, 0), impl=impl)
+    o_c, l_c = binding.bdlm_lse_merge([p[0] for p in parts], [p[1] for p in parts])
+    o_n, l_n = binding.bdlm_lse_merge([p[2] for p in parts] + [diag[2]], [p[3] for p in parts] + [diag[3]])
+    torch.cuda.synchronize()
+    full_ref = orc.attn_forward(*[x[n] for n in pu.NAMES6], M)
+    full_gpu = pu.gpu_fwd(g, M, impl=impl)
+    for got, want, unsh, name in zip((o_c, l_c, o_n, l_n), full_ref, full_gpu, ["oc", "lc", "on", "ln"]):
+        tol = pu.TOL_LSE if name[0] == "l" else pu.TOL_O
+        assert np.abs(synth.to_f64(got) - want).max() <= tol, name
+        assert np.abs(synth.to_f64(got) - synth.to_f64(unsh)).max() <= tol, name
+
+
+def test_merge_kernel_matches_oracle_merge():
+    """bdlm_lse_merge alone: bf16 and fp32 partials, empty (-inf) rows, all-empty rows."""
+    rng = np.random.default_rng(5)
+    B, L, H, d, n = 2, 300, 3, 64, 5
+    for dtype in (torch.bfloat16, torch.float32):
+        os_ = [torch.tensor(rng.normal(size=(B, L, H, d)), dtype=dtype) for _ in range(n)]
+        ls = [torch.tensor(rng.normal(size=(B, H, L)) * 4, dtype=torch.float32) for _ in range(n)]
+        ls[1][:, :, :50] = -float("inf")
+        for l in ls:
+            l[:, :, 100:110] = -float("inf")     # rows empty in every partial
+        o, l = binding.bdlm_lse_merge([t.cuda() for t in os_], [t.cuda() for t in ls])
+        torch.cuda.synchronize()
+        ro, rl = orc.lse_merge([synth.to_f64(t) for t in os_], [synth.to_f64(t) for t in ls])
+        got_l = synth.to_f64(l)
+        assert (np.isneginf(got_l) == np.isneginf(rl)).all()
+        fin = np.isfinite(rl)
+        assert np.abs(got_l[fin] - rl[fin]).max() <= 1e-5
+        assert np.abs(synth.to_f64(o) - ro).max() <= 2e-2   # bf16 output rounding of |O| up to ~4
+        assert np.abs(synth.to_f64(o)[:, 100:110]).max() == 0
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_backward_is_bitwise_reproducible(impl):
+    w = Workload("repro", 1, 4, 2, 128, 384, 32)
+    g = pu.to_cuda(synth.make_inputs(w, "cpu"))
+    out = pu.gpu_fwd(g, w.block_size, impl=impl)
+    a = [t.clone() for t in pu.gpu_bwd(g, out, w.block_size, impl=impl)]
+    b = pu.gpu_bwd(g, out, w.block_size, impl=impl)
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
+
+
+def test_skipping_a_stream():
+    w = Workload("skip", 1, 2, 1, 128, 256, 32)
+    g = pu.to_cuda(synth.make_inputs(w, "cpu", with_grad=False))
+    full = pu.gpu_fwd(g, w.block_size)
+    only_n = binding.bdlm_attn_fwd(None, g["k_clean"], g["v_clean"], g["q_noisy"], g["k_noisy"], g["v_noisy"], w.block_size)
+    only_c = binding.bdlm_attn_fwd(g["q_clean"], g["k_clean"], g["v_clean"], None, None, None, w.block_size)
+    assert only_n[0] is None and torch.equal(only_n[2], full[2]) and torch.equal(only_n[3], full[3])
+    assert only_c[2] is None and torch.equal(only_c[0], full[0]) and torch.equal(only_c[1], full[1])
