@@ -1,0 +1,356 @@
+#!/usr/bin/env python
+"""Benchmark of the BDLM attention layer (forward + backward) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 32k] [--impl ours|reference]
+
+A step is one forward plus one backward of the whole layer over one batch of seeded
+synthetic inputs.  `value` counts FLOPs of unmasked (query, key) pairs only
+(14 * d per pair: 4d forward, 10d backward).  Prints ONE JSON line on rank 0.
+
+With N > 1 (launched by torch.distributed.run) every rank runs an independent replica on its
+own GPU: the layer as specified does not shard and has no collective, so the aggregate is
+N replicas ("replicas only", weak scaling); ranks only meet at the timing barriers.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2609_19242_b200 import synth  # noqa: E402
+
+METRIC = "BDLM attn fwd+bwd TFLOP/s (unmasked FLOPs)"
+UNIT = "TFLOP/s"
+NAMES6 = ["q_clean", "k_clean", "v_clean", "q_noisy", "k_noisy", "v_noisy"]
+
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant
+# kernel, from the ncu captures summarised under profiles/ ; keyed by (workload, kernel).
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"bf16_tflops": float(p["bf16_tflops"]), "bf16_tflops_sustained": float(p["bf16_tflops_sustained"]),
+                "hbm_gbs": float(p["hbm_gbs"]), "source": "measured"}
+    return {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-i", str(self.index), "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.thread.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def physical_gpu_index(local):
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        parts = [p for p in vis.split(",") if p != ""]
+        if local < len(parts) and parts[local].isdigit():
+            return int(parts[local])
+    return local
+
+
+# ------------------------------------------------------------------------------------------
+# reference arm / cpu baseline: the fp64 oracle on a bounded sample of the workload
+# ------------------------------------------------------------------------------------------
+def oracle_sample(w, inp_cpu, rows_per_stream, seed):
+    """Runs the oracle (forward + backward) for `rows_per_stream` sampled query rows of one
+    (batch 0, head 0) per stream.  Returns (seconds, FLOPs of the visible pairs of those rows)."""
+    from oracle import bdlm_oracle as orc
+    M = w.block_size
+    kv = {n: synth.to_f64(inp_cpu[n][0, :, 0]) for n in ("k_clean", "v_clean", "k_noisy", "v_noisy")}
+    rng = np.random.default_rng(seed)
+    flops = 0
+    t0 = time.perf_counter()
+    for s, (qn, dn) in enumerate((("q_clean", "do_clean"), ("q_noisy", "do_noisy"))):
+        rows = np.sort(rng.choice(w.L, size=min(rows_per_stream, w.L), replace=False))
+        q_rows = synth.to_f64(inp_cpu[qn][0, rows, 0])
+        do_rows = synth.to_f64(inp_cpu[dn][0, rows, 0])
+        orc.attn_rows(s, rows, q_rows, kv["k_clean"], kv["v_clean"], kv["k_noisy"], kv["v_noisy"], M, do_rows=do_rows)
+        pairs = (rows + 1).sum() if s == 0 else ((rows // M + 1) * M).sum()
+        flops += 14 * w.d * int(pairs)
+    return time.perf_counter() - t0, flops
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [i.get("num_threads", 1) for i in threadpool_info() if i.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return len(os.sched_getaffinity(0))
+
+
+def cpu_inputs_for_oracle(w):
+    """bf16 inputs of (batch 0, head 0 / KV head 0) only, on the host, same recipe as the GPU's."""
+    small = synth.small(w, batch=1, H=1, H_kv=1)
+    return synth.make_inputs(small, "cpu")
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    inp = cpu_inputs_for_oracle(w)
+    rows = args.oracle_rows
+    for i in range(args.warmup):
+        oracle_sample(w, inp, max(8, rows // 8), seed=100 + i)
+    t_tot, f_tot = 0.0, 0
+    for i in range(args.steps):
+        t, f = oracle_sample(w, inp, rows, seed=i)
+        t_tot += t
+        f_tot += f
+    val = f_tot / t_tot / 1e12
+    cores = blas_threads()
+    sample = f"{rows} sampled query rows per stream of (batch 0, head 0) per step, fwd+bwd, fp64"
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_tot / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": w.name, "batch": w.batch, "H": w.H, "H_kv": w.H_kv,
+                                            "d": w.d, "L": w.L, "block_size": w.block_size},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------
+def run_ours(args, w):
+    from paper_2609_19242_b200 import binding
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    peaks = load_peaks()
+    M = w.block_size
+    g = synth.make_inputs(synth.small(w, seed=w.seed + rank), "cuda")
+    p = binding.make_params(w.batch, w.L, M, w.H, w.H_kv, w.d)
+    ws = torch.empty(max(16, binding.bdlm_workspace_bytes(p, binding.BDLM_WS_BWD)), dtype=torch.uint8, device="cuda")
+    fwd_out = tuple(t for t in (torch.empty_like(g["q_clean"]),
+                                torch.empty(w.batch, w.H, w.L, dtype=torch.float32, device="cuda"),
+                                torch.empty_like(g["q_noisy"]),
+                                torch.empty(w.batch, w.H, w.L, dtype=torch.float32, device="cuda")))
+    grads = tuple(torch.empty_like(g[n]) for n in NAMES6)
+    impl = args.kernel_impl
+
+    def fwd():
+        binding.bdlm_attn_fwd(*[g[n] for n in NAMES6], M, out=fwd_out, impl=impl)
+
+    def bwd(passes=0):
+        binding.bdlm_attn_bwd(*[g[n] for n in NAMES6], fwd_out[0], fwd_out[1], fwd_out[2], fwd_out[3],
+                              g["do_clean"], g["do_noisy"], M, out=grads, workspace=ws, impl=impl, passes=passes)
+
+    for _ in range(args.warmup):
+        fwd()
+        bwd()
+    torch.cuda.synchronize()
+    if binding.bdlm_get_device_status() != 0:
+        raise RuntimeError("device-side wait timed out during warm-up")
+
+    # ---- timed region: K steps, device time, events between the kernels of a step -------------
+    K = args.steps
+    names = ["fwd", "bwd_dsum", "bwd_dkdv", "bwd_dq"]
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(len(names) + 1)] for _ in range(K)]
+    sampler = ClockSampler(physical_gpu_index(local))
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    barrier()
+    e_start, e_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e_start.record()
+    for i in range(K):
+        ev[i][0].record()
+        fwd()
+        ev[i][1].record()
+        bwd(binding.PASS_DSUM)
+        ev[i][2].record()
+        bwd(binding.PASS_DKDV)
+        ev[i][3].record()
+        bwd(binding.PASS_DQ)
+        ev[i][4].record()
+    e_stop.record()
+    barrier()
+    ms_total = e_start.elapsed_time(e_stop)
+    clocks = sampler.stop() if rank == 0 else None
+    if binding.bdlm_get_device_status() != 0:
+        raise RuntimeError("device-side wait timed out during the timed region")
+    if world > 1:
+        t = torch.tensor([ms_total], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    per_kernel_ms = {n: float(np.mean([ev[i][j].elapsed_time(ev[i][j + 1]) for i in range(K)])) for j, n in enumerate(names)}
+
+    f_fwd, f_bwd = w.flops()
+    ms_step = ms_total / K
+    value = world * (f_fwd + f_bwd) / (ms_step * 1e-3) / 1e12
+
+    # ---- end to end through the public call with HOST buffers (pinned), copies inside ---------
+    e2e = None
+    if rank == 0 or world > 1:
+        host_in = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True).copy_(v) for k, v in g.items()}
+        host_out = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in fwd_out + grads]
+        h2d = sum(t.numel() * t.element_size() for t in host_in.values())
+        d2h = sum(t.numel() * t.element_size() for t in host_out)
+
+        def e2e_step():
+            for k_, v in host_in.items():
+                g[k_].copy_(v, non_blocking=True)
+            fwd()
+            bwd()
+            for dst, src in zip(host_out, fwd_out + grads):
+                dst.copy_(src, non_blocking=True)
+
+        e2e_step()
+        barrier()
+        n_e2e = max(1, min(K, 5))
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(n_e2e):
+            e2e_step()
+        b.record()
+        barrier()
+        ms_e2e = a.elapsed_time(b) / n_e2e
+        if world > 1:
+            t = torch.tensor([ms_e2e], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e2e = float(t.item())
+        e2e = {"value": world * (f_fwd + f_bwd) / (ms_e2e * 1e-3) / 1e12, "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e}
+        del host_in, host_out
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (tensor-bound: algorithmic FLOPs / device time) -------
+    # The counted backward is 5 GEMMs per pair (S, dP, dV, dK, dQ = 10d FLOPs).  The dK/dV pass owns
+    # four of them (8d); the dQ pass owns dQ (2d) -- its recomputation of S and dP is not counted.
+    algo_flops = {"fwd": f_fwd, "bwd_dkdv": f_bwd * 0.8, "bwd_dq": f_bwd * 0.2, "bwd_dsum": 0.0}
+    dom = max(("fwd", "bwd_dkdv", "bwd_dq"), key=lambda n: per_kernel_ms[n])
+    peak = peaks["bf16_tflops_sustained"] if ms_step * K > 1000.0 else peaks["bf16_tflops"]
+    achieved = algo_flops[dom] / (per_kernel_ms[dom] * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": achieved / peak, "peak_source": peaks["source"] +
+                (" sustained" if peak == peaks["bf16_tflops_sustained"] else " burst"),
+                "traffic": NCU_TRAFFIC_BYTES.get((w.name, dom)),
+                "per_kernel_ms": per_kernel_ms,
+                "per_kernel_tflops": {n: (algo_flops[n] / (per_kernel_ms[n] * 1e-3) / 1e12) for n in names}}
+
+    # ---- CPU baseline: the oracle on a bounded sample, on this machine's host cores ---------------
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        inp = cpu_inputs_for_oracle(w)
+        oracle_sample(w, inp, 8, seed=99)
+        t, f = oracle_sample(w, inp, args.oracle_rows, seed=0)
+        cpu = {"value": f / t / 1e12, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+               "sample": f"{args.oracle_rows} sampled query rows per stream of (batch 0, head 0), fwd+bwd, fp64, {t:.1f} s"}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": w.name, "batch": w.batch, "H": w.H, "H_kv": w.H_kv, "d": w.d, "L": w.L,
+                       "block_size": w.block_size, "rope_theta": w.rope_theta, "parallelism": "replicas only",
+                       "l2": "inputs larger than L2 (q/k/v/dO of one step exceed 126 MB)",
+                       "kernel_impl": {0: "auto", 1: "portable", 2: "tcgen05"}[impl]},
+            "pct_of_bf16_peak": {"measured_burst": 100 * value / world / peaks["bf16_tflops"],
+                                 "measured_sustained": 100 * value / world / peaks["bf16_tflops_sustained"],
+                                 "nominal_2250": 100 * value / world / 2250.0, "source": peaks["source"]},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": 5 * K, "roofline": roofline, "cpu_baseline": cpu}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="32k", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--kernel-impl", type=int, default=0, help="0 auto, 1 portable mma.sync, 2 tcgen05")
+    ap.add_argument("--oracle-rows", type=int, default=768)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = synth.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -54,8 +54,13 @@ typedef struct {
   int32_t kv_range_set;        /* 0: ignore kv_begin/kv_end (full range); 1: use them (may be empty) */
   int32_t include_noisy_diag;  /* 1: noisy queries also attend their own noisy block; 0: clean-shard partial only */
   int32_t impl;                /* 0: automatic; 1: force the portable mma.sync kernels; 2: force the tcgen05 kernels */
-  int32_t reserved[5];
+  int32_t bwd_passes;          /* backward only: 0 = all passes; otherwise a bit set of BDLM_BWD_PASS_* to run
+                                  (lets a caller time the passes separately; each pass needs the earlier ones'
+                                  results from a previous call with the same workspace) */
+  int32_t reserved[4];
 } bdlm_params;
+
+enum { BDLM_BWD_PASS_DSUM = 1, BDLM_BWD_PASS_DKDV = 2, BDLM_BWD_PASS_DQ = 4 };
 
 enum { BDLM_WS_FWD = 0, BDLM_WS_BWD = 1 };
 

@@ -16,6 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libbdlm_attn.so")
 
 BDLM_WS_FWD, BDLM_WS_BWD = 0, 1
 IMPL_AUTO, IMPL_PORTABLE, IMPL_TCGEN05 = 0, 1, 2
+PASS_DSUM, PASS_DKDV, PASS_DQ = 1, 2, 4
 
 EXPORTS = ("bdlm_workspace_bytes", "bdlm_attn_fwd", "bdlm_attn_bwd", "bdlm_lse_merge",
            "bdlm_status_string", "bdlm_get_device_status")
@@ -33,7 +34,8 @@ class BdlmParams(ctypes.Structure):
                 ("scale", ctypes.c_float), ("clean_mask_mode", ctypes.c_int32),
                 ("kv_begin", ctypes.c_int32), ("kv_end", ctypes.c_int32),
                 ("kv_range_set", ctypes.c_int32), ("include_noisy_diag", ctypes.c_int32),
-                ("impl", ctypes.c_int32), ("reserved", ctypes.c_int32 * 5)]
+                ("impl", ctypes.c_int32), ("bwd_passes", ctypes.c_int32),
+                ("reserved", ctypes.c_int32 * 4)]
 
 
 _lib = None
@@ -73,7 +75,7 @@ bdlm_status_string = status_string
 
 
 def make_params(batch, L, block_size, H, H_kv, d, scale=0.0, clean_mask_mode=0, kv_range=None,
-                include_noisy_diag=True, impl=IMPL_AUTO) -> BdlmParams:
+                include_noisy_diag=True, impl=IMPL_AUTO, bwd_passes=0) -> BdlmParams:
     p = BdlmParams()
     p.batch, p.L, p.block_size, p.H, p.H_kv, p.d = batch, L, block_size, H, H_kv, d
     p.scale = float(scale)
@@ -84,6 +86,7 @@ def make_params(batch, L, block_size, H, H_kv, d, scale=0.0, clean_mask_mode=0, 
         p.kv_begin, p.kv_end, p.kv_range_set = int(kv_range[0]), int(kv_range[1]), 1
     p.include_noisy_diag = 1 if include_noisy_diag else 0
     p.impl = impl
+    p.bwd_passes = bwd_passes
     return p
 
 
@@ -132,9 +135,10 @@ def bdlm_attn_fwd(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, block_si
 
 def bdlm_attn_bwd(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, o_clean, lse_clean,
                   o_noisy, lse_noisy, do_clean, do_noisy, block_size, *, out=None, workspace=None,
-                  scale=0.0, clean_mask_mode=0, impl=IMPL_AUTO):
+                  scale=0.0, clean_mask_mode=0, impl=IMPL_AUTO, passes=0):
     """Backward of the layer.  Returns (dq_clean, dk_clean, dv_clean, dq_noisy, dk_noisy, dv_noisy)."""
-    p = _shape_params(q_clean, k_clean, block_size, scale=scale, clean_mask_mode=clean_mask_mode, impl=impl)
+    p = _shape_params(q_clean, k_clean, block_size, scale=scale, clean_mask_mode=clean_mask_mode, impl=impl,
+                      bwd_passes=passes)
     if out is None:
         out = tuple(torch.empty_like(t) for t in (q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy))
     need = bdlm_workspace_bytes(p, BDLM_WS_BWD)

@@ -19,6 +19,7 @@ int check_params(const bdlm_params* p) {
   if (p->H % p->H_kv != 0 || p->L % p->block_size != 0) return BDLM_ERR_INVALID_ARG;
   if (p->clean_mask_mode != 0 && p->clean_mask_mode != 1) return BDLM_ERR_INVALID_ARG;
   if (p->impl < 0 || p->impl > 2) return BDLM_ERR_INVALID_ARG;
+  if (p->bwd_passes < 0 || p->bwd_passes > 7) return BDLM_ERR_INVALID_ARG;
   if (!(p->scale >= 0.f) || isinf(p->scale)) return BDLM_ERR_INVALID_ARG;
   if (p->kv_range_set) {
     if (p->kv_begin < 0 || p->kv_end < p->kv_begin || p->kv_end > p->L) return BDLM_ERR_INVALID_ARG;
@@ -150,13 +151,15 @@ int bdlm_attn_bwd(const bdlm_params* p,
 
   const bool tc_ok = tc_bwd_supported(a);
   if (p->impl == 2 && !tc_ok) return BDLM_ERR_UNSUPPORTED;
-  cudaError_t e = launch_dsum(a, ds_c, ds_n, st);
+  const int passes = p->bwd_passes ? p->bwd_passes : 7;
+  cudaError_t e = cudaSuccess;
+  if (passes & BDLM_BWD_PASS_DSUM) e = launch_dsum(a, ds_c, ds_n, st);
   if (e != cudaSuccess) return BDLM_ERR_CUDA;
   if (tc_ok && p->impl != 1) {
     void* extra = static_cast<char*>(workspace) + 2 * dsum_bytes(p);
-    e = launch_tc_bwd(a, extra, st);
+    e = launch_tc_bwd(a, extra, passes, st);
   } else {
-    e = launch_portable_bwd(a, st);
+    e = launch_portable_bwd(a, passes, st);
   }
   return e == cudaSuccess ? BDLM_OK : BDLM_ERR_CUDA;
 }

@@ -66,7 +66,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 // Launchers (host).  Each enqueues on `st` and returns the launch's cudaError_t.
 cudaError_t launch_portable_fwd(const KArgs& a, cudaStream_t st);
-cudaError_t launch_portable_bwd(const KArgs& a, cudaStream_t st);
+cudaError_t launch_portable_bwd(const KArgs& a, int passes, cudaStream_t st);
 cudaError_t launch_dsum(const KArgs& a, float* dsum_clean, float* dsum_noisy, cudaStream_t st);
 cudaError_t launch_merge(int n, int batch, int L, int H, int d, const void* const* o_parts,
                          const float* const* lse_parts, int dtype, void* o_out, float* lse_out,

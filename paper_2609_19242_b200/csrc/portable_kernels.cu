@@ -469,9 +469,9 @@ cudaError_t launch_portable_fwd(const KArgs& a, cudaStream_t st) {
   return cudaGetLastError();
 }
 
-cudaError_t launch_portable_bwd(const KArgs& a, cudaStream_t st) {
-  cudaError_t e;
-  {
+cudaError_t launch_portable_bwd(const KArgs& a, int passes, cudaStream_t st) {
+  cudaError_t e = cudaSuccess;
+  if (passes & BDLM_BWD_PASS_DKDV) {
     dim3 grid((a.L + BQ - 1) / BQ, a.Hkv, a.batch * 2);
     size_t smem = (size_t)(2 * BQ + 2 * BQ2) * (a.d + PAD) * sizeof(bf16) + 4 * BQ2 * sizeof(float);
     if (a.d == 128) {
@@ -483,7 +483,7 @@ cudaError_t launch_portable_bwd(const KArgs& a, cudaStream_t st) {
     }
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
-  {
+  if (passes & BDLM_BWD_PASS_DQ) {
     dim3 grid((a.L + BQ - 1) / BQ, a.H, a.batch * 2);
     size_t smem = (size_t)(2 * BQ + 2 * BK) * (a.d + PAD) * sizeof(bf16);
     if (a.d == 128) {
@@ -493,8 +493,9 @@ cudaError_t launch_portable_bwd(const KArgs& a, cudaStream_t st) {
       if ((e = set_smem(portable_dq_kernel<64>, smem)) != cudaSuccess) return e;
       portable_dq_kernel<64><<<grid, NTHREADS, smem, st>>>(a);
     }
+    e = cudaGetLastError();
   }
-  return cudaGetLastError();
+  return e;
 }
 
 }  // namespace bdlm

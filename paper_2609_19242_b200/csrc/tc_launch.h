@@ -11,6 +11,6 @@ bool tc_fwd_supported(const KArgs& a);
 bool tc_bwd_supported(const KArgs& a);
 size_t tc_bwd_extra_workspace(const bdlm_params* p);
 cudaError_t launch_tc_fwd(const KArgs& a, cudaStream_t st);
-cudaError_t launch_tc_bwd(const KArgs& a, void* extra_ws, cudaStream_t st);
+cudaError_t launch_tc_bwd(const KArgs& a, void* extra_ws, int passes, cudaStream_t st);
 
 }  // namespace bdlm
