@@ -21,6 +21,9 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+}  // namespace
+
+namespace {
 EncodeTiledFn encode_fn() {
   static EncodeTiledFn fn = [] {
     void* p = nullptr;
@@ -32,8 +35,12 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
+}  // namespace
+
+bool tc_encoder_available() { return encode_fn() != nullptr; }
+
 // [batch, L, heads, 128] bf16 viewed as 3-D (heads*128, L, batch); box = 64 columns x `rows` rows.
-bool make_map(CUtensorMap* m, const void* ptr, int heads, int L, int batch, int rows) {
+bool tc_make_map(CUtensorMap* m, const void* ptr, int heads, int L, int batch, int rows) {
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr || ptr == nullptr) return false;
   cuuint64_t gdim[3] = {(cuuint64_t)heads * 128, (cuuint64_t)L, (cuuint64_t)batch};
@@ -46,10 +53,14 @@ bool make_map(CUtensorMap* m, const void* ptr, int heads, int L, int batch, int 
   return r == CUDA_SUCCESS;
 }
 
+namespace {
 // ---------------------------------------------------------------- forward kernel
 constexpr uint32_t IDESC_QK = make_idesc(128, 128, false, false);
 constexpr uint32_t IDESC_PV = make_idesc(128, 128, false, true);
 constexpr int TILE_BYTES = 2 * PANEL_BYTES;   // 128 x 128 bf16
+#ifndef BDLM_P_IN_TMEM
+#define BDLM_P_IN_TMEM 1
+#endif
 constexpr int FWD_SMEM = 6 * TILE_BYTES + 128 + 1024;   // Q, 2x(K,V), P, barriers, alignment slack
 
 __global__ void __launch_bounds__(128, 1)
@@ -160,6 +171,21 @@ tc_fwd_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restri
     const float corr = exp2f(m - mb);
     m = m_new;
     float psum = 0.f;
+#if BDLM_P_IN_TMEM
+    // P (bf16 pairs) overwrites the first 64 columns of this row's S in tensor memory
+#pragma unroll
+    for (int c32 = 0; c32 < 2; ++c32) {
+      uint32_t pk[32];
+#pragma unroll
+      for (int e = 0; e < 32; ++e) {
+        const float p0 = exp2f(__uint_as_float(sr[c32 * 64 + 2 * e]) - mb);
+        const float p1 = exp2f(__uint_as_float(sr[c32 * 64 + 2 * e + 1]) - mb);
+        psum += p0 + p1;
+        pk[e] = pack_bf16(p0, p1);
+      }
+      tmem_st32(tS + c32 * 32, pk);
+    }
+#else
     uint8_t* prow = sm + (sP - base);
 #pragma unroll
     for (int c8 = 0; c8 < 16; ++c8) {
@@ -170,6 +196,7 @@ tc_fwd_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restri
       v.x = pack_bf16(p[0], p[1]); v.y = pack_bf16(p[2], p[3]); v.z = pack_bf16(p[4], p[5]); v.w = pack_bf16(p[6], p[7]);
       *reinterpret_cast<uint4*>(prow + sw128_offset(tid, c8 * 8)) = v;
     }
+#endif
     l = l * corr + psum;
     if (t > 0) {   // rescale the running output (the previous PV MMA has completed)
 #pragma unroll
@@ -181,8 +208,8 @@ tc_fwd_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restri
         for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * corr);
         tmem_st32(tO + c * 32, o);
       }
-      tmem_wait_st();
     }
+    tmem_wait_st();
     tc_fence_before();
     fence_async_smem();
     if (__syncthreads_or(fail)) { fail = true; break; }
@@ -190,9 +217,14 @@ tc_fwd_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restri
       tc_fence_after();
 #pragma unroll
       for (int kk = 0; kk < 8; ++kk) {
+#if BDLM_P_IN_TMEM
+        mma_ts(tmem + 128, tmem + kk * 8, smem_desc(sV + kk * 2048, PANEL_BYTES, 1024), IDESC_PV,
+               (t > 0 || kk > 0) ? 1u : 0u);
+#else
         const uint32_t aoff = (kk >> 2) * PANEL_BYTES + (kk & 3) * 32;
         mma_ss(tmem + 128, smem_desc(sP + aoff, 16, 1024), smem_desc(sV + kk * 2048, PANEL_BYTES, 1024), IDESC_PV,
                (t > 0 || kk > 0) ? 1u : 0u);
+#endif
       }
       mma_commit(bar_o);
     }
@@ -235,16 +267,14 @@ tc_fwd_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restri
 bool tc_fwd_supported(const KArgs& a) {
   return a.d == 128 && a.L % TILE == 0 && encode_fn() != nullptr;
 }
-bool tc_bwd_supported(const KArgs&) { return false; }
-size_t tc_bwd_extra_workspace(const bdlm_params*) { return 0; }
 
 cudaError_t launch_tc_fwd(const KArgs& a, cudaStream_t st) {
   FwdMaps maps;
   for (int s = 0; s < 2; ++s) {
     const void* q = a.q[s] ? (const void*)a.q[s] : (const void*)a.q[1 - s];
-    if (!make_map(&maps.q[s], q, a.H, a.L, a.batch, TILE)) return cudaErrorInvalidValue;
-    if (!make_map(&maps.k[s], a.k[s], a.Hkv, a.L, a.batch, TILE)) return cudaErrorInvalidValue;
-    if (!make_map(&maps.v[s], a.v[s], a.Hkv, a.L, a.batch, TILE)) return cudaErrorInvalidValue;
+    if (!tc_make_map(&maps.q[s], q, a.H, a.L, a.batch, TILE)) return cudaErrorInvalidValue;
+    if (!tc_make_map(&maps.k[s], a.k[s], a.Hkv, a.L, a.batch, TILE)) return cudaErrorInvalidValue;
+    if (!tc_make_map(&maps.v[s], a.v[s], a.Hkv, a.L, a.batch, TILE)) return cudaErrorInvalidValue;
   }
   int* status = device_status_ptr();
   if (status == nullptr) return cudaErrorUnknown;
@@ -254,7 +284,5 @@ cudaError_t launch_tc_fwd(const KArgs& a, cudaStream_t st) {
   tc_fwd_kernel<<<grid, 128, FWD_SMEM, st>>>(maps, a, status);
   return cudaGetLastError();
 }
-
-cudaError_t launch_tc_bwd(const KArgs&, void*, int, cudaStream_t) { return cudaErrorNotSupported; }
 
 }  // namespace bdlm

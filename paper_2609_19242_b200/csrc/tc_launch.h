@@ -1,11 +1,17 @@
 // Host-side interface of the tcgen05 (5th-generation tensor core) kernels.
 #pragma once
+#include <cuda.h>
+
 #include "bdlm_common.cuh"
 
 namespace bdlm {
 
 // Address of the device status word that bounded waits report to (nullptr on failure).
 int* device_status_ptr();
+
+bool tc_encoder_available();
+// Tensor map over a [batch, L, heads, 128] bf16 tensor, box = 64 columns x `rows` rows, 128-byte swizzle.
+bool tc_make_map(CUtensorMap* m, const void* ptr, int heads, int L, int batch, int rows);
 
 bool tc_fwd_supported(const KArgs& a);
 bool tc_bwd_supported(const KArgs& a);
