@@ -262,6 +262,258 @@ tc_fwd_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restri
   if (warp == 0) tmem_dealloc(tmem, 256);
 }
 
+
+// ---------------------------------------------------------------- forward, warp-specialised
+// One CTA = one 128-row query tile of TWO query heads of the same KV group (same stream, same
+// rows, so the same key tiles and the same masks).  Warp 8 loads Q of both heads once and
+// streams K/V tiles through a 2-stage ring; warp 9 issues tcgen05.mma; warpgroup w (warps
+// 4w..4w+3) runs the online softmax of head w, one thread per row, writes P (bf16) over its S
+// columns in tensor memory and rescales its O accumulator only when the running maximum grew
+// by more than 2^8 (the stale maximum is exact in the final LSE and normalisation).
+constexpr int FWD2_THREADS = 320;
+constexpr int FWD2_BARS = 6 * TILE_BYTES;                 // Q_A, Q_B, two (K, V) stages
+constexpr int FWD2_SMEM = FWD2_BARS + 256 + 1024;
+
+__global__ void __launch_bounds__(FWD2_THREADS, 1)
+tc_fwd2_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t sQ = base, sK0 = base + 2 * TILE_BYTES;   // stage s: K at sK0 + s*2*TILE, V after it
+  const uint32_t bars = base + FWD2_BARS;
+  const uint32_t bar_q = bars, bar_k_full = bars + 8 /*[2]*/, bar_v_full = bars + 24 /*[2]*/, bar_kv_empty = bars + 40 /*[2]*/,
+                 bar_s = bars + 56 /*[2]*/, bar_p = bars + 72 /*[2]*/, bar_o = bars + 88 /*[2]*/;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + FWD2_BARS + 128);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + FWD2_BARS + 136);
+
+  const int qs = blockIdx.z & 1, b = blockIdx.z >> 1;
+  if (a.q[qs] == nullptr) return;
+  const int h0 = blockIdx.y * 2, hk = h0 / a.G;
+  const int q0 = (gridDim.x - 1 - blockIdx.x) * TILE;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  int seg_lo[2], ntile[2], lo_last[2], hi_first[2];
+#pragma unroll
+  for (int ks = 0; ks < 2; ++ks) {
+    int lo_f, hi_f, lo_l, hi_l;
+    visible_interval(qs, ks, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_f, hi_f);
+    visible_interval(qs, ks, q0 + TILE - 1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_l, hi_l);
+    seg_lo[ks] = lo_f; lo_last[ks] = lo_l; hi_first[ks] = hi_f;
+    ntile[ks] = hi_l > lo_f ? (hi_l - lo_f + TILE - 1) / TILE : 0;
+  }
+  const int nt = ntile[0] + ntile[1];
+  auto tile_ks = [&](int t) { return t < ntile[0] ? 0 : 1; };
+  auto tile_k0 = [&](int t) { return t < ntile[0] ? seg_lo[0] + t * TILE : seg_lo[1] + (t - ntile[0]) * TILE; };
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar_q, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar_k_full + 8 * i, 1); mbar_init(bar_v_full + 8 * i, 1); mbar_init(bar_kv_empty + 8 * i, 1);
+      mbar_init(bar_s + 8 * i, 1); mbar_init(bar_p + 8 * i, 128); mbar_init(bar_o + 8 * i, 1);
+    }
+    *abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 8) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  // TMEM columns: [0,128) S/P head A   [128,256) S/P head B   [256,384) O head A   [384,512) O head B
+
+  if (warp == 8) {
+    if (lane == 0 && nt > 0) {
+      mbar_expect_tx(bar_q, 2 * TILE_BYTES);
+      tma_load_3d(sQ, &maps.q[qs], bar_q, h0 * 128, q0, b);
+      tma_load_3d(sQ + PANEL_BYTES, &maps.q[qs], bar_q, h0 * 128 + 64, q0, b);
+      tma_load_3d(sQ + TILE_BYTES, &maps.q[qs], bar_q, h0 * 128 + 128, q0, b);
+      tma_load_3d(sQ + TILE_BYTES + PANEL_BYTES, &maps.q[qs], bar_q, h0 * 128 + 192, q0, b);
+      bool ok = true;
+      for (int t = 0; t < nt && ok; ++t) {
+        const int s = t & 1;
+        if (t >= 2) ok = mbar_wait_abortable(bar_kv_empty + 8 * s, ((t >> 1) - 1) & 1, abort_flag);
+        if (!ok) break;
+        const int ks = tile_ks(t), k0 = tile_k0(t);
+        const uint32_t dK = sK0 + s * 2 * TILE_BYTES, dV = dK + TILE_BYTES;
+        mbar_expect_tx(bar_k_full + 8 * s, TILE_BYTES);
+        tma_load_3d(dK, &maps.k[ks], bar_k_full + 8 * s, hk * 128, k0, b);
+        tma_load_3d(dK + PANEL_BYTES, &maps.k[ks], bar_k_full + 8 * s, hk * 128 + 64, k0, b);
+        mbar_expect_tx(bar_v_full + 8 * s, TILE_BYTES);
+        tma_load_3d(dV, &maps.v[ks], bar_v_full + 8 * s, hk * 128, k0, b);
+        tma_load_3d(dV + PANEL_BYTES, &maps.v[ks], bar_v_full + 8 * s, hk * 128 + 64, k0, b);
+      }
+    }
+  } else if (warp == 9) {
+    if (lane == 0 && nt > 0) {
+      auto issue_qk = [&](int w, uint32_t kt) {
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+          const uint32_t off = (kk >> 2) * PANEL_BYTES + (kk & 3) * 32;
+          mma_ss(tmem + w * 128, smem_desc(sQ + w * TILE_BYTES + off, 16, 1024), smem_desc(kt + off, 16, 1024), IDESC_QK, kk > 0);
+        }
+        mma_commit(bar_s + 8 * w);
+      };
+      bool ok = mbar_wait_abortable(bar_q, 0, abort_flag);
+      ok = ok && mbar_wait_abortable(bar_k_full, 0, abort_flag);
+      if (ok) {
+        tc_fence_after();
+        issue_qk(0, sK0);
+        issue_qk(1, sK0);
+      }
+      for (int t = 0; t < nt && ok; ++t) {
+        const int s = t & 1;
+        const uint32_t cV = sK0 + s * 2 * TILE_BYTES + TILE_BYTES;
+        const uint32_t nK = sK0 + (s ^ 1) * 2 * TILE_BYTES;
+        for (int w = 0; w < 2 && ok; ++w) {
+          ok = mbar_wait_abortable(bar_p + 8 * w, t & 1, abort_flag);
+          if (ok && w == 0) ok = mbar_wait_abortable(bar_v_full + 8 * s, (t >> 1) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk)
+            mma_ts(tmem + 256 + w * 128, tmem + w * 128 + kk * 8, smem_desc(cV + kk * 2048, PANEL_BYTES, 1024), IDESC_PV,
+                   (t > 0 || kk > 0) ? 1u : 0u);
+          mma_commit(bar_o + 8 * w);
+          if (w == 1) mma_commit(bar_kv_empty + 8 * s);
+          if (t + 1 < nt) {
+            if (w == 0) ok = mbar_wait_abortable(bar_k_full + 8 * (s ^ 1), ((t + 1) >> 1) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            issue_qk(w, nK);
+          }
+        }
+      }
+    }
+  } else {
+    const int w = warp >> 2;
+    const int r = (warp & 3) * 32 + lane;
+    const int row = q0 + r;
+    const int h = h0 + w;
+    const uint32_t tS = tmem + ((uint32_t)((warp & 3) * 32) << 16) + w * 128;
+    const uint32_t tO = tmem + ((uint32_t)((warp & 3) * 32) << 16) + 256 + w * 128;
+    int rlo[2], rhi[2];
+#pragma unroll
+    for (int ks = 0; ks < 2; ++ks) visible_interval(qs, ks, row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo[ks], rhi[ks]);
+    float m_ref = -INFINITY, l = 0.f;
+    bool ok = true;
+    for (int t = 0; t < nt; ++t) {
+      const int ks = tile_ks(t), k0 = tile_k0(t);
+      ok = mbar_wait_abortable(bar_s + 8 * w, t & 1, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const bool need_mask = (k0 < lo_last[ks]) || (k0 + TILE > hi_first[ks]);
+      // pass 1: row maximum of the raw scores (scale > 0 commutes with max); S is re-read in pass 2
+      float mx = -INFINITY;
+#pragma unroll
+      for (int c2 = 0; c2 < 2; ++c2) {
+        uint32_t v0[32], v1[32];
+        tmem_ld32(tS + c2 * 64, v0); tmem_ld32(tS + c2 * 64 + 32, v1);
+        tmem_wait_ld();
+        if (need_mask) {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            const int j0 = k0 + c2 * 64 + e, j1 = j0 + 32;
+            if (j0 >= rlo[ks] && j0 < rhi[ks]) mx = fmaxf(mx, __uint_as_float(v0[e]));
+            if (j1 >= rlo[ks] && j1 < rhi[ks]) mx = fmaxf(mx, __uint_as_float(v1[e]));
+          }
+        } else {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) mx = fmaxf(mx, fmaxf(__uint_as_float(v0[e]), __uint_as_float(v1[e])));
+        }
+      }
+      mx *= a.scale_log2;   // -inf stays -inf
+      const float m_new = fmaxf(m_ref, mx);
+      const bool grow = m_new > m_ref + 8.0f;
+      if (__any_sync(0xffffffffu, grow)) {
+        const float mb_new = (m_new == -INFINITY) ? 0.f : m_new;
+        const float corr = exp2f(m_ref - mb_new);
+        m_ref = m_new;
+        l *= corr;
+        if (t > 0) {
+          ok = mbar_wait_abortable(bar_o + 8 * w, (t - 1) & 1, abort_flag);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            uint32_t o[32];
+            tmem_ld32(tO + c * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * corr);
+            tmem_st32(tO + c * 32, o);
+          }
+        }
+      }
+      const float mb = (m_ref == -INFINITY) ? 0.f : m_ref;
+      // pass 2: p = exp2(s * scale - m), packed to bf16 pairs over the first 64 columns of S
+      float psum = 0.f;
+#pragma unroll
+      for (int c2 = 0; c2 < 2; ++c2) {
+        uint32_t v0[32], v1[32], pk[32];
+        tmem_ld32(tS + c2 * 64, v0); tmem_ld32(tS + c2 * 64 + 32, v1);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          float p0 = exp2f(fmaf(__uint_as_float(v0[2 * e]), a.scale_log2, -mb));
+          float p1 = exp2f(fmaf(__uint_as_float(v0[2 * e + 1]), a.scale_log2, -mb));
+          float p2 = exp2f(fmaf(__uint_as_float(v1[2 * e]), a.scale_log2, -mb));
+          float p3 = exp2f(fmaf(__uint_as_float(v1[2 * e + 1]), a.scale_log2, -mb));
+          if (need_mask) {
+            const int j = k0 + c2 * 64 + 2 * e;
+            p0 = (j >= rlo[ks] && j < rhi[ks]) ? p0 : 0.f;
+            p1 = (j + 1 >= rlo[ks] && j + 1 < rhi[ks]) ? p1 : 0.f;
+            p2 = (j + 32 >= rlo[ks] && j + 32 < rhi[ks]) ? p2 : 0.f;
+            p3 = (j + 33 >= rlo[ks] && j + 33 < rhi[ks]) ? p3 : 0.f;
+          }
+          psum += (p0 + p1) + (p2 + p3);
+          pk[e] = pack_bf16(p0, p1);
+          pk[16 + e] = pack_bf16(p2, p3);
+        }
+        // the second pass over columns [64, 128) must not be clobbered: P of the first 64 columns
+        // lands in TMEM columns [0, 32), which pass 2 has already consumed
+        tmem_st32(tS + c2 * 32, pk);
+      }
+      l += psum;
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar_p + 8 * w);
+    }
+    if (ok && nt > 0) {
+      ok = mbar_wait_abortable(bar_o + 8 * w, (nt - 1) & 1, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+    }
+    if (ok) {
+      tc_fence_after();
+      const float inv = l > 0.f ? 1.f / l : 0.f;
+      bf16* orow = a.o[qs] + (((int64_t)b * a.L + row) * a.H + h) * 128;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t o[32];
+        if (nt > 0) { tmem_ld32(tO + c * 32, o); tmem_wait_ld(); }
+#pragma unroll
+        for (int e8 = 0; e8 < 4; ++e8) {
+          uint4 v;
+          uint32_t* pv = reinterpret_cast<uint32_t*>(&v);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float x0 = nt > 0 ? __uint_as_float(o[e8 * 8 + 2 * e]) * inv : 0.f;
+            const float x1 = nt > 0 ? __uint_as_float(o[e8 * 8 + 2 * e + 1]) * inv : 0.f;
+            pv[e] = pack_bf16(x0, x1);
+          }
+          *reinterpret_cast<uint4*>(orow + c * 32 + e8 * 8) = v;
+        }
+      }
+      a.lse[qs][((int64_t)b * a.H + h) * a.L + row] = l > 0.f ? (m_ref + log2f(l)) * LN2 : -INFINITY;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) atomicExch(status, (int)BDLM_ERR_DEVICE_TIMEOUT);
+  if (warp == 8) tmem_dealloc(tmem, 512);
+}
+
 }  // namespace
 
 bool tc_fwd_supported(const KArgs& a) {
@@ -280,6 +532,13 @@ cudaError_t launch_tc_fwd(const KArgs& a, cudaStream_t st) {
   if (status == nullptr) return cudaErrorUnknown;
   cudaError_t e = cudaFuncSetAttribute(tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM);
   if (e != cudaSuccess) return e;
+  if (a.G % 2 == 0) {   // two heads of one KV group per CTA
+    e = cudaFuncSetAttribute(tc_fwd2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD2_SMEM);
+    if (e != cudaSuccess) return e;
+    dim3 grid2(a.L / TILE, a.H / 2, a.batch * 2);
+    tc_fwd2_kernel<<<grid2, FWD2_THREADS, FWD2_SMEM, st>>>(maps, a, status);
+    return cudaGetLastError();
+  }
   dim3 grid(a.L / TILE, a.H, a.batch * 2);
   tc_fwd_kernel<<<grid, 128, FWD_SMEM, st>>>(maps, a, status);
   return cudaGetLastError();
