@@ -126,6 +126,19 @@ const char* bdlm_status_string(int status);
  */
 int bdlm_get_device_status(void* cuda_stream);
 
+/*
+ * Tracing (no counterpart in the paper; the paper reports GPU spans in its appendix K only).
+ * When a device buffer of at least BDLM_TRACE_SLOTS 64-bit counters is set, the tensor-core
+ * kernels add, per CTA and role, the clock cycles spent waiting and computing:
+ *   slot = kernel * 16 + counter, kernel 0 = forward, 1 = dK/dV pass, 2 = dQ pass;
+ *   counters 0..7 belong to compute warp 0 (0 steps, 1..5 waits/compute phases in kernel order,
+ *   6 total), 8..11 to the MMA thread (8 total, 9..11 waits), 12..13 to the producer (12 total,
+ *   13 wait for a free stage).
+ * Pass NULL to switch tracing off (the default).  The caller zeroes and reads the buffer.
+ */
+enum { BDLM_TRACE_SLOTS = 64 };
+int bdlm_set_trace_buffer(void* device_counters, size_t bytes);
+
 #ifdef __cplusplus
 }
 #endif

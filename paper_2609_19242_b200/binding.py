@@ -19,7 +19,8 @@ IMPL_AUTO, IMPL_PORTABLE, IMPL_TCGEN05 = 0, 1, 2
 PASS_DSUM, PASS_DKDV, PASS_DQ = 1, 2, 4
 
 EXPORTS = ("bdlm_workspace_bytes", "bdlm_attn_fwd", "bdlm_attn_bwd", "bdlm_lse_merge",
-           "bdlm_status_string", "bdlm_get_device_status")
+           "bdlm_status_string", "bdlm_get_device_status", "bdlm_set_trace_buffer")
+TRACE_SLOTS = 64
 
 
 class BdlmError(RuntimeError):
@@ -63,6 +64,8 @@ def lib():
         L.bdlm_status_string.argtypes = [ctypes.c_int]
         L.bdlm_get_device_status.restype = ctypes.c_int
         L.bdlm_get_device_status.argtypes = [vp]
+        L.bdlm_set_trace_buffer.restype = ctypes.c_int
+        L.bdlm_set_trace_buffer.argtypes = [vp, ctypes.c_size_t]
         _lib = L
     return _lib
 
@@ -177,3 +180,14 @@ def bdlm_lse_merge(o_partials, lse_partials, *, out=None):
 
 def bdlm_get_device_status() -> int:
     return int(lib().bdlm_get_device_status(_stream()))
+
+
+def bdlm_set_trace_buffer(counters) -> None:
+    """Switch kernel tracing on (an int64 CUDA tensor of TRACE_SLOTS zeros) or off (None)."""
+    if counters is None:
+        rc = lib().bdlm_set_trace_buffer(None, 0)
+    else:
+        assert counters.is_cuda and counters.dtype == torch.int64 and counters.numel() >= TRACE_SLOTS
+        rc = lib().bdlm_set_trace_buffer(_ptr(counters), counters.numel() * 8)
+    if rc != 0:
+        raise BdlmError(rc, "bdlm_set_trace_buffer")

@@ -10,6 +10,7 @@ namespace bdlm {
 namespace {
 
 __device__ int g_device_status = 0;
+unsigned long long* g_trace = nullptr;   // host-side copy of the trace buffer pointer
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -42,6 +43,7 @@ void fill(KArgs& a, const bdlm_params* p) {
     a.q[s] = a.k[s] = a.v[s] = nullptr; a.o[s] = nullptr; a.lse[s] = nullptr;
     a.dout[s] = nullptr; a.dsum[s] = nullptr; a.dq[s] = a.dk[s] = a.dv[s] = nullptr;
   }
+  a.trace = g_trace;
 }
 
 bool is_sm100() {
@@ -179,6 +181,13 @@ int bdlm_lse_merge(int32_t n_partials, int32_t batch, int32_t L, int32_t H, int3
   cudaError_t e = launch_merge(n_partials, batch, L, H, d, o_partials, lse_partials, partial_dtype,
                                o_out, lse_out, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? BDLM_OK : BDLM_ERR_CUDA;
+}
+
+int bdlm_set_trace_buffer(void* device_counters, size_t bytes) {
+  if (device_counters != nullptr && (bytes < BDLM_TRACE_SLOTS * sizeof(unsigned long long) || !aligned16(device_counters)))
+    return BDLM_ERR_INVALID_ARG;
+  g_trace = static_cast<unsigned long long*>(device_counters);
+  return BDLM_OK;
 }
 
 const char* bdlm_status_string(int status) {

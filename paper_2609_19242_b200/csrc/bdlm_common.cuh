@@ -32,6 +32,7 @@ struct KArgs {
   __nv_bfloat16* dq[2];
   __nv_bfloat16* dk[2];
   __nv_bfloat16* dv[2];
+  unsigned long long* trace;   // optional cycle counters (bdlm_set_trace_buffer), else nullptr
 };
 
 // Visible key interval [lo, hi) of query row i (stream qs) inside key stream ks

@@ -62,26 +62,27 @@ __device__ __forceinline__ void store_row_chunk(bf16* dst, const uint32_t (&v)[3
 // =============================================================================================
 // dK/dV pass
 // =============================================================================================
-constexpr int DKDV_ARR = 6 * TILE_BYTES;            // after K, V and two (Q, dO) stages
-constexpr int DKDV_BARS = DKDV_ARR + 4096 + 64;
-constexpr int DKDV_SMEM = DKDV_BARS + 256 + 1024;
+// Shared memory: K, V (resident), a 3-stage Q ring (a Q tile is read first by S^T and last by
+// dK, so it lives longest), a 2-stage dO ring with the LSE and D rows of the same query tile.
+constexpr int DKDV_Q0 = 2 * TILE_BYTES;
+constexpr int DKDV_DO0 = 5 * TILE_BYTES;
+constexpr int DKDV_ARR = 7 * TILE_BYTES;            // lse_s[2][128], d_s[2][128]
+constexpr int DKDV_BARS = DKDV_ARR + 2048;
+constexpr int DKDV_SMEM = DKDV_BARS + 160;
 
 struct QStep { int qs, h, q0; };
 
 __global__ void __launch_bounds__(BWD_THREADS, 1)
 tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restrict__ status) {
-  extern __shared__ uint8_t smem_raw[];
-  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t sK = base, sV = base + TILE_BYTES, sQ0 = base + 2 * TILE_BYTES;   // stage s: Q at sQ0 + s*2*TILE, dO after it
+  extern __shared__ __align__(1024) uint8_t sm[];
+  const uint32_t base = smem_u32(sm);
+  const uint32_t sK = base, sV = base + TILE_BYTES, sQ0 = base + DKDV_Q0, sdO0 = base + DKDV_DO0;
   float* lse_s = reinterpret_cast<float*>(sm + DKDV_ARR);          // [2][128], log2 units
   float* d_s = lse_s + 256;                                        // [2][128]
-  int* vlo_s = reinterpret_cast<int*>(d_s + 256);                  // [2][128] visible key interval of each query column
-  int* vhi_s = vlo_s + 256;
-  int* flag_s = reinterpret_cast<int*>(sm + DKDV_ARR + 4096);      // [2] tile needs masking
   const uint32_t bars = base + DKDV_BARS;
-  const uint32_t bar_kv = bars, bar_qdo_full = bars + 8 /*[2]*/, bar_qdo_empty = bars + 24 /*[2]*/,
-                 bar_st = bars + 40, bar_dpt = bars + 48, bar_pt = bars + 56, bar_dst = bars + 64, bar_done = bars + 72;
+  const uint32_t bar_kv = bars, bar_q_full = bars + 8 /*[3]*/, bar_q_empty = bars + 32 /*[3]*/,
+                 bar_do_full = bars + 56 /*[2]*/, bar_do_empty = bars + 72 /*[2]*/,
+                 bar_st = bars + 88, bar_dpt = bars + 96, bar_pt = bars + 104, bar_dst = bars + 112, bar_done = bars + 120;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + DKDV_BARS + 128);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + DKDV_BARS + 136);
 
@@ -113,13 +114,13 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
   };
 
   if (threadIdx.x == 0) {
+    if (base & 1023u) *abort_flag = 1; else *abort_flag = 0;   // swizzled tiles need a 1024-byte aligned base
     mbar_init(bar_kv, 1);
-    mbar_init(bar_qdo_full, 1); mbar_init(bar_qdo_full + 8, 1);
-    mbar_init(bar_qdo_empty, 1); mbar_init(bar_qdo_empty + 8, 1);
+    for (int i = 0; i < 3; ++i) { mbar_init(bar_q_full + 8 * i, 1); mbar_init(bar_q_empty + 8 * i, 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_do_full + 8 * i, 2); mbar_init(bar_do_empty + 8 * i, 1); }   // dO full: TMA bytes + LSE/D rows
     mbar_init(bar_st, 1); mbar_init(bar_dpt, 1);
     mbar_init(bar_pt, 256); mbar_init(bar_dst, 256);
     mbar_init(bar_done, 1);
-    *abort_flag = 0;
     fence_mbar_init();
   }
   if (warp == 8) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
@@ -127,9 +128,12 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  const bool bad_base = (*abort_flag != 0);
   // TMEM columns: [0,128) S^T / P^T   [128,256) dP^T / dS^T   [256,384) dV   [384,512) dK
 
-  if (warp == 8) {
+  if (bad_base) {
+    // fall through to the common exit
+  } else if (warp == 8) {
     // ------------------------------------------------------------------ producer
     if (lane == 0) {
       mbar_expect_tx(bar_kv, 2 * TILE_BYTES);
@@ -137,66 +141,75 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       tma_tile(sV, &maps.v[ks], bar_kv, hk * 128, k0, b);
     }
     bool ok = true;
+    long long w_empty = 0;
+    const long long t_begin = clock64();
     for (int i = 0; i < nsteps && ok; ++i) {
-      const int s = i & 1;
-      if (i >= 2) ok = mbar_wait_abortable(bar_qdo_empty + 8 * s, ((i >> 1) - 1) & 1, abort_flag);
+      const int sq = i % 3, sd = i & 1;
+      const QStep st = step_of(i);
+      if (i >= 3) ok = mbar_wait_timed(bar_q_empty + 8 * sq, ((i / 3) - 1) & 1, abort_flag, w_empty);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
-      const QStep st = step_of(i);
+      if (lane == 0) {
+        mbar_expect_tx(bar_q_full + 8 * sq, TILE_BYTES);
+        tma_tile(sQ0 + sq * TILE_BYTES, &maps.q[st.qs], bar_q_full + 8 * sq, st.h * 128, st.q0, b);
+      }
+      if (i >= 2) ok = mbar_wait_timed(bar_do_empty + 8 * sd, ((i >> 1) - 1) & 1, abort_flag, w_empty);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      if (lane == 0) {
+        mbar_expect_tx(bar_do_full + 8 * sd, TILE_BYTES);   // one arrival of two; the LSE/D rows follow
+        tma_tile(sdO0 + sd * TILE_BYTES, &maps.dout[st.qs], bar_do_full + 8 * sd, st.h * 128, st.q0, b);
+      }
       const float* lsep = a.lse[st.qs] + ((int64_t)b * a.H + st.h) * L + st.q0;
       const float* dsp = a.dsum[st.qs] + ((int64_t)b * a.H + st.h) * L + st.q0;
-      bool need = false;
-#pragma unroll
-      for (int c4 = 0; c4 < 4; ++c4) {
-        const int c = lane + 32 * c4;
-        const float z = lsep[c];
-        int lo, hi;
-        visible_interval(st.qs, ks, st.q0 + c, M, a.mode, a.kv_begin, a.kv_end, a.diag, lo, hi);
-        lse_s[s * 128 + c] = isfinite(z) ? z * LOG2E : INFINITY;
-        d_s[s * 128 + c] = dsp[c];
-        vlo_s[s * 128 + c] = lo;
-        vhi_s[s * 128 + c] = hi;
-        need |= (lo > k0) || (hi < k0 + TILE);
+      {
+        const float4 z = reinterpret_cast<const float4*>(lsep)[lane];
+        const float4 dd = reinterpret_cast<const float4*>(dsp)[lane];
+        float4 z2;
+        z2.x = isfinite(z.x) ? z.x * LOG2E : INFINITY; z2.y = isfinite(z.y) ? z.y * LOG2E : INFINITY;
+        z2.z = isfinite(z.z) ? z.z * LOG2E : INFINITY; z2.w = isfinite(z.w) ? z.w * LOG2E : INFINITY;
+        reinterpret_cast<float4*>(lse_s + sd * 128)[lane] = z2;
+        reinterpret_cast<float4*>(d_s + sd * 128)[lane] = dd;
       }
-      need = __any_sync(0xffffffffu, need);
-      if (lane == 0) flag_s[s] = need ? 1 : 0;
       __syncwarp();
-      if (lane == 0) {
-        const uint32_t bar = bar_qdo_full + 8 * s;
-        const uint32_t dQ = sQ0 + s * 2 * TILE_BYTES;
-        mbar_expect_tx(bar, 2 * TILE_BYTES);
-        tma_tile(dQ, &maps.q[st.qs], bar, st.h * 128, st.q0, b);
-        tma_tile(dQ + TILE_BYTES, &maps.dout[st.qs], bar, st.h * 128, st.q0, b);
-      }
+      if (lane == 0) mbar_arrive(bar_do_full + 8 * sd);
     }
+    if (lane == 0) { trace_add(a.trace, 16 + 12, clock64() - t_begin); trace_add(a.trace, 16 + 13, w_empty); }
   } else if (warp == 9) {
     // ------------------------------------------------------------------ MMA issuer (one thread)
     if (lane == 0 && nsteps > 0) {
+      long long w_pt = 0, w_q = 0, w_dst = 0;
+      const long long t_begin = clock64();
       bool ok = mbar_wait_abortable(bar_kv, 0, abort_flag);
-      ok = ok && mbar_wait_abortable(bar_qdo_full, 0, abort_flag);
+      ok = ok && mbar_wait_abortable(bar_q_full, 0, abort_flag);
       if (ok) {
         tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) mma_ss(tmem, kmajor_desc(sK, kk), kmajor_desc(sQ0, kk), IDESC_KK, kk > 0);
         mma_commit(bar_st);
+      }
+      ok = ok && mbar_wait_abortable(bar_do_full, 0, abort_flag);
+      if (ok) {
+        tc_fence_after();
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) mma_ss(tmem + 128, kmajor_desc(sV, kk), kmajor_desc(sQ0 + TILE_BYTES, kk), IDESC_KK, kk > 0);
+        for (int kk = 0; kk < 8; ++kk) mma_ss(tmem + 128, kmajor_desc(sV, kk), kmajor_desc(sdO0, kk), IDESC_KK, kk > 0);
         mma_commit(bar_dpt);
       }
       for (int i = 0; i < nsteps && ok; ++i) {
-        const int s = i & 1;
-        const uint32_t cQ = sQ0 + s * 2 * TILE_BYTES, cdO = cQ + TILE_BYTES;
-        const uint32_t nQ = sQ0 + (s ^ 1) * 2 * TILE_BYTES, ndO = nQ + TILE_BYTES;
+        const int sq = i % 3, sd = i & 1, nq = (i + 1) % 3;
+        const uint32_t cQ = sQ0 + sq * TILE_BYTES, cdO = sdO0 + sd * TILE_BYTES;
+        const uint32_t nQ = sQ0 + nq * TILE_BYTES, ndO = sdO0 + (sd ^ 1) * TILE_BYTES;
         // dV += P^T dO_i   (P^T: this lane's 64+64 bf16 pairs at columns [0,32) and [64,96))
-        ok = mbar_wait_abortable(bar_pt, i & 1, abort_flag);
+        ok = mbar_wait_timed(bar_pt, i & 1, abort_flag, w_pt);
         if (!ok) break;
         tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)
           mma_ts(tmem + 256, tmem + (kk < 4 ? kk * 8 : 64 + (kk - 4) * 8), mnmajor_desc(cdO, kk), IDESC_KM, (i > 0 || kk > 0) ? 1u : 0u);
+        mma_commit(bar_do_empty + 8 * sd);
         // S^T of the next step may start as soon as its Q is in shared memory
         if (i + 1 < nsteps) {
-          ok = mbar_wait_abortable(bar_qdo_full + 8 * (s ^ 1), ((i + 1) >> 1) & 1, abort_flag);
+          ok = mbar_wait_timed(bar_q_full + 8 * nq, ((i + 1) / 3) & 1, abort_flag, w_q);
           if (!ok) break;
           tc_fence_after();
 #pragma unroll
@@ -204,20 +217,25 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
           mma_commit(bar_st);
         }
         // dK += dS^T Q_i
-        ok = mbar_wait_abortable(bar_dst, i & 1, abort_flag);
+        ok = mbar_wait_timed(bar_dst, i & 1, abort_flag, w_dst);
         if (!ok) break;
         tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)
           mma_ts(tmem + 384, tmem + 128 + (kk < 4 ? kk * 8 : 64 + (kk - 4) * 8), mnmajor_desc(cQ, kk), IDESC_KM, (i > 0 || kk > 0) ? 1u : 0u);
-        mma_commit(bar_qdo_empty + 8 * s);
+        mma_commit(bar_q_empty + 8 * sq);
         if (i + 1 < nsteps) {
+          ok = mbar_wait_timed(bar_do_full + 8 * (sd ^ 1), ((i + 1) >> 1) & 1, abort_flag, w_q);
+          if (!ok) break;
+          tc_fence_after();
 #pragma unroll
           for (int kk = 0; kk < 8; ++kk) mma_ss(tmem + 128, kmajor_desc(sV, kk), kmajor_desc(ndO, kk), IDESC_KK, kk > 0);
           mma_commit(bar_dpt);
         }
       }
       mma_commit(bar_done);
+      trace_add(a.trace, 16 + 8, clock64() - t_begin); trace_add(a.trace, 16 + 9, w_pt);
+      trace_add(a.trace, 16 + 10, w_q); trace_add(a.trace, 16 + 11, w_dst);
     }
   } else {
     // ------------------------------------------------------------------ compute warpgroups
@@ -226,11 +244,29 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
     const int j = k0 + r;
     const uint32_t tl = tmem + ((uint32_t)((warp & 3) * 32) << 16);
     const int c0 = w * 64;
+    // query rows that see key j, per query stream (section 3.2 read from the key's side)
+    int vq_lo[2], vq_hi[2];
+    if (ks == CLEAN) {
+      vq_lo[CLEAN] = (a.mode == 0) ? j : (j / M) * M; vq_hi[CLEAN] = L;
+      vq_lo[NOISY] = (j / M + 1) * M; vq_hi[NOISY] = L;
+    } else {
+      vq_lo[CLEAN] = 0; vq_hi[CLEAN] = 0;
+      vq_lo[NOISY] = (j / M) * M; vq_hi[NOISY] = vq_lo[NOISY] + M;
+    }
+    const int vqc_lo = vq_lo[CLEAN], vqc_hi = vq_hi[CLEAN], vqn_lo = vq_lo[NOISY], vqn_hi = vq_hi[NOISY];
     bool ok = true;
+    long long w_st = 0, w_dpt = 0;
+    const long long t_begin = clock64();
     for (int i = 0; i < nsteps; ++i) {
-      const int s = i & 1;
-      ok = mbar_wait_abortable(bar_qdo_full + 8 * s, (i >> 1) & 1, abort_flag);
-      ok = ok && mbar_wait_abortable(bar_st, i & 1, abort_flag);
+      const int sd = i & 1;
+      const QStep st = step_of(i);
+      // the tile needs masking unless every query row of it sees every key of this key tile
+      int lo_a, hi_a, lo_b, hi_b;
+      visible_interval(st.qs, ks, st.q0, M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_a, hi_a);
+      visible_interval(st.qs, ks, st.q0 + TILE - 1, M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_b, hi_b);
+      const bool need_mask = (lo_b > k0) || (hi_a < k0 + TILE);
+      ok = mbar_wait_timed(bar_do_full + 8 * sd, (i >> 1) & 1, abort_flag, w_st);
+      ok = ok && mbar_wait_timed(bar_st, i & 1, abort_flag, w_st);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -240,13 +276,18 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
         tmem_ld32(tl + c0, c[0]); tmem_ld32(tl + c0 + 32, c[1]);
         tmem_wait_ld();
       }
-      const bool need_mask = flag_s[s] != 0;
-      const float* lz = lse_s + s * 128 + c0;
+      const float* lz = lse_s + sd * 128 + c0;
+      if (!need_mask) {
 #pragma unroll
-      for (int c = 0; c < 64; ++c) {
-        float p = exp2f(__uint_as_float(x[c]) * a.scale_log2 - lz[c]);
-        if (need_mask) p = (j >= vlo_s[s * 128 + c0 + c] && j < vhi_s[s * 128 + c0 + c]) ? p : 0.f;
-        x[c] = __float_as_uint(p);
+        for (int c = 0; c < 64; ++c) x[c] = __float_as_uint(exp2f(fmaf(__uint_as_float(x[c]), a.scale_log2, -lz[c])));
+      } else {
+        // visible columns of this thread's key row inside the tile: [vlo, vhi)
+        const int vlo = (st.qs == CLEAN ? vqc_lo : vqn_lo) - st.q0 - c0, vhi = (st.qs == CLEAN ? vqc_hi : vqn_hi) - st.q0 - c0;
+#pragma unroll
+        for (int c = 0; c < 64; ++c) {
+          const float p = exp2f(fmaf(__uint_as_float(x[c]), a.scale_log2, -lz[c]));
+          x[c] = __float_as_uint((c >= vlo && c < vhi) ? p : 0.f);
+        }
       }
       {
         uint32_t pk[32];
@@ -258,7 +299,7 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       tc_fence_before();
       mbar_arrive(bar_pt);
 
-      ok = mbar_wait_abortable(bar_dpt, i & 1, abort_flag);
+      ok = mbar_wait_timed(bar_dpt, i & 1, abort_flag, w_dpt);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -267,7 +308,7 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
         uint32_t (*c)[32] = reinterpret_cast<uint32_t (*)[32]>(y);
         tmem_ld32(tl + 128 + c0, c[0]); tmem_ld32(tl + 128 + c0 + 32, c[1]);
         tmem_wait_ld();
-        const float* dz = d_s + s * 128 + c0;
+        const float* dz = d_s + sd * 128 + c0;
         uint32_t pk[32];
 #pragma unroll
         for (int e = 0; e < 32; ++e) {
@@ -280,6 +321,10 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       }
       tc_fence_before();
       mbar_arrive(bar_dst);
+    }
+    if (warp == 0 && lane == 0) {
+      trace_add(a.trace, 16 + 0, nsteps); trace_add(a.trace, 16 + 1, w_st); trace_add(a.trace, 16 + 2, w_dpt);
+      trace_add(a.trace, 16 + 6, clock64() - t_begin);
     }
     // epilogue: warpgroup 0 writes dV, warpgroup 1 writes dK (scaled)
     if (ok && nsteps > 0) {
@@ -311,18 +356,22 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
 // =============================================================================================
 // dQ pass
 // =============================================================================================
-constexpr int DQ_BARS = 6 * TILE_BYTES;             // Q, dO, two (K, V) stages
-constexpr int DQ_SMEM = DQ_BARS + 256 + 1024;
+// Shared memory: Q, dO (resident), a 3-stage K ring (a K tile is read first by S and last by dQ) and
+// a 2-stage V ring.
+constexpr int DQ_K0 = 2 * TILE_BYTES;
+constexpr int DQ_V0 = 5 * TILE_BYTES;
+constexpr int DQ_BARS = 7 * TILE_BYTES;
+constexpr int DQ_SMEM = DQ_BARS + 160;
 
 __global__ void __launch_bounds__(BWD_THREADS, 1)
 tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restrict__ status) {
-  extern __shared__ uint8_t smem_raw[];
-  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t sQ = base, sdO = base + TILE_BYTES, sK0 = base + 2 * TILE_BYTES;   // stage s: K at sK0 + s*2*TILE, V after it
+  extern __shared__ __align__(1024) uint8_t sm[];
+  const uint32_t base = smem_u32(sm);
+  const uint32_t sQ = base, sdO = base + TILE_BYTES, sK0 = base + DQ_K0, sV0 = base + DQ_V0;
   const uint32_t bars = base + DQ_BARS;
-  const uint32_t bar_qdo = bars, bar_kv_full = bars + 8 /*[2]*/, bar_kv_empty = bars + 24 /*[2]*/,
-                 bar_s = bars + 40 /*[2]*/, bar_dp = bars + 56, bar_ds = bars + 64, bar_done = bars + 72;
+  const uint32_t bar_qdo = bars, bar_k_full = bars + 8 /*[3]*/, bar_k_empty = bars + 32 /*[3]*/,
+                 bar_v_full = bars + 56 /*[2]*/, bar_v_empty = bars + 72 /*[2]*/,
+                 bar_s = bars + 88 /*[2]*/, bar_dp = bars + 104, bar_ds = bars + 112, bar_done = bars + 120;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + DQ_BARS + 128);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + DQ_BARS + 136);
 
@@ -332,26 +381,27 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
   const int L = a.L;
 
   // key tiles visible from this query tile: clean segment, then noisy segment
-  int seg_lo[2], ntile[2], lo_last[2], hi_first[2];
-#pragma unroll
-  for (int ks = 0; ks < 2; ++ks) {
+  int lo0, lo1, nt0, nt1, lo_last0, lo_last1, hi_first0, hi_first1;
+  {
     int lo_f, hi_f, lo_l, hi_l;
-    visible_interval(qs, ks, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_f, hi_f);
-    visible_interval(qs, ks, q0 + TILE - 1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_l, hi_l);
-    seg_lo[ks] = lo_f; lo_last[ks] = lo_l; hi_first[ks] = hi_f;
-    ntile[ks] = hi_l > lo_f ? (hi_l - lo_f + TILE - 1) / TILE : 0;
+    visible_interval(qs, 0, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_f, hi_f);
+    visible_interval(qs, 0, q0 + TILE - 1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_l, hi_l);
+    lo0 = lo_f; lo_last0 = lo_l; hi_first0 = hi_f; nt0 = hi_l > lo_f ? (hi_l - lo_f + TILE - 1) / TILE : 0;
+    visible_interval(qs, 1, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_f, hi_f);
+    visible_interval(qs, 1, q0 + TILE - 1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_l, hi_l);
+    lo1 = lo_f; lo_last1 = lo_l; hi_first1 = hi_f; nt1 = hi_l > lo_f ? (hi_l - lo_f + TILE - 1) / TILE : 0;
   }
-  const int nsteps = ntile[0] + ntile[1];
-  auto tile_ks = [&](int i) { return i < ntile[0] ? 0 : 1; };
-  auto tile_k0 = [&](int i) { return i < ntile[0] ? seg_lo[0] + i * TILE : seg_lo[1] + (i - ntile[0]) * TILE; };
+  const int nsteps = nt0 + nt1;
+  auto tile_ks = [&](int i) { return i < nt0 ? 0 : 1; };
+  auto tile_k0 = [&](int i) { return i < nt0 ? lo0 + i * TILE : lo1 + (i - nt0) * TILE; };
 
   if (threadIdx.x == 0) {
+    if (base & 1023u) *abort_flag = 1; else *abort_flag = 0;
     mbar_init(bar_qdo, 1);
-    mbar_init(bar_kv_full, 1); mbar_init(bar_kv_full + 8, 1);
-    mbar_init(bar_kv_empty, 1); mbar_init(bar_kv_empty + 8, 1);
+    for (int i = 0; i < 3; ++i) { mbar_init(bar_k_full + 8 * i, 1); mbar_init(bar_k_empty + 8 * i, 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_v_full + 8 * i, 1); mbar_init(bar_v_empty + 8 * i, 1); }
     mbar_init(bar_s, 1); mbar_init(bar_s + 8, 1);
     mbar_init(bar_dp, 1); mbar_init(bar_ds, 256); mbar_init(bar_done, 1);
-    *abort_flag = 0;
     fence_mbar_init();
   }
   if (warp == 8) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
@@ -359,66 +409,86 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  const bool bad_base = (*abort_flag != 0);
   // TMEM columns: [0,128) S even / dS   [128,256) dP   [256,384) dQ   [384,512) S odd / dS
   auto s_col = [&](int i) { return (i & 1) ? 384u : 0u; };
 
-  if (warp == 8) {
+  if (bad_base) {
+    // fall through to the common exit
+  } else if (warp == 8) {
     if (lane == 0 && nsteps > 0) {
       mbar_expect_tx(bar_qdo, 2 * TILE_BYTES);
       tma_tile(sQ, &maps.q[qs], bar_qdo, h * 128, q0, b);
       tma_tile(sdO, &maps.dout[qs], bar_qdo, h * 128, q0, b);
       bool ok = true;
+      long long w_empty = 0;
+      const long long t_begin = clock64();
       for (int i = 0; i < nsteps && ok; ++i) {
-        const int s = i & 1;
-        if (i >= 2) ok = mbar_wait_abortable(bar_kv_empty + 8 * s, ((i >> 1) - 1) & 1, abort_flag);
-        if (!ok) break;
+        const int sk = i % 3, sv = i & 1;
         const int ks = tile_ks(i), k0 = tile_k0(i);
-        const uint32_t bar = bar_kv_full + 8 * s, dK = sK0 + s * 2 * TILE_BYTES;
-        mbar_expect_tx(bar, 2 * TILE_BYTES);
-        tma_tile(dK, &maps.k[ks], bar, hk * 128, k0, b);
-        tma_tile(dK + TILE_BYTES, &maps.v[ks], bar, hk * 128, k0, b);
+        if (i >= 3) ok = mbar_wait_timed(bar_k_empty + 8 * sk, ((i / 3) - 1) & 1, abort_flag, w_empty);
+        if (!ok) break;
+        mbar_expect_tx(bar_k_full + 8 * sk, TILE_BYTES);
+        tma_tile(sK0 + sk * TILE_BYTES, &maps.k[ks], bar_k_full + 8 * sk, hk * 128, k0, b);
+        if (i >= 2) ok = mbar_wait_timed(bar_v_empty + 8 * sv, ((i >> 1) - 1) & 1, abort_flag, w_empty);
+        if (!ok) break;
+        mbar_expect_tx(bar_v_full + 8 * sv, TILE_BYTES);
+        tma_tile(sV0 + sv * TILE_BYTES, &maps.v[ks], bar_v_full + 8 * sv, hk * 128, k0, b);
       }
+      trace_add(a.trace, 32 + 12, clock64() - t_begin); trace_add(a.trace, 32 + 13, w_empty);
     }
   } else if (warp == 9) {
     if (lane == 0 && nsteps > 0) {
+      long long w_kv = 0, w_ds = 0;
+      const long long t_begin = clock64();
       bool ok = mbar_wait_abortable(bar_qdo, 0, abort_flag);
-      ok = ok && mbar_wait_abortable(bar_kv_full, 0, abort_flag);
+      ok = ok && mbar_wait_abortable(bar_k_full, 0, abort_flag);
       if (ok) {
         tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) mma_ss(tmem, kmajor_desc(sQ, kk), kmajor_desc(sK0, kk), IDESC_KK, kk > 0);
         mma_commit(bar_s);
+      }
+      ok = ok && mbar_wait_abortable(bar_v_full, 0, abort_flag);
+      if (ok) {
+        tc_fence_after();
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) mma_ss(tmem + 128, kmajor_desc(sdO, kk), kmajor_desc(sK0 + TILE_BYTES, kk), IDESC_KK, kk > 0);
+        for (int kk = 0; kk < 8; ++kk) mma_ss(tmem + 128, kmajor_desc(sdO, kk), kmajor_desc(sV0, kk), IDESC_KK, kk > 0);
         mma_commit(bar_dp);
+        mma_commit(bar_v_empty);
       }
       for (int i = 0; i < nsteps && ok; ++i) {
-        const int s = i & 1;
-        const uint32_t cK = sK0 + s * 2 * TILE_BYTES;
-        const uint32_t nK = sK0 + (s ^ 1) * 2 * TILE_BYTES, nV = nK + TILE_BYTES;
+        const uint32_t cK = sK0 + (i % 3) * TILE_BYTES;
         if (i + 1 < nsteps) {   // S of the next key tile into the other S buffer
-          ok = mbar_wait_abortable(bar_kv_full + 8 * (s ^ 1), ((i + 1) >> 1) & 1, abort_flag);
+          const int nk = (i + 1) % 3;
+          ok = mbar_wait_timed(bar_k_full + 8 * nk, ((i + 1) / 3) & 1, abort_flag, w_kv);
           if (!ok) break;
           tc_fence_after();
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk) mma_ss(tmem + s_col(i + 1), kmajor_desc(sQ, kk), kmajor_desc(nK, kk), IDESC_KK, kk > 0);
-          mma_commit(bar_s + 8 * (s ^ 1));
+          for (int kk = 0; kk < 8; ++kk) mma_ss(tmem + s_col(i + 1), kmajor_desc(sQ, kk), kmajor_desc(sK0 + nk * TILE_BYTES, kk), IDESC_KK, kk > 0);
+          mma_commit(bar_s + 8 * ((i + 1) & 1));
         }
         // dQ += dS_i K_i   (dS: bf16 pairs at columns [0,32) and [64,96) of this step's S buffer)
-        ok = mbar_wait_abortable(bar_ds, i & 1, abort_flag);
+        ok = mbar_wait_timed(bar_ds, i & 1, abort_flag, w_ds);
         if (!ok) break;
         tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)
           mma_ts(tmem + 256, tmem + s_col(i) + (kk < 4 ? kk * 8 : 64 + (kk - 4) * 8), mnmajor_desc(cK, kk), IDESC_KM, (i > 0 || kk > 0) ? 1u : 0u);
-        mma_commit(bar_kv_empty + 8 * s);
+        mma_commit(bar_k_empty + 8 * (i % 3));
         if (i + 1 < nsteps) {
+          const int nv = (i + 1) & 1;
+          ok = mbar_wait_timed(bar_v_full + 8 * nv, ((i + 1) >> 1) & 1, abort_flag, w_kv);
+          if (!ok) break;
+          tc_fence_after();
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk) mma_ss(tmem + 128, kmajor_desc(sdO, kk), kmajor_desc(nV, kk), IDESC_KK, kk > 0);
+          for (int kk = 0; kk < 8; ++kk) mma_ss(tmem + 128, kmajor_desc(sdO, kk), kmajor_desc(sV0 + nv * TILE_BYTES, kk), IDESC_KK, kk > 0);
           mma_commit(bar_dp);
+          mma_commit(bar_v_empty + 8 * nv);
         }
       }
       mma_commit(bar_done);
+      trace_add(a.trace, 32 + 8, clock64() - t_begin); trace_add(a.trace, 32 + 9, w_kv); trace_add(a.trace, 32 + 10, w_ds);
     }
   } else {
     const int w = warp >> 2;
@@ -432,34 +502,46 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
       if (isfinite(z)) lse2 = z * LOG2E;
       dsum = a.dsum[qs][((int64_t)b * a.H + h) * L + row];
     }
-    int rlo[2], rhi[2];
-#pragma unroll
-    for (int ks = 0; ks < 2; ++ks) visible_interval(qs, ks, row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo[ks], rhi[ks]);
+    int rlo0, rhi0, rlo1, rhi1;
+    visible_interval(qs, 0, row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo0, rhi0);
+    visible_interval(qs, 1, row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo1, rhi1);
     bool ok = true;
+    long long w_s = 0, w_dp = 0, c_ld = 0, c_exp = 0, c_ds = 0;
+    Stopwatch sw;
+    const long long t_begin = clock64();
     for (int i = 0; i < nsteps; ++i) {
       const int ks = tile_ks(i), k0 = tile_k0(i);
-      ok = mbar_wait_abortable(bar_s + 8 * (i & 1), (i >> 1) & 1, abort_flag);
+      ok = mbar_wait_timed(bar_s + 8 * (i & 1), (i >> 1) & 1, abort_flag, w_s);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
       const uint32_t ts = tl + s_col(i) + c0;
       uint32_t x[64];
+      sw.start();
       {
         uint32_t (*c)[32] = reinterpret_cast<uint32_t (*)[32]>(x);
         tmem_ld32(ts, c[0]); tmem_ld32(ts + 32, c[1]);
         tmem_wait_ld();
       }
-      const bool need_mask = (k0 < lo_last[ks]) || (k0 + TILE > hi_first[ks]);
+      sw.lap(c_ld);
+      const bool need_mask = ks == 0 ? (k0 < lo_last0 || k0 + TILE > hi_first0) : (k0 < lo_last1 || k0 + TILE > hi_first1);
+      if (!need_mask) {
 #pragma unroll
-      for (int c = 0; c < 64; ++c) {
-        float p = exp2f(__uint_as_float(x[c]) * a.scale_log2 - lse2);
-        if (need_mask) { const int jj = k0 + c0 + c; p = (jj >= rlo[ks] && jj < rhi[ks]) ? p : 0.f; }
-        x[c] = __float_as_uint(p);
+        for (int c = 0; c < 64; ++c) x[c] = __float_as_uint(exp2f(fmaf(__uint_as_float(x[c]), a.scale_log2, -lse2)));
+      } else {
+        const int vlo = (ks == 0 ? rlo0 : rlo1) - k0 - c0, vhi = (ks == 0 ? rhi0 : rhi1) - k0 - c0;
+#pragma unroll
+        for (int c = 0; c < 64; ++c) {
+          const float p = exp2f(fmaf(__uint_as_float(x[c]), a.scale_log2, -lse2));
+          x[c] = __float_as_uint((c >= vlo && c < vhi) ? p : 0.f);
+        }
       }
-      ok = mbar_wait_abortable(bar_dp, i & 1, abort_flag);
+      sw.lap(c_exp);
+      ok = mbar_wait_timed(bar_dp, i & 1, abort_flag, w_dp);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
+      sw.start();
       {
         uint32_t y[64];
         uint32_t (*c)[32] = reinterpret_cast<uint32_t (*)[32]>(y);
@@ -477,6 +559,12 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
       }
       tc_fence_before();
       mbar_arrive(bar_ds);
+      sw.lap(c_ds);
+    }
+    if (warp == 0 && lane == 0) {
+      trace_add(a.trace, 32 + 0, nsteps); trace_add(a.trace, 32 + 1, w_s); trace_add(a.trace, 32 + 2, w_dp);
+      trace_add(a.trace, 32 + 6, clock64() - t_begin);
+      trace_add(a.trace, 32 + 3, c_ld); trace_add(a.trace, 32 + 4, c_exp); trace_add(a.trace, 32 + 5, c_ds);
     }
     if (ok && nsteps > 0) {
       ok = mbar_wait_abortable(bar_done, 0, abort_flag);

@@ -65,6 +65,24 @@ __device__ __forceinline__ bool mbar_wait_abortable(uint32_t bar, uint32_t parit
   return true;
 }
 
+__device__ __forceinline__ bool mbar_wait_timed(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long& acc) {
+  const long long t0 = clock64();
+  const bool ok = mbar_wait_abortable(bar, parity, abort_flag);
+  acc += clock64() - t0;
+  return ok;
+}
+
+// Cycle accounting for the optional trace buffer: a role keeps a few local counters and adds
+// them to the global slots once, when it leaves its loop.
+struct Stopwatch {
+  long long t;
+  __device__ __forceinline__ void start() { t = clock64(); }
+  __device__ __forceinline__ void lap(long long& acc) { const long long n = clock64(); acc += n - t; t = n; }
+};
+__device__ __forceinline__ void trace_add(unsigned long long* trace, int slot, long long v) {
+  if (trace != nullptr) atomicAdd(trace + slot, static_cast<unsigned long long>(v));
+}
+
 // ---------------------------------------------------------------- fences
 __device__ __forceinline__ void fence_async_smem() {   // generic-proxy smem writes -> async proxy (MMA / TMA)
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");

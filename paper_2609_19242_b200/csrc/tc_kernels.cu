@@ -263,6 +263,25 @@ tc_fwd_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restri
 }
 
 
+// Key tiles visible from one 128-row query tile: a clean segment then a noisy segment, each a run
+// of 128-key tiles starting at the first visible key; scalars only (no indexed arrays).
+struct TileSched {
+  int lo0, lo1, nt0, nt1, lo_last0, lo_last1, hi_first0, hi_first1;
+  __device__ __forceinline__ void init(int qs, int q0, const KArgs& a) {
+    int lo_f, hi_f, lo_l, hi_l;
+    visible_interval(qs, 0, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_f, hi_f);
+    visible_interval(qs, 0, q0 + TILE - 1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_l, hi_l);
+    lo0 = lo_f; lo_last0 = lo_l; hi_first0 = hi_f; nt0 = hi_l > lo_f ? (hi_l - lo_f + TILE - 1) / TILE : 0;
+    visible_interval(qs, 1, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_f, hi_f);
+    visible_interval(qs, 1, q0 + TILE - 1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_l, hi_l);
+    lo1 = lo_f; lo_last1 = lo_l; hi_first1 = hi_f; nt1 = hi_l > lo_f ? (hi_l - lo_f + TILE - 1) / TILE : 0;
+  }
+  // a tile needs per-element masking unless every row of the query tile sees all of its 128 keys
+  __device__ __forceinline__ bool need_mask(int ks, int k0) const {
+    return ks == 0 ? (k0 < lo_last0 || k0 + TILE > hi_first0) : (k0 < lo_last1 || k0 + TILE > hi_first1);
+  }
+};
+
 // ---------------------------------------------------------------- forward, warp-specialised
 // One CTA = one 128-row query tile of TWO query heads of the same KV group (same stream, same
 // rows, so the same key tiles and the same masks).  Warp 8 loads Q of both heads once and
@@ -292,18 +311,11 @@ tc_fwd2_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
   const int q0 = (gridDim.x - 1 - blockIdx.x) * TILE;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-  int seg_lo[2], ntile[2], lo_last[2], hi_first[2];
-#pragma unroll
-  for (int ks = 0; ks < 2; ++ks) {
-    int lo_f, hi_f, lo_l, hi_l;
-    visible_interval(qs, ks, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_f, hi_f);
-    visible_interval(qs, ks, q0 + TILE - 1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_l, hi_l);
-    seg_lo[ks] = lo_f; lo_last[ks] = lo_l; hi_first[ks] = hi_f;
-    ntile[ks] = hi_l > lo_f ? (hi_l - lo_f + TILE - 1) / TILE : 0;
-  }
-  const int nt = ntile[0] + ntile[1];
-  auto tile_ks = [&](int t) { return t < ntile[0] ? 0 : 1; };
-  auto tile_k0 = [&](int t) { return t < ntile[0] ? seg_lo[0] + t * TILE : seg_lo[1] + (t - ntile[0]) * TILE; };
+  TileSched sch;
+  sch.init(qs, q0, a);
+  const int nt = sch.nt0 + sch.nt1;
+  auto tile_ks = [&](int t) { return t < sch.nt0 ? 0 : 1; };
+  auto tile_k0 = [&](int t) { return t < sch.nt0 ? sch.lo0 + t * TILE : sch.lo1 + (t - sch.nt0) * TILE; };
 
   if (threadIdx.x == 0) {
     mbar_init(bar_q, 1);
@@ -329,9 +341,11 @@ tc_fwd2_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
       tma_load_3d(sQ + TILE_BYTES, &maps.q[qs], bar_q, h0 * 128 + 128, q0, b);
       tma_load_3d(sQ + TILE_BYTES + PANEL_BYTES, &maps.q[qs], bar_q, h0 * 128 + 192, q0, b);
       bool ok = true;
+      long long w_empty = 0;
+      const long long t_begin = clock64();
       for (int t = 0; t < nt && ok; ++t) {
         const int s = t & 1;
-        if (t >= 2) ok = mbar_wait_abortable(bar_kv_empty + 8 * s, ((t >> 1) - 1) & 1, abort_flag);
+        if (t >= 2) ok = mbar_wait_timed(bar_kv_empty + 8 * s, ((t >> 1) - 1) & 1, abort_flag, w_empty);
         if (!ok) break;
         const int ks = tile_ks(t), k0 = tile_k0(t);
         const uint32_t dK = sK0 + s * 2 * TILE_BYTES, dV = dK + TILE_BYTES;
@@ -342,6 +356,7 @@ tc_fwd2_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
         tma_load_3d(dV, &maps.v[ks], bar_v_full + 8 * s, hk * 128, k0, b);
         tma_load_3d(dV + PANEL_BYTES, &maps.v[ks], bar_v_full + 8 * s, hk * 128 + 64, k0, b);
       }
+      trace_add(a.trace, 12, clock64() - t_begin); trace_add(a.trace, 13, w_empty);
     }
   } else if (warp == 9) {
     if (lane == 0 && nt > 0) {
@@ -353,6 +368,8 @@ tc_fwd2_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
         }
         mma_commit(bar_s + 8 * w);
       };
+      long long w_p = 0, w_v = 0, w_k = 0;
+      const long long t_begin = clock64();
       bool ok = mbar_wait_abortable(bar_q, 0, abort_flag);
       ok = ok && mbar_wait_abortable(bar_k_full, 0, abort_flag);
       if (ok) {
@@ -365,8 +382,8 @@ tc_fwd2_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
         const uint32_t cV = sK0 + s * 2 * TILE_BYTES + TILE_BYTES;
         const uint32_t nK = sK0 + (s ^ 1) * 2 * TILE_BYTES;
         for (int w = 0; w < 2 && ok; ++w) {
-          ok = mbar_wait_abortable(bar_p + 8 * w, t & 1, abort_flag);
-          if (ok && w == 0) ok = mbar_wait_abortable(bar_v_full + 8 * s, (t >> 1) & 1, abort_flag);
+          ok = mbar_wait_timed(bar_p + 8 * w, t & 1, abort_flag, w_p);
+          if (ok && w == 0) ok = mbar_wait_timed(bar_v_full + 8 * s, (t >> 1) & 1, abort_flag, w_v);
           if (!ok) break;
           tc_fence_after();
 #pragma unroll
@@ -376,13 +393,14 @@ tc_fwd2_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
           mma_commit(bar_o + 8 * w);
           if (w == 1) mma_commit(bar_kv_empty + 8 * s);
           if (t + 1 < nt) {
-            if (w == 0) ok = mbar_wait_abortable(bar_k_full + 8 * (s ^ 1), ((t + 1) >> 1) & 1, abort_flag);
+            if (w == 0) ok = mbar_wait_timed(bar_k_full + 8 * (s ^ 1), ((t + 1) >> 1) & 1, abort_flag, w_k);
             if (!ok) break;
             tc_fence_after();
             issue_qk(w, nK);
           }
         }
       }
+      trace_add(a.trace, 8, clock64() - t_begin); trace_add(a.trace, 9, w_p); trace_add(a.trace, 10, w_v); trace_add(a.trace, 11, w_k);
     }
   } else {
     const int w = warp >> 2;
@@ -391,18 +409,23 @@ tc_fwd2_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
     const int h = h0 + w;
     const uint32_t tS = tmem + ((uint32_t)((warp & 3) * 32) << 16) + w * 128;
     const uint32_t tO = tmem + ((uint32_t)((warp & 3) * 32) << 16) + 256 + w * 128;
-    int rlo[2], rhi[2];
-#pragma unroll
-    for (int ks = 0; ks < 2; ++ks) visible_interval(qs, ks, row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo[ks], rhi[ks]);
+    int rlo0, rhi0, rlo1, rhi1;
+    visible_interval(qs, 0, row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo0, rhi0);
+    visible_interval(qs, 1, row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo1, rhi1);
     float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
+    long long w_s = 0, w_o = 0, c_p1 = 0, c_p2ld = 0, c_p2 = 0;
+    Stopwatch sw;
+    const long long t_begin = clock64();
     for (int t = 0; t < nt; ++t) {
       const int ks = tile_ks(t), k0 = tile_k0(t);
-      ok = mbar_wait_abortable(bar_s + 8 * w, t & 1, abort_flag);
+      ok = mbar_wait_timed(bar_s + 8 * w, t & 1, abort_flag, w_s);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const bool need_mask = (k0 < lo_last[ks]) || (k0 + TILE > hi_first[ks]);
+      const bool need_mask = sch.need_mask(ks, k0);
+      const int vlo = (ks == 0 ? rlo0 : rlo1) - k0, vhi = (ks == 0 ? rhi0 : rhi1) - k0;   // visible columns [vlo, vhi) of this tile
+      sw.start();
       // pass 1: row maximum of the raw scores (scale > 0 commutes with max); S is re-read in pass 2
       float mx = -INFINITY;
 #pragma unroll
@@ -413,9 +436,9 @@ tc_fwd2_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
         if (need_mask) {
 #pragma unroll
           for (int e = 0; e < 32; ++e) {
-            const int j0 = k0 + c2 * 64 + e, j1 = j0 + 32;
-            if (j0 >= rlo[ks] && j0 < rhi[ks]) mx = fmaxf(mx, __uint_as_float(v0[e]));
-            if (j1 >= rlo[ks] && j1 < rhi[ks]) mx = fmaxf(mx, __uint_as_float(v1[e]));
+            const int j0 = c2 * 64 + e, j1 = j0 + 32;
+            mx = fmaxf(mx, (j0 >= vlo && j0 < vhi) ? __uint_as_float(v0[e]) : -INFINITY);
+            mx = fmaxf(mx, (j1 >= vlo && j1 < vhi) ? __uint_as_float(v1[e]) : -INFINITY);
           }
         } else {
 #pragma unroll
@@ -423,6 +446,7 @@ tc_fwd2_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
         }
       }
       mx *= a.scale_log2;   // -inf stays -inf
+      sw.lap(c_p1);
       const float m_new = fmaxf(m_ref, mx);
       const bool grow = m_new > m_ref + 8.0f;
       if (__any_sync(0xffffffffu, grow)) {
@@ -431,7 +455,7 @@ tc_fwd2_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
         m_ref = m_new;
         l *= corr;
         if (t > 0) {
-          ok = mbar_wait_abortable(bar_o + 8 * w, (t - 1) & 1, abort_flag);
+          ok = mbar_wait_timed(bar_o + 8 * w, (t - 1) & 1, abort_flag, w_o);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
@@ -447,6 +471,7 @@ tc_fwd2_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
         }
       }
       const float mb = (m_ref == -INFINITY) ? 0.f : m_ref;
+      sw.start();
       // pass 2: p = exp2(s * scale - m), packed to bf16 pairs over the first 64 columns of S
       float psum = 0.f;
 #pragma unroll
@@ -454,31 +479,48 @@ tc_fwd2_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
         uint32_t v0[32], v1[32], pk[32];
         tmem_ld32(tS + c2 * 64, v0); tmem_ld32(tS + c2 * 64 + 32, v1);
         tmem_wait_ld();
+        sw.lap(c_p2ld);
+        if (!need_mask) {
 #pragma unroll
-        for (int e = 0; e < 16; ++e) {
-          float p0 = exp2f(fmaf(__uint_as_float(v0[2 * e]), a.scale_log2, -mb));
-          float p1 = exp2f(fmaf(__uint_as_float(v0[2 * e + 1]), a.scale_log2, -mb));
-          float p2 = exp2f(fmaf(__uint_as_float(v1[2 * e]), a.scale_log2, -mb));
-          float p3 = exp2f(fmaf(__uint_as_float(v1[2 * e + 1]), a.scale_log2, -mb));
-          if (need_mask) {
-            const int j = k0 + c2 * 64 + 2 * e;
-            p0 = (j >= rlo[ks] && j < rhi[ks]) ? p0 : 0.f;
-            p1 = (j + 1 >= rlo[ks] && j + 1 < rhi[ks]) ? p1 : 0.f;
-            p2 = (j + 32 >= rlo[ks] && j + 32 < rhi[ks]) ? p2 : 0.f;
-            p3 = (j + 33 >= rlo[ks] && j + 33 < rhi[ks]) ? p3 : 0.f;
+          for (int e = 0; e < 16; ++e) {
+            const float p0 = exp2f(fmaf(__uint_as_float(v0[2 * e]), a.scale_log2, -mb));
+            const float p1 = exp2f(fmaf(__uint_as_float(v0[2 * e + 1]), a.scale_log2, -mb));
+            const float p2 = exp2f(fmaf(__uint_as_float(v1[2 * e]), a.scale_log2, -mb));
+            const float p3 = exp2f(fmaf(__uint_as_float(v1[2 * e + 1]), a.scale_log2, -mb));
+            psum += (p0 + p1) + (p2 + p3);
+            pk[e] = pack_bf16(p0, p1);
+            pk[16 + e] = pack_bf16(p2, p3);
           }
-          psum += (p0 + p1) + (p2 + p3);
-          pk[e] = pack_bf16(p0, p1);
-          pk[16 + e] = pack_bf16(p2, p3);
+        } else {
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const int j = c2 * 64 + 2 * e;
+            float p0 = exp2f(fmaf(__uint_as_float(v0[2 * e]), a.scale_log2, -mb));
+            float p1 = exp2f(fmaf(__uint_as_float(v0[2 * e + 1]), a.scale_log2, -mb));
+            float p2 = exp2f(fmaf(__uint_as_float(v1[2 * e]), a.scale_log2, -mb));
+            float p3 = exp2f(fmaf(__uint_as_float(v1[2 * e + 1]), a.scale_log2, -mb));
+            p0 = (j >= vlo && j < vhi) ? p0 : 0.f;
+            p1 = (j + 1 >= vlo && j + 1 < vhi) ? p1 : 0.f;
+            p2 = (j + 32 >= vlo && j + 32 < vhi) ? p2 : 0.f;
+            p3 = (j + 33 >= vlo && j + 33 < vhi) ? p3 : 0.f;
+            psum += (p0 + p1) + (p2 + p3);
+            pk[e] = pack_bf16(p0, p1);
+            pk[16 + e] = pack_bf16(p2, p3);
+          }
         }
         // the second pass over columns [64, 128) must not be clobbered: P of the first 64 columns
         // lands in TMEM columns [0, 32), which pass 2 has already consumed
         tmem_st32(tS + c2 * 32, pk);
+        sw.lap(c_p2);
       }
       l += psum;
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(bar_p + 8 * w);
+    }
+    if (warp == 0 && lane == 0) {
+      trace_add(a.trace, 0, nt); trace_add(a.trace, 1, w_s); trace_add(a.trace, 2, w_o); trace_add(a.trace, 6, clock64() - t_begin);
+      trace_add(a.trace, 3, c_p1); trace_add(a.trace, 4, c_p2ld); trace_add(a.trace, 5, c_p2);
     }
     if (ok && nt > 0) {
       ok = mbar_wait_abortable(bar_o + 8 * w, (nt - 1) & 1, abort_flag);
