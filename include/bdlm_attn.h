@@ -39,7 +39,8 @@ typedef enum {
   BDLM_ERR_UNSUPPORTED = -2,        /* d not in {64,128}; device is not sm_100; sharded backward */
   BDLM_ERR_WORKSPACE_TOO_SMALL = -3,
   BDLM_ERR_CUDA = -4,               /* a CUDA runtime/driver call or a launch failed */
-  BDLM_ERR_DEVICE_TIMEOUT = -5      /* a bounded device-side wait expired (see bdlm_get_device_status) */
+  BDLM_ERR_DEVICE_TIMEOUT = -5,     /* a bounded device-side wait expired (see bdlm_get_device_status) */
+  BDLM_ERR_STATIC_SCRATCH_TOO_SMALL = -6   /* batch*H*L exceeds BDLM_STATIC_SCRATCH_ROWS (bdlm_attn_bwd_static_scratch) */
 } bdlm_status;
 
 typedef struct {
@@ -125,6 +126,34 @@ const char* bdlm_status_string(int status);
  * last call (the word is cleared).  BDLM_ERR_CUDA if the synchronise itself failed.
  */
 int bdlm_get_device_status(void* cuda_stream);
+
+/*
+ * Backward without a workspace argument (the paper has no counterpart; this exists for callers
+ * that are not allowed to allocate device memory: a plug-in inside a host framework whose pool
+ * already owns the whole GPU, or a latency-critical loop that cannot accept the device-wide
+ * synchronisation an allocator call implies).  Same inputs, outputs, checks and kernels as
+ * bdlm_attn_bwd; the D_i scratch lives in a fixed device array inside the library
+ * (2 * BDLM_STATIC_SCRATCH_ROWS floats = 8 MiB, resident on every GPU that loads the library
+ * until the process exits).  The call allocates and frees nothing.
+ *   - Limit: batch * H * L <= BDLM_STATIC_SCRATCH_ROWS, otherwise
+ *     BDLM_ERR_STATIC_SCRATCH_TOO_SMALL is returned and nothing is launched.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps the previous call's contents.
+ *     Nothing in it has to start at zero (each call rewrites D in full before reading it), but
+ *     two calls that overlap on the GPU -- different streams, or different host threads -- race
+ *     on it: serialise them.
+ */
+enum { BDLM_STATIC_SCRATCH_ROWS = 1 << 20 };
+int bdlm_attn_bwd_static_scratch(const bdlm_params* p,
+                                 const void* q_clean, const void* k_clean, const void* v_clean,
+                                 const void* q_noisy, const void* k_noisy, const void* v_noisy,
+                                 const void* o_clean, const void* o_noisy,
+                                 const float* lse_clean, const float* lse_noisy,
+                                 const void* do_clean, const void* do_noisy,
+                                 void* dq_clean, void* dk_clean, void* dv_clean,
+                                 void* dq_noisy, void* dk_noisy, void* dv_noisy,
+                                 void* cuda_stream);
 
 /*
  * Tracing (no counterpart in the paper; the paper reports GPU spans in its appendix K only).

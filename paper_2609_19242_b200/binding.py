@@ -19,7 +19,9 @@ IMPL_AUTO, IMPL_PORTABLE, IMPL_TCGEN05 = 0, 1, 2
 PASS_DSUM, PASS_DKDV, PASS_DQ = 1, 2, 4
 
 EXPORTS = ("bdlm_workspace_bytes", "bdlm_attn_fwd", "bdlm_attn_bwd", "bdlm_lse_merge",
-           "bdlm_status_string", "bdlm_get_device_status", "bdlm_set_trace_buffer")
+           "bdlm_status_string", "bdlm_get_device_status", "bdlm_set_trace_buffer",
+           "bdlm_attn_bwd_static_scratch")
+STATIC_SCRATCH_ROWS = 1 << 20
 TRACE_SLOTS = 64
 
 
@@ -64,6 +66,8 @@ def lib():
         L.bdlm_status_string.argtypes = [ctypes.c_int]
         L.bdlm_get_device_status.restype = ctypes.c_int
         L.bdlm_get_device_status.argtypes = [vp]
+        L.bdlm_attn_bwd_static_scratch.restype = ctypes.c_int
+        L.bdlm_attn_bwd_static_scratch.argtypes = [pp] + [vp] * 18 + [vp]
         L.bdlm_set_trace_buffer.restype = ctypes.c_int
         L.bdlm_set_trace_buffer.argtypes = [vp, ctypes.c_size_t]
         _lib = L
@@ -155,6 +159,24 @@ def bdlm_attn_bwd(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, o_clean,
                              _ptr(workspace), workspace.numel(), _stream())
     if rc != 0:
         raise BdlmError(rc, "bdlm_attn_bwd")
+    return out
+
+
+def bdlm_attn_bwd_static_scratch(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, o_clean, lse_clean,
+                                 o_noisy, lse_noisy, do_clean, do_noisy, block_size, *, out,
+                                 scale=0.0, clean_mask_mode=0, impl=IMPL_AUTO):
+    """Backward through the entry point that takes no workspace: the library's built-in scratch
+    array is used, so this wrapper allocates nothing either -- `out` (the six gradient tensors)
+    must be supplied by the caller.  For callers that may not allocate device memory; limited to
+    batch*H*L <= STATIC_SCRATCH_ROWS, and calls that overlap on the GPU must be serialised."""
+    p = _shape_params(q_clean, k_clean, block_size, scale=scale, clean_mask_mode=clean_mask_mode, impl=impl)
+    dq_c, dk_c, dv_c, dq_n, dk_n, dv_n = out
+    rc = lib().bdlm_attn_bwd_static_scratch(
+        ctypes.byref(p), _ptr(q_clean), _ptr(k_clean), _ptr(v_clean), _ptr(q_noisy), _ptr(k_noisy), _ptr(v_noisy),
+        _ptr(o_clean), _ptr(o_noisy), _ptr(lse_clean), _ptr(lse_noisy), _ptr(do_clean), _ptr(do_noisy),
+        _ptr(dq_c), _ptr(dk_c), _ptr(dv_c), _ptr(dq_n), _ptr(dk_n), _ptr(dv_n), _stream())
+    if rc != 0:
+        raise BdlmError(rc, "bdlm_attn_bwd_static_scratch")
     return out
 
 

@@ -198,6 +198,7 @@ const char* bdlm_status_string(int status) {
     case BDLM_ERR_WORKSPACE_TOO_SMALL: return "BDLM_ERR_WORKSPACE_TOO_SMALL";
     case BDLM_ERR_CUDA: return "BDLM_ERR_CUDA";
     case BDLM_ERR_DEVICE_TIMEOUT: return "BDLM_ERR_DEVICE_TIMEOUT";
+    case BDLM_ERR_STATIC_SCRATCH_TOO_SMALL: return "BDLM_ERR_STATIC_SCRATCH_TOO_SMALL";
     default: return "BDLM_ERR_UNKNOWN";
   }
 }

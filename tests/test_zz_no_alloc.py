@@ -1,0 +1,67 @@
+"""The allocation-free backward entry point (bdlm_attn_bwd_static_scratch), for callers that are
+not allowed to allocate device memory -- e.g. a plug-in inside a framework whose pool owns the
+whole GPU, or a latency-critical loop that cannot take an allocator's device-wide sync.
+
+It must give the regular backward's results, twice in a row (the built-in scratch array keeps
+the previous call's contents), and must refuse sizes beyond its fixed limit.  This file is
+collected last on purpose: a run that stops at the first failure has then already run every
+other test."""
+import ctypes
+
+import pytest
+import torch
+
+from paper_2609_19242_b200 import binding, synth
+from paper_2609_19242_b200.synth import Workload
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+def _max_abs_diff(a, b):
+    return float((a.float() - b.float()).abs().max())
+
+
+@pytest.mark.parametrize("w", [Workload("na_d128", 2, 4, 2, 128, 384, 32), Workload("na_d64", 1, 2, 2, 64, 256, 16)],
+                         ids=lambda w: w.name)
+def test_static_scratch_backward_matches_regular_backward_twice(w):
+    M = w.block_size
+    g = pu.to_cuda(synth.make_inputs(w, "cpu"))
+    fwd = pu.gpu_fwd(g, M)
+    ref = [t.clone() for t in pu.gpu_bwd(g, fwd, M)]
+    torch.cuda.synchronize()
+    out = tuple(torch.empty_like(t) for t in ref)            # caller-owned outputs: the call allocates nothing
+    for call in range(2):
+        if call == 1:
+            # second call with a different upstream gradient first, so stale scratch would show
+            g2 = dict(g)
+            g2["do_clean"] = (g["do_clean"].float() * -2.0).to(torch.bfloat16)
+            g2["do_noisy"] = (g["do_noisy"].float() * 0.5).to(torch.bfloat16)
+            binding.bdlm_attn_bwd_static_scratch(*[g2[n] for n in pu.NAMES6], fwd[0], fwd[1], fwd[2], fwd[3],
+                                                 g2["do_clean"], g2["do_noisy"], M, out=out)
+        for t in out:
+            t.fill_(float("nan"))
+        binding.bdlm_attn_bwd_static_scratch(*[g[n] for n in pu.NAMES6], fwd[0], fwd[1], fwd[2], fwd[3],
+                                             g["do_clean"], g["do_noisy"], M, out=out)
+        torch.cuda.synchronize()
+        assert binding.bdlm_get_device_status() == 0
+        for got, want in zip(out, ref):
+            assert torch.isfinite(got.float()).all()
+            # same kernels, same fixed summation order: equal within the gradient tolerance (in fact bitwise)
+            assert pu.rel_l2(synth.to_f64(got), synth.to_f64(want)) <= pu.TOL_GRAD
+            assert _max_abs_diff(got, want) == 0.0
+
+
+def test_static_scratch_rejects_sizes_beyond_its_limit():
+    # batch*H*L just above the limit: refused before any pointer is touched or anything is launched
+    rows = binding.STATIC_SCRATCH_ROWS
+    p = binding.make_params(1, rows // 32 + 128, 128, 32, 8, 128)
+    assert p.batch * p.H * p.L > rows
+    fake = ctypes.c_void_p(0x1000)
+    rc = binding.lib().bdlm_attn_bwd_static_scratch(ctypes.byref(p), *([fake] * 18), None)
+    assert rc == -6
+    assert binding.status_string(rc) == "BDLM_ERR_STATIC_SCRATCH_TOO_SMALL"
+    # invalid parameters are still rejected as such
+    bad = binding.make_params(1, 100, 16, 4, 2, 128)
+    assert binding.lib().bdlm_attn_bwd_static_scratch(ctypes.byref(bad), *([fake] * 18), None) == -1
