@@ -35,7 +35,14 @@ NAMES6 = ["q_clean", "k_clean", "v_clean", "q_noisy", "k_noisy", "v_noisy"]
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant
 # kernel, from the ncu captures summarised under profiles/ ; keyed by (workload, kernel).
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    ("8k", "fwd"): 209513728 + 105072640,
+    ("8k", "bwd_dkdv"): 416072192 + 51993088,
+    ("8k", "bwd_dq"): 365939200 + 111330560,
+}
+TRAFFIC_NOTE = ("ncu DRAM bytes were captured on the 8k workload only (profiles/tc_kernels_8k_ncu_full.md); "
+                "DRAM traffic of these L2-resident, tensor-bound kernels does not grow in proportion to the "
+                "units processed, so no figure is extrapolated to other workloads")
 
 
 def load_peaks():
@@ -303,7 +310,7 @@ def run_ours(args, w):
     roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                 "frac": achieved / peak, "peak_source": peaks["source"] +
                 (" sustained" if peak == peaks["bf16_tflops_sustained"] else " burst"),
-                "traffic": NCU_TRAFFIC_BYTES.get((w.name, dom)),
+                "traffic": NCU_TRAFFIC_BYTES.get((w.name, dom)), "traffic_note": TRAFFIC_NOTE,
                 "per_kernel_ms": per_kernel_ms,
                 "per_kernel_tflops": {n: (algo_flops[n] / (per_kernel_ms[n] * 1e-3) / 1e12) for n in names}}
 
