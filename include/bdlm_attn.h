@@ -165,7 +165,7 @@ int bdlm_attn_bwd_static_scratch(const bdlm_params* p,
  *   13 wait for a free stage).
  * Pass NULL to switch tracing off (the default).  The caller zeroes and reads the buffer.
  */
-enum { BDLM_TRACE_SLOTS = 64 };
+enum { BDLM_TRACE_SLOTS = 256 };
 int bdlm_set_trace_buffer(void* device_counters, size_t bytes);
 
 #ifdef __cplusplus

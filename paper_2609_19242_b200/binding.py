@@ -22,7 +22,7 @@ EXPORTS = ("bdlm_workspace_bytes", "bdlm_attn_fwd", "bdlm_attn_bwd", "bdlm_lse_m
            "bdlm_status_string", "bdlm_get_device_status", "bdlm_set_trace_buffer",
            "bdlm_attn_bwd_static_scratch")
 STATIC_SCRATCH_ROWS = 1 << 20
-TRACE_SLOTS = 64
+TRACE_SLOTS = 256
 
 
 class BdlmError(RuntimeError):

@@ -180,58 +180,54 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
     if (lane == 0 && nsteps > 0) {
       long long w_pt = 0, w_q = 0, w_dst = 0;
       const long long t_begin = clock64();
+      const uint32_t k_lo = desc_lo_k(sK), v_lo = desc_lo_k(sV);
+      const uint32_t qk_lo0 = desc_lo_k(sQ0), qm_lo0 = desc_lo_mn(sQ0);       // Q ring, as K-major B (S^T) / MN-major B (dK)
+      const uint32_t dok_lo0 = desc_lo_k(sdO0), dom_lo0 = desc_lo_mn(sdO0);   // dO ring, as K-major B (dP^T) / MN-major B (dV)
       bool ok = mbar_wait_abortable(bar_kv, 0, abort_flag);
       ok = ok && mbar_wait_abortable(bar_q_full, 0, abort_flag);
       if (ok) {
         tc_fence_after();
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk) mma_ss(tmem, kmajor_desc(sK, kk), kmajor_desc(sQ0, kk), IDESC_KK, kk > 0);
+        gemm_ss(tmem, k_lo, qk_lo0, IDESC_KK, 0u);
         mma_commit(bar_st);
       }
       ok = ok && mbar_wait_abortable(bar_do_full, 0, abort_flag);
       if (ok) {
         tc_fence_after();
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk) mma_ss(tmem + 128, kmajor_desc(sV, kk), kmajor_desc(sdO0, kk), IDESC_KK, kk > 0);
+        gemm_ss(tmem + 128, v_lo, dok_lo0, IDESC_KK, 0u);
         mma_commit(bar_dpt);
       }
+      int sq = 0;   // i % 3
       for (int i = 0; i < nsteps && ok; ++i) {
-        const int sq = i % 3, sd = i & 1, nq = (i + 1) % 3;
-        const uint32_t cQ = sQ0 + sq * TILE_BYTES, cdO = sdO0 + sd * TILE_BYTES;
-        const uint32_t nQ = sQ0 + nq * TILE_BYTES, ndO = sdO0 + (sd ^ 1) * TILE_BYTES;
+        const int sd = i & 1, nq = (sq == 2) ? 0 : sq + 1;
+        const uint32_t acc = i > 0 ? 1u : 0u;
         // dV += P^T dO_i   (P^T: this lane's 64+64 bf16 pairs at columns [0,32) and [64,96))
-        ok = mbar_wait_timed(bar_pt, i & 1, abort_flag, w_pt);
+        ok = mbar_wait_lean(bar_pt, i & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk)
-          mma_ts(tmem + 256, tmem + (kk < 4 ? kk * 8 : 64 + (kk - 4) * 8), mnmajor_desc(cdO, kk), IDESC_KM, (i > 0 || kk > 0) ? 1u : 0u);
+        gemm_ts_mn<true>(tmem + 256, tmem, dom_lo0 + sd * TILE_LO, IDESC_KM, acc);
         mma_commit(bar_do_empty + 8 * sd);
         // S^T of the next step may start as soon as its Q is in shared memory
         if (i + 1 < nsteps) {
-          ok = mbar_wait_timed(bar_q_full + 8 * nq, ((i + 1) / 3) & 1, abort_flag, w_q);
+          ok = mbar_wait_lean(bar_q_full + 8 * nq, ((i + 1) / 3) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk) mma_ss(tmem, kmajor_desc(sK, kk), kmajor_desc(nQ, kk), IDESC_KK, kk > 0);
+          gemm_ss(tmem, k_lo, qk_lo0 + nq * TILE_LO, IDESC_KK, 0u);
           mma_commit(bar_st);
         }
         // dK += dS^T Q_i
-        ok = mbar_wait_timed(bar_dst, i & 1, abort_flag, w_dst);
+        ok = mbar_wait_lean(bar_dst, i & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk)
-          mma_ts(tmem + 384, tmem + 128 + (kk < 4 ? kk * 8 : 64 + (kk - 4) * 8), mnmajor_desc(cQ, kk), IDESC_KM, (i > 0 || kk > 0) ? 1u : 0u);
+        gemm_ts_mn<true>(tmem + 384, tmem + 128, qm_lo0 + sq * TILE_LO, IDESC_KM, acc);
         mma_commit(bar_q_empty + 8 * sq);
         if (i + 1 < nsteps) {
-          ok = mbar_wait_timed(bar_do_full + 8 * (sd ^ 1), ((i + 1) >> 1) & 1, abort_flag, w_q);
+          ok = mbar_wait_lean(bar_do_full + 8 * (sd ^ 1), ((i + 1) >> 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk) mma_ss(tmem + 128, kmajor_desc(sV, kk), kmajor_desc(ndO, kk), IDESC_KK, kk > 0);
+          gemm_ss(tmem + 128, v_lo, dok_lo0 + (sd ^ 1) * TILE_LO, IDESC_KK, 0u);
           mma_commit(bar_dpt);
         }
+        sq = nq;
       }
       mma_commit(bar_done);
       trace_add(a.trace, 16 + 8, clock64() - t_begin); trace_add(a.trace, 16 + 9, w_pt);
@@ -356,12 +352,28 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
 // =============================================================================================
 // dQ pass
 // =============================================================================================
-// Shared memory: Q, dO (resident), a 3-stage K ring (a K tile is read first by S and last by dQ) and
-// a 2-stage V ring.
+// Q and dO of the CTA's query tile are copied once from shared memory into tensor memory (bf16
+// pairs, one row per lane) and serve as TMEM-resident A operands, so S = Q K^T and dP = dO V^T
+// read only K / V from shared memory.  Shared memory: Q, dO staging, a 3-stage K ring (a K tile
+// is read first by S and last by dQ) and a 2-stage V ring.
 constexpr int DQ_K0 = 2 * TILE_BYTES;
 constexpr int DQ_V0 = 5 * TILE_BYTES;
 constexpr int DQ_BARS = 7 * TILE_BYTES;
-constexpr int DQ_SMEM = DQ_BARS + 160;
+constexpr int DQ_SMEM = DQ_BARS + 192;
+
+// Copy row `r` of a swizzled [128 x 128] bf16 tile into 64 TMEM columns (this thread's lane).
+__device__ __forceinline__ void row_smem_to_tmem(const uint8_t* tile, int r, uint32_t taddr) {
+#pragma unroll
+  for (int half = 0; half < 2; ++half) {
+    uint32_t v[32];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      const uint4 u = *reinterpret_cast<const uint4*>(tile + half * PANEL_BYTES + r * 128 + ((c ^ (r & 7)) << 4));
+      v[4 * c] = u.x; v[4 * c + 1] = u.y; v[4 * c + 2] = u.z; v[4 * c + 3] = u.w;
+    }
+    tmem_st32(taddr + half * 32, v);
+  }
+}
 
 __global__ void __launch_bounds__(BWD_THREADS, 1)
 tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restrict__ status) {
@@ -371,9 +383,10 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
   const uint32_t bars = base + DQ_BARS;
   const uint32_t bar_qdo = bars, bar_k_full = bars + 8 /*[3]*/, bar_k_empty = bars + 32 /*[3]*/,
                  bar_v_full = bars + 56 /*[2]*/, bar_v_empty = bars + 72 /*[2]*/,
-                 bar_s = bars + 88 /*[2]*/, bar_dp = bars + 104, bar_ds = bars + 112, bar_done = bars + 120;
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + DQ_BARS + 128);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + DQ_BARS + 136);
+                 bar_s = bars + 88, bar_sfree = bars + 96, bar_dp = bars + 104, bar_ds = bars + 112,
+                 bar_done = bars + 120, bar_aready = bars + 128;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + DQ_BARS + 144);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + DQ_BARS + 152);
 
   const int qs = blockIdx.z & 1, b = blockIdx.z >> 1, h = blockIdx.y, hk = h / a.G;
   const int q0 = (gridDim.x - 1 - blockIdx.x) * TILE;
@@ -400,8 +413,8 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
     mbar_init(bar_qdo, 1);
     for (int i = 0; i < 3; ++i) { mbar_init(bar_k_full + 8 * i, 1); mbar_init(bar_k_empty + 8 * i, 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(bar_v_full + 8 * i, 1); mbar_init(bar_v_empty + 8 * i, 1); }
-    mbar_init(bar_s, 1); mbar_init(bar_s + 8, 1);
-    mbar_init(bar_dp, 1); mbar_init(bar_ds, 256); mbar_init(bar_done, 1);
+    mbar_init(bar_s, 1); mbar_init(bar_sfree, 256);
+    mbar_init(bar_dp, 1); mbar_init(bar_ds, 256); mbar_init(bar_done, 1); mbar_init(bar_aready, 256);
     fence_mbar_init();
   }
   if (warp == 8) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
@@ -410,8 +423,8 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   const bool bad_base = (*abort_flag != 0);
-  // TMEM columns: [0,128) S even / dS   [128,256) dP   [256,384) dQ   [384,512) S odd / dS
-  auto s_col = [&](int i) { return (i & 1) ? 384u : 0u; };
+  // TMEM columns: [0,64) Q (bf16 pairs)  [64,128) dO (bf16 pairs)  [128,256) S  [256,384) dP / dS  [384,512) dQ
+  constexpr uint32_t C_Q = 0, C_DO = 64, C_S = 128, C_DP = 256, C_DQ = 384;
 
   if (bad_base) {
     // fall through to the common exit
@@ -439,56 +452,55 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
     }
   } else if (warp == 9) {
     if (lane == 0 && nsteps > 0) {
-      long long w_kv = 0, w_ds = 0;
+      long long w_kv = 0, w_ds = 0, w_sf = 0;
       const long long t_begin = clock64();
-      bool ok = mbar_wait_abortable(bar_qdo, 0, abort_flag);
+      const uint32_t kk_lo0 = desc_lo_k(sK0), km_lo0 = desc_lo_mn(sK0);   // K ring as K-major B (S) / MN-major B (dQ)
+      const uint32_t vk_lo0 = desc_lo_k(sV0);
+      bool ok = mbar_wait_abortable(bar_aready, 0, abort_flag);
       ok = ok && mbar_wait_abortable(bar_k_full, 0, abort_flag);
       if (ok) {
         tc_fence_after();
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk) mma_ss(tmem, kmajor_desc(sQ, kk), kmajor_desc(sK0, kk), IDESC_KK, kk > 0);
+        gemm_ts(tmem + C_S, tmem + C_Q, kk_lo0, IDESC_KK, 0u);
         mma_commit(bar_s);
       }
       ok = ok && mbar_wait_abortable(bar_v_full, 0, abort_flag);
       if (ok) {
         tc_fence_after();
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk) mma_ss(tmem + 128, kmajor_desc(sdO, kk), kmajor_desc(sV0, kk), IDESC_KK, kk > 0);
+        gemm_ts(tmem + C_DP, tmem + C_DO, vk_lo0, IDESC_KK, 0u);
         mma_commit(bar_dp);
         mma_commit(bar_v_empty);
       }
+      int sk = 0;   // i % 3
       for (int i = 0; i < nsteps && ok; ++i) {
-        const uint32_t cK = sK0 + (i % 3) * TILE_BYTES;
-        if (i + 1 < nsteps) {   // S of the next key tile into the other S buffer
-          const int nk = (i + 1) % 3;
-          ok = mbar_wait_timed(bar_k_full + 8 * nk, ((i + 1) / 3) & 1, abort_flag, w_kv);
+        const int nk = (sk == 2) ? 0 : sk + 1;
+        if (i + 1 < nsteps) {   // S of the next key tile, once both warpgroups have read S of this one
+          ok = mbar_wait_lean(bar_sfree, i & 1, abort_flag);
+          ok = ok && mbar_wait_lean(bar_k_full + 8 * nk, ((i + 1) / 3) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk) mma_ss(tmem + s_col(i + 1), kmajor_desc(sQ, kk), kmajor_desc(sK0 + nk * TILE_BYTES, kk), IDESC_KK, kk > 0);
-          mma_commit(bar_s + 8 * ((i + 1) & 1));
+          gemm_ts(tmem + C_S, tmem + C_Q, kk_lo0 + nk * TILE_LO, IDESC_KK, 0u);
+          mma_commit(bar_s);
         }
-        // dQ += dS_i K_i   (dS: bf16 pairs at columns [0,32) and [64,96) of this step's S buffer)
-        ok = mbar_wait_timed(bar_ds, i & 1, abort_flag, w_ds);
+        // dQ += dS_i K_i   (dS: bf16 pairs at columns [0,32) and [64,96) of the dP region)
+        ok = mbar_wait_lean(bar_ds, i & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk)
-          mma_ts(tmem + 256, tmem + s_col(i) + (kk < 4 ? kk * 8 : 64 + (kk - 4) * 8), mnmajor_desc(cK, kk), IDESC_KM, (i > 0 || kk > 0) ? 1u : 0u);
-        mma_commit(bar_k_empty + 8 * (i % 3));
+        gemm_ts_mn<true>(tmem + C_DQ, tmem + C_DP, km_lo0 + sk * TILE_LO, IDESC_KM, i > 0 ? 1u : 0u);
+        mma_commit(bar_k_empty + 8 * sk);
         if (i + 1 < nsteps) {
           const int nv = (i + 1) & 1;
-          ok = mbar_wait_timed(bar_v_full + 8 * nv, ((i + 1) >> 1) & 1, abort_flag, w_kv);
+          ok = mbar_wait_lean(bar_v_full + 8 * nv, ((i + 1) >> 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk) mma_ss(tmem + 128, kmajor_desc(sdO, kk), kmajor_desc(sV0 + nv * TILE_BYTES, kk), IDESC_KK, kk > 0);
+          gemm_ts(tmem + C_DP, tmem + C_DO, vk_lo0 + nv * TILE_LO, IDESC_KK, 0u);
           mma_commit(bar_dp);
           mma_commit(bar_v_empty + 8 * nv);
         }
+        sk = nk;
       }
       mma_commit(bar_done);
       trace_add(a.trace, 32 + 8, clock64() - t_begin); trace_add(a.trace, 32 + 9, w_kv); trace_add(a.trace, 32 + 10, w_ds);
+      trace_add(a.trace, 32 + 11, w_sf);
     }
   } else {
     const int w = warp >> 2;
@@ -509,20 +521,31 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
     long long w_s = 0, w_dp = 0, c_ld = 0, c_exp = 0, c_ds = 0;
     Stopwatch sw;
     const long long t_begin = clock64();
-    for (int i = 0; i < nsteps; ++i) {
+    if (nsteps > 0) {   // stage the A operands: warpgroup 0 copies Q, warpgroup 1 copies dO
+      ok = mbar_wait_abortable(bar_qdo, 0, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (ok) {
+        row_smem_to_tmem(sm + (w == 0 ? 0 : TILE_BYTES), r, tl + (w == 0 ? C_Q : C_DO));
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar_aready);
+      }
+    }
+    for (int i = 0; i < nsteps && ok; ++i) {
       const int ks = tile_ks(i), k0 = tile_k0(i);
-      ok = mbar_wait_timed(bar_s + 8 * (i & 1), (i >> 1) & 1, abort_flag, w_s);
+      ok = mbar_wait_timed(bar_s, i & 1, abort_flag, w_s);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const uint32_t ts = tl + s_col(i) + c0;
       uint32_t x[64];
       sw.start();
       {
         uint32_t (*c)[32] = reinterpret_cast<uint32_t (*)[32]>(x);
-        tmem_ld32(ts, c[0]); tmem_ld32(ts + 32, c[1]);
+        tmem_ld32(tl + C_S + c0, c[0]); tmem_ld32(tl + C_S + c0 + 32, c[1]);
         tmem_wait_ld();
       }
+      tc_fence_before();
+      mbar_arrive(bar_sfree);
       sw.lap(c_ld);
       const bool need_mask = ks == 0 ? (k0 < lo_last0 || k0 + TILE > hi_first0) : (k0 < lo_last1 || k0 + TILE > hi_first1);
       if (!need_mask) {
@@ -545,7 +568,7 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
       {
         uint32_t y[64];
         uint32_t (*c)[32] = reinterpret_cast<uint32_t (*)[32]>(y);
-        tmem_ld32(tl + 128 + c0, c[0]); tmem_ld32(tl + 128 + c0 + 32, c[1]);
+        tmem_ld32(tl + C_DP + c0, c[0]); tmem_ld32(tl + C_DP + c0 + 32, c[1]);
         tmem_wait_ld();
         uint32_t pk[32];
 #pragma unroll
@@ -554,7 +577,7 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
           const float d1 = __uint_as_float(x[2 * e + 1]) * (__uint_as_float(y[2 * e + 1]) - dsum);
           pk[e] = pack_bf16(d0, d1);
         }
-        tmem_st32(ts, pk);
+        tmem_st32(tl + C_DP + c0, pk);
         tmem_wait_st();
       }
       tc_fence_before();
@@ -576,7 +599,7 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
         uint32_t v[32];
-        if (nsteps > 0) { tmem_ld32(tl + 256 + c0 + c * 32, v); tmem_wait_ld(); }
+        if (nsteps > 0) { tmem_ld32(tl + C_DQ + c0 + c * 32, v); tmem_wait_ld(); }
         else {
 #pragma unroll
           for (int e = 0; e < 32; ++e) v[e] = 0u;

@@ -65,6 +65,13 @@ __device__ __forceinline__ bool mbar_wait_abortable(uint32_t bar, uint32_t parit
   return true;
 }
 
+// Lean wait for the MMA-issuing thread: its instruction stream is the critical path, so the common case
+// (barrier already complete) must cost a single try_wait.
+__device__ __forceinline__ bool mbar_wait_lean(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_abortable(bar, parity, abort_flag);
+}
+
 __device__ __forceinline__ bool mbar_wait_timed(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long& acc) {
   const long long t0 = clock64();
   const bool ok = mbar_wait_abortable(bar, parity, abort_flag);
@@ -175,6 +182,39 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
 __host__ __device__ constexpr uint32_t make_idesc(int M, int N, bool a_mn_major, bool b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16) |
          (static_cast<uint32_t>(N >> 3) << 17) | (static_cast<uint32_t>(M >> 4) << 24);
+}
+
+// The MMA-issuing thread is a single scalar instruction stream: a 128x128x16 MMA occupies the
+// tensor pipe for 64 clocks, so the issue path must cost well under that per instruction.
+// Descriptors are therefore kept as a precomputed low word per tile (address field + LBO) plus a
+// constant high word, and the k-slice offsets are compile-time constants added to the low word.
+constexpr uint32_t DESC_HI = 0x40004040u;   // SBO = 1024 B (>>4 = 0x40), version 1 (bit 46), SWIZZLE_128B (2 << 61)
+__device__ __forceinline__ uint32_t desc_lo_k(uint32_t addr) { return ((addr & 0x3FFFFu) >> 4) | (1u << 16); }
+__device__ __forceinline__ uint32_t desc_lo_mn(uint32_t addr) {
+  return ((addr & 0x3FFFFu) >> 4) | (static_cast<uint32_t>(PANEL_BYTES >> 4) << 16);
+}
+__device__ __forceinline__ uint64_t desc64(uint32_t lo) { return (static_cast<uint64_t>(DESC_HI) << 32) | lo; }
+__host__ __device__ constexpr uint32_t koff(int kk) { return (kk >> 2) * (PANEL_BYTES >> 4) + (kk & 3) * 2; }   // K-major slice
+__host__ __device__ constexpr uint32_t moff(int kk) { return kk * 128; }                                        // MN-major slice (16 rows)
+constexpr uint32_t TILE_LO = (2 * PANEL_BYTES) >> 4;   // low-word stride between consecutive 32 KB tiles
+
+// D (+)= A B^T, A and B both K-major tiles in shared memory (8 k-slices of 16).
+__device__ __forceinline__ void gemm_ss(uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t acc_first) {
+#pragma unroll
+  for (int kk = 0; kk < 8; ++kk) mma_ss(d, desc64(a_lo + koff(kk)), desc64(b_lo + koff(kk)), idesc, kk == 0 ? acc_first : 1u);
+}
+// A = 64 contiguous TMEM columns of bf16 pairs, B K-major tile in shared memory.
+__device__ __forceinline__ void gemm_ts(uint32_t d, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc, uint32_t acc_first) {
+#pragma unroll
+  for (int kk = 0; kk < 8; ++kk) mma_ts(d, a_tmem + kk * 8, desc64(b_lo + koff(kk)), idesc, kk == 0 ? acc_first : 1u);
+}
+// A = bf16 pairs in TMEM, B MN-major tile ([contraction row][128 columns]) in shared memory.  `split`: the A
+// pairs of contraction indices 64..127 sit 64 columns after those of 0..63 (two warpgroups wrote them).
+template <bool SPLIT>
+__device__ __forceinline__ void gemm_ts_mn(uint32_t d, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc, uint32_t acc_first) {
+#pragma unroll
+  for (int kk = 0; kk < 8; ++kk)
+    mma_ts(d, a_tmem + (SPLIT ? (kk < 4 ? kk * 8 : 64 + (kk - 4) * 8) : kk * 8), desc64(b_lo + moff(kk)), idesc, kk == 0 ? acc_first : 1u);
 }
 
 // Byte offset of element (row, col) inside a [128 x 128] bf16 tile stored as two swizzled panels

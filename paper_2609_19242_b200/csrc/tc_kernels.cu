@@ -360,44 +360,48 @@ tc_fwd2_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
     }
   } else if (warp == 9) {
     if (lane == 0 && nt > 0) {
-      auto issue_qk = [&](int w, uint32_t kt) {
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
-          const uint32_t off = (kk >> 2) * PANEL_BYTES + (kk & 3) * 32;
-          mma_ss(tmem + w * 128, smem_desc(sQ + w * TILE_BYTES + off, 16, 1024), smem_desc(kt + off, 16, 1024), IDESC_QK, kk > 0);
-        }
-        mma_commit(bar_s + 8 * w);
-      };
+      const uint32_t qa_lo = desc_lo_k(sQ), qb_lo = qa_lo + TILE_LO;
+      const uint32_t k_lo0 = desc_lo_k(sK0), v_lo0 = desc_lo_mn(sK0 + TILE_BYTES);
       long long w_p = 0, w_v = 0, w_k = 0;
       const long long t_begin = clock64();
       bool ok = mbar_wait_abortable(bar_q, 0, abort_flag);
       ok = ok && mbar_wait_abortable(bar_k_full, 0, abort_flag);
       if (ok) {
         tc_fence_after();
-        issue_qk(0, sK0);
-        issue_qk(1, sK0);
+        gemm_ss(tmem, qa_lo, k_lo0, IDESC_QK, 0u);
+        mma_commit(bar_s);
+        gemm_ss(tmem + 128, qb_lo, k_lo0, IDESC_QK, 0u);
+        mma_commit(bar_s + 8);
       }
       for (int t = 0; t < nt && ok; ++t) {
         const int s = t & 1;
-        const uint32_t cV = sK0 + s * 2 * TILE_BYTES + TILE_BYTES;
-        const uint32_t nK = sK0 + (s ^ 1) * 2 * TILE_BYTES;
-        for (int w = 0; w < 2 && ok; ++w) {
-          ok = mbar_wait_timed(bar_p + 8 * w, t & 1, abort_flag, w_p);
-          if (ok && w == 0) ok = mbar_wait_timed(bar_v_full + 8 * s, (t >> 1) & 1, abort_flag, w_v);
+        const uint32_t cv_lo = v_lo0 + s * 2 * TILE_LO;
+        const uint32_t nk_lo = k_lo0 + (s ^ 1) * 2 * TILE_LO;
+        const uint32_t acc = t > 0 ? 1u : 0u;
+        // head A
+        ok = mbar_wait_lean(bar_p, t & 1, abort_flag);
+        ok = ok && mbar_wait_lean(bar_v_full + 8 * s, (t >> 1) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        gemm_ts_mn<false>(tmem + 256, tmem, cv_lo, IDESC_PV, acc);
+        mma_commit(bar_o);
+        if (t + 1 < nt) {
+          ok = mbar_wait_lean(bar_k_full + 8 * (s ^ 1), ((t + 1) >> 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk)
-            mma_ts(tmem + 256 + w * 128, tmem + w * 128 + kk * 8, smem_desc(cV + kk * 2048, PANEL_BYTES, 1024), IDESC_PV,
-                   (t > 0 || kk > 0) ? 1u : 0u);
-          mma_commit(bar_o + 8 * w);
-          if (w == 1) mma_commit(bar_kv_empty + 8 * s);
-          if (t + 1 < nt) {
-            if (w == 0) ok = mbar_wait_timed(bar_k_full + 8 * (s ^ 1), ((t + 1) >> 1) & 1, abort_flag, w_k);
-            if (!ok) break;
-            tc_fence_after();
-            issue_qk(w, nK);
-          }
+          gemm_ss(tmem, qa_lo, nk_lo, IDESC_QK, 0u);
+          mma_commit(bar_s);
+        }
+        // head B
+        ok = mbar_wait_lean(bar_p + 8, t & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        gemm_ts_mn<false>(tmem + 384, tmem + 128, cv_lo, IDESC_PV, acc);
+        mma_commit(bar_o + 8);
+        mma_commit(bar_kv_empty + 8 * s);
+        if (t + 1 < nt) {
+          gemm_ss(tmem + 128, qb_lo, nk_lo, IDESC_QK, 0u);
+          mma_commit(bar_s + 8);
         }
       }
       trace_add(a.trace, 8, clock64() - t_begin); trace_add(a.trace, 9, w_p); trace_add(a.trace, 10, w_v); trace_add(a.trace, 11, w_k);
