@@ -152,14 +152,27 @@ def cpu_inputs_for_oracle(w):
     return synth.make_inputs(small, "cpu")
 
 
+def timed_oracle_sample(w, inp, target_seconds, max_rows):
+    """Calibrates on a small sample, then runs one sample sized for about `target_seconds` of CPU work."""
+    oracle_sample(w, inp, 8, seed=99)                      # warm-up (BLAS threads, page faults)
+    t_cal, _ = oracle_sample(w, inp, 64, seed=98)
+    rows = int(min(max_rows, max(64, 64 * target_seconds / max(t_cal, 1e-3))))
+    t, f = oracle_sample(w, inp, rows, seed=0)
+    return rows, t, f
+
+
 def run_reference(args, w):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     inp = cpu_inputs_for_oracle(w)
-    rows = args.oracle_rows
+    # each step is a bounded sample; the whole run is sized to end within a few minutes
+    oracle_sample(w, inp, 8, seed=99)
+    t_cal, _ = oracle_sample(w, inp, 64, seed=98)
+    per_step_s = min(20.0, 120.0 / max(1, args.steps + args.warmup))
+    rows = args.oracle_rows if args.oracle_rows > 0 else int(min(w.L, max(64, 64 * per_step_s / max(t_cal, 1e-3))))
     for i in range(args.warmup):
-        oracle_sample(w, inp, max(8, rows // 8), seed=100 + i)
+        oracle_sample(w, inp, rows, seed=100 + i)
     t_tot, f_tot = 0.0, 0
     for i in range(args.steps):
         t, f = oracle_sample(w, inp, rows, seed=i)
@@ -177,6 +190,21 @@ def run_reference(args, w):
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
+
+
+def max_over_ranks(value_ms, device, world):
+    """Slowest rank's time (every multi-GPU number is the max over ranks)."""
+    if world <= 1:
+        return float(value_ms)
+    import torch.distributed as dist
+    t = torch.tensor([float(value_ms)], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_tflops(flops_per_replica, ms_per_step, world):
+    """Whole-job throughput of `world` independent replicas that each do `flops_per_replica` per step."""
+    return world * flops_per_replica / (ms_per_step * 1e-3) / 1e12
 
 
 # ------------------------------------------------------------------------------------------
@@ -251,15 +279,12 @@ def run_ours(args, w):
     clocks = sampler.stop() if rank == 0 else None
     if binding.bdlm_get_device_status() != 0:
         raise RuntimeError("device-side wait timed out during the timed region")
-    if world > 1:
-        t = torch.tensor([ms_total], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, "cuda", world)
     per_kernel_ms = {n: float(np.mean([ev[i][j].elapsed_time(ev[i][j + 1]) for i in range(K)])) for j, n in enumerate(names)}
 
     f_fwd, f_bwd = w.flops()
     ms_step = ms_total / K
-    value = world * (f_fwd + f_bwd) / (ms_step * 1e-3) / 1e12
+    value = aggregate_tflops(f_fwd + f_bwd, ms_step, world)
 
     # ---- end to end through the public call with HOST buffers (pinned), copies inside ---------
     e2e = None
@@ -287,11 +312,8 @@ def run_ours(args, w):
         b.record()
         barrier()
         ms_e2e = a.elapsed_time(b) / n_e2e
-        if world > 1:
-            t = torch.tensor([ms_e2e], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
-        e2e = {"value": world * (f_fwd + f_bwd) / (ms_e2e * 1e-3) / 1e12, "unit": UNIT,
+        ms_e2e = max_over_ranks(ms_e2e, "cuda", world)
+        e2e = {"value": aggregate_tflops(f_fwd + f_bwd, ms_e2e, world), "unit": UNIT,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e}
         del host_in, host_out
 
@@ -318,10 +340,14 @@ def run_ours(args, w):
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
         inp = cpu_inputs_for_oracle(w)
-        oracle_sample(w, inp, 8, seed=99)
-        t, f = oracle_sample(w, inp, args.oracle_rows, seed=0)
+        if args.oracle_rows > 0:
+            oracle_sample(w, inp, 8, seed=99)
+            rows = args.oracle_rows
+            t, f = oracle_sample(w, inp, rows, seed=0)
+        else:
+            rows, t, f = timed_oracle_sample(w, inp, 40.0, w.L)
         cpu = {"value": f / t / 1e12, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
-               "sample": f"{args.oracle_rows} sampled query rows per stream of (batch 0, head 0), fwd+bwd, fp64, {t:.1f} s"}
+               "sample": f"{rows} sampled query rows per stream of (batch 0, head 0), fwd+bwd, fp64, {t:.1f} s"}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -347,7 +373,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="32k", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--kernel-impl", type=int, default=0, help="0 auto, 1 portable mma.sync, 2 tcgen05")
-    ap.add_argument("--oracle-rows", type=int, default=768)
+    ap.add_argument("--oracle-rows", type=int, default=0, help="rows per stream in the oracle sample; 0 = size it for ~15 s")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     w = synth.WORKLOADS[args.workload]
