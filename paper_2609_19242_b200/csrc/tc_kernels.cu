@@ -283,27 +283,33 @@ struct TileSched {
 };
 
 // ---------------------------------------------------------------- forward, warp-specialised
-// One CTA = one 128-row query tile of TWO query heads of the same KV group (same stream, same
-// rows, so the same key tiles and the same masks).  Warp 8 loads Q of both heads once and
-// streams K/V tiles through a 2-stage ring; warp 9 issues tcgen05.mma; warpgroup w (warps
-// 4w..4w+3) runs the online softmax of head w, one thread per row, writes P (bf16) over its S
-// columns in tensor memory and rescales its O accumulator only when the running maximum grew
-// by more than 2^8 (the stale maximum is exact in the final LSE and normalisation).
-constexpr int FWD2_THREADS = 320;
-constexpr int FWD2_BARS = 6 * TILE_BYTES;                 // Q_A, Q_B, two (K, V) stages
-constexpr int FWD2_SMEM = FWD2_BARS + 256 + 1024;
+// One CTA = one 128-row query tile of TWO query heads of the same KV group (same stream, same rows, so
+// the same key tiles and the same masks).  Warp 16 loads Q of both heads once and streams K/V tiles through
+// a 2-stage ring; warp 17 issues tcgen05.mma (QK^T from shared memory, PV with P as a TMEM operand);
+// warps 0-15 run the online softmax, two warpgroups per head, each owning one half of the 128 score
+// columns of every row (with one warpgroup per head a single warp per scheduler runs the whole row, about
+// 2300 clocks per tile; two bring it close to the exponential unit's floor).  The halves exchange their
+// partial row maximum through shared memory once per tile and add their partial row sums once at the end.
+// P (bf16) overwrites the S columns it was computed from; O is rescaled only when the running maximum
+// grew by more than 2^8 (the stale maximum is exact in the final LSE and normalisation).
+constexpr int FWD2H_THREADS = 576;                          // 16 softmax warps, producer warp, MMA warp
+constexpr int FWD2H_MX = 6 * TILE_BYTES;                    // mx_s[2][2][2][128] floats, then ls_s[2][2][128]
+constexpr int FWD2H_BARS = FWD2H_MX + 4096 + 2048;
+constexpr int FWD2H_SMEM = FWD2H_BARS + 256 + 1024;
 
-__global__ void __launch_bounds__(FWD2_THREADS, 1)
-tc_fwd2_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restrict__ status) {
+__global__ void __launch_bounds__(FWD2H_THREADS, 1)
+tc_fwd2h_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t sQ = base, sK0 = base + 2 * TILE_BYTES;   // stage s: K at sK0 + s*2*TILE, V after it
-  const uint32_t bars = base + FWD2_BARS;
+  float* mx_s = reinterpret_cast<float*>(sm + FWD2H_MX);    // [tile parity][head][half][row]
+  float* ls_s = mx_s + 1024;                               // [head][half][row]
+  const uint32_t bars = base + FWD2H_BARS;
   const uint32_t bar_q = bars, bar_k_full = bars + 8 /*[2]*/, bar_v_full = bars + 24 /*[2]*/, bar_kv_empty = bars + 40 /*[2]*/,
                  bar_s = bars + 56 /*[2]*/, bar_p = bars + 72 /*[2]*/, bar_o = bars + 88 /*[2]*/;
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + FWD2_BARS + 128);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + FWD2_BARS + 136);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + FWD2H_BARS + 128);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + FWD2H_BARS + 136);
 
   const int qs = blockIdx.z & 1, b = blockIdx.z >> 1;
   if (a.q[qs] == nullptr) return;
@@ -321,19 +327,19 @@ tc_fwd2_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
     mbar_init(bar_q, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar_k_full + 8 * i, 1); mbar_init(bar_v_full + 8 * i, 1); mbar_init(bar_kv_empty + 8 * i, 1);
-      mbar_init(bar_s + 8 * i, 1); mbar_init(bar_p + 8 * i, 128); mbar_init(bar_o + 8 * i, 1);
+      mbar_init(bar_s + 8 * i, 1); mbar_init(bar_p + 8 * i, 256); mbar_init(bar_o + 8 * i, 1);
     }
     *abort_flag = 0;
     fence_mbar_init();
   }
-  if (warp == 8) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
+  if (warp == 16) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   // TMEM columns: [0,128) S/P head A   [128,256) S/P head B   [256,384) O head A   [384,512) O head B
 
-  if (warp == 8) {
+  if (warp == 16) {
     if (lane == 0 && nt > 0) {
       mbar_expect_tx(bar_q, 2 * TILE_BYTES);
       tma_load_3d(sQ, &maps.q[qs], bar_q, h0 * 128, q0, b);
@@ -341,11 +347,9 @@ tc_fwd2_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
       tma_load_3d(sQ + TILE_BYTES, &maps.q[qs], bar_q, h0 * 128 + 128, q0, b);
       tma_load_3d(sQ + TILE_BYTES + PANEL_BYTES, &maps.q[qs], bar_q, h0 * 128 + 192, q0, b);
       bool ok = true;
-      long long w_empty = 0;
-      const long long t_begin = clock64();
       for (int t = 0; t < nt && ok; ++t) {
         const int s = t & 1;
-        if (t >= 2) ok = mbar_wait_timed(bar_kv_empty + 8 * s, ((t >> 1) - 1) & 1, abort_flag, w_empty);
+        if (t >= 2) ok = mbar_wait_abortable(bar_kv_empty + 8 * s, ((t >> 1) - 1) & 1, abort_flag);
         if (!ok) break;
         const int ks = tile_ks(t), k0 = tile_k0(t);
         const uint32_t dK = sK0 + s * 2 * TILE_BYTES, dV = dK + TILE_BYTES;
@@ -356,14 +360,11 @@ tc_fwd2_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
         tma_load_3d(dV, &maps.v[ks], bar_v_full + 8 * s, hk * 128, k0, b);
         tma_load_3d(dV + PANEL_BYTES, &maps.v[ks], bar_v_full + 8 * s, hk * 128 + 64, k0, b);
       }
-      trace_add(a.trace, 12, clock64() - t_begin); trace_add(a.trace, 13, w_empty);
     }
-  } else if (warp == 9) {
+  } else if (warp == 17) {
     if (lane == 0 && nt > 0) {
       const uint32_t qa_lo = desc_lo_k(sQ), qb_lo = qa_lo + TILE_LO;
       const uint32_t k_lo0 = desc_lo_k(sK0), v_lo0 = desc_lo_mn(sK0 + TILE_BYTES);
-      long long w_p = 0, w_v = 0, w_k = 0;
-      const long long t_begin = clock64();
       bool ok = mbar_wait_abortable(bar_q, 0, abort_flag);
       ok = ok && mbar_wait_abortable(bar_k_full, 0, abort_flag);
       if (ok) {
@@ -378,12 +379,12 @@ tc_fwd2_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
         const uint32_t cv_lo = v_lo0 + s * 2 * TILE_LO;
         const uint32_t nk_lo = k_lo0 + (s ^ 1) * 2 * TILE_LO;
         const uint32_t acc = t > 0 ? 1u : 0u;
-        // head A
+        // head A   (P: bf16 pairs at columns [0,32) and [64,96) of the head's S region)
         ok = mbar_wait_lean(bar_p, t & 1, abort_flag);
         ok = ok && mbar_wait_lean(bar_v_full + 8 * s, (t >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        gemm_ts_mn<false>(tmem + 256, tmem, cv_lo, IDESC_PV, acc);
+        gemm_ts_mn<true>(tmem + 256, tmem, cv_lo, IDESC_PV, acc);
         mma_commit(bar_o);
         if (t + 1 < nt) {
           ok = mbar_wait_lean(bar_k_full + 8 * (s ^ 1), ((t + 1) >> 1) & 1, abort_flag);
@@ -396,7 +397,7 @@ tc_fwd2_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
         ok = mbar_wait_lean(bar_p + 8, t & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        gemm_ts_mn<false>(tmem + 384, tmem + 128, cv_lo, IDESC_PV, acc);
+        gemm_ts_mn<true>(tmem + 384, tmem + 128, cv_lo, IDESC_PV, acc);
         mma_commit(bar_o + 8);
         mma_commit(bar_kv_empty + 8 * s);
         if (t + 1 < nt) {
@@ -404,67 +405,70 @@ tc_fwd2_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
           mma_commit(bar_s + 8);
         }
       }
-      trace_add(a.trace, 8, clock64() - t_begin); trace_add(a.trace, 9, w_p); trace_add(a.trace, 10, w_v); trace_add(a.trace, 11, w_k);
     }
   } else {
-    const int w = warp >> 2;
+    const int g = warp >> 2, w = g >> 1, hc = g & 1;      // head, column half
     const int r = (warp & 3) * 32 + lane;
     const int row = q0 + r;
     const int h = h0 + w;
-    const uint32_t tS = tmem + ((uint32_t)((warp & 3) * 32) << 16) + w * 128;
-    const uint32_t tO = tmem + ((uint32_t)((warp & 3) * 32) << 16) + 256 + w * 128;
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t tS = tmem + lane_base + w * 128 + hc * 64;          // this thread's 64 score columns
+    const uint32_t tO = tmem + lane_base + 256 + w * 128 + hc * 64;    // and its 64 output columns
     int rlo0, rhi0, rlo1, rhi1;
     visible_interval(qs, 0, row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo0, rhi0);
     visible_interval(qs, 1, row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo1, rhi1);
     float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
-    long long w_s = 0, w_o = 0, c_p1 = 0, c_p2ld = 0, c_p2 = 0;
-    Stopwatch sw;
+    long long w_s = 0;
     const long long t_begin = clock64();
     for (int t = 0; t < nt; ++t) {
       const int ks = tile_ks(t), k0 = tile_k0(t);
-      ok = mbar_wait_timed(bar_s + 8 * w, t & 1, abort_flag, w_s);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
+      // After a failed (timed-out) wait this warpgroup keeps walking the loop without touching tensor memory,
+      // so that it still meets its partner at every named barrier: the failure path must end, never hang.
+      if (ok) {
+        ok = mbar_wait_timed(bar_s + 8 * w, t & 1, abort_flag, w_s);
+        ok = __all_sync(0xffffffffu, ok);
+      }
       tc_fence_after();
       const bool need_mask = sch.need_mask(ks, k0);
-      const int vlo = (ks == 0 ? rlo0 : rlo1) - k0, vhi = (ks == 0 ? rhi0 : rhi1) - k0;   // visible columns [vlo, vhi) of this tile
-      sw.start();
-      // pass 1: row maximum of the raw scores (scale > 0 commutes with max); S is re-read in pass 2
+      const int vlo = (ks == 0 ? rlo0 : rlo1) - k0 - hc * 64, vhi = (ks == 0 ? rhi0 : rhi1) - k0 - hc * 64;
+      // pass 1: maximum of this half row, exchanged with the other half
       float mx = -INFINITY;
-#pragma unroll
-      for (int c2 = 0; c2 < 2; ++c2) {
+      if (ok) {
         uint32_t v0[32], v1[32];
-        tmem_ld32(tS + c2 * 64, v0); tmem_ld32(tS + c2 * 64 + 32, v1);
+        tmem_ld32(tS, v0); tmem_ld32(tS + 32, v1);
         tmem_wait_ld();
         if (need_mask) {
 #pragma unroll
           for (int e = 0; e < 32; ++e) {
-            const int j0 = c2 * 64 + e, j1 = j0 + 32;
-            mx = fmaxf(mx, (j0 >= vlo && j0 < vhi) ? __uint_as_float(v0[e]) : -INFINITY);
-            mx = fmaxf(mx, (j1 >= vlo && j1 < vhi) ? __uint_as_float(v1[e]) : -INFINITY);
+            mx = fmaxf(mx, (e >= vlo && e < vhi) ? __uint_as_float(v0[e]) : -INFINITY);
+            mx = fmaxf(mx, (e + 32 >= vlo && e + 32 < vhi) ? __uint_as_float(v1[e]) : -INFINITY);
           }
         } else {
 #pragma unroll
           for (int e = 0; e < 32; ++e) mx = fmaxf(mx, fmaxf(__uint_as_float(v0[e]), __uint_as_float(v1[e])));
         }
       }
-      mx *= a.scale_log2;   // -inf stays -inf
-      sw.lap(c_p1);
+      mx *= a.scale_log2;
+      float* slot = mx_s + (((t & 1) * 2 + w) * 2) * 128;
+      slot[hc * 128 + r] = mx;
+      asm volatile("bar.sync %0, %1;" ::"r"(1 + w), "r"(256) : "memory");
+      mx = fmaxf(mx, slot[(hc ^ 1) * 128 + r]);
+      if (!ok) continue;
       const float m_new = fmaxf(m_ref, mx);
       const bool grow = m_new > m_ref + 8.0f;
-      if (__any_sync(0xffffffffu, grow)) {
+      if (__any_sync(0xffffffffu, grow)) {   // same decision in both halves: same rows, same m_ref, same m_new
         const float mb_new = (m_new == -INFINITY) ? 0.f : m_new;
         const float corr = exp2f(m_ref - mb_new);
         m_ref = m_new;
         l *= corr;
         if (t > 0) {
-          ok = mbar_wait_timed(bar_o + 8 * w, (t - 1) & 1, abort_flag, w_o);
+          ok = mbar_wait_abortable(bar_o + 8 * w, (t - 1) & 1, abort_flag);
           ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
+          if (!ok) continue;
           tc_fence_after();
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
+          for (int c = 0; c < 2; ++c) {
             uint32_t o[32];
             tmem_ld32(tO + c * 32, o);
             tmem_wait_ld();
@@ -475,15 +479,12 @@ tc_fwd2_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
         }
       }
       const float mb = (m_ref == -INFINITY) ? 0.f : m_ref;
-      sw.start();
-      // pass 2: p = exp2(s * scale - m), packed to bf16 pairs over the first 64 columns of S
+      // pass 2: p = exp2(s * scale - m) for this half row; bf16 pairs over its own first 32 columns
       float psum = 0.f;
-#pragma unroll
-      for (int c2 = 0; c2 < 2; ++c2) {
+      {
         uint32_t v0[32], v1[32], pk[32];
-        tmem_ld32(tS + c2 * 64, v0); tmem_ld32(tS + c2 * 64 + 32, v1);
+        tmem_ld32(tS, v0); tmem_ld32(tS + 32, v1);
         tmem_wait_ld();
-        sw.lap(c_p2ld);
         if (!need_mask) {
 #pragma unroll
           for (int e = 0; e < 16; ++e) {
@@ -498,7 +499,7 @@ tc_fwd2_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
         } else {
 #pragma unroll
           for (int e = 0; e < 16; ++e) {
-            const int j = c2 * 64 + 2 * e;
+            const int j = 2 * e;
             float p0 = exp2f(fmaf(__uint_as_float(v0[2 * e]), a.scale_log2, -mb));
             float p1 = exp2f(fmaf(__uint_as_float(v0[2 * e + 1]), a.scale_log2, -mb));
             float p2 = exp2f(fmaf(__uint_as_float(v1[2 * e]), a.scale_log2, -mb));
@@ -512,30 +513,28 @@ tc_fwd2_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
             pk[16 + e] = pack_bf16(p2, p3);
           }
         }
-        // the second pass over columns [64, 128) must not be clobbered: P of the first 64 columns
-        // lands in TMEM columns [0, 32), which pass 2 has already consumed
-        tmem_st32(tS + c2 * 32, pk);
-        sw.lap(c_p2);
+        tmem_st32(tS, pk);
       }
       l += psum;
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(bar_p + 8 * w);
     }
-    if (warp == 0 && lane == 0) {
-      trace_add(a.trace, 0, nt); trace_add(a.trace, 1, w_s); trace_add(a.trace, 2, w_o); trace_add(a.trace, 6, clock64() - t_begin);
-      trace_add(a.trace, 3, c_p1); trace_add(a.trace, 4, c_p2ld); trace_add(a.trace, 5, c_p2);
-    }
+    if (warp == 0 && lane == 0) { trace_add(a.trace, 0, nt); trace_add(a.trace, 1, w_s); trace_add(a.trace, 6, clock64() - t_begin); }
+    // total row sum = sum of the two halves (both kept the same reference maximum)
+    ls_s[(w * 2 + hc) * 128 + r] = l;
+    asm volatile("bar.sync %0, %1;" ::"r"(1 + w), "r"(256) : "memory");
+    const float l_tot = l + ls_s[(w * 2 + (hc ^ 1)) * 128 + r];
     if (ok && nt > 0) {
       ok = mbar_wait_abortable(bar_o + 8 * w, (nt - 1) & 1, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
     }
     if (ok) {
       tc_fence_after();
-      const float inv = l > 0.f ? 1.f / l : 0.f;
-      bf16* orow = a.o[qs] + (((int64_t)b * a.L + row) * a.H + h) * 128;
+      const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
+      bf16* orow = a.o[qs] + (((int64_t)b * a.L + row) * a.H + h) * 128 + hc * 64;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < 2; ++c) {
         uint32_t o[32];
         if (nt > 0) { tmem_ld32(tO + c * 32, o); tmem_wait_ld(); }
 #pragma unroll
@@ -551,13 +550,13 @@ tc_fwd2_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
           *reinterpret_cast<uint4*>(orow + c * 32 + e8 * 8) = v;
         }
       }
-      a.lse[qs][((int64_t)b * a.H + h) * a.L + row] = l > 0.f ? (m_ref + log2f(l)) * LN2 : -INFINITY;
+      if (hc == 0) a.lse[qs][((int64_t)b * a.H + h) * a.L + row] = l_tot > 0.f ? (m_ref + log2f(l_tot)) * LN2 : -INFINITY;
     }
   }
   tc_fence_before();
   __syncthreads();
   if (threadIdx.x == 0 && *abort_flag) atomicExch(status, (int)BDLM_ERR_DEVICE_TIMEOUT);
-  if (warp == 8) tmem_dealloc(tmem, 512);
+  if (warp == 16) tmem_dealloc(tmem, 512);
 }
 
 }  // namespace
@@ -578,11 +577,11 @@ cudaError_t launch_tc_fwd(const KArgs& a, cudaStream_t st) {
   if (status == nullptr) return cudaErrorUnknown;
   cudaError_t e = cudaFuncSetAttribute(tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM);
   if (e != cudaSuccess) return e;
-  if (a.G % 2 == 0) {   // two heads of one KV group per CTA
-    e = cudaFuncSetAttribute(tc_fwd2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD2_SMEM);
+  if (a.G % 2 == 0) {   // two heads of one KV group per CTA, four softmax warpgroups
+    e = cudaFuncSetAttribute(tc_fwd2h_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD2H_SMEM);
     if (e != cudaSuccess) return e;
-    dim3 grid2(a.L / TILE, a.H / 2, a.batch * 2);
-    tc_fwd2_kernel<<<grid2, FWD2_THREADS, FWD2_SMEM, st>>>(maps, a, status);
+    dim3 grid4(a.L / TILE, a.H / 2, a.batch * 2);
+    tc_fwd2h_kernel<<<grid4, FWD2H_THREADS, FWD2H_SMEM, st>>>(maps, a, status);
     return cudaGetLastError();
   }
   dim3 grid(a.L / TILE, a.H, a.batch * 2);
