@@ -58,7 +58,12 @@ typedef struct {
   int32_t bwd_passes;          /* backward only: 0 = all passes; otherwise a bit set of BDLM_BWD_PASS_* to run
                                   (lets a caller time the passes separately; each pass needs the earlier ones'
                                   results from a previous call with the same workspace) */
-  int32_t reserved[4];
+  int32_t bwd_single_pass;     /* backward only: 0 = dK/dV pass + dQ pass, fixed summation order, bitwise reproducible;
+                                  1 = one pass: dQ is accumulated by the dK/dV kernel with fp32 atomic adds (5 GEMMs per
+                                  tile pair instead of 7; dQ is then reproducible only up to fp32 summation order).
+                                  Needs the larger workspace bdlm_workspace_bytes reports for this setting; falls back to
+                                  the two-pass path when the tensor-core kernels do not take the shape. */
+  int32_t reserved[3];
 } bdlm_params;
 
 enum { BDLM_BWD_PASS_DSUM = 1, BDLM_BWD_PASS_DKDV = 2, BDLM_BWD_PASS_DQ = 4 };

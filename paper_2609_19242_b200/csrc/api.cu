@@ -21,6 +21,7 @@ int check_params(const bdlm_params* p) {
   if (p->clean_mask_mode != 0 && p->clean_mask_mode != 1) return BDLM_ERR_INVALID_ARG;
   if (p->impl < 0 || p->impl > 2) return BDLM_ERR_INVALID_ARG;
   if (p->bwd_passes < 0 || p->bwd_passes > 7) return BDLM_ERR_INVALID_ARG;
+  if (p->bwd_single_pass != 0 && p->bwd_single_pass != 1) return BDLM_ERR_INVALID_ARG;
   if (!(p->scale >= 0.f) || isinf(p->scale)) return BDLM_ERR_INVALID_ARG;
   if (p->kv_range_set) {
     if (p->kv_begin < 0 || p->kv_end < p->kv_begin || p->kv_end > p->L) return BDLM_ERR_INVALID_ARG;
@@ -44,6 +45,7 @@ void fill(KArgs& a, const bdlm_params* p) {
     a.dout[s] = nullptr; a.dsum[s] = nullptr; a.dq[s] = a.dk[s] = a.dv[s] = nullptr;
   }
   a.trace = g_trace;
+  a.single_pass = 0; a.dq32[0] = a.dq32[1] = nullptr;
 }
 
 bool is_sm100() {
@@ -153,6 +155,7 @@ int bdlm_attn_bwd(const bdlm_params* p,
 
   const bool tc_ok = tc_bwd_supported(a);
   if (p->impl == 2 && !tc_ok) return BDLM_ERR_UNSUPPORTED;
+  a.single_pass = (p->bwd_single_pass && tc_ok && p->impl != 1) ? 1 : 0;
   const int passes = p->bwd_passes ? p->bwd_passes : 7;
   cudaError_t e = cudaSuccess;
   if (passes & BDLM_BWD_PASS_DSUM) e = launch_dsum(a, ds_c, ds_n, st);

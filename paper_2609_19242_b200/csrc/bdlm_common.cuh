@@ -33,6 +33,8 @@ struct KArgs {
   __nv_bfloat16* dk[2];
   __nv_bfloat16* dv[2];
   unsigned long long* trace;   // optional cycle counters (bdlm_set_trace_buffer), else nullptr
+  int single_pass;             // backward: dQ accumulated in the dK/dV kernel through fp32 atomics
+  float* dq32[2];              // fp32 dQ accumulators [batch, L, H, d] (single-pass backward), else nullptr
 };
 
 // Visible key interval [lo, hi) of query row i (stream qs) inside key stream ks

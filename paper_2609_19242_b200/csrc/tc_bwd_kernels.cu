@@ -117,7 +117,7 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
     if (base & 1023u) *abort_flag = 1; else *abort_flag = 0;   // swizzled tiles need a 1024-byte aligned base
     mbar_init(bar_kv, 1);
     for (int i = 0; i < 3; ++i) { mbar_init(bar_q_full + 8 * i, 1); mbar_init(bar_q_empty + 8 * i, 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(bar_do_full + 8 * i, 2); mbar_init(bar_do_empty + 8 * i, 1); }   // dO full: TMA bytes + LSE/D rows
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_do_full + 8 * i, 2); mbar_init(bar_do_empty + 8 * i, 9); }   // full: TMA bytes + LSE/D rows; empty: dV done + 8 warps done with the D rows
     mbar_init(bar_st, 1); mbar_init(bar_dpt, 1);
     mbar_init(bar_pt, 256); mbar_init(bar_dst, 256);
     mbar_init(bar_done, 1);
@@ -317,6 +317,8 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       }
       tc_fence_before();
       mbar_arrive(bar_dst);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_do_empty + 8 * sd);   // this warp is done with the stage's D rows
     }
     if (warp == 0 && lane == 0) {
       trace_add(a.trace, 16 + 0, nsteps); trace_add(a.trace, 16 + 1, w_st); trace_add(a.trace, 16 + 2, w_dpt);
@@ -614,14 +616,361 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
   if (warp == 8) tmem_dealloc(tmem, 512);
 }
 
+
+// =============================================================================================
+// single-pass backward: the dK/dV kernel also produces dQ
+// =============================================================================================
+// Same CTA unit and S^T / P^T / dV pipeline as tc_dkdv_kernel, but dS^T goes to a shared-memory tile
+// instead of tensor memory.  There it is the K-major A operand of dK += dS^T Q and the MN-major B
+// operand of dQ^T = K^T dS^T (K, resident, is the MN-major A operand), whose 128x128 fp32 result
+// lands in the tensor-memory columns dP^T has just vacated.  The compute warps add that tile to an
+// fp32 dQ buffer with red.global.add (a warp's 32 lanes are 32 consecutive head-dim elements of one
+// query row: one 128-byte atomic per instruction).  5 GEMMs and one exp phase per tile pair instead of
+// the 7 + 2 of the two-pass backward; dQ depends on the order the key tiles' atomics arrive in.
+// Shared memory: K, V, Q ring x2, dO ring x2 (+ LSE, D rows), dS^T.
+constexpr int P1_Q0 = 2 * TILE_BYTES;
+constexpr int P1_DO0 = 4 * TILE_BYTES;
+constexpr int P1_DS = 6 * TILE_BYTES;
+constexpr int P1_ARR = 7 * TILE_BYTES;            // lse_s[2][128], d_s[2][128]
+constexpr int P1_BARS = P1_ARR + 2048;
+constexpr int P1_SMEM = P1_BARS + 160;
+constexpr uint32_t IDESC_MM = make_idesc(128, 128, true, true);   // A and B both MN-major
+
+__global__ void __launch_bounds__(BWD_THREADS, 1)
+tc_bwd1p_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restrict__ status) {
+  extern __shared__ __align__(1024) uint8_t sm[];
+  const uint32_t base = smem_u32(sm);
+  const uint32_t sK = base, sV = base + TILE_BYTES, sQ0 = base + P1_Q0, sdO0 = base + P1_DO0, sDS = base + P1_DS;
+  float* lse_s = reinterpret_cast<float*>(sm + P1_ARR);            // [2][128], log2 units
+  float* d_s = lse_s + 256;                                        // [2][128]
+  const uint32_t bars = base + P1_BARS;
+  const uint32_t bar_kv = bars, bar_q_full = bars + 8 /*[2]*/, bar_q_empty = bars + 24 /*[2]*/,
+                 bar_do_full = bars + 40 /*[2]*/, bar_do_empty = bars + 56 /*[2]*/,
+                 bar_st = bars + 72, bar_dpt = bars + 80, bar_pt = bars + 88, bar_dst = bars + 96,
+                 bar_dqf = bars + 104, bar_dqr = bars + 112, bar_done = bars + 120;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + P1_BARS + 128);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + P1_BARS + 136);
+
+  const int ks = blockIdx.z & 1, b = blockIdx.z >> 1, hk = blockIdx.y;
+  const int k0 = blockIdx.x * TILE;   // key tile 0 has the most query tiles: scheduled first
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int L = a.L, M = a.M, NT = L / TILE;
+
+  int tA0, nA, tB0 = 0, nB = 0;
+  if (ks == CLEAN) {
+    const int qa_lo = (a.mode == 0) ? k0 : (k0 / M) * M;
+    tA0 = qa_lo / TILE; nA = NT - tA0;
+    const int qb_lo = (k0 / M + 1) * M;
+    if (qb_lo < L) { tB0 = qb_lo / TILE; nB = NT - tB0; }
+  } else {
+    const int lo = (k0 / M) * M, hi = min(L, ((k0 + TILE - 1) / M + 1) * M);
+    tA0 = lo / TILE; nA = (hi + TILE - 1) / TILE - tA0;
+  }
+  const int per_head = nA + nB;
+  const int nsteps = per_head * a.G;
+  auto step_of = [&](int i) {
+    QStep s;
+    const int hh = i / per_head, r = i - hh * per_head;
+    s.h = hk * a.G + hh;
+    if (r < nA) { s.qs = (ks == NOISY) ? NOISY : CLEAN; s.q0 = (tA0 + r) * TILE; }
+    else { s.qs = NOISY; s.q0 = (tB0 + r - nA) * TILE; }
+    return s;
+  };
+
+  if (threadIdx.x == 0) {
+    if (base & 1023u) *abort_flag = 1; else *abort_flag = 0;
+    mbar_init(bar_kv, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar_q_full + 8 * i, 1); mbar_init(bar_q_empty + 8 * i, 1);
+      mbar_init(bar_do_full + 8 * i, 2); mbar_init(bar_do_empty + 8 * i, 9);   // empty: dV done + 8 warps done with the D rows
+    }
+    mbar_init(bar_st, 1); mbar_init(bar_dpt, 1); mbar_init(bar_pt, 256); mbar_init(bar_dst, 256);
+    mbar_init(bar_dqf, 1); mbar_init(bar_dqr, 256); mbar_init(bar_done, 1);
+    fence_mbar_init();
+  }
+  if (warp == 8) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const bool bad_base = (*abort_flag != 0);
+  // TMEM columns: [0,128) S^T / P^T   [128,256) dP^T, then dQ^T   [256,384) dV   [384,512) dK
+
+  if (bad_base) {
+    // fall through to the common exit
+  } else if (warp == 8) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0) {
+      mbar_expect_tx(bar_kv, 2 * TILE_BYTES);
+      tma_tile(sK, &maps.k[ks], bar_kv, hk * 128, k0, b);
+      tma_tile(sV, &maps.v[ks], bar_kv, hk * 128, k0, b);
+    }
+    bool ok = true;
+    long long w_empty = 0;
+    const long long t_begin = clock64();
+    for (int i = 0; i < nsteps && ok; ++i) {
+      const int sd = i & 1;
+      const QStep st = step_of(i);
+      if (i >= 2) ok = mbar_wait_timed(bar_q_empty + 8 * sd, ((i >> 1) - 1) & 1, abort_flag, w_empty);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      if (lane == 0) {
+        mbar_expect_tx(bar_q_full + 8 * sd, TILE_BYTES);
+        tma_tile(sQ0 + sd * TILE_BYTES, &maps.q[st.qs], bar_q_full + 8 * sd, st.h * 128, st.q0, b);
+      }
+      if (i >= 2) ok = mbar_wait_timed(bar_do_empty + 8 * sd, ((i >> 1) - 1) & 1, abort_flag, w_empty);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      if (lane == 0) {
+        mbar_expect_tx(bar_do_full + 8 * sd, TILE_BYTES);   // one arrival of two; the LSE/D rows follow
+        tma_tile(sdO0 + sd * TILE_BYTES, &maps.dout[st.qs], bar_do_full + 8 * sd, st.h * 128, st.q0, b);
+      }
+      const float* lsep = a.lse[st.qs] + ((int64_t)b * a.H + st.h) * L + st.q0;
+      const float* dsp = a.dsum[st.qs] + ((int64_t)b * a.H + st.h) * L + st.q0;
+      {
+        const float4 z = reinterpret_cast<const float4*>(lsep)[lane];
+        const float4 dd = reinterpret_cast<const float4*>(dsp)[lane];
+        float4 z2;
+        z2.x = isfinite(z.x) ? z.x * LOG2E : INFINITY; z2.y = isfinite(z.y) ? z.y * LOG2E : INFINITY;
+        z2.z = isfinite(z.z) ? z.z * LOG2E : INFINITY; z2.w = isfinite(z.w) ? z.w * LOG2E : INFINITY;
+        reinterpret_cast<float4*>(lse_s + sd * 128)[lane] = z2;
+        reinterpret_cast<float4*>(d_s + sd * 128)[lane] = dd;
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_do_full + 8 * sd);
+    }
+    if (lane == 0) { trace_add(a.trace, 16 + 12, clock64() - t_begin); trace_add(a.trace, 16 + 13, w_empty); }
+  } else if (warp == 9) {
+    // ------------------------------------------------------------------ MMA issuer (one thread)
+    if (lane == 0 && nsteps > 0) {
+      const long long t_begin = clock64();
+      const uint32_t k_lo = desc_lo_k(sK), v_lo = desc_lo_k(sV), kt_lo = desc_lo_mn(sK);
+      const uint32_t qk_lo0 = desc_lo_k(sQ0), qm_lo0 = desc_lo_mn(sQ0);
+      const uint32_t dok_lo0 = desc_lo_k(sdO0), dom_lo0 = desc_lo_mn(sdO0);
+      const uint32_t dsk_lo = desc_lo_k(sDS), dsm_lo = desc_lo_mn(sDS);
+      bool ok = mbar_wait_abortable(bar_kv, 0, abort_flag);
+      ok = ok && mbar_wait_abortable(bar_q_full, 0, abort_flag);
+      if (ok) {
+        tc_fence_after();
+        gemm_ss(tmem, k_lo, qk_lo0, IDESC_KK, 0u);
+        mma_commit(bar_st);
+      }
+      ok = ok && mbar_wait_abortable(bar_do_full, 0, abort_flag);
+      if (ok) {
+        tc_fence_after();
+        gemm_ss(tmem + 128, v_lo, dok_lo0, IDESC_KK, 0u);
+        mma_commit(bar_dpt);
+      }
+      for (int i = 0; i < nsteps && ok; ++i) {
+        const int sd = i & 1;
+        const uint32_t acc = i > 0 ? 1u : 0u;
+        // dV += P^T dO_i
+        ok = mbar_wait_lean(bar_pt, i & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        gemm_ts_mn<true>(tmem + 256, tmem, dom_lo0 + sd * TILE_LO, IDESC_KM, acc);
+        mma_commit(bar_do_empty + 8 * sd);
+        if (i + 1 < nsteps) {   // S^T of the next step
+          ok = mbar_wait_lean(bar_q_full + 8 * (sd ^ 1), ((i + 1) >> 1) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          gemm_ss(tmem, k_lo, qk_lo0 + (sd ^ 1) * TILE_LO, IDESC_KK, 0u);
+          mma_commit(bar_st);
+        }
+        // dS^T(i) is in shared memory: dQ^T = K^T dS^T into the columns dP^T(i) occupied, then dK += dS^T Q_i
+        ok = mbar_wait_lean(bar_dst, i & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        gemm_ss_mm(tmem + 128, kt_lo, dsm_lo, IDESC_MM, 0u);
+        mma_commit(bar_dqf);
+        gemm_ss_km(tmem + 384, dsk_lo, qm_lo0 + sd * TILE_LO, IDESC_KM, acc);
+        mma_commit(bar_q_empty + 8 * sd);
+        if (i + 1 < nsteps) {   // dP^T of the next step, once dQ^T(i) has been read out of those columns
+          ok = mbar_wait_lean(bar_dqr, i & 1, abort_flag);
+          ok = ok && mbar_wait_lean(bar_do_full + 8 * (sd ^ 1), ((i + 1) >> 1) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          gemm_ss(tmem + 128, v_lo, dok_lo0 + (sd ^ 1) * TILE_LO, IDESC_KK, 0u);
+          mma_commit(bar_dpt);
+        }
+      }
+      mma_commit(bar_done);
+      trace_add(a.trace, 16 + 8, clock64() - t_begin);
+    }
+  } else {
+    // ------------------------------------------------------------------ compute warpgroups
+    const int w = warp >> 2;                                   // column half: query columns [64w, 64w+64)
+    const int r = (warp & 3) * 32 + lane;                      // TMEM lane: key row of S^T/dP^T, head-dim index of dQ^T
+    const int j = k0 + r;
+    const uint32_t tl = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+    const int c0 = w * 64;
+    int vqc_lo, vqc_hi, vqn_lo, vqn_hi;   // query rows that see key j, per query stream
+    if (ks == CLEAN) {
+      vqc_lo = (a.mode == 0) ? j : (j / M) * M; vqc_hi = L;
+      vqn_lo = (j / M + 1) * M; vqn_hi = L;
+    } else {
+      vqc_lo = 0; vqc_hi = 0;
+      vqn_lo = (j / M) * M; vqn_hi = vqn_lo + M;
+    }
+    bool ok = true;
+    long long w_st = 0, w_dpt = 0, w_dqf = 0;
+    const long long t_begin = clock64();
+    uint32_t x[64];   // P^T of the step in flight (fp32), kept from phase 1 to phase 2
+
+    // phase 1 of step i: P^T = exp2(S^T * scale - LSE) on visible pairs, bf16 pairs back into the S^T columns
+    auto phase1 = [&](int i) {
+      const int sd = i & 1;
+      const QStep st = step_of(i);
+      int lo_a, hi_a, lo_b, hi_b;
+      visible_interval(st.qs, ks, st.q0, M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_a, hi_a);
+      visible_interval(st.qs, ks, st.q0 + TILE - 1, M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_b, hi_b);
+      const bool need_mask = (lo_b > k0) || (hi_a < k0 + TILE);
+      ok = mbar_wait_timed(bar_do_full + 8 * sd, (i >> 1) & 1, abort_flag, w_st);
+      ok = ok && mbar_wait_timed(bar_st, i & 1, abort_flag, w_st);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) return;
+      tc_fence_after();
+      {
+        uint32_t (*c)[32] = reinterpret_cast<uint32_t (*)[32]>(x);
+        tmem_ld32(tl + c0, c[0]); tmem_ld32(tl + c0 + 32, c[1]);
+        tmem_wait_ld();
+      }
+      const float* lz = lse_s + sd * 128 + c0;
+      if (!need_mask) {
+#pragma unroll
+        for (int c = 0; c < 64; ++c) x[c] = __float_as_uint(exp2f(fmaf(__uint_as_float(x[c]), a.scale_log2, -lz[c])));
+      } else {
+        const int vlo = (st.qs == CLEAN ? vqc_lo : vqn_lo) - st.q0 - c0, vhi = (st.qs == CLEAN ? vqc_hi : vqn_hi) - st.q0 - c0;
+#pragma unroll
+        for (int c = 0; c < 64; ++c) {
+          const float p = exp2f(fmaf(__uint_as_float(x[c]), a.scale_log2, -lz[c]));
+          x[c] = __float_as_uint((c >= vlo && c < vhi) ? p : 0.f);
+        }
+      }
+      uint32_t pk[32];
+#pragma unroll
+      for (int e = 0; e < 32; ++e) pk[e] = pack_bf16(__uint_as_float(x[2 * e]), __uint_as_float(x[2 * e + 1]));
+      tmem_st32(tl + c0, pk);
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar_pt);
+    };
+
+    if (nsteps > 0) phase1(0);
+    for (int i = 0; i < nsteps && ok; ++i) {
+      const int sd = i & 1;
+      // phase 2: dS^T = P^T * (dP^T - D), bf16, into the shared-memory tile (row = key, this half's 64 query columns)
+      ok = mbar_wait_timed(bar_dpt, i & 1, abort_flag, w_dpt);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      {
+        uint32_t y[64];
+        uint32_t (*c)[32] = reinterpret_cast<uint32_t (*)[32]>(y);
+        tmem_ld32(tl + 128 + c0, c[0]); tmem_ld32(tl + 128 + c0 + 32, c[1]);
+        tmem_wait_ld();
+        const float* dz = d_s + sd * 128 + c0;
+        uint8_t* rowp = sm + P1_DS + w * PANEL_BYTES + r * 128;
+#pragma unroll
+        for (int c8 = 0; c8 < 8; ++c8) {
+          uint4 v;
+          uint32_t* pv = reinterpret_cast<uint32_t*>(&v);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int c = c8 * 8 + 2 * e;
+            const float d0 = __uint_as_float(x[c]) * (__uint_as_float(y[c]) - dz[c]);
+            const float d1 = __uint_as_float(x[c + 1]) * (__uint_as_float(y[c + 1]) - dz[c + 1]);
+            pv[e] = pack_bf16(d0, d1);
+          }
+          *reinterpret_cast<uint4*>(rowp + ((c8 ^ (r & 7)) << 4)) = v;
+        }
+      }
+      tc_fence_before();
+      fence_async_smem();
+      mbar_arrive(bar_dst);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_do_empty + 8 * sd);   // this warp is done with the stage's D rows
+
+      // phase 1 of the next step runs before this step's dQ^T read-out: dQ^T(i) is still being computed
+      if (i + 1 < nsteps) { phase1(i + 1); if (!ok) break; }
+
+      // read-out: dQ[q, h, d] += scale * dQ^T[d, q]; this thread is head-dim element d = r of the step's query rows
+      ok = mbar_wait_timed(bar_dqf, i & 1, abort_flag, w_dqf);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      {
+        const QStep st = step_of(i);
+        float* dst = a.dq32[st.qs] + (((int64_t)b * L + st.q0 + c0) * a.H + st.h) * 128 + r;
+        const int64_t qstride = (int64_t)a.H * 128;
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t v[32];
+          tmem_ld32(tl + 128 + c0 + c * 32, v);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) atomicAdd(dst + (c * 32 + e) * qstride, __uint_as_float(v[e]) * a.scale);
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(bar_dqr);
+    }
+    if (warp == 0 && lane == 0) {
+      trace_add(a.trace, 16 + 0, nsteps); trace_add(a.trace, 16 + 1, w_st); trace_add(a.trace, 16 + 2, w_dpt);
+      trace_add(a.trace, 16 + 3, w_dqf); trace_add(a.trace, 16 + 6, clock64() - t_begin);
+    }
+    // epilogue: warpgroup 0 writes dV, warpgroup 1 writes dK (scaled)
+    if (ok && nsteps > 0) {
+      ok = mbar_wait_abortable(bar_done, 0, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+    }
+    if (ok) {
+      tc_fence_after();
+      bf16* dst = (w == 0 ? a.dv[ks] : a.dk[ks]) + (((int64_t)b * L + j) * a.Hkv + hk) * 128;
+      const float sc = (w == 0) ? 1.f : a.scale;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t v[32];
+        tmem_ld32(tl + 256 + w * 128 + c * 32, v);
+        tmem_wait_ld();
+        store_row_chunk(dst + c * 32, v, sc);
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) atomicExch(status, (int)BDLM_ERR_DEVICE_TIMEOUT);
+  if (warp == 8) tmem_dealloc(tmem, 512);
+}
+
+// fp32 dQ accumulator -> bf16 dQ
+__global__ void __launch_bounds__(256) dq_convert_kernel(const float* __restrict__ src, bf16* __restrict__ dst, int64_t n8) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += (int64_t)gridDim.x * blockDim.x) {
+    const float4 u = reinterpret_cast<const float4*>(src)[2 * i], v = reinterpret_cast<const float4*>(src)[2 * i + 1];
+    uint4 o;
+    o.x = pack_bf16(u.x, u.y); o.y = pack_bf16(u.z, u.w); o.z = pack_bf16(v.x, v.y); o.w = pack_bf16(v.z, v.w);
+    reinterpret_cast<uint4*>(dst)[i] = o;
+  }
+}
+
 }  // namespace
 
 bool tc_bwd_supported(const KArgs& a) {
   return a.d == 128 && a.L % TILE == 0 && tc_encoder_available();
 }
-size_t tc_bwd_extra_workspace(const bdlm_params*) { return 0; }
+// fp32 dQ accumulators of the single-pass backward: one [batch, L, H, 128] tensor per stream
+size_t tc_bwd_extra_workspace(const bdlm_params* p) {
+  if (!p->bwd_single_pass || p->d != 128 || p->L % TILE != 0 || p->impl == 1) return 0;
+  return 2 * (size_t)p->batch * p->L * p->H * 128 * sizeof(float);
+}
 
-cudaError_t launch_tc_bwd(const KArgs& a, void*, int passes, cudaStream_t st) {
+cudaError_t launch_tc_bwd(const KArgs& a_in, void* extra_ws, int passes, cudaStream_t st) {
+  KArgs a = a_in;
+  const size_t dq32_elems = (size_t)a.batch * a.L * a.H * 128;
+  if (a.single_pass) {
+    a.dq32[0] = static_cast<float*>(extra_ws);
+    a.dq32[1] = a.dq32[0] + dq32_elems;
+  }
   BwdMaps maps;
   for (int s = 0; s < 2; ++s) {
     if (!tc_make_map(&maps.q[s], a.q[s], a.H, a.L, a.batch, TILE)) return cudaErrorInvalidValue;
@@ -632,6 +981,21 @@ cudaError_t launch_tc_bwd(const KArgs& a, void*, int passes, cudaStream_t st) {
   int* status = device_status_ptr();
   if (status == nullptr) return cudaErrorUnknown;
   cudaError_t e;
+  if (a.single_pass) {
+    // one kernel produces dK, dV and (through fp32 atomics) dQ; it runs for the DKDV pass bit, the DQ bit is a no-op
+    if (passes & BDLM_BWD_PASS_DKDV) {
+      if ((e = cudaMemsetAsync(a.dq32[0], 0, 2 * dq32_elems * sizeof(float), st)) != cudaSuccess) return e;
+      if ((e = cudaFuncSetAttribute(tc_bwd1p_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P1_SMEM)) != cudaSuccess) return e;
+      dim3 grid(a.L / TILE, a.Hkv, a.batch * 2);
+      tc_bwd1p_kernel<<<grid, BWD_THREADS, P1_SMEM, st>>>(maps, a, status);
+      if ((e = cudaGetLastError()) != cudaSuccess) return e;
+      for (int s2 = 0; s2 < 2; ++s2) {
+        dq_convert_kernel<<<148 * 8, 256, 0, st>>>(a.dq32[s2], a.dq[s2], (int64_t)(dq32_elems / 8));
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+      }
+    }
+    return cudaSuccess;
+  }
   if (passes & BDLM_BWD_PASS_DKDV) {
     if ((e = cudaFuncSetAttribute(tc_dkdv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DKDV_SMEM)) != cudaSuccess) return e;
     dim3 grid(a.L / TILE, a.Hkv, a.batch * 2);

@@ -217,6 +217,17 @@ __device__ __forceinline__ void gemm_ts_mn(uint32_t d, uint32_t a_tmem, uint32_t
     mma_ts(d, a_tmem + (SPLIT ? (kk < 4 ? kk * 8 : 64 + (kk - 4) * 8) : kk * 8), desc64(b_lo + moff(kk)), idesc, kk == 0 ? acc_first : 1u);
 }
 
+// A K-major tile and B MN-major tile, both in shared memory.
+__device__ __forceinline__ void gemm_ss_km(uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t acc_first) {
+#pragma unroll
+  for (int kk = 0; kk < 8; ++kk) mma_ss(d, desc64(a_lo + koff(kk)), desc64(b_lo + moff(kk)), idesc, kk == 0 ? acc_first : 1u);
+}
+// A and B both MN-major tiles ([contraction row][128 columns]) in shared memory: D = A^T-tile x B-tile.
+__device__ __forceinline__ void gemm_ss_mm(uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t acc_first) {
+#pragma unroll
+  for (int kk = 0; kk < 8; ++kk) mma_ss(d, desc64(a_lo + moff(kk)), desc64(b_lo + moff(kk)), idesc, kk == 0 ? acc_first : 1u);
+}
+
 // Byte offset of element (row, col) inside a [128 x 128] bf16 tile stored as two swizzled panels
 // (panel = 64 columns): the layout TMA writes with SWIZZLE_128B and the MMA reads.
 __device__ __forceinline__ uint32_t sw128_offset(int row, int col) {

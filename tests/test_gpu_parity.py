@@ -114,3 +114,26 @@ def test_skipping_a_stream():
     only_c = binding.bdlm_attn_fwd(g["q_clean"], g["k_clean"], g["v_clean"], None, None, None, w.block_size)
     assert only_n[0] is None and torch.equal(only_n[2], full[2]) and torch.equal(only_n[3], full[3])
     assert only_c[2] is None and torch.equal(only_c[0], full[0]) and torch.equal(only_c[1], full[1])
+
+
+@pytest.mark.parametrize("w", [Workload("sp_3tiles", 2, 4, 2, 128, 384, 32), Workload("sp_m256", 1, 4, 1, 128, 512, 256),
+                               Workload("sp_m16", 1, 2, 2, 128, 512, 16)], ids=lambda w: w.name)
+def test_single_pass_backward_matches_oracle_and_two_pass(w):
+    """The opt-in one-kernel backward (dQ through fp32 atomics): same tolerances against the oracle; dK and
+    dV come from the same fixed-order accumulation as the two-pass kernels, so they are bitwise equal."""
+    inp = synth.make_inputs(w, "cpu")
+    g = pu.to_cuda(inp)
+    x = pu.f64(inp)
+    M = w.block_size
+    out = pu.gpu_fwd(g, M)
+    two = [t.clone() for t in pu.gpu_bwd(g, out, M)]
+    one = pu.gpu_bwd(g, out, M, single_pass=True)
+    torch.cuda.synchronize()
+    assert binding.bdlm_get_device_status() == 0
+    gref = orc.attn_backward(*[x[n] for n in pu.NAMES6], x["do_clean"], x["do_noisy"], M)
+    for got, want in zip(one, gref):
+        assert pu.rel_l2(synth.to_f64(got), want) <= pu.TOL_GRAD
+    for i in (1, 2, 4, 5):
+        assert torch.equal(one[i], two[i])
+    p = binding.make_params(w.batch, w.L, M, w.H, w.H_kv, w.d, bwd_single_pass=True)
+    assert binding.bdlm_workspace_bytes(p, binding.BDLM_WS_BWD) >= 2 * w.batch * w.L * w.H * w.d * 4
