@@ -44,20 +44,25 @@ NOISY = 1
 # visibility (the mask, written out)
 # --------------------------------------------------------------------------------------
 def visible_rows(stream, rows, L, M, clean_mask_mode=0, kv_begin=0, kv_end=None,
-                 include_noisy_diag=True):
+                 include_noisy_diag=True, window=0):
     """Boolean visibility [len(rows), 2L] of the concatenated key axis (clean keys 0..L-1
     then noisy keys L..2L-1) for the given query rows of one stream.
 
     Section 3.2 / Eqs. correctness-clean-attention, correctness-corrupted-attention.
     `kv_begin:kv_end` restricts the clean keys to one context shard (set C_r of Eq.
     correctness-clean-partition); `include_noisy_diag=False` drops the noisy keys, which
-    leaves the clean-shard partial of a noisy query.
+    leaves the clean-shard partial of a noisy query.  `window` = W > 0 is the sliding-window
+    variant of a layer (appendix K mentions 1,024-token windows; the paper does not spell the
+    mask out, so this is a reading): a clean key j is visible to a query at position i of either
+    stream only if additionally i - j < W; the noisy keys of the own block are unaffected.
     """
     if kv_end is None:
         kv_end = L
     i = np.asarray(rows, dtype=np.int64)[:, None]
     j = np.arange(L, dtype=np.int64)[None, :]
     in_shard = (j >= kv_begin) & (j < kv_end)
+    if window and window > 0:
+        in_shard = in_shard & (i - j < window)
     if stream == CLEAN:
         if clean_mask_mode == 0:
             to_clean = j <= i
@@ -72,11 +77,11 @@ def visible_rows(stream, rows, L, M, clean_mask_mode=0, kv_begin=0, kv_end=None,
     return np.concatenate([to_clean & in_shard, to_noisy], axis=1)
 
 
-def visibility_2L(L, M, clean_mask_mode=0, kv_begin=0, kv_end=None, include_noisy_diag=True):
+def visibility_2L(L, M, clean_mask_mode=0, kv_begin=0, kv_end=None, include_noisy_diag=True, window=0):
     """The explicit 2L x 2L mask: rows 0..L-1 clean queries, rows L..2L-1 noisy queries."""
     allrows = np.arange(L)
-    top = visible_rows(CLEAN, allrows, L, M, clean_mask_mode, kv_begin, kv_end, include_noisy_diag)
-    bot = visible_rows(NOISY, allrows, L, M, clean_mask_mode, kv_begin, kv_end, include_noisy_diag)
+    top = visible_rows(CLEAN, allrows, L, M, clean_mask_mode, kv_begin, kv_end, include_noisy_diag, window)
+    bot = visible_rows(NOISY, allrows, L, M, clean_mask_mode, kv_begin, kv_end, include_noisy_diag, window)
     return np.concatenate([top, bot], axis=0)
 
 
@@ -124,7 +129,7 @@ def _check_shapes(q_clean, k_clean, q_noisy, k_noisy, M):
 # --------------------------------------------------------------------------------------
 def attn_forward(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, block_size,
                  scale=None, clean_mask_mode=0, kv_begin=0, kv_end=None,
-                 include_noisy_diag=True, row_chunk=2048):
+                 include_noisy_diag=True, row_chunk=2048, window=0):
     """Forward of the BDLM attention layer (Eqs. correctness-clean-attention,
     correctness-corrupted-attention; scale 1/sqrt(d_h) per Eq. context-parallel-attention).
     Returns (o_clean, lse_clean, o_noisy, lse_noisy)."""
@@ -145,7 +150,7 @@ def attn_forward(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, block_siz
                 for r0 in range(0, L, row_chunk):
                     rows = np.arange(r0, min(L, r0 + row_chunk))
                     vis = visible_rows(stream, rows, L, M, clean_mask_mode, kv_begin, kv_end,
-                                       include_noisy_diag)
+                                       include_noisy_diag, window)
                     oo, ll, _ = _masked_attention(qs[stream][b, rows, h], k2, v2, vis, scale)
                     o[stream][b, rows, h] = oo
                     lse[stream][b, h, rows] = ll
@@ -153,7 +158,7 @@ def attn_forward(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, block_siz
 
 
 def attn_backward(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, do_clean, do_noisy,
-                  block_size, scale=None, clean_mask_mode=0, row_chunk=2048):
+                  block_size, scale=None, clean_mask_mode=0, row_chunk=2048, window=0):
     """Backward of the layer for the scalar sum(O*dO) (Algorithm 2; Eqs.
     correctness-corrupted-gradient, correctness-clean-gradient, correctness-query-gradient).
     Returns (dq_clean, dk_clean, dv_clean, dq_noisy, dk_noisy, dv_noisy)."""
@@ -175,7 +180,7 @@ def attn_backward(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, do_clean
             for stream in (CLEAN, NOISY):
                 for r0 in range(0, L, row_chunk):
                     rows = np.arange(r0, min(L, r0 + row_chunk))
-                    vis = visible_rows(stream, rows, L, M, clean_mask_mode)
+                    vis = visible_rows(stream, rows, L, M, clean_mask_mode, window=window)
                     qq = qs[stream][b, rows, h]
                     _, _, p = _masked_attention(qq, k2, v2, vis, scale)
                     gq, gk, gv = _masked_attention_grad(qq, k2, v2, p, dos[stream][b, rows, h], scale)
@@ -222,7 +227,7 @@ def lse_merge(o_partials, lse_partials):
 # --------------------------------------------------------------------------------------
 def attn_rows(stream, rows, q_rows, k_clean, v_clean, k_noisy, v_noisy, block_size,
               do_rows=None, scale=None, clean_mask_mode=0, kv_begin=0, kv_end=None,
-              include_noisy_diag=True, row_chunk=128):
+              include_noisy_diag=True, row_chunk=128, window=0):
     """The same definition evaluated for selected query rows of one (batch, head).
 
     q_rows/do_rows [n, d] belong to `rows` of `stream`; k_*/v_* are that head's KV head,
@@ -246,7 +251,7 @@ def attn_rows(stream, rows, q_rows, k_clean, v_clean, k_noisy, v_noisy, block_si
     for c0 in range(0, n, row_chunk):
         sel = order[c0:c0 + row_chunk]
         vis = visible_rows(stream, rows[sel], L, M, clean_mask_mode, kv_begin, kv_end,
-                           include_noisy_diag)
+                           include_noisy_diag, window)
         cols = np.nonzero(vis.any(axis=0))[0]
         kc = np.concatenate([k_clean[cols[cols < L]], k_noisy[cols[cols >= L] - L]], axis=0)
         vc = np.concatenate([v_clean[cols[cols < L]], v_noisy[cols[cols >= L] - L]], axis=0)
@@ -268,7 +273,7 @@ def attn_rows(stream, rows, q_rows, k_clean, v_clean, k_noisy, v_noisy, block_si
 # --------------------------------------------------------------------------------------
 # counting (used for FLOP accounting and the appendix-B pins)
 # --------------------------------------------------------------------------------------
-def visible_pair_counts(L, M, clean_mask_mode=0):
+def visible_pair_counts(L, M, clean_mask_mode=0, window=0):
     """(clean pairs, noisy pairs) counted from the explicit mask, per (batch, head)."""
-    vis = visibility_2L(L, M, clean_mask_mode)
+    vis = visibility_2L(L, M, clean_mask_mode, window=window)
     return int(vis[:L].sum()), int(vis[L:].sum())

@@ -413,3 +413,90 @@ def test_sampled_rows_equal_full_oracle(mode):
         assert np.allclose(rn["dk_noisy"], g[4][0, :, 0], atol=1e-13)
         assert np.allclose(rn["dv_noisy"], g[5][0, :, 0], atol=1e-13)
         assert np.abs(rc["dk_noisy"]).max() == 0
+
+
+# ------------------------------------------------------------------ sliding-window variant
+@pytest.mark.parametrize("L,M,W", [(32, 4, 8), (48, 8, 5), (24, 6, 6), (32, 8, 100), (40, 1, 7)])
+def test_window_mask_counts_and_shape(L, M, W):
+    """Reading of the sliding-window layers (appendix K): clean key j visible to position i only if i - j < W.
+    Clean row i then sees min(i+1, W) keys; noisy row i of block b sees its M noisy keys plus the clean keys
+    of (i-W, bM); with W >= L the mask is the unwindowed one."""
+    vis = orc.visibility_2L(L, M, window=W)
+    for i in range(L):
+        b = i // M
+        assert vis[i, :L].sum() == min(i + 1, W)
+        lo = max(0, i - W + 1)
+        assert vis[L + i, :L].sum() == max(0, b * M - lo)
+        if b * M > lo:
+            assert vis[L + i, lo:b * M].all()
+        assert vis[L + i, L:].sum() == M
+        assert not vis[i, L:].any()
+    if W >= L:
+        assert (vis == orc.visibility_2L(L, M)).all()
+    c, n = orc.visible_pair_counts(L, M, window=W)
+    assert c == sum(min(i + 1, W) for i in range(L))
+
+
+def test_window_clean_stream_is_library_sliding_window_attention():
+    """M = 1: the clean stream under a window is ordinary causal sliding-window attention; compared with
+    torch SDPA given a band mask built here by loops, values and autograd gradients."""
+    B, L, H, d, M, W = 1, 40, 2, 8, 1, 6
+    t = _inputs(B, L, H, H, d, seed=41)
+    band = torch.zeros(L, L, dtype=torch.bool)
+    for i in range(L):
+        for j in range(L):
+            band[i, j] = (j <= i) and (i - j < W)
+    tq, tk, tv = (torch.tensor(np.moveaxis(x[0], 1, 0)[None], dtype=torch.float64, requires_grad=True)
+                  for x in (t["qc"], t["kc"], t["vc"]))
+    o_ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, attn_mask=band)
+    names = ["qc", "kc", "vc", "qn", "kn", "vn"]
+    oc, lc, on, ln = orc.attn_forward(*[t[n] for n in names], M, window=W)
+    assert np.allclose(oc[0], np.moveaxis(o_ref[0].detach().numpy(), 0, 1), atol=1e-12)
+    g = orc.attn_backward(*[t[n] for n in names], t["doc"], np.zeros_like(t["don"]), M, window=W)
+    (o_ref * torch.tensor(np.moveaxis(t["doc"][0], 1, 0)[None])).sum().backward()
+    for got, ref in zip(g[:3], (tq, tk, tv)):
+        assert np.allclose(got[0], np.moveaxis(ref.grad[0].numpy(), 0, 1), atol=1e-11)
+
+
+def test_window_against_brute_force_and_rows():
+    """General windowed case against per-row loops over the visible set, and the sampled-row path."""
+    B, L, H, Hkv, d, M, W = 1, 24, 2, 1, 4, 6, 9
+    t = _inputs(B, L, H, Hkv, d, seed=43)
+    names = ["qc", "kc", "vc", "qn", "kn", "vn"]
+    oc, lc, on, ln = orc.attn_forward(*[t[n] for n in names], M, window=W)
+    sc = 1 / math.sqrt(d)
+    for h in range(H):
+        for i in range(L):
+            blk = i // M
+            for stream, q, o_got, l_got in (("c", t["qc"], oc, lc), ("n", t["qn"], on, ln)):
+                if stream == "c":
+                    keys = [("c", j) for j in range(max(0, i - W + 1), i + 1)]
+                else:
+                    keys = [("c", j) for j in range(max(0, i - W + 1), blk * M)] + [("n", j) for j in range(blk * M, (blk + 1) * M)]
+                a = np.array([sc * np.dot(q[0, i, h], t["k" + s][0, j, 0]) for s, j in keys])
+                w_ = np.exp(a - a.max())
+                o = sum(wj * t["v" + s][0, j, 0] for wj, (s, j) in zip(w_ / w_.sum(), keys))
+                assert np.allclose(o_got[0, i, h], o, atol=1e-12)
+                assert abs(l_got[0, h, i] - (a.max() + math.log(w_.sum()))) < 1e-12
+    rows = np.array([0, 5, 6, 13, 23])
+    full_g = None
+    for h in range(H):
+        r = orc.attn_rows(orc.NOISY, rows, t["qn"][0, rows, h], t["kc"][0, :, 0], t["vc"][0, :, 0],
+                          t["kn"][0, :, 0], t["vn"][0, :, 0], M, window=W)
+        assert np.allclose(r["o"], on[0, rows, h], atol=1e-13) and np.allclose(r["lse"], ln[0, h, rows], atol=1e-13)
+    # gradients by central differences under the window
+    g = orc.attn_backward(*[t[n] for n in names], t["doc"], t["don"], M, window=W)
+
+    def loss(tt):
+        a_, _, b_, _ = orc.attn_forward(*[tt[n] for n in names], M, window=W)
+        return (a_ * t["doc"]).sum() + (b_ * t["don"]).sum()
+    rng = np.random.default_rng(1)
+    for name, grad in zip(names, g):
+        for _ in range(6):
+            idx = tuple(int(rng.integers(0, s_)) for s_ in t[name].shape)
+            tp = {k: v.copy() for k, v in t.items()}
+            tm = {k: v.copy() for k, v in t.items()}
+            tp[name][idx] += 1e-5
+            tm[name][idx] -= 1e-5
+            fd = (loss(tp) - loss(tm)) / 2e-5
+            assert abs(fd - grad[idx]) <= 1e-6 * max(1.0, abs(fd))
