@@ -7,6 +7,8 @@
  *   - clean query i      sees clean keys 0..i                     (clean_mask_mode 0)
  *   - noisy query i      sees noisy keys of its own block (bidirectional) and the clean
  *                        keys of all earlier blocks: j < floor(i/block_size)*block_size
+ *   - sliding-window layers (appendix K of the paper mentions 1,024-token windows) restrict the clean keys
+ *     further to i - j < window (`window` parameter; the paper does not spell this mask out)
  * Scores are q.k * scale (scale = 1/sqrt(d), Eq. context-parallel-attention), softmax is
  * taken over the visible keys, LSE is the natural-log row log-sum-exp of the scaled scores.
  * Partials over disjoint key sets are combined exactly by Eq. csbp-lse-merge.
@@ -63,7 +65,9 @@ typedef struct {
                                   tile pair instead of 7; dQ is then reproducible only up to fp32 summation order).
                                   Needs the larger workspace bdlm_workspace_bytes reports for this setting; falls back to
                                   the two-pass path when the tensor-core kernels do not take the shape. */
-  int32_t reserved[3];
+  int32_t window;              /* sliding-window layers: > 0 = a clean key j is visible to the query at position i (of either
+                                  stream) only if additionally i - j < window; the noisy own block is unaffected.  0 = none. */
+  int32_t reserved[2];
 } bdlm_params;
 
 enum { BDLM_BWD_PASS_DSUM = 1, BDLM_BWD_PASS_DKDV = 2, BDLM_BWD_PASS_DQ = 4 };

@@ -38,7 +38,7 @@ class BdlmParams(ctypes.Structure):
                 ("kv_begin", ctypes.c_int32), ("kv_end", ctypes.c_int32),
                 ("kv_range_set", ctypes.c_int32), ("include_noisy_diag", ctypes.c_int32),
                 ("impl", ctypes.c_int32), ("bwd_passes", ctypes.c_int32), ("bwd_single_pass", ctypes.c_int32),
-                ("reserved", ctypes.c_int32 * 3)]
+                ("window", ctypes.c_int32), ("reserved", ctypes.c_int32 * 2)]
 
 
 _lib = None
@@ -82,7 +82,7 @@ bdlm_status_string = status_string
 
 
 def make_params(batch, L, block_size, H, H_kv, d, scale=0.0, clean_mask_mode=0, kv_range=None,
-                include_noisy_diag=True, impl=IMPL_AUTO, bwd_passes=0, bwd_single_pass=False) -> BdlmParams:
+                include_noisy_diag=True, impl=IMPL_AUTO, bwd_passes=0, bwd_single_pass=False, window=0) -> BdlmParams:
     p = BdlmParams()
     p.batch, p.L, p.block_size, p.H, p.H_kv, p.d = batch, L, block_size, H, H_kv, d
     p.scale = float(scale)
@@ -95,6 +95,7 @@ def make_params(batch, L, block_size, H, H_kv, d, scale=0.0, clean_mask_mode=0, 
     p.impl = impl
     p.bwd_passes = bwd_passes
     p.bwd_single_pass = 1 if bwd_single_pass else 0
+    p.window = int(window)
     return p
 
 
@@ -120,13 +121,13 @@ def bdlm_workspace_bytes(params: BdlmParams, which: int) -> int:
 
 def bdlm_attn_fwd(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, block_size, *,
                   out=None, scale=0.0, clean_mask_mode=0, kv_range=None, include_noisy_diag=True,
-                  impl=IMPL_AUTO):
+                  impl=IMPL_AUTO, window=0):
     """Forward of the layer.  Tensors: q [batch,L,H,d], k/v [batch,L,H_kv,d], bf16, on one CUDA
     device.  Either q may be None (that stream is skipped).  Returns
     (o_clean, lse_clean, o_noisy, lse_noisy); `out` may supply those four tensors."""
     qref = q_clean if q_clean is not None else q_noisy
     p = _shape_params(qref, k_clean, block_size, scale=scale, clean_mask_mode=clean_mask_mode,
-                      kv_range=kv_range, include_noisy_diag=include_noisy_diag, impl=impl)
+                      kv_range=kv_range, include_noisy_diag=include_noisy_diag, impl=impl, window=window)
     dev = qref.device
     if out is None:
         mk_o = lambda q: None if q is None else torch.empty_like(q)
@@ -143,12 +144,12 @@ def bdlm_attn_fwd(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, block_si
 
 def bdlm_attn_bwd(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, o_clean, lse_clean,
                   o_noisy, lse_noisy, do_clean, do_noisy, block_size, *, out=None, workspace=None,
-                  scale=0.0, clean_mask_mode=0, impl=IMPL_AUTO, passes=0, single_pass=False):
+                  scale=0.0, clean_mask_mode=0, impl=IMPL_AUTO, passes=0, single_pass=False, window=0):
     """Backward of the layer.  Returns (dq_clean, dk_clean, dv_clean, dq_noisy, dk_noisy, dv_noisy).
     `single_pass=True` selects the one-kernel backward (dQ by fp32 atomics: faster, dQ not bitwise
     reproducible)."""
     p = _shape_params(q_clean, k_clean, block_size, scale=scale, clean_mask_mode=clean_mask_mode, impl=impl,
-                      bwd_passes=passes, bwd_single_pass=single_pass)
+                      bwd_passes=passes, bwd_single_pass=single_pass, window=window)
     if out is None:
         out = tuple(torch.empty_like(t) for t in (q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy))
     need = bdlm_workspace_bytes(p, BDLM_WS_BWD)

@@ -22,6 +22,7 @@ int check_params(const bdlm_params* p) {
   if (p->impl < 0 || p->impl > 2) return BDLM_ERR_INVALID_ARG;
   if (p->bwd_passes < 0 || p->bwd_passes > 7) return BDLM_ERR_INVALID_ARG;
   if (p->bwd_single_pass != 0 && p->bwd_single_pass != 1) return BDLM_ERR_INVALID_ARG;
+  if (p->window < 0) return BDLM_ERR_INVALID_ARG;
   if (!(p->scale >= 0.f) || isinf(p->scale)) return BDLM_ERR_INVALID_ARG;
   if (p->kv_range_set) {
     if (p->kv_begin < 0 || p->kv_end < p->kv_begin || p->kv_end > p->L) return BDLM_ERR_INVALID_ARG;
@@ -40,6 +41,7 @@ void fill(KArgs& a, const bdlm_params* p) {
   a.kv_begin = p->kv_range_set ? p->kv_begin : 0;
   a.kv_end = p->kv_range_set ? p->kv_end : p->L;
   a.diag = p->include_noisy_diag ? 1 : 0;
+  a.window = p->window;
   for (int s = 0; s < 2; ++s) {
     a.q[s] = a.k[s] = a.v[s] = nullptr; a.o[s] = nullptr; a.lse[s] = nullptr;
     a.dout[s] = nullptr; a.dsum[s] = nullptr; a.dq[s] = a.dk[s] = a.dv[s] = nullptr;

@@ -21,6 +21,7 @@ struct KArgs {
   int mode;           // clean_mask_mode
   int kv_begin, kv_end;
   int diag;           // include_noisy_diag
+  int window;         // sliding window over clean keys (0 = none)
   const __nv_bfloat16* q[2];
   const __nv_bfloat16* k[2];
   const __nv_bfloat16* v[2];
@@ -42,7 +43,9 @@ struct KArgs {
 // the noisy keys of its own block).  Every row's visible set per key stream is one interval.
 __device__ __forceinline__ void visible_interval(int qs, int ks, int i, int M, int mode,
                                                  int kv_begin, int kv_end, int diag,
-                                                 int& lo, int& hi) {
+                                                 int& lo, int& hi, int window) {
+  // sliding-window layers: a clean key j is visible to position i only if i - j < window (0 = no window)
+  if (ks == CLEAN && window > 0) kv_begin = max(kv_begin, i - window + 1);
   if (qs == CLEAN) {
     if (ks == CLEAN) {
       lo = kv_begin;

@@ -93,12 +93,12 @@ __global__ void __launch_bounds__(NTHREADS) portable_fwd_kernel(const KArgs a) {
 
   for (int ks = 0; ks < 2; ++ks) {
     int seg_lo, seg_hi, tmp;
-    visible_interval(qs, ks, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, seg_lo, tmp);
-    visible_interval(qs, ks, last_row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, tmp, seg_hi);
+    visible_interval(qs, ks, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, seg_lo, tmp, a.window);
+    visible_interval(qs, ks, last_row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, tmp, seg_hi, a.window);
     if (seg_hi <= seg_lo) continue;
     int rlo0 = 0, rhi0 = 0, rlo1 = 0, rhi1 = 0;
-    if (r0 < L) visible_interval(qs, ks, r0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo0, rhi0);
-    if (r1 < L) visible_interval(qs, ks, r1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo1, rhi1);
+    if (r0 < L) visible_interval(qs, ks, r0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo0, rhi0, a.window);
+    if (r1 < L) visible_interval(qs, ks, r1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo1, rhi1, a.window);
     const bf16* kbase = a.k[ks] + ((int64_t)b * L * a.Hkv + hk) * D;
     const bf16* vbase = a.v[ks] + ((int64_t)b * L * a.Hkv + hk) * D;
 
@@ -229,12 +229,12 @@ __global__ void __launch_bounds__(NTHREADS) portable_dq_kernel(const KArgs a) {
 
   for (int ks = 0; ks < 2; ++ks) {
     int seg_lo, seg_hi, tmp;
-    visible_interval(qs, ks, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, seg_lo, tmp);
-    visible_interval(qs, ks, last_row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, tmp, seg_hi);
+    visible_interval(qs, ks, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, seg_lo, tmp, a.window);
+    visible_interval(qs, ks, last_row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, tmp, seg_hi, a.window);
     if (seg_hi <= seg_lo) continue;
     int rlo0 = 0, rhi0 = 0, rlo1 = 0, rhi1 = 0;
-    if (r0 < L) visible_interval(qs, ks, r0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo0, rhi0);
-    if (r1 < L) visible_interval(qs, ks, r1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo1, rhi1);
+    if (r0 < L) visible_interval(qs, ks, r0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo0, rhi0, a.window);
+    if (r1 < L) visible_interval(qs, ks, r1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo1, rhi1, a.window);
     const bf16* kbase = a.k[ks] + ((int64_t)b * L * a.Hkv + hk) * D;
     const bf16* vbase = a.v[ks] + ((int64_t)b * L * a.Hkv + hk) * D;
 
@@ -343,10 +343,10 @@ __global__ void __launch_bounds__(NTHREADS) portable_dkdv_kernel(const KArgs a) 
     if (qs == CLEAN) {
       if (ks == NOISY) continue;
       q_lo = (a.mode == 0) ? k0 : (k0 / M) * M;
-      q_hi = L;
+      q_hi = (a.window > 0) ? min(L, k_last + a.window) : L;
     } else if (ks == CLEAN) {
       q_lo = (k0 / M + 1) * M;
-      q_hi = L;
+      q_hi = (a.window > 0) ? min(L, k_last + a.window) : L;
     } else {
       q_lo = (k0 / M) * M;
       q_hi = min(L, (k_last / M + 1) * M);
@@ -368,7 +368,7 @@ __global__ void __launch_bounds__(NTHREADS) portable_dkdv_kernel(const KArgs a) 
             float zz = lsep[i];
             z = isfinite(zz) ? zz * LOG2E : INFINITY;
             dd = dsp[i];
-            visible_interval(qs, ks, i, M, a.mode, a.kv_begin, a.kv_end, a.diag, lo, hi);
+            visible_interval(qs, ks, i, M, a.mode, a.kv_begin, a.kv_end, a.diag, lo, hi, a.window);
           }
           lse_s[threadIdx.x] = z; d_s[threadIdx.x] = dd;
           vlo_s[threadIdx.x] = lo; vhi_s[threadIdx.x] = hi;

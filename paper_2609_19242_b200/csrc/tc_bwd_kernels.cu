@@ -95,9 +95,11 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
   int tA0, nA, tB0 = 0, nB = 0;
   if (ks == CLEAN) {
     const int qa_lo = (a.mode == 0) ? k0 : (k0 / M) * M;
-    tA0 = qa_lo / TILE; nA = NT - tA0;
+    // with a sliding window the last query row that sees a key of this tile is k0 + TILE - 1 + window - 1
+    const int t_end = (a.window > 0) ? min(NT, (min(L, k0 + TILE - 1 + a.window) + TILE - 1) / TILE) : NT;
+    tA0 = qa_lo / TILE; nA = t_end - tA0;
     const int qb_lo = (k0 / M + 1) * M;
-    if (qb_lo < L) { tB0 = qb_lo / TILE; nB = NT - tB0; }
+    if (qb_lo < L) { tB0 = qb_lo / TILE; nB = max(0, t_end - tB0); }
   } else {
     const int lo = (k0 / M) * M, hi = min(L, ((k0 + TILE - 1) / M + 1) * M);
     tA0 = lo / TILE; nA = (hi + TILE - 1) / TILE - tA0;
@@ -243,8 +245,9 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
     // query rows that see key j, per query stream (section 3.2 read from the key's side)
     int vq_lo[2], vq_hi[2];
     if (ks == CLEAN) {
-      vq_lo[CLEAN] = (a.mode == 0) ? j : (j / M) * M; vq_hi[CLEAN] = L;
-      vq_lo[NOISY] = (j / M + 1) * M; vq_hi[NOISY] = L;
+      const int q_end = (a.window > 0) ? min(L, j + a.window) : L;
+      vq_lo[CLEAN] = (a.mode == 0) ? j : (j / M) * M; vq_hi[CLEAN] = q_end;
+      vq_lo[NOISY] = (j / M + 1) * M; vq_hi[NOISY] = q_end;
     } else {
       vq_lo[CLEAN] = 0; vq_hi[CLEAN] = 0;
       vq_lo[NOISY] = (j / M) * M; vq_hi[NOISY] = vq_lo[NOISY] + M;
@@ -258,8 +261,8 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       const QStep st = step_of(i);
       // the tile needs masking unless every query row of it sees every key of this key tile
       int lo_a, hi_a, lo_b, hi_b;
-      visible_interval(st.qs, ks, st.q0, M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_a, hi_a);
-      visible_interval(st.qs, ks, st.q0 + TILE - 1, M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_b, hi_b);
+      visible_interval(st.qs, ks, st.q0, M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_a, hi_a, a.window);
+      visible_interval(st.qs, ks, st.q0 + TILE - 1, M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_b, hi_b, a.window);
       const bool need_mask = (lo_b > k0) || (hi_a < k0 + TILE);
       ok = mbar_wait_timed(bar_do_full + 8 * sd, (i >> 1) & 1, abort_flag, w_st);
       ok = ok && mbar_wait_timed(bar_st, i & 1, abort_flag, w_st);
@@ -399,11 +402,11 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
   int lo0, lo1, nt0, nt1, lo_last0, lo_last1, hi_first0, hi_first1;
   {
     int lo_f, hi_f, lo_l, hi_l;
-    visible_interval(qs, 0, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_f, hi_f);
-    visible_interval(qs, 0, q0 + TILE - 1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_l, hi_l);
+    visible_interval(qs, 0, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_f, hi_f, a.window);
+    visible_interval(qs, 0, q0 + TILE - 1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_l, hi_l, a.window);
     lo0 = lo_f; lo_last0 = lo_l; hi_first0 = hi_f; nt0 = hi_l > lo_f ? (hi_l - lo_f + TILE - 1) / TILE : 0;
-    visible_interval(qs, 1, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_f, hi_f);
-    visible_interval(qs, 1, q0 + TILE - 1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_l, hi_l);
+    visible_interval(qs, 1, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_f, hi_f, a.window);
+    visible_interval(qs, 1, q0 + TILE - 1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_l, hi_l, a.window);
     lo1 = lo_f; lo_last1 = lo_l; hi_first1 = hi_f; nt1 = hi_l > lo_f ? (hi_l - lo_f + TILE - 1) / TILE : 0;
   }
   const int nsteps = nt0 + nt1;
@@ -517,8 +520,8 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
       dsum = a.dsum[qs][((int64_t)b * a.H + h) * L + row];
     }
     int rlo0, rhi0, rlo1, rhi1;
-    visible_interval(qs, 0, row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo0, rhi0);
-    visible_interval(qs, 1, row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo1, rhi1);
+    visible_interval(qs, 0, row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo0, rhi0, a.window);
+    visible_interval(qs, 1, row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo1, rhi1, a.window);
     bool ok = true;
     long long w_s = 0, w_dp = 0, c_ld = 0, c_exp = 0, c_ds = 0;
     Stopwatch sw;
@@ -659,9 +662,11 @@ tc_bwd1p_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __rest
   int tA0, nA, tB0 = 0, nB = 0;
   if (ks == CLEAN) {
     const int qa_lo = (a.mode == 0) ? k0 : (k0 / M) * M;
-    tA0 = qa_lo / TILE; nA = NT - tA0;
+    // with a sliding window the last query row that sees a key of this tile is k0 + TILE - 1 + window - 1
+    const int t_end = (a.window > 0) ? min(NT, (min(L, k0 + TILE - 1 + a.window) + TILE - 1) / TILE) : NT;
+    tA0 = qa_lo / TILE; nA = t_end - tA0;
     const int qb_lo = (k0 / M + 1) * M;
-    if (qb_lo < L) { tB0 = qb_lo / TILE; nB = NT - tB0; }
+    if (qb_lo < L) { tB0 = qb_lo / TILE; nB = max(0, t_end - tB0); }
   } else {
     const int lo = (k0 / M) * M, hi = min(L, ((k0 + TILE - 1) / M + 1) * M);
     tA0 = lo / TILE; nA = (hi + TILE - 1) / TILE - tA0;
@@ -806,8 +811,9 @@ tc_bwd1p_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __rest
     const int c0 = w * 64;
     int vqc_lo, vqc_hi, vqn_lo, vqn_hi;   // query rows that see key j, per query stream
     if (ks == CLEAN) {
-      vqc_lo = (a.mode == 0) ? j : (j / M) * M; vqc_hi = L;
-      vqn_lo = (j / M + 1) * M; vqn_hi = L;
+      const int q_end = (a.window > 0) ? min(L, j + a.window) : L;
+      vqc_lo = (a.mode == 0) ? j : (j / M) * M; vqc_hi = q_end;
+      vqn_lo = (j / M + 1) * M; vqn_hi = q_end;
     } else {
       vqc_lo = 0; vqc_hi = 0;
       vqn_lo = (j / M) * M; vqn_hi = vqn_lo + M;
@@ -822,8 +828,8 @@ tc_bwd1p_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __rest
       const int sd = i & 1;
       const QStep st = step_of(i);
       int lo_a, hi_a, lo_b, hi_b;
-      visible_interval(st.qs, ks, st.q0, M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_a, hi_a);
-      visible_interval(st.qs, ks, st.q0 + TILE - 1, M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_b, hi_b);
+      visible_interval(st.qs, ks, st.q0, M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_a, hi_a, a.window);
+      visible_interval(st.qs, ks, st.q0 + TILE - 1, M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_b, hi_b, a.window);
       const bool need_mask = (lo_b > k0) || (hi_a < k0 + TILE);
       ok = mbar_wait_timed(bar_do_full + 8 * sd, (i >> 1) & 1, abort_flag, w_st);
       ok = ok && mbar_wait_timed(bar_st, i & 1, abort_flag, w_st);

@@ -99,11 +99,11 @@ tc_fwd_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restri
 #pragma unroll
   for (int ks = 0; ks < 2; ++ks) {
     int lo_f, hi_f, lo_l, hi_l;
-    visible_interval(qs, ks, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_f, hi_f);
-    visible_interval(qs, ks, q0 + TILE - 1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_l, hi_l);
+    visible_interval(qs, ks, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_f, hi_f, a.window);
+    visible_interval(qs, ks, q0 + TILE - 1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_l, hi_l, a.window);
     seg_lo[ks] = lo_f; seg_hi[ks] = hi_l; lo_last[ks] = lo_l; hi_first[ks] = hi_f;
     ntile[ks] = seg_hi[ks] > seg_lo[ks] ? (seg_hi[ks] - seg_lo[ks] + TILE - 1) / TILE : 0;
-    visible_interval(qs, ks, row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo[ks], rhi[ks]);
+    visible_interval(qs, ks, row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo[ks], rhi[ks], a.window);
   }
   const int nt = ntile[0] + ntile[1];
 
@@ -269,11 +269,11 @@ struct TileSched {
   int lo0, lo1, nt0, nt1, lo_last0, lo_last1, hi_first0, hi_first1;
   __device__ __forceinline__ void init(int qs, int q0, const KArgs& a) {
     int lo_f, hi_f, lo_l, hi_l;
-    visible_interval(qs, 0, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_f, hi_f);
-    visible_interval(qs, 0, q0 + TILE - 1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_l, hi_l);
+    visible_interval(qs, 0, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_f, hi_f, a.window);
+    visible_interval(qs, 0, q0 + TILE - 1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_l, hi_l, a.window);
     lo0 = lo_f; lo_last0 = lo_l; hi_first0 = hi_f; nt0 = hi_l > lo_f ? (hi_l - lo_f + TILE - 1) / TILE : 0;
-    visible_interval(qs, 1, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_f, hi_f);
-    visible_interval(qs, 1, q0 + TILE - 1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_l, hi_l);
+    visible_interval(qs, 1, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_f, hi_f, a.window);
+    visible_interval(qs, 1, q0 + TILE - 1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_l, hi_l, a.window);
     lo1 = lo_f; lo_last1 = lo_l; hi_first1 = hi_f; nt1 = hi_l > lo_f ? (hi_l - lo_f + TILE - 1) / TILE : 0;
   }
   // a tile needs per-element masking unless every row of the query tile sees all of its 128 keys
@@ -415,8 +415,8 @@ tc_fwd2h_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __rest
     const uint32_t tS = tmem + lane_base + w * 128 + hc * 64;          // this thread's 64 score columns
     const uint32_t tO = tmem + lane_base + 256 + w * 128 + hc * 64;    // and its 64 output columns
     int rlo0, rhi0, rlo1, rhi1;
-    visible_interval(qs, 0, row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo0, rhi0);
-    visible_interval(qs, 1, row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo1, rhi1);
+    visible_interval(qs, 0, row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo0, rhi0, a.window);
+    visible_interval(qs, 1, row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo1, rhi1, a.window);
     float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
     long long w_s = 0;

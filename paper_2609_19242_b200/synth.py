@@ -29,12 +29,19 @@ class Workload:
     rope_theta: float = 0.0   # > 0: rotate q and k before rounding to bf16
     kv_shards: int = 1        # > 1: forward is also run as that many clean-K/V shard partials
     seed: int = 0
+    window: int = 0           # > 0: sliding-window layer, clean key j visible only if i - j < window
 
     def pairs_per_head(self):
         """Unmasked (query, key) pairs per (batch, query head): clean L(L+1)/2 and noisy
-        L(L+M)/2 (appendix B, Eq. aligned-rank-work with P = 1)."""
-        L, M = self.L, self.block_size
-        return L * (L + 1) // 2, L * (L + M) // 2
+        L(L+M)/2 (appendix B, Eq. aligned-rank-work with P = 1); with a sliding window the
+        clean keys of row i are cut to the last `window` positions up to i."""
+        L, M, W = self.L, self.block_size, self.window
+        if W <= 0:
+            return L * (L + 1) // 2, L * (L + M) // 2
+        i = np.arange(L, dtype=np.int64)
+        clean = np.minimum(i + 1, W).sum()
+        noisy = (M + np.maximum(0, (i // M) * M - np.maximum(0, i - W + 1))).sum()
+        return int(clean), int(noisy)
 
     def flops(self):
         """(forward, backward) FLOPs over unmasked pairs only: 4d and 10d per pair."""
@@ -51,6 +58,8 @@ WORKLOADS = {
     "256k": Workload("256k", 1, 32, 8, 128, 262144, 16),
     # paper-shaped block size (appendix J uses 128..1024, default 256); not a BASELINE config
     "32k_m256": Workload("32k_m256", 1, 32, 8, 128, 32768, 256, rope_theta=5e5),
+    # sliding-window layer of a hybrid model (appendix K: 1,024-token windows); not a BASELINE config
+    "32k_w1024": Workload("32k_w1024", 1, 32, 8, 128, 32768, 64, rope_theta=5e5, window=1024),
 }
 
 
@@ -115,6 +124,8 @@ def sample_rows(w: Workload, n: int, seed: int, extra=()):
         step = L // w.kv_shards
         for s in range(1, w.kv_shards):
             fixed += [s * step - 1, s * step, s * step + M]
+    if w.window > 0:
+        fixed += [w.window - 2, w.window - 1, w.window, w.window + M]
     fixed += list(extra)
     rows = sorted({r for r in fixed if 0 <= r < L})
     rows = rows[:n]

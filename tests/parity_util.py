@@ -48,9 +48,9 @@ def check_full(w, impl, mode=0, check_bwd=True, inp=None):
     g = to_cuda(inp)
     x = f64(inp)
     M = w.block_size
-    out = gpu_fwd(g, M, clean_mask_mode=mode, impl=impl)
+    out = gpu_fwd(g, M, clean_mask_mode=mode, impl=impl, window=w.window)
     torch.cuda.synchronize()
-    ref = orc.attn_forward(*[x[n] for n in NAMES6], M, clean_mask_mode=mode)
+    ref = orc.attn_forward(*[x[n] for n in NAMES6], M, clean_mask_mode=mode, window=w.window)
     for got, want, name in zip(out, ref, ["o_clean", "lse_clean", "o_noisy", "lse_noisy"]):
         gotn = synth.to_f64(got)
         assert np.isfinite(gotn).all(), name
@@ -58,9 +58,10 @@ def check_full(w, impl, mode=0, check_bwd=True, inp=None):
         assert err <= (TOL_LSE if "lse" in name else TOL_O), (name, err)
     if not check_bwd:
         return
-    grads = gpu_bwd(g, out, M, clean_mask_mode=mode, impl=impl)
+    grads = gpu_bwd(g, out, M, clean_mask_mode=mode, impl=impl, window=w.window)
     torch.cuda.synchronize()
-    gref = orc.attn_backward(*[x[n] for n in NAMES6], x["do_clean"], x["do_noisy"], M, clean_mask_mode=mode)
+    gref = orc.attn_backward(*[x[n] for n in NAMES6], x["do_clean"], x["do_noisy"], M, clean_mask_mode=mode,
+                             window=w.window)
     for got, want, name in zip(grads, gref, ["dq_clean", "dk_clean", "dv_clean", "dq_noisy", "dk_noisy", "dv_noisy"]):
         gotn = synth.to_f64(got)
         assert np.isfinite(gotn).all(), name
@@ -79,7 +80,7 @@ def check_sampled(w, impl, n_rows=256, g=None, fwd_out=None, check_bwd=True, rep
     if g is None:
         g = synth.make_inputs(w, "cuda")
     if fwd_out is None:
-        fwd_out = gpu_fwd(g, M, impl=impl)
+        fwd_out = gpu_fwd(g, M, impl=impl, window=w.window)
     torch.cuda.synchronize()
     G = w.H // w.H_kv
     rows_of = {}
@@ -89,13 +90,13 @@ def check_sampled(w, impl, n_rows=256, g=None, fwd_out=None, check_bwd=True, rep
                 rows_of[(b, h, s)] = synth.sample_rows(w, n_rows, seed=1000 * b + 10 * h + s)
     grads = grads_sp = None
     if check_bwd:
-        grads = gpu_bwd(g, fwd_out, M, impl=impl)
+        grads = gpu_bwd(g, fwd_out, M, impl=impl, window=w.window)
         do_sp = [torch.zeros_like(g["do_clean"]), torch.zeros_like(g["do_noisy"])]
         for (b, h, s), rows in rows_of.items():
             r = torch.from_numpy(rows).cuda()
             src = g["do_clean"] if s == 0 else g["do_noisy"]
             do_sp[s][b, r, h] = src[b, r, h]
-        grads_sp = gpu_bwd(g, fwd_out, M, do_clean=do_sp[0], do_noisy=do_sp[1], impl=impl)
+        grads_sp = gpu_bwd(g, fwd_out, M, do_clean=do_sp[0], do_noisy=do_sp[1], impl=impl, window=w.window)
         torch.cuda.synchronize()
         assert binding.bdlm_get_device_status() == 0
     worst = {"o": 0.0, "lse": 0.0, "dq": 0.0, "dk": 0.0, "dv": 0.0}
@@ -114,7 +115,7 @@ def check_sampled(w, impl, n_rows=256, g=None, fwd_out=None, check_bwd=True, rep
                     q_rows = synth.to_f64(g[qn[s]][b, rt, h])
                     do_rows = synth.to_f64(g[don[s]][b, rt, h]) if check_bwd else None
                     ref = orc.attn_rows(s, rows, q_rows, kv["k_clean"], kv["v_clean"], kv["k_noisy"],
-                                        kv["v_noisy"], M, do_rows=do_rows)
+                                        kv["v_noisy"], M, do_rows=do_rows, window=w.window)
                     o_got = synth.to_f64(fwd_out[2 * s][b, rt, h])
                     l_got = synth.to_f64(fwd_out[2 * s + 1][b, h, rt])
                     worst["o"] = max(worst["o"], float(np.abs(o_got - ref["o"]).max()))

@@ -34,6 +34,45 @@ def test_forward_backward_match_oracle(w, impl):
     pu.check_full(w, impl)
 
 
+WINDOWED = [
+    Workload("w1", 1, 2, 1, 128, 256, 32, window=1),
+    Workload("w7_m1", 1, 2, 2, 64, 160, 1, window=7),
+    Workload("w_lt_block", 1, 2, 1, 128, 512, 64, window=40),
+    Workload("w100_ragged", 1, 4, 2, 128, 456, 8, window=100),
+    Workload("w128", 1, 2, 1, 128, 640, 32, window=128),
+    Workload("w129", 1, 2, 1, 128, 640, 32, window=129),
+    Workload("w300_m128", 2, 4, 2, 128, 768, 128, window=300),
+    Workload("w_ge_L", 1, 2, 1, 64, 384, 16, window=1000),
+]
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("w", WINDOWED, ids=lambda w: w.name)
+def test_sliding_window_matches_oracle(w, impl):
+    """Sliding-window layers: clean keys limited to i - j < window, forward and backward."""
+    pu.check_full(w, impl)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_sliding_window_mode_1_and_shards(impl):
+    """The window composes with the whole-own-block clean mask and with a clean-key shard range."""
+    pu.check_full(Workload("w_mode1", 1, 2, 1, 128, 384, 32, window=70), impl, mode=1)
+    w = Workload("w_shard", 1, 2, 1, 128, 512, 32, window=150)
+    inp = synth.make_inputs(w, "cpu", with_grad=False)
+    g = pu.to_cuda(inp)
+    x = pu.f64(inp)
+    for a, b in [(0, 200), (200, 512), (300, 301)]:
+        out = pu.gpu_fwd(g, w.block_size, kv_range=(a, b), include_noisy_diag=False, impl=impl, window=w.window)
+        ref = orc.attn_forward(*[x[n] for n in pu.NAMES6], w.block_size, kv_begin=a, kv_end=b,
+                               include_noisy_diag=False, window=w.window)
+        for got, want in zip(out, ref):
+            gotn = synth.to_f64(got)
+            assert not np.isnan(gotn).any()
+            assert (np.isneginf(gotn) == np.isneginf(want)).all()
+            fin = np.isfinite(want)
+            assert np.abs(gotn[fin] - want[fin]).max() <= pu.TOL_O
+
+
 @pytest.mark.parametrize("impl", IMPLS)
 def test_clean_mask_mode_1(impl):
     pu.check_full(Workload("mode1", 1, 2, 1, 128, 384, 32), impl, mode=1)
@@ -117,7 +156,8 @@ def test_skipping_a_stream():
 
 
 @pytest.mark.parametrize("w", [Workload("sp_3tiles", 2, 4, 2, 128, 384, 32), Workload("sp_m256", 1, 4, 1, 128, 512, 256),
-                               Workload("sp_m16", 1, 2, 2, 128, 512, 16)], ids=lambda w: w.name)
+                               Workload("sp_m16", 1, 2, 2, 128, 512, 16),
+                               Workload("sp_w200", 1, 2, 1, 128, 768, 32, window=200)], ids=lambda w: w.name)
 def test_single_pass_backward_matches_oracle_and_two_pass(w):
     """The opt-in one-kernel backward (dQ through fp32 atomics): same tolerances against the oracle; dK and
     dV come from the same fixed-order accumulation as the two-pass kernels, so they are bitwise equal."""
@@ -125,12 +165,12 @@ def test_single_pass_backward_matches_oracle_and_two_pass(w):
     g = pu.to_cuda(inp)
     x = pu.f64(inp)
     M = w.block_size
-    out = pu.gpu_fwd(g, M)
-    two = [t.clone() for t in pu.gpu_bwd(g, out, M)]
-    one = pu.gpu_bwd(g, out, M, single_pass=True)
+    out = pu.gpu_fwd(g, M, window=w.window)
+    two = [t.clone() for t in pu.gpu_bwd(g, out, M, window=w.window)]
+    one = pu.gpu_bwd(g, out, M, single_pass=True, window=w.window)
     torch.cuda.synchronize()
     assert binding.bdlm_get_device_status() == 0
-    gref = orc.attn_backward(*[x[n] for n in pu.NAMES6], x["do_clean"], x["do_noisy"], M)
+    gref = orc.attn_backward(*[x[n] for n in pu.NAMES6], x["do_clean"], x["do_noisy"], M, window=w.window)
     for got, want in zip(one, gref):
         assert pu.rel_l2(synth.to_f64(got), want) <= pu.TOL_GRAD
     for i in (1, 2, 4, 5):

@@ -12,7 +12,7 @@ import parity_util as pu
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("name", ["8k", "32k", "32k_m256"])
+@pytest.mark.parametrize("name", ["8k", "32k", "32k_m256", "32k_w1024"])
 def test_sampled_rows_full_size(name):
     w = WORKLOADS[name]
     worst = pu.check_sampled(w, binding.IMPL_AUTO)
