@@ -131,8 +131,13 @@ def oracle_sample(w, inp_cpu, rows_per_stream, seed):
         rows = np.sort(rng.choice(w.L, size=min(rows_per_stream, w.L), replace=False))
         q_rows = synth.to_f64(inp_cpu[qn][0, rows, 0])
         do_rows = synth.to_f64(inp_cpu[dn][0, rows, 0])
-        orc.attn_rows(s, rows, q_rows, kv["k_clean"], kv["v_clean"], kv["k_noisy"], kv["v_noisy"], M, do_rows=do_rows)
-        pairs = (rows + 1).sum() if s == 0 else ((rows // M + 1) * M).sum()
+        orc.attn_rows(s, rows, q_rows, kv["k_clean"], kv["v_clean"], kv["k_noisy"], kv["v_noisy"], M, do_rows=do_rows,
+                      window=w.window)
+        if w.window > 0:
+            lo = np.maximum(0, rows - w.window + 1)
+            pairs = (rows + 1 - lo).sum() if s == 0 else (M + np.maximum(0, (rows // M) * M - lo)).sum()
+        else:
+            pairs = (rows + 1).sum() if s == 0 else ((rows // M + 1) * M).sum()
         flops += 14 * w.d * int(pairs)
     return time.perf_counter() - t0, flops
 
@@ -185,7 +190,7 @@ def run_reference(args, w):
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_tot / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
             "data": "synthetic", "config": {"workload": w.name, "batch": w.batch, "H": w.H, "H_kv": w.H_kv,
-                                            "d": w.d, "L": w.L, "block_size": w.block_size},
+                                            "d": w.d, "L": w.L, "block_size": w.block_size, "window": w.window},
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -239,11 +244,12 @@ def run_ours(args, w):
     impl = args.kernel_impl
 
     def fwd():
-        binding.bdlm_attn_fwd(*[g[n] for n in NAMES6], M, out=fwd_out, impl=impl)
+        binding.bdlm_attn_fwd(*[g[n] for n in NAMES6], M, out=fwd_out, impl=impl, window=w.window)
 
     def bwd(passes=0):
         binding.bdlm_attn_bwd(*[g[n] for n in NAMES6], fwd_out[0], fwd_out[1], fwd_out[2], fwd_out[3],
-                              g["do_clean"], g["do_noisy"], M, out=grads, workspace=ws, impl=impl, passes=passes)
+                              g["do_clean"], g["do_noisy"], M, out=grads, workspace=ws, impl=impl, passes=passes,
+                              window=w.window)
 
     for _ in range(args.warmup):
         fwd()
@@ -353,7 +359,7 @@ def run_ours(args, w):
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": w.name, "batch": w.batch, "H": w.H, "H_kv": w.H_kv, "d": w.d, "L": w.L,
-                       "block_size": w.block_size, "rope_theta": w.rope_theta, "parallelism": "replicas only",
+                       "block_size": w.block_size, "window": w.window, "rope_theta": w.rope_theta, "parallelism": "replicas only",
                        "l2": "inputs larger than L2 (q/k/v/dO of one step exceed 126 MB)",
                        "kernel_impl": {0: "auto", 1: "portable", 2: "tcgen05"}[impl]},
             "pct_of_bf16_peak": {"measured_burst": 100 * value / world / peaks["bf16_tflops"],
