@@ -62,27 +62,33 @@ __device__ __forceinline__ void store_row_chunk(bf16* dst, const uint32_t (&v)[3
 // =============================================================================================
 // dK/dV pass
 // =============================================================================================
-// Shared memory: K, V (resident), a 3-stage Q ring (a Q tile is read first by S^T and last by
-// dK, so it lives longest), a 2-stage dO ring with the LSE and D rows of the same query tile.
+// Shared memory: K, V (resident), a 2-stage Q ring, a 2-stage dO ring with the LSE and D rows of
+// the same query tile, and one tile for P^T.  P^T goes to the tensor core through shared memory
+// rather than through the S^T columns of tensor memory: the S^T columns are then free as soon as
+// the compute warps hold S^T(i) in registers, so S^T(i+1) is computed while exp(i) runs, and the
+// compute warps never wait for the tensor core in steady state.
 constexpr int DKDV_Q0 = 2 * TILE_BYTES;
-constexpr int DKDV_DO0 = 5 * TILE_BYTES;
+constexpr int DKDV_DO0 = 4 * TILE_BYTES;
+constexpr int DKDV_P = 6 * TILE_BYTES;
 constexpr int DKDV_ARR = 7 * TILE_BYTES;            // lse_s[2][128], d_s[2][128]
 constexpr int DKDV_BARS = DKDV_ARR + 2048;
-constexpr int DKDV_SMEM = DKDV_BARS + 160;
+constexpr int DKDV_SMEM = DKDV_BARS + 176;
 
 struct QStep { int qs, h, q0; };
 
+template <bool TR>
 __global__ void __launch_bounds__(BWD_THREADS, 1)
 tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restrict__ status) {
   extern __shared__ __align__(1024) uint8_t sm[];
   const uint32_t base = smem_u32(sm);
-  const uint32_t sK = base, sV = base + TILE_BYTES, sQ0 = base + DKDV_Q0, sdO0 = base + DKDV_DO0;
+  const uint32_t sK = base, sV = base + TILE_BYTES, sQ0 = base + DKDV_Q0, sdO0 = base + DKDV_DO0, sP = base + DKDV_P;
   float* lse_s = reinterpret_cast<float*>(sm + DKDV_ARR);          // [2][128], log2 units
   float* d_s = lse_s + 256;                                        // [2][128]
   const uint32_t bars = base + DKDV_BARS;
-  const uint32_t bar_kv = bars, bar_q_full = bars + 8 /*[3]*/, bar_q_empty = bars + 32 /*[3]*/,
-                 bar_do_full = bars + 56 /*[2]*/, bar_do_empty = bars + 72 /*[2]*/,
-                 bar_st = bars + 88, bar_dpt = bars + 96, bar_pt = bars + 104, bar_dst = bars + 112, bar_done = bars + 120;
+  const uint32_t bar_kv = bars, bar_q_full = bars + 8 /*[2]*/, bar_q_empty = bars + 24 /*[2]*/,
+                 bar_do_full = bars + 40 /*[2]*/, bar_do_empty = bars + 56 /*[2]*/,
+                 bar_st = bars + 72, bar_sfree = bars + 80, bar_dpt = bars + 88, bar_pt = bars + 96,
+                 bar_pfree = bars + 104, bar_dst = bars + 112, bar_done = bars + 120;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + DKDV_BARS + 128);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + DKDV_BARS + 136);
 
@@ -106,22 +112,24 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
   }
   const int per_head = nA + nB;
   const int nsteps = per_head * a.G;
-  auto step_of = [&](int i) {
+  // steps are walked in order by every role: (head of the group, tile index inside the head) counters, no division
+  int it_r = 0, it_h = hk * a.G;
+  auto step_cur = [&]() {
     QStep s;
-    const int hh = i / per_head, r = i - hh * per_head;
-    s.h = hk * a.G + hh;
-    if (r < nA) { s.qs = (ks == NOISY) ? NOISY : CLEAN; s.q0 = (tA0 + r) * TILE; }
-    else { s.qs = NOISY; s.q0 = (tB0 + r - nA) * TILE; }
+    s.h = it_h;
+    if (it_r < nA) { s.qs = (ks == NOISY) ? NOISY : CLEAN; s.q0 = (tA0 + it_r) * TILE; }
+    else { s.qs = NOISY; s.q0 = (tB0 + it_r - nA) * TILE; }
     return s;
   };
+  auto step_next = [&]() { if (++it_r == per_head) { it_r = 0; ++it_h; } };
 
   if (threadIdx.x == 0) {
     if (base & 1023u) *abort_flag = 1; else *abort_flag = 0;   // swizzled tiles need a 1024-byte aligned base
     mbar_init(bar_kv, 1);
-    for (int i = 0; i < 3; ++i) { mbar_init(bar_q_full + 8 * i, 1); mbar_init(bar_q_empty + 8 * i, 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_q_full + 8 * i, 1); mbar_init(bar_q_empty + 8 * i, 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(bar_do_full + 8 * i, 2); mbar_init(bar_do_empty + 8 * i, 9); }   // full: TMA bytes + LSE/D rows; empty: dV done + 8 warps done with the D rows
-    mbar_init(bar_st, 1); mbar_init(bar_dpt, 1);
-    mbar_init(bar_pt, 256); mbar_init(bar_dst, 256);
+    mbar_init(bar_st, 1); mbar_init(bar_dpt, 1); mbar_init(bar_pfree, 1);
+    mbar_init(bar_sfree, 256); mbar_init(bar_pt, 256); mbar_init(bar_dst, 256);
     mbar_init(bar_done, 1);
     fence_mbar_init();
   }
@@ -131,7 +139,7 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   const bool bad_base = (*abort_flag != 0);
-  // TMEM columns: [0,128) S^T / P^T   [128,256) dP^T / dS^T   [256,384) dV   [384,512) dK
+  // TMEM columns: [0,128) S^T   [128,256) dP^T / dS^T   [256,384) dV   [384,512) dK
 
   if (bad_base) {
     // fall through to the common exit
@@ -144,18 +152,19 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
     }
     bool ok = true;
     long long w_empty = 0;
-    const long long t_begin = clock64();
+    const long long t_begin = tick<TR>();
     for (int i = 0; i < nsteps && ok; ++i) {
-      const int sq = i % 3, sd = i & 1;
-      const QStep st = step_of(i);
-      if (i >= 3) ok = mbar_wait_timed(bar_q_empty + 8 * sq, ((i / 3) - 1) & 1, abort_flag, w_empty);
+      const int sd = i & 1;
+      const QStep st = step_cur();
+      step_next();
+      if (i >= 2) ok = mbar_wait_timed<TR>(bar_q_empty + 8 * sd, ((i >> 1) - 1) & 1, abort_flag, w_empty);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       if (lane == 0) {
-        mbar_expect_tx(bar_q_full + 8 * sq, TILE_BYTES);
-        tma_tile(sQ0 + sq * TILE_BYTES, &maps.q[st.qs], bar_q_full + 8 * sq, st.h * 128, st.q0, b);
+        mbar_expect_tx(bar_q_full + 8 * sd, TILE_BYTES);
+        tma_tile(sQ0 + sd * TILE_BYTES, &maps.q[st.qs], bar_q_full + 8 * sd, st.h * 128, st.q0, b);
       }
-      if (i >= 2) ok = mbar_wait_timed(bar_do_empty + 8 * sd, ((i >> 1) - 1) & 1, abort_flag, w_empty);
+      if (i >= 2) ok = mbar_wait_timed<TR>(bar_do_empty + 8 * sd, ((i >> 1) - 1) & 1, abort_flag, w_empty);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       if (lane == 0) {
@@ -176,13 +185,13 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_do_full + 8 * sd);
     }
-    if (lane == 0) { trace_add(a.trace, 16 + 12, clock64() - t_begin); trace_add(a.trace, 16 + 13, w_empty); }
+    if (lane == 0) { trace_add(a.trace, 16 + 12, tick<TR>() - t_begin); trace_add(a.trace, 16 + 13, w_empty); }
   } else if (warp == 9) {
     // ------------------------------------------------------------------ MMA issuer (one thread)
     if (lane == 0 && nsteps > 0) {
-      long long w_pt = 0, w_q = 0, w_dst = 0;
-      const long long t_begin = clock64();
-      const uint32_t k_lo = desc_lo_k(sK), v_lo = desc_lo_k(sV);
+      long long w_pt = 0, w_sf = 0, w_dst = 0;
+      const long long t_begin = tick<TR>();
+      const uint32_t k_lo = desc_lo_k(sK), v_lo = desc_lo_k(sV), p_lo = desc_lo_k(sP);
       const uint32_t qk_lo0 = desc_lo_k(sQ0), qm_lo0 = desc_lo_mn(sQ0);       // Q ring, as K-major B (S^T) / MN-major B (dK)
       const uint32_t dok_lo0 = desc_lo_k(sdO0), dom_lo0 = desc_lo_mn(sdO0);   // dO ring, as K-major B (dP^T) / MN-major B (dV)
       bool ok = mbar_wait_abortable(bar_kv, 0, abort_flag);
@@ -198,42 +207,43 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
         gemm_ss(tmem + 128, v_lo, dok_lo0, IDESC_KK, 0u);
         mma_commit(bar_dpt);
       }
-      int sq = 0;   // i % 3
       for (int i = 0; i < nsteps && ok; ++i) {
-        const int sd = i & 1, nq = (sq == 2) ? 0 : sq + 1;
+        const int sd = i & 1, sn = sd ^ 1;
         const uint32_t acc = i > 0 ? 1u : 0u;
-        // dV += P^T dO_i   (P^T: this lane's 64+64 bf16 pairs at columns [0,32) and [64,96))
-        ok = mbar_wait_lean(bar_pt, i & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        gemm_ts_mn<true>(tmem + 256, tmem, dom_lo0 + sd * TILE_LO, IDESC_KM, acc);
-        mma_commit(bar_do_empty + 8 * sd);
-        // S^T of the next step may start as soon as its Q is in shared memory
+        // S^T of the next step: its columns are free once every compute thread holds S^T(i) in registers
         if (i + 1 < nsteps) {
-          ok = mbar_wait_lean(bar_q_full + 8 * nq, ((i + 1) / 3) & 1, abort_flag);
+          ok = mbar_wait_timed<TR>(bar_sfree, i & 1, abort_flag, w_sf);
+          ok = ok && mbar_wait_lean(bar_q_full + 8 * sn, ((i + 1) >> 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          gemm_ss(tmem, k_lo, qk_lo0 + nq * TILE_LO, IDESC_KK, 0u);
+          gemm_ss(tmem, k_lo, qk_lo0 + sn * TILE_LO, IDESC_KK, 0u);
           mma_commit(bar_st);
         }
-        // dK += dS^T Q_i
-        ok = mbar_wait_lean(bar_dst, i & 1, abort_flag);
+        // dV += P^T dO_i   (P^T from shared memory, K-major: row = key, contraction = query)
+        ok = mbar_wait_timed<TR>(bar_pt, i & 1, abort_flag, w_pt);
         if (!ok) break;
         tc_fence_after();
-        gemm_ts_mn<true>(tmem + 384, tmem + 128, qm_lo0 + sq * TILE_LO, IDESC_KM, acc);
-        mma_commit(bar_q_empty + 8 * sq);
+        gemm_ss_km(tmem + 256, p_lo, dom_lo0 + sd * TILE_LO, IDESC_KM, acc);
+        mma_commit(bar_do_empty + 8 * sd);
+        mma_commit(bar_pfree);
+        // dK += dS^T Q_i   (dS^T: this lane's 64+64 bf16 pairs at columns 128+[0,32) and 128+[64,96))
+        ok = mbar_wait_timed<TR>(bar_dst, i & 1, abort_flag, w_dst);
+        if (!ok) break;
+        tc_fence_after();
+        gemm_ts_mn<true>(tmem + 384, tmem + 128, qm_lo0 + sd * TILE_LO, IDESC_KM, acc);
+        mma_commit(bar_q_empty + 8 * sd);
+        // dP^T of the next step follows dK in the pipe, so it cannot overwrite dS^T(i) early
         if (i + 1 < nsteps) {
-          ok = mbar_wait_lean(bar_do_full + 8 * (sd ^ 1), ((i + 1) >> 1) & 1, abort_flag);
+          ok = mbar_wait_lean(bar_do_full + 8 * sn, ((i + 1) >> 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          gemm_ss(tmem + 128, v_lo, dok_lo0 + (sd ^ 1) * TILE_LO, IDESC_KK, 0u);
+          gemm_ss(tmem + 128, v_lo, dok_lo0 + sn * TILE_LO, IDESC_KK, 0u);
           mma_commit(bar_dpt);
         }
-        sq = nq;
       }
       mma_commit(bar_done);
-      trace_add(a.trace, 16 + 8, clock64() - t_begin); trace_add(a.trace, 16 + 9, w_pt);
-      trace_add(a.trace, 16 + 10, w_q); trace_add(a.trace, 16 + 11, w_dst);
+      trace_add(a.trace, 16 + 8, tick<TR>() - t_begin); trace_add(a.trace, 16 + 9, w_pt);
+      trace_add(a.trace, 16 + 10, w_sf); trace_add(a.trace, 16 + 11, w_dst);
     }
   } else {
     // ------------------------------------------------------------------ compute warpgroups
@@ -242,6 +252,7 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
     const int j = k0 + r;
     const uint32_t tl = tmem + ((uint32_t)((warp & 3) * 32) << 16);
     const int c0 = w * 64;
+    uint8_t* prow = sm + DKDV_P + w * PANEL_BYTES + r * 128;   // this thread's 128-byte row of the P^T tile
     // query rows that see key j, per query stream (section 3.2 read from the key's side)
     int vq_lo[2], vq_hi[2];
     if (ks == CLEAN) {
@@ -253,67 +264,116 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       vq_lo[NOISY] = (j / M) * M; vq_hi[NOISY] = vq_lo[NOISY] + M;
     }
     const int vqc_lo = vq_lo[CLEAN], vqc_hi = vq_hi[CLEAN], vqn_lo = vq_lo[NOISY], vqn_hi = vq_hi[NOISY];
+    // a query tile [q0, q0+128) needs no masking iff every key row of this tile sees all of it: the visible-query
+    // interval is monotone in the key, so the last key's lower bound and the first key's upper bound decide
+    int fullc_lo, fullc_hi, fulln_lo, fulln_hi;
+    {
+      const int jl = k0 + TILE - 1;
+      if (ks == CLEAN) {
+        fullc_lo = (a.mode == 0) ? jl : (jl / M) * M; fullc_hi = (a.window > 0) ? min(L, k0 + a.window) : L;
+        fulln_lo = (jl / M + 1) * M; fulln_hi = fullc_hi;
+      } else {
+        fullc_lo = 0; fullc_hi = 0;
+        fulln_lo = (jl / M) * M; fulln_hi = (k0 / M) * M + M;
+      }
+    }
     bool ok = true;
-    long long w_st = 0, w_dpt = 0;
-    const long long t_begin = clock64();
+    long long w_st = 0, w_dpt = 0, w_pf = 0, c_exp = 0, c_ds = 0, c_ld = 0, c_math = 0;
+    const long long t_begin = tick<TR>();
     for (int i = 0; i < nsteps; ++i) {
       const int sd = i & 1;
-      const QStep st = step_of(i);
-      // the tile needs masking unless every query row of it sees every key of this key tile
-      int lo_a, hi_a, lo_b, hi_b;
-      visible_interval(st.qs, ks, st.q0, M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_a, hi_a, a.window);
-      visible_interval(st.qs, ks, st.q0 + TILE - 1, M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_b, hi_b, a.window);
-      const bool need_mask = (lo_b > k0) || (hi_a < k0 + TILE);
-      ok = mbar_wait_timed(bar_do_full + 8 * sd, (i >> 1) & 1, abort_flag, w_st);
-      ok = ok && mbar_wait_timed(bar_st, i & 1, abort_flag, w_st);
+      const QStep st = step_cur();
+      step_next();
+      const bool need_mask = (st.qs == CLEAN) ? (st.q0 < fullc_lo || st.q0 + TILE > fullc_hi)
+                                              : (st.q0 < fulln_lo || st.q0 + TILE > fulln_hi);
+      ok = mbar_wait_timed<TR>(bar_do_full + 8 * sd, (i >> 1) & 1, abort_flag, w_st);
+      ok = ok && mbar_wait_timed<TR>(bar_st, i & 1, abort_flag, w_st);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
+      const long long t0 = tick<TR>();
       uint32_t x[64];
       {
         uint32_t (*c)[32] = reinterpret_cast<uint32_t (*)[32]>(x);
         tmem_ld32(tl + c0, c[0]); tmem_ld32(tl + c0 + 32, c[1]);
         tmem_wait_ld();
       }
-      const float* lz = lse_s + sd * 128 + c0;
+      tc_fence_before();
+      mbar_arrive(bar_sfree);   // S^T(i) is in registers: the tensor core may overwrite its columns
+      const long long t0b = tick<TR>();
+      c_ld += t0b - t0;
+      const float4* lz4 = reinterpret_cast<const float4*>(lse_s + sd * 128 + c0);
       if (!need_mask) {
 #pragma unroll
-        for (int c = 0; c < 64; ++c) x[c] = __float_as_uint(exp2f(fmaf(__uint_as_float(x[c]), a.scale_log2, -lz[c])));
+        for (int c8 = 0; c8 < 8; ++c8) {
+          const float4 za = lz4[2 * c8], zb = lz4[2 * c8 + 1];
+          float* xf = reinterpret_cast<float*>(x) + 8 * c8;
+          xf[0] = exp2f(fmaf(xf[0], a.scale_log2, -za.x));
+          xf[1] = exp2f(fmaf(xf[1], a.scale_log2, -za.y));
+          xf[2] = exp2f(fmaf(xf[2], a.scale_log2, -za.z));
+          xf[3] = exp2f(fmaf(xf[3], a.scale_log2, -za.w));
+          xf[4] = exp2f(fmaf(xf[4], a.scale_log2, -zb.x));
+          xf[5] = exp2f(fmaf(xf[5], a.scale_log2, -zb.y));
+          xf[6] = exp2f(fmaf(xf[6], a.scale_log2, -zb.z));
+          xf[7] = exp2f(fmaf(xf[7], a.scale_log2, -zb.w));
+        }
       } else {
         // visible columns of this thread's key row inside the tile: [vlo, vhi)
         const int vlo = (st.qs == CLEAN ? vqc_lo : vqn_lo) - st.q0 - c0, vhi = (st.qs == CLEAN ? vqc_hi : vqn_hi) - st.q0 - c0;
 #pragma unroll
-        for (int c = 0; c < 64; ++c) {
-          const float p = exp2f(fmaf(__uint_as_float(x[c]), a.scale_log2, -lz[c]));
-          x[c] = __float_as_uint((c >= vlo && c < vhi) ? p : 0.f);
+        for (int c4 = 0; c4 < 16; ++c4) {
+          const float4 z = lz4[c4];
+          const float zz[4] = {z.x, z.y, z.z, z.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int c = 4 * c4 + e;
+            const float p = exp2f(fmaf(__uint_as_float(x[c]), a.scale_log2, -zz[e]));
+            x[c] = __float_as_uint((c >= vlo && c < vhi) ? p : 0.f);
+          }
         }
       }
-      {
-        uint32_t pk[32];
-#pragma unroll
-        for (int e = 0; e < 32; ++e) pk[e] = pack_bf16(__uint_as_float(x[2 * e]), __uint_as_float(x[2 * e + 1]));
-        tmem_st32(tl + c0, pk);
-        tmem_wait_st();
+      c_math += tick<TR>() - t0b;
+      // P^T(i) as bf16 into the shared-memory tile, once dV(i-1) has finished reading P^T(i-1)
+      if (i > 0) {
+        ok = mbar_wait_timed<TR>(bar_pfree, (i - 1) & 1, abort_flag, w_pf);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
       }
-      tc_fence_before();
+#pragma unroll
+      for (int c8 = 0; c8 < 8; ++c8) {
+        uint4 v;
+        v.x = pack_bf16(__uint_as_float(x[c8 * 8 + 0]), __uint_as_float(x[c8 * 8 + 1]));
+        v.y = pack_bf16(__uint_as_float(x[c8 * 8 + 2]), __uint_as_float(x[c8 * 8 + 3]));
+        v.z = pack_bf16(__uint_as_float(x[c8 * 8 + 4]), __uint_as_float(x[c8 * 8 + 5]));
+        v.w = pack_bf16(__uint_as_float(x[c8 * 8 + 6]), __uint_as_float(x[c8 * 8 + 7]));
+        *reinterpret_cast<uint4*>(prow + ((c8 ^ (r & 7)) << 4)) = v;
+      }
+      fence_async_smem();
       mbar_arrive(bar_pt);
+      const long long t1 = tick<TR>();
+      c_exp += t1 - t0;
 
-      ok = mbar_wait_timed(bar_dpt, i & 1, abort_flag, w_dpt);
+      ok = mbar_wait_timed<TR>(bar_dpt, i & 1, abort_flag, w_dpt);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
+      const long long t2 = tick<TR>();
       {
         uint32_t y[64];
         uint32_t (*c)[32] = reinterpret_cast<uint32_t (*)[32]>(y);
         tmem_ld32(tl + 128 + c0, c[0]); tmem_ld32(tl + 128 + c0 + 32, c[1]);
         tmem_wait_ld();
-        const float* dz = d_s + sd * 128 + c0;
+        const float4* dz4 = reinterpret_cast<const float4*>(d_s + sd * 128 + c0);
         uint32_t pk[32];
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          const float d0 = __uint_as_float(x[2 * e]) * (__uint_as_float(y[2 * e]) - dz[2 * e]);
-          const float d1 = __uint_as_float(x[2 * e + 1]) * (__uint_as_float(y[2 * e + 1]) - dz[2 * e + 1]);
-          pk[e] = pack_bf16(d0, d1);
+        for (int c4 = 0; c4 < 16; ++c4) {
+          const float4 dd = dz4[c4];
+          const float d0 = __uint_as_float(x[4 * c4 + 0]) * (__uint_as_float(y[4 * c4 + 0]) - dd.x);
+          const float d1 = __uint_as_float(x[4 * c4 + 1]) * (__uint_as_float(y[4 * c4 + 1]) - dd.y);
+          const float d2 = __uint_as_float(x[4 * c4 + 2]) * (__uint_as_float(y[4 * c4 + 2]) - dd.z);
+          const float d3 = __uint_as_float(x[4 * c4 + 3]) * (__uint_as_float(y[4 * c4 + 3]) - dd.w);
+          pk[2 * c4] = pack_bf16(d0, d1);
+          pk[2 * c4 + 1] = pack_bf16(d2, d3);
         }
         tmem_st32(tl + 128 + c0, pk);
         tmem_wait_st();
@@ -322,10 +382,13 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       mbar_arrive(bar_dst);
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_do_empty + 8 * sd);   // this warp is done with the stage's D rows
+      c_ds += tick<TR>() - t2;
     }
     if (warp == 0 && lane == 0) {
       trace_add(a.trace, 16 + 0, nsteps); trace_add(a.trace, 16 + 1, w_st); trace_add(a.trace, 16 + 2, w_dpt);
-      trace_add(a.trace, 16 + 6, clock64() - t_begin);
+      trace_add(a.trace, 16 + 3, w_pf); trace_add(a.trace, 16 + 4, c_exp); trace_add(a.trace, 16 + 5, c_ds);
+      trace_add(a.trace, 16 + 6, tick<TR>() - t_begin);
+      trace_add(a.trace, 16 + 14, c_ld); trace_add(a.trace, 16 + 15, c_math);
     }
     // epilogue: warpgroup 0 writes dV, warpgroup 1 writes dK (scaled)
     if (ok && nsteps > 0) {
@@ -380,6 +443,7 @@ __device__ __forceinline__ void row_smem_to_tmem(const uint8_t* tile, int r, uin
   }
 }
 
+template <bool TR>
 __global__ void __launch_bounds__(BWD_THREADS, 1)
 tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restrict__ status) {
   extern __shared__ __align__(1024) uint8_t sm[];
@@ -440,25 +504,25 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
       tma_tile(sdO, &maps.dout[qs], bar_qdo, h * 128, q0, b);
       bool ok = true;
       long long w_empty = 0;
-      const long long t_begin = clock64();
+      const long long t_begin = tick<TR>();
       for (int i = 0; i < nsteps && ok; ++i) {
         const int sk = i % 3, sv = i & 1;
         const int ks = tile_ks(i), k0 = tile_k0(i);
-        if (i >= 3) ok = mbar_wait_timed(bar_k_empty + 8 * sk, ((i / 3) - 1) & 1, abort_flag, w_empty);
+        if (i >= 3) ok = mbar_wait_timed<TR>(bar_k_empty + 8 * sk, ((i / 3) - 1) & 1, abort_flag, w_empty);
         if (!ok) break;
         mbar_expect_tx(bar_k_full + 8 * sk, TILE_BYTES);
         tma_tile(sK0 + sk * TILE_BYTES, &maps.k[ks], bar_k_full + 8 * sk, hk * 128, k0, b);
-        if (i >= 2) ok = mbar_wait_timed(bar_v_empty + 8 * sv, ((i >> 1) - 1) & 1, abort_flag, w_empty);
+        if (i >= 2) ok = mbar_wait_timed<TR>(bar_v_empty + 8 * sv, ((i >> 1) - 1) & 1, abort_flag, w_empty);
         if (!ok) break;
         mbar_expect_tx(bar_v_full + 8 * sv, TILE_BYTES);
         tma_tile(sV0 + sv * TILE_BYTES, &maps.v[ks], bar_v_full + 8 * sv, hk * 128, k0, b);
       }
-      trace_add(a.trace, 32 + 12, clock64() - t_begin); trace_add(a.trace, 32 + 13, w_empty);
+      trace_add(a.trace, 32 + 12, tick<TR>() - t_begin); trace_add(a.trace, 32 + 13, w_empty);
     }
   } else if (warp == 9) {
     if (lane == 0 && nsteps > 0) {
       long long w_kv = 0, w_ds = 0, w_sf = 0;
-      const long long t_begin = clock64();
+      const long long t_begin = tick<TR>();
       const uint32_t kk_lo0 = desc_lo_k(sK0), km_lo0 = desc_lo_mn(sK0);   // K ring as K-major B (S) / MN-major B (dQ)
       const uint32_t vk_lo0 = desc_lo_k(sV0);
       bool ok = mbar_wait_abortable(bar_aready, 0, abort_flag);
@@ -504,7 +568,7 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
         sk = nk;
       }
       mma_commit(bar_done);
-      trace_add(a.trace, 32 + 8, clock64() - t_begin); trace_add(a.trace, 32 + 9, w_kv); trace_add(a.trace, 32 + 10, w_ds);
+      trace_add(a.trace, 32 + 8, tick<TR>() - t_begin); trace_add(a.trace, 32 + 9, w_kv); trace_add(a.trace, 32 + 10, w_ds);
       trace_add(a.trace, 32 + 11, w_sf);
     }
   } else {
@@ -524,8 +588,8 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
     visible_interval(qs, 1, row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo1, rhi1, a.window);
     bool ok = true;
     long long w_s = 0, w_dp = 0, c_ld = 0, c_exp = 0, c_ds = 0;
-    Stopwatch sw;
-    const long long t_begin = clock64();
+    Stopwatch<TR> sw;
+    const long long t_begin = tick<TR>();
     if (nsteps > 0) {   // stage the A operands: warpgroup 0 copies Q, warpgroup 1 copies dO
       ok = mbar_wait_abortable(bar_qdo, 0, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
@@ -538,7 +602,7 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
     }
     for (int i = 0; i < nsteps && ok; ++i) {
       const int ks = tile_ks(i), k0 = tile_k0(i);
-      ok = mbar_wait_timed(bar_s, i & 1, abort_flag, w_s);
+      ok = mbar_wait_timed<TR>(bar_s, i & 1, abort_flag, w_s);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -555,7 +619,17 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
       const bool need_mask = ks == 0 ? (k0 < lo_last0 || k0 + TILE > hi_first0) : (k0 < lo_last1 || k0 + TILE > hi_first1);
       if (!need_mask) {
 #pragma unroll
-        for (int c = 0; c < 64; ++c) x[c] = __float_as_uint(exp2f(fmaf(__uint_as_float(x[c]), a.scale_log2, -lse2)));
+        for (int c8 = 0; c8 < 8; ++c8) {
+          float* xf = reinterpret_cast<float*>(x) + 8 * c8;
+          xf[0] = exp2f(fmaf(xf[0], a.scale_log2, -lse2));
+          xf[1] = exp2f(fmaf(xf[1], a.scale_log2, -lse2));
+          xf[2] = exp2f(fmaf(xf[2], a.scale_log2, -lse2));
+          xf[3] = exp2f(fmaf(xf[3], a.scale_log2, -lse2));
+          xf[4] = exp2f(fmaf(xf[4], a.scale_log2, -lse2));
+          xf[5] = exp2f(fmaf(xf[5], a.scale_log2, -lse2));
+          xf[6] = exp2f(fmaf(xf[6], a.scale_log2, -lse2));
+          xf[7] = exp2f(fmaf(xf[7], a.scale_log2, -lse2));
+        }
       } else {
         const int vlo = (ks == 0 ? rlo0 : rlo1) - k0 - c0, vhi = (ks == 0 ? rhi0 : rhi1) - k0 - c0;
 #pragma unroll
@@ -565,7 +639,7 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
         }
       }
       sw.lap(c_exp);
-      ok = mbar_wait_timed(bar_dp, i & 1, abort_flag, w_dp);
+      ok = mbar_wait_timed<TR>(bar_dp, i & 1, abort_flag, w_dp);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -591,7 +665,7 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
     }
     if (warp == 0 && lane == 0) {
       trace_add(a.trace, 32 + 0, nsteps); trace_add(a.trace, 32 + 1, w_s); trace_add(a.trace, 32 + 2, w_dp);
-      trace_add(a.trace, 32 + 6, clock64() - t_begin);
+      trace_add(a.trace, 32 + 6, tick<TR>() - t_begin);
       trace_add(a.trace, 32 + 3, c_ld); trace_add(a.trace, 32 + 4, c_exp); trace_add(a.trace, 32 + 5, c_ds);
     }
     if (ok && nsteps > 0) {
@@ -639,6 +713,7 @@ constexpr int P1_BARS = P1_ARR + 2048;
 constexpr int P1_SMEM = P1_BARS + 160;
 constexpr uint32_t IDESC_MM = make_idesc(128, 128, true, true);   // A and B both MN-major
 
+template <bool TR>
 __global__ void __launch_bounds__(BWD_THREADS, 1)
 tc_bwd1p_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restrict__ status) {
   extern __shared__ __align__(1024) uint8_t sm[];
@@ -712,18 +787,18 @@ tc_bwd1p_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __rest
     }
     bool ok = true;
     long long w_empty = 0;
-    const long long t_begin = clock64();
+    const long long t_begin = tick<TR>();
     for (int i = 0; i < nsteps && ok; ++i) {
       const int sd = i & 1;
       const QStep st = step_of(i);
-      if (i >= 2) ok = mbar_wait_timed(bar_q_empty + 8 * sd, ((i >> 1) - 1) & 1, abort_flag, w_empty);
+      if (i >= 2) ok = mbar_wait_timed<TR>(bar_q_empty + 8 * sd, ((i >> 1) - 1) & 1, abort_flag, w_empty);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       if (lane == 0) {
         mbar_expect_tx(bar_q_full + 8 * sd, TILE_BYTES);
         tma_tile(sQ0 + sd * TILE_BYTES, &maps.q[st.qs], bar_q_full + 8 * sd, st.h * 128, st.q0, b);
       }
-      if (i >= 2) ok = mbar_wait_timed(bar_do_empty + 8 * sd, ((i >> 1) - 1) & 1, abort_flag, w_empty);
+      if (i >= 2) ok = mbar_wait_timed<TR>(bar_do_empty + 8 * sd, ((i >> 1) - 1) & 1, abort_flag, w_empty);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       if (lane == 0) {
@@ -744,11 +819,11 @@ tc_bwd1p_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __rest
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_do_full + 8 * sd);
     }
-    if (lane == 0) { trace_add(a.trace, 16 + 12, clock64() - t_begin); trace_add(a.trace, 16 + 13, w_empty); }
+    if (lane == 0) { trace_add(a.trace, 16 + 12, tick<TR>() - t_begin); trace_add(a.trace, 16 + 13, w_empty); }
   } else if (warp == 9) {
     // ------------------------------------------------------------------ MMA issuer (one thread)
     if (lane == 0 && nsteps > 0) {
-      const long long t_begin = clock64();
+      const long long t_begin = tick<TR>();
       const uint32_t k_lo = desc_lo_k(sK), v_lo = desc_lo_k(sV), kt_lo = desc_lo_mn(sK);
       const uint32_t qk_lo0 = desc_lo_k(sQ0), qm_lo0 = desc_lo_mn(sQ0);
       const uint32_t dok_lo0 = desc_lo_k(sdO0), dom_lo0 = desc_lo_mn(sdO0);
@@ -800,7 +875,7 @@ tc_bwd1p_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __rest
         }
       }
       mma_commit(bar_done);
-      trace_add(a.trace, 16 + 8, clock64() - t_begin);
+      trace_add(a.trace, 16 + 8, tick<TR>() - t_begin);
     }
   } else {
     // ------------------------------------------------------------------ compute warpgroups
@@ -820,7 +895,7 @@ tc_bwd1p_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __rest
     }
     bool ok = true;
     long long w_st = 0, w_dpt = 0, w_dqf = 0;
-    const long long t_begin = clock64();
+    const long long t_begin = tick<TR>();
     uint32_t x[64];   // P^T of the step in flight (fp32), kept from phase 1 to phase 2
 
     // phase 1 of step i: P^T = exp2(S^T * scale - LSE) on visible pairs, bf16 pairs back into the S^T columns
@@ -831,8 +906,8 @@ tc_bwd1p_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __rest
       visible_interval(st.qs, ks, st.q0, M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_a, hi_a, a.window);
       visible_interval(st.qs, ks, st.q0 + TILE - 1, M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_b, hi_b, a.window);
       const bool need_mask = (lo_b > k0) || (hi_a < k0 + TILE);
-      ok = mbar_wait_timed(bar_do_full + 8 * sd, (i >> 1) & 1, abort_flag, w_st);
-      ok = ok && mbar_wait_timed(bar_st, i & 1, abort_flag, w_st);
+      ok = mbar_wait_timed<TR>(bar_do_full + 8 * sd, (i >> 1) & 1, abort_flag, w_st);
+      ok = ok && mbar_wait_timed<TR>(bar_st, i & 1, abort_flag, w_st);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) return;
       tc_fence_after();
@@ -866,7 +941,7 @@ tc_bwd1p_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __rest
     for (int i = 0; i < nsteps && ok; ++i) {
       const int sd = i & 1;
       // phase 2: dS^T = P^T * (dP^T - D), bf16, into the shared-memory tile (row = key, this half's 64 query columns)
-      ok = mbar_wait_timed(bar_dpt, i & 1, abort_flag, w_dpt);
+      ok = mbar_wait_timed<TR>(bar_dpt, i & 1, abort_flag, w_dpt);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -901,7 +976,7 @@ tc_bwd1p_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __rest
       if (i + 1 < nsteps) { phase1(i + 1); if (!ok) break; }
 
       // read-out: dQ[q, h, d] += scale * dQ^T[d, q]; this thread is head-dim element d = r of the step's query rows
-      ok = mbar_wait_timed(bar_dqf, i & 1, abort_flag, w_dqf);
+      ok = mbar_wait_timed<TR>(bar_dqf, i & 1, abort_flag, w_dqf);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -923,7 +998,7 @@ tc_bwd1p_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __rest
     }
     if (warp == 0 && lane == 0) {
       trace_add(a.trace, 16 + 0, nsteps); trace_add(a.trace, 16 + 1, w_st); trace_add(a.trace, 16 + 2, w_dpt);
-      trace_add(a.trace, 16 + 3, w_dqf); trace_add(a.trace, 16 + 6, clock64() - t_begin);
+      trace_add(a.trace, 16 + 3, w_dqf); trace_add(a.trace, 16 + 6, tick<TR>() - t_begin);
     }
     // epilogue: warpgroup 0 writes dV, warpgroup 1 writes dK (scaled)
     if (ok && nsteps > 0) {
@@ -991,9 +1066,10 @@ cudaError_t launch_tc_bwd(const KArgs& a_in, void* extra_ws, int passes, cudaStr
     // one kernel produces dK, dV and (through fp32 atomics) dQ; it runs for the DKDV pass bit, the DQ bit is a no-op
     if (passes & BDLM_BWD_PASS_DKDV) {
       if ((e = cudaMemsetAsync(a.dq32[0], 0, 2 * dq32_elems * sizeof(float), st)) != cudaSuccess) return e;
-      if ((e = cudaFuncSetAttribute(tc_bwd1p_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P1_SMEM)) != cudaSuccess) return e;
+      auto kern = a.trace ? tc_bwd1p_kernel<true> : tc_bwd1p_kernel<false>;
+      if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, P1_SMEM)) != cudaSuccess) return e;
       dim3 grid(a.L / TILE, a.Hkv, a.batch * 2);
-      tc_bwd1p_kernel<<<grid, BWD_THREADS, P1_SMEM, st>>>(maps, a, status);
+      kern<<<grid, BWD_THREADS, P1_SMEM, st>>>(maps, a, status);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
       for (int s2 = 0; s2 < 2; ++s2) {
         dq_convert_kernel<<<148 * 8, 256, 0, st>>>(a.dq32[s2], a.dq[s2], (int64_t)(dq32_elems / 8));
@@ -1003,15 +1079,17 @@ cudaError_t launch_tc_bwd(const KArgs& a_in, void* extra_ws, int passes, cudaStr
     return cudaSuccess;
   }
   if (passes & BDLM_BWD_PASS_DKDV) {
-    if ((e = cudaFuncSetAttribute(tc_dkdv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DKDV_SMEM)) != cudaSuccess) return e;
+    auto kern = a.trace ? tc_dkdv_kernel<true> : tc_dkdv_kernel<false>;
+    if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, DKDV_SMEM)) != cudaSuccess) return e;
     dim3 grid(a.L / TILE, a.Hkv, a.batch * 2);
-    tc_dkdv_kernel<<<grid, BWD_THREADS, DKDV_SMEM, st>>>(maps, a, status);
+    kern<<<grid, BWD_THREADS, DKDV_SMEM, st>>>(maps, a, status);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
   if (passes & BDLM_BWD_PASS_DQ) {
-    if ((e = cudaFuncSetAttribute(tc_dq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DQ_SMEM)) != cudaSuccess) return e;
+    auto kern = a.trace ? tc_dq_kernel<true> : tc_dq_kernel<false>;
+    if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, DQ_SMEM)) != cudaSuccess) return e;
     dim3 grid(a.L / TILE, a.H, a.batch * 2);
-    tc_dq_kernel<<<grid, BWD_THREADS, DQ_SMEM, st>>>(maps, a, status);
+    kern<<<grid, BWD_THREADS, DQ_SMEM, st>>>(maps, a, status);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
   return cudaSuccess;

@@ -72,19 +72,33 @@ __device__ __forceinline__ bool mbar_wait_lean(uint32_t bar, uint32_t parity, vo
   return mbar_wait_abortable(bar, parity, abort_flag);
 }
 
+// Reading the clock costs tens of cycles on a path that is otherwise a handful of instructions, so the cycle
+// accounting is compiled in only for the traced instantiation of a kernel (TR = true).
+template <bool TR>
+__device__ __forceinline__ long long tick() {
+  if constexpr (TR) return clock64(); else return 0;
+}
+template <bool TR>
 __device__ __forceinline__ bool mbar_wait_timed(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long& acc) {
-  const long long t0 = clock64();
-  const bool ok = mbar_wait_abortable(bar, parity, abort_flag);
-  acc += clock64() - t0;
-  return ok;
+  if constexpr (TR) {
+    const long long t0 = clock64();
+    const bool ok = mbar_wait_abortable(bar, parity, abort_flag);
+    acc += clock64() - t0;
+    return ok;
+  } else {
+    return mbar_wait_lean(bar, parity, abort_flag);
+  }
 }
 
 // Cycle accounting for the optional trace buffer: a role keeps a few local counters and adds
 // them to the global slots once, when it leaves its loop.
+template <bool TR>
 struct Stopwatch {
   long long t;
-  __device__ __forceinline__ void start() { t = clock64(); }
-  __device__ __forceinline__ void lap(long long& acc) { const long long n = clock64(); acc += n - t; t = n; }
+  __device__ __forceinline__ void start() { if constexpr (TR) t = clock64(); }
+  __device__ __forceinline__ void lap(long long& acc) {
+    if constexpr (TR) { const long long n = clock64(); acc += n - t; t = n; }
+  }
 };
 __device__ __forceinline__ void trace_add(unsigned long long* trace, int slot, long long v) {
   if (trace != nullptr) atomicAdd(trace + slot, static_cast<unsigned long long>(v));

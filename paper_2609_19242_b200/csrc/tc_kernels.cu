@@ -297,6 +297,7 @@ constexpr int FWD2H_MX = 6 * TILE_BYTES;                    // mx_s[2][2][2][128
 constexpr int FWD2H_BARS = FWD2H_MX + 4096 + 2048;
 constexpr int FWD2H_SMEM = FWD2H_BARS + 256 + 1024;
 
+template <bool TR>
 __global__ void __launch_bounds__(FWD2H_THREADS, 1)
 tc_fwd2h_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
@@ -420,13 +421,13 @@ tc_fwd2h_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __rest
     float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
     long long w_s = 0;
-    const long long t_begin = clock64();
+    const long long t_begin = tick<TR>();
     for (int t = 0; t < nt; ++t) {
       const int ks = tile_ks(t), k0 = tile_k0(t);
       // After a failed (timed-out) wait this warpgroup keeps walking the loop without touching tensor memory,
       // so that it still meets its partner at every named barrier: the failure path must end, never hang.
       if (ok) {
-        ok = mbar_wait_timed(bar_s + 8 * w, t & 1, abort_flag, w_s);
+        ok = mbar_wait_timed<TR>(bar_s + 8 * w, t & 1, abort_flag, w_s);
         ok = __all_sync(0xffffffffu, ok);
       }
       tc_fence_after();
@@ -520,7 +521,7 @@ tc_fwd2h_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __rest
       tc_fence_before();
       mbar_arrive(bar_p + 8 * w);
     }
-    if (warp == 0 && lane == 0) { trace_add(a.trace, 0, nt); trace_add(a.trace, 1, w_s); trace_add(a.trace, 6, clock64() - t_begin); }
+    if (warp == 0 && lane == 0) { trace_add(a.trace, 0, nt); trace_add(a.trace, 1, w_s); trace_add(a.trace, 6, tick<TR>() - t_begin); }
     // total row sum = sum of the two halves (both kept the same reference maximum)
     ls_s[(w * 2 + hc) * 128 + r] = l;
     asm volatile("bar.sync %0, %1;" ::"r"(1 + w), "r"(256) : "memory");
@@ -578,10 +579,11 @@ cudaError_t launch_tc_fwd(const KArgs& a, cudaStream_t st) {
   cudaError_t e = cudaFuncSetAttribute(tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM);
   if (e != cudaSuccess) return e;
   if (a.G % 2 == 0) {   // two heads of one KV group per CTA, four softmax warpgroups
-    e = cudaFuncSetAttribute(tc_fwd2h_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD2H_SMEM);
+    auto kern = a.trace ? tc_fwd2h_kernel<true> : tc_fwd2h_kernel<false>;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD2H_SMEM);
     if (e != cudaSuccess) return e;
     dim3 grid4(a.L / TILE, a.H / 2, a.batch * 2);
-    tc_fwd2h_kernel<<<grid4, FWD2H_THREADS, FWD2H_SMEM, st>>>(maps, a, status);
+    kern<<<grid4, FWD2H_THREADS, FWD2H_SMEM, st>>>(maps, a, status);
     return cudaGetLastError();
   }
   dim3 grid(a.L / TILE, a.H, a.batch * 2);
