@@ -73,11 +73,15 @@ constexpr int DKDV_P = 6 * TILE_BYTES;
 constexpr int DKDV_ARR = 7 * TILE_BYTES;            // lse_s[2][128], d_s[2][128]
 constexpr int DKDV_BARS = DKDV_ARR + 2048;
 constexpr int DKDV_SMEM = DKDV_BARS + 176;
+constexpr int DKDV_NWG = 2;                          // compute warpgroups; each owns 128 / NWG query columns of every key row
+constexpr int DKDV_CW = 128 / DKDV_NWG;
+constexpr int DKDV_THREADS = (4 * DKDV_NWG + 2) * 32;
+constexpr int DKDV_PRODUCER = 4 * DKDV_NWG, DKDV_ISSUER = 4 * DKDV_NWG + 1;
 
 struct QStep { int qs, h, q0; };
 
 template <bool TR>
-__global__ void __launch_bounds__(BWD_THREADS, 1)
+__global__ void __launch_bounds__(DKDV_THREADS, 1)
 tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restrict__ status) {
   extern __shared__ __align__(1024) uint8_t sm[];
   const uint32_t base = smem_u32(sm);
@@ -127,13 +131,13 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
     if (base & 1023u) *abort_flag = 1; else *abort_flag = 0;   // swizzled tiles need a 1024-byte aligned base
     mbar_init(bar_kv, 1);
     for (int i = 0; i < 2; ++i) { mbar_init(bar_q_full + 8 * i, 1); mbar_init(bar_q_empty + 8 * i, 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(bar_do_full + 8 * i, 2); mbar_init(bar_do_empty + 8 * i, 9); }   // full: TMA bytes + LSE/D rows; empty: dV done + 8 warps done with the D rows
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_do_full + 8 * i, 2); mbar_init(bar_do_empty + 8 * i, 1 + 4 * DKDV_NWG); }   // full: TMA bytes + LSE/D rows; empty: dV done + every compute warp done with the D rows
     mbar_init(bar_st, 1); mbar_init(bar_dpt, 1); mbar_init(bar_pfree, 1);
-    mbar_init(bar_sfree, 256); mbar_init(bar_pt, 256); mbar_init(bar_dst, 256);
+    mbar_init(bar_sfree, 128 * DKDV_NWG); mbar_init(bar_pt, 128 * DKDV_NWG); mbar_init(bar_dst, 128 * DKDV_NWG);
     mbar_init(bar_done, 1);
     fence_mbar_init();
   }
-  if (warp == 8) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
+  if (warp == DKDV_PRODUCER) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -143,7 +147,7 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
 
   if (bad_base) {
     // fall through to the common exit
-  } else if (warp == 8) {
+  } else if (warp == DKDV_PRODUCER) {
     // ------------------------------------------------------------------ producer
     if (lane == 0) {
       mbar_expect_tx(bar_kv, 2 * TILE_BYTES);
@@ -186,7 +190,7 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       if (lane == 0) mbar_arrive(bar_do_full + 8 * sd);
     }
     if (lane == 0) { trace_add(a.trace, 16 + 12, tick<TR>() - t_begin); trace_add(a.trace, 16 + 13, w_empty); }
-  } else if (warp == 9) {
+  } else if (warp == DKDV_ISSUER) {
     // ------------------------------------------------------------------ MMA issuer (one thread)
     if (lane == 0 && nsteps > 0) {
       long long w_pt = 0, w_sf = 0, w_dst = 0;
@@ -226,11 +230,11 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
         gemm_ss_km(tmem + 256, p_lo, dom_lo0 + sd * TILE_LO, IDESC_KM, acc);
         mma_commit(bar_do_empty + 8 * sd);
         mma_commit(bar_pfree);
-        // dK += dS^T Q_i   (dS^T: this lane's 64+64 bf16 pairs at columns 128+[0,32) and 128+[64,96))
+        // dK += dS^T Q_i   (dS^T: bf16 pairs, each warpgroup's share at the start of its own dP^T columns)
         ok = mbar_wait_timed<TR>(bar_dst, i & 1, abort_flag, w_dst);
         if (!ok) break;
         tc_fence_after();
-        gemm_ts_mn<true>(tmem + 384, tmem + 128, qm_lo0 + sd * TILE_LO, IDESC_KM, acc);
+        gemm_ts_mn_cw<DKDV_CW>(tmem + 384, tmem + 128, qm_lo0 + sd * TILE_LO, IDESC_KM, acc);
         mma_commit(bar_q_empty + 8 * sd);
         // dP^T of the next step follows dK in the pipe, so it cannot overwrite dS^T(i) early
         if (i + 1 < nsteps) {
@@ -247,12 +251,14 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
     }
   } else {
     // ------------------------------------------------------------------ compute warpgroups
-    const int w = warp >> 2;                                   // column half: query columns [64w, 64w+64)
+    constexpr int CW = DKDV_CW;
+    const int w = warp >> 2;                                   // column share: query columns [CW w, CW w + CW)
     const int r = (warp & 3) * 32 + lane;                      // TMEM lane = key row of the tile
     const int j = k0 + r;
     const uint32_t tl = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-    const int c0 = w * 64;
-    uint8_t* prow = sm + DKDV_P + w * PANEL_BYTES + r * 128;   // this thread's 128-byte row of the P^T tile
+    const int c0 = w * CW;
+    uint8_t* prow = sm + DKDV_P + (c0 >> 6) * PANEL_BYTES + r * 128;   // this thread's row of the P^T tile (panel of its columns)
+    const int pch0 = (c0 & 63) >> 3;                           // its first 16-byte chunk in that row
     // query rows that see key j, per query stream (section 3.2 read from the key's side)
     int vq_lo[2], vq_hi[2];
     if (ks == CLEAN) {
@@ -292,10 +298,11 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       if (!ok) break;
       tc_fence_after();
       const long long t0 = tick<TR>();
-      uint32_t x[64];
+      uint32_t x[CW];
       {
         uint32_t (*c)[32] = reinterpret_cast<uint32_t (*)[32]>(x);
-        tmem_ld32(tl + c0, c[0]); tmem_ld32(tl + c0 + 32, c[1]);
+#pragma unroll
+        for (int q = 0; q < CW / 32; ++q) tmem_ld32(tl + c0 + 32 * q, c[q]);
         tmem_wait_ld();
       }
       tc_fence_before();
@@ -305,7 +312,7 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       const float4* lz4 = reinterpret_cast<const float4*>(lse_s + sd * 128 + c0);
       if (!need_mask) {
 #pragma unroll
-        for (int c8 = 0; c8 < 8; ++c8) {
+        for (int c8 = 0; c8 < CW / 8; ++c8) {
           const float4 za = lz4[2 * c8], zb = lz4[2 * c8 + 1];
           float* xf = reinterpret_cast<float*>(x) + 8 * c8;
           xf[0] = exp2f(fmaf(xf[0], a.scale_log2, -za.x));
@@ -321,7 +328,7 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
         // visible columns of this thread's key row inside the tile: [vlo, vhi)
         const int vlo = (st.qs == CLEAN ? vqc_lo : vqn_lo) - st.q0 - c0, vhi = (st.qs == CLEAN ? vqc_hi : vqn_hi) - st.q0 - c0;
 #pragma unroll
-        for (int c4 = 0; c4 < 16; ++c4) {
+        for (int c4 = 0; c4 < CW / 4; ++c4) {
           const float4 z = lz4[c4];
           const float zz[4] = {z.x, z.y, z.z, z.w};
 #pragma unroll
@@ -340,13 +347,13 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
         if (!ok) break;
       }
 #pragma unroll
-      for (int c8 = 0; c8 < 8; ++c8) {
+      for (int c8 = 0; c8 < CW / 8; ++c8) {
         uint4 v;
         v.x = pack_bf16(__uint_as_float(x[c8 * 8 + 0]), __uint_as_float(x[c8 * 8 + 1]));
         v.y = pack_bf16(__uint_as_float(x[c8 * 8 + 2]), __uint_as_float(x[c8 * 8 + 3]));
         v.z = pack_bf16(__uint_as_float(x[c8 * 8 + 4]), __uint_as_float(x[c8 * 8 + 5]));
         v.w = pack_bf16(__uint_as_float(x[c8 * 8 + 6]), __uint_as_float(x[c8 * 8 + 7]));
-        *reinterpret_cast<uint4*>(prow + ((c8 ^ (r & 7)) << 4)) = v;
+        *reinterpret_cast<uint4*>(prow + (((pch0 + c8) ^ (r & 7)) << 4)) = v;
       }
       fence_async_smem();
       mbar_arrive(bar_pt);
@@ -359,14 +366,15 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       tc_fence_after();
       const long long t2 = tick<TR>();
       {
-        uint32_t y[64];
+        uint32_t y[CW];
         uint32_t (*c)[32] = reinterpret_cast<uint32_t (*)[32]>(y);
-        tmem_ld32(tl + 128 + c0, c[0]); tmem_ld32(tl + 128 + c0 + 32, c[1]);
+#pragma unroll
+        for (int q = 0; q < CW / 32; ++q) tmem_ld32(tl + 128 + c0 + 32 * q, c[q]);
         tmem_wait_ld();
         const float4* dz4 = reinterpret_cast<const float4*>(d_s + sd * 128 + c0);
-        uint32_t pk[32];
+        uint32_t pk[CW / 2];
 #pragma unroll
-        for (int c4 = 0; c4 < 16; ++c4) {
+        for (int c4 = 0; c4 < CW / 4; ++c4) {
           const float4 dd = dz4[c4];
           const float d0 = __uint_as_float(x[4 * c4 + 0]) * (__uint_as_float(y[4 * c4 + 0]) - dd.x);
           const float d1 = __uint_as_float(x[4 * c4 + 1]) * (__uint_as_float(y[4 * c4 + 1]) - dd.y);
@@ -375,7 +383,8 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
           pk[2 * c4] = pack_bf16(d0, d1);
           pk[2 * c4 + 1] = pack_bf16(d2, d3);
         }
-        tmem_st32(tl + 128 + c0, pk);
+        if constexpr (CW == 64) tmem_st32(tl + 128 + c0, reinterpret_cast<uint32_t (&)[32]>(pk));
+        else tmem_st16(tl + 128 + c0, reinterpret_cast<uint32_t (&)[16]>(pk));
         tmem_wait_st();
       }
       tc_fence_before();
@@ -390,19 +399,22 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       trace_add(a.trace, 16 + 6, tick<TR>() - t_begin);
       trace_add(a.trace, 16 + 14, c_ld); trace_add(a.trace, 16 + 15, c_math);
     }
-    // epilogue: warpgroup 0 writes dV, warpgroup 1 writes dK (scaled)
+    // epilogue: the 256 accumulator columns (dV, then dK) are shared out evenly over the warpgroups
     if (ok && nsteps > 0) {
       ok = mbar_wait_abortable(bar_done, 0, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
     }
     if (ok) {
       tc_fence_after();
-      bf16* dst = (w == 0 ? a.dv[ks] : a.dk[ks]) + (((int64_t)b * L + j) * a.Hkv + hk) * 128;
-      const float sc = (w == 0) ? 1.f : a.scale;
+      constexpr int EW = 256 / DKDV_NWG;                       // accumulator columns per thread
+      const int acol = w * EW;                                 // first of them, in [0, 256)
+      const bool is_dk = acol >= 128;
+      bf16* dst = (is_dk ? a.dk[ks] : a.dv[ks]) + (((int64_t)b * L + j) * a.Hkv + hk) * 128 + (acol & 127);
+      const float sc = is_dk ? a.scale : 1.f;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < EW / 32; ++c) {
         uint32_t v[32];
-        if (nsteps > 0) { tmem_ld32(tl + 256 + w * 128 + c * 32, v); tmem_wait_ld(); }
+        if (nsteps > 0) { tmem_ld32(tl + 256 + acol + c * 32, v); tmem_wait_ld(); }
         else {
 #pragma unroll
           for (int e = 0; e < 32; ++e) v[e] = 0u;
@@ -414,7 +426,7 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
   tc_fence_before();
   __syncthreads();
   if (threadIdx.x == 0 && *abort_flag) atomicExch(status, (int)BDLM_ERR_DEVICE_TIMEOUT);
-  if (warp == 8) tmem_dealloc(tmem, 512);
+  if (warp == DKDV_PRODUCER) tmem_dealloc(tmem, 512);
 }
 
 // =============================================================================================
@@ -521,7 +533,7 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
     }
   } else if (warp == 9) {
     if (lane == 0 && nsteps > 0) {
-      long long w_kv = 0, w_ds = 0, w_sf = 0;
+      long long w_kv = 0, w_ds = 0, w_sf = 0, t_issue = 0;
       const long long t_begin = tick<TR>();
       const uint32_t kk_lo0 = desc_lo_k(sK0), km_lo0 = desc_lo_mn(sK0);   // K ring as K-major B (S) / MN-major B (dQ)
       const uint32_t vk_lo0 = desc_lo_k(sV0);
@@ -543,33 +555,39 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
       for (int i = 0; i < nsteps && ok; ++i) {
         const int nk = (sk == 2) ? 0 : sk + 1;
         if (i + 1 < nsteps) {   // S of the next key tile, once both warpgroups have read S of this one
-          ok = mbar_wait_lean(bar_sfree, i & 1, abort_flag);
-          ok = ok && mbar_wait_lean(bar_k_full + 8 * nk, ((i + 1) / 3) & 1, abort_flag);
+          ok = mbar_wait_timed<TR>(bar_sfree, i & 1, abort_flag, w_sf);
+          ok = ok && mbar_wait_timed<TR>(bar_k_full + 8 * nk, ((i + 1) / 3) & 1, abort_flag, w_kv);
           if (!ok) break;
           tc_fence_after();
+          const long long g0 = tick<TR>();
           gemm_ts(tmem + C_S, tmem + C_Q, kk_lo0 + nk * TILE_LO, IDESC_KK, 0u);
           mma_commit(bar_s);
+          t_issue += tick<TR>() - g0;
         }
         // dQ += dS_i K_i   (dS: bf16 pairs at columns [0,32) and [64,96) of the dP region)
-        ok = mbar_wait_lean(bar_ds, i & 1, abort_flag);
+        ok = mbar_wait_timed<TR>(bar_ds, i & 1, abort_flag, w_ds);
         if (!ok) break;
         tc_fence_after();
+        const long long g1 = tick<TR>();
         gemm_ts_mn<true>(tmem + C_DQ, tmem + C_DP, km_lo0 + sk * TILE_LO, IDESC_KM, i > 0 ? 1u : 0u);
         mma_commit(bar_k_empty + 8 * sk);
+        t_issue += tick<TR>() - g1;
         if (i + 1 < nsteps) {
           const int nv = (i + 1) & 1;
-          ok = mbar_wait_lean(bar_v_full + 8 * nv, ((i + 1) >> 1) & 1, abort_flag);
+          ok = mbar_wait_timed<TR>(bar_v_full + 8 * nv, ((i + 1) >> 1) & 1, abort_flag, w_kv);
           if (!ok) break;
           tc_fence_after();
+          const long long g2 = tick<TR>();
           gemm_ts(tmem + C_DP, tmem + C_DO, vk_lo0 + nv * TILE_LO, IDESC_KK, 0u);
           mma_commit(bar_dp);
           mma_commit(bar_v_empty + 8 * nv);
+          t_issue += tick<TR>() - g2;
         }
         sk = nk;
       }
       mma_commit(bar_done);
       trace_add(a.trace, 32 + 8, tick<TR>() - t_begin); trace_add(a.trace, 32 + 9, w_kv); trace_add(a.trace, 32 + 10, w_ds);
-      trace_add(a.trace, 32 + 11, w_sf);
+      trace_add(a.trace, 32 + 11, w_sf); trace_add(a.trace, 32 + 14, t_issue);
     }
   } else {
     const int w = warp >> 2;
@@ -1082,7 +1100,7 @@ cudaError_t launch_tc_bwd(const KArgs& a_in, void* extra_ws, int passes, cudaStr
     auto kern = a.trace ? tc_dkdv_kernel<true> : tc_dkdv_kernel<false>;
     if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, DKDV_SMEM)) != cudaSuccess) return e;
     dim3 grid(a.L / TILE, a.Hkv, a.batch * 2);
-    kern<<<grid, BWD_THREADS, DKDV_SMEM, st>>>(maps, a, status);
+    kern<<<grid, DKDV_THREADS, DKDV_SMEM, st>>>(maps, a, status);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
   if (passes & BDLM_BWD_PASS_DQ) {

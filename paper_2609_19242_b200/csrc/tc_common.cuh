@@ -174,7 +174,14 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]),
         "r"(taddr) : "memory");
 }
-// 16 packed-bf16 columns variant is not needed; 32-column accesses cover every use here.
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"
+      ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(taddr) : "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -224,6 +231,14 @@ __device__ __forceinline__ void gemm_ts(uint32_t d, uint32_t a_tmem, uint32_t b_
 }
 // A = bf16 pairs in TMEM, B MN-major tile ([contraction row][128 columns]) in shared memory.  `split`: the A
 // pairs of contraction indices 64..127 sit 64 columns after those of 0..63 (two warpgroups wrote them).
+// A = bf16 pairs in TMEM written by warpgroups that each own CW of the 128 contraction indices: the pairs of
+// index c sit at column (c / CW) * CW + (c % CW) / 2.  B MN-major tile in shared memory.
+template <int CW>
+__device__ __forceinline__ void gemm_ts_mn_cw(uint32_t d, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc, uint32_t acc_first) {
+#pragma unroll
+  for (int kk = 0; kk < 8; ++kk)
+    mma_ts(d, a_tmem + ((kk * 16) / CW) * CW + ((kk * 16) % CW) / 2, desc64(b_lo + moff(kk)), idesc, kk == 0 ? acc_first : 1u);
+}
 template <bool SPLIT>
 __device__ __forceinline__ void gemm_ts_mn(uint32_t d, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc, uint32_t acc_first) {
 #pragma unroll
