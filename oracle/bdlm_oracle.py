@@ -30,7 +30,10 @@ lse is [batch, H, L]; everything float64.  Rows and keys are 0-indexed.
 
 All functions here are pinned by tests/test_oracle_*.py against closed forms, the
 paper's mask-count formulas (appendix B), library attention in special cases, finite
-differences and an independent per-row brute force.
+differences and an independent per-row brute force.  The packed form at the end of the file
+(one rank's launches under Algorithms 1 and 2; DFlash2-style blocks of appendix E) is pinned
+by tests/test_oracle_packed_pins.py: per-row brute force, finite differences, the identity
+"ranks' results add up to the unsharded layer" and the work-balance counts of appendix B.
 """
 from __future__ import annotations
 
@@ -277,3 +280,155 @@ def visible_pair_counts(L, M, clean_mask_mode=0, window=0):
     """(clean pairs, noisy pairs) counted from the explicit mask, per (batch, head)."""
     vis = visibility_2L(L, M, clean_mask_mode, window=window)
     return int(vis[:L].sum()), int(vis[L:].sum())
+
+
+# --------------------------------------------------------------------------------------
+# packed form: what one rank of the CSBP schedule launches, and DFlash2-style blocks
+# --------------------------------------------------------------------------------------
+# Algorithm 1 / Algorithm 2 give a rank (a) a run of consecutive clean query positions
+# (one piece of its context shard) and (b) a list of complete corrupted blocks, packed one
+# after the other; both attend the full gathered clean K/V, whose keys keep their original
+# positions.  Appendix E (Eq. dflash2-block-attention) has the same shape with sampled
+# blocks: block b is the token at position a_b followed by M-1 masked tokens, attends its own
+# M keys bidirectionally and the clean ("target-feature") keys at positions < a_b.  Both are
+# described by one table: block_prefix[b] = number of leading clean keys block b sees
+# (b_index * M for a BDLM block, a_b for a DFlash2 block).  Packed row i belongs to packed
+# block i // M and stands at position block_prefix[i // M] + i % M (used by the window only).
+def visible_rows_packed(stream, rows, Lk, M, n_blocks, block_prefix=None, clean_q_pos0=0,
+                        clean_mask_mode=0, kv_begin=0, kv_end=None, include_noisy_diag=True,
+                        window=0):
+    """Boolean visibility [len(rows), Lk + n_blocks*M]: clean keys 0..Lk-1 (by position), then
+    the packed noisy keys.  `rows` index the packed query tensor of `stream`: clean row i is
+    the clean token at position clean_q_pos0 + i; noisy row i is token i % M of packed block
+    i // M."""
+    if kv_end is None:
+        kv_end = Lk
+    Ln = n_blocks * M
+    if block_prefix is None:
+        block_prefix = np.arange(n_blocks, dtype=np.int64) * M
+    block_prefix = np.asarray(block_prefix, dtype=np.int64)
+    i = np.asarray(rows, dtype=np.int64)[:, None]
+    j = np.arange(Lk, dtype=np.int64)[None, :]
+    in_shard = (j >= kv_begin) & (j < kv_end)
+    if stream == CLEAN:
+        pos = clean_q_pos0 + i
+        to_clean = (j <= pos) if clean_mask_mode == 0 else ((j // M) <= (pos // M))
+        to_noisy = np.zeros((i.shape[0], Ln), dtype=bool)
+    else:
+        pfx = block_prefix[i // M]
+        pos = pfx + i % M
+        to_clean = j < pfx
+        jj = np.arange(Ln, dtype=np.int64)[None, :]
+        to_noisy = (jj // M) == (i // M)
+        if not include_noisy_diag:
+            to_noisy = np.zeros_like(to_noisy)
+    if window and window > 0:
+        in_shard = in_shard & (pos - j < window)
+    return np.concatenate([to_clean & in_shard, to_noisy], axis=1)
+
+
+def attn_packed(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, block_size,
+                do_clean=None, do_noisy=None, block_prefix=None, clean_q_pos0=0, scale=None,
+                clean_mask_mode=0, kv_begin=0, kv_end=None, include_noisy_diag=True, window=0,
+                row_chunk=1024):
+    """Forward (and, when a dO is given, backward for sum(O*dO)) of the packed form.
+
+    q_clean [B, Lq, H, d] or None: clean queries at positions clean_q_pos0 .. +Lq-1.
+    q_noisy [B, n_blocks*M, H, d] or None: packed blocks; k_noisy/v_noisy [B, n_blocks*M, Hkv, d].
+    k_clean/v_clean [B, Lk, Hkv, d]: every clean key, by position.
+    Returns a dict: o_clean, lse_clean, o_noisy, lse_noisy (present when that q is given) and,
+    with gradients, dq_clean, dq_noisy, dk_clean, dv_clean (this call's contribution for every
+    clean key: Algorithm 2 reduce-scatters exactly these), dk_noisy, dv_noisy."""
+    M = block_size
+    B, Lk, Hkv, d = k_clean.shape
+    Ln = k_noisy.shape[1]
+    assert Ln % M == 0
+    nb = Ln // M
+    if scale is None:
+        scale = 1.0 / np.sqrt(d)
+    qs = [q_clean, q_noisy]
+    dos = [do_clean, do_noisy]
+    names = ["clean", "noisy"]
+    out = {}
+    want_grad = do_clean is not None or do_noisy is not None
+    if want_grad:
+        dk2 = np.zeros((B, Lk + Ln, Hkv, d))
+        dv2 = np.zeros((B, Lk + Ln, Hkv, d))
+    for stream in (CLEAN, NOISY):
+        q = qs[stream]
+        if q is None:
+            continue
+        _, Lq, H, _ = q.shape
+        G = H // Hkv
+        o = np.zeros((B, Lq, H, d))
+        lse = np.zeros((B, H, Lq))
+        dq = np.zeros((B, Lq, H, d)) if dos[stream] is not None else None
+        for b in range(B):
+            for h in range(H):
+                hk = h // G
+                k2 = np.concatenate([k_clean[b, :, hk], k_noisy[b, :, hk]], axis=0)
+                v2 = np.concatenate([v_clean[b, :, hk], v_noisy[b, :, hk]], axis=0)
+                for r0 in range(0, Lq, row_chunk):
+                    rows = np.arange(r0, min(Lq, r0 + row_chunk))
+                    vis = visible_rows_packed(stream, rows, Lk, M, nb, block_prefix, clean_q_pos0,
+                                              clean_mask_mode, kv_begin, kv_end, include_noisy_diag, window)
+                    qq = q[b, rows, h]
+                    oo, ll, p = _masked_attention(qq, k2, v2, vis, scale)
+                    o[b, rows, h] = oo
+                    lse[b, h, rows] = ll
+                    if dq is not None:
+                        gq, gk, gv = _masked_attention_grad(qq, k2, v2, p, dos[stream][b, rows, h], scale)
+                        dq[b, rows, h] = gq
+                        dk2[b, :, hk] += gk
+                        dv2[b, :, hk] += gv
+        out["o_" + names[stream]] = o
+        out["lse_" + names[stream]] = lse
+        if dq is not None:
+            out["dq_" + names[stream]] = dq
+    if want_grad:
+        out["dk_clean"], out["dk_noisy"] = dk2[:, :Lk], dk2[:, Lk:]
+        out["dv_clean"], out["dv_noisy"] = dv2[:, :Lk], dv2[:, Lk:]
+    return out
+
+
+def attn_rows_packed(stream, rows, q_rows, k_clean, v_clean, k_noisy, v_noisy, block_size,
+                     do_rows=None, block_prefix=None, clean_q_pos0=0, scale=None, clean_mask_mode=0,
+                     window=0, row_chunk=128):
+    """Packed form for selected query rows of one (batch, head): the counterpart of `attn_rows`.
+    k_clean/v_clean [Lk, d], k_noisy/v_noisy [n_blocks*M, d] are that head's KV head.  Returns `o`,
+    `lse` and, with do_rows, `dq` and the rows' contributions dk_clean/dv_clean [Lk, d],
+    dk_noisy/dv_noisy [n_blocks*M, d]."""
+    M = block_size
+    Lk, d = k_clean.shape
+    Ln = k_noisy.shape[0]
+    nb = Ln // M
+    if scale is None:
+        scale = 1.0 / np.sqrt(d)
+    rows = np.asarray(rows, dtype=np.int64)
+    n = rows.shape[0]
+    out = {"o": np.zeros((n, d)), "lse": np.zeros(n)}
+    want_grad = do_rows is not None
+    if want_grad:
+        out["dq"] = np.zeros((n, d))
+        dk2 = np.zeros((Lk + Ln, d))
+        dv2 = np.zeros((Lk + Ln, d))
+    order = np.argsort(rows, kind="stable")
+    for c0 in range(0, n, row_chunk):
+        sel = order[c0:c0 + row_chunk]
+        vis = visible_rows_packed(stream, rows[sel], Lk, M, nb, block_prefix, clean_q_pos0,
+                                  clean_mask_mode, window=window)
+        cols = np.nonzero(vis.any(axis=0))[0]
+        kc = np.concatenate([k_clean[cols[cols < Lk]], k_noisy[cols[cols >= Lk] - Lk]], axis=0)
+        vc = np.concatenate([v_clean[cols[cols < Lk]], v_noisy[cols[cols >= Lk] - Lk]], axis=0)
+        oo, ll, p = _masked_attention(q_rows[sel], kc, vc, vis[:, cols], scale)
+        out["o"][sel] = oo
+        out["lse"][sel] = ll
+        if want_grad:
+            gq, gk, gv = _masked_attention_grad(q_rows[sel], kc, vc, p, do_rows[sel], scale)
+            out["dq"][sel] = gq
+            dk2[cols] += gk
+            dv2[cols] += gv
+    if want_grad:
+        out["dk_clean"], out["dk_noisy"] = dk2[:Lk], dk2[Lk:]
+        out["dv_clean"], out["dv_noisy"] = dv2[:Lk], dv2[Lk:]
+    return out
