@@ -127,6 +127,16 @@ def oracle_sample(w, inp_cpu, rows_per_stream, seed):
     rng = np.random.default_rng(seed)
     flops = 0
     t0 = time.perf_counter()
+    if w.packed:   # DFlash2-style blocks: noisy queries only, per-block prefix table
+        anchors = w.anchors()
+        Ln = w.n_blocks * M
+        rows = np.sort(rng.choice(Ln, size=min(2 * rows_per_stream, Ln), replace=False))
+        q_rows = synth.to_f64(inp_cpu["q_noisy"][0, rows, 0])
+        do_rows = synth.to_f64(inp_cpu["do_noisy"][0, rows, 0])
+        orc.attn_rows_packed(1, rows, q_rows, kv["k_clean"], kv["v_clean"], kv["k_noisy"], kv["v_noisy"], M,
+                             do_rows=do_rows, block_prefix=anchors)
+        flops = 14 * w.d * int((M + anchors[rows // M]).sum())
+        return time.perf_counter() - t0, flops
     for s, (qn, dn) in enumerate((("q_clean", "do_clean"), ("q_noisy", "do_noisy"))):
         rows = np.sort(rng.choice(w.L, size=min(rows_per_stream, w.L), replace=False))
         q_rows = synth.to_f64(inp_cpu[qn][0, rows, 0])
@@ -190,7 +200,7 @@ def run_reference(args, w):
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_tot / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
             "data": "synthetic", "config": {"workload": w.name, "batch": w.batch, "H": w.H, "H_kv": w.H_kv,
-                                            "d": w.d, "L": w.L, "block_size": w.block_size, "window": w.window},
+                                            "d": w.d, "L": w.L, "block_size": w.block_size, "window": w.window, "n_blocks": w.n_blocks},
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -234,22 +244,49 @@ def run_ours(args, w):
     peaks = load_peaks()
     M = w.block_size
     g = synth.make_inputs(synth.small(w, seed=w.seed + rank), "cuda")
-    p = binding.make_params(w.batch, w.L, M, w.H, w.H_kv, w.d)
-    ws = torch.empty(max(16, binding.bdlm_workspace_bytes(p, binding.BDLM_WS_BWD)), dtype=torch.uint8, device="cuda")
-    fwd_out = tuple(t for t in (torch.empty_like(g["q_clean"]),
-                                torch.empty(w.batch, w.H, w.L, dtype=torch.float32, device="cuda"),
-                                torch.empty_like(g["q_noisy"]),
-                                torch.empty(w.batch, w.H, w.L, dtype=torch.float32, device="cuda")))
-    grads = tuple(torch.empty_like(g[n]) for n in NAMES6)
     impl = args.kernel_impl
 
+    def like(t):
+        return None if t is None else torch.empty_like(t)
+
+    def lse_like(q):
+        return None if q is None else torch.empty(w.batch, w.H, q.shape[1], dtype=torch.float32, device="cuda")
+
+    def make_buffers(gg):
+        """Outputs, gradients and workspace of one step for the inputs `gg`."""
+        fo = (like(gg["q_clean"]), lse_like(gg["q_clean"]), like(gg["q_noisy"]), lse_like(gg["q_noisy"]))
+        gr = tuple(like(gg[n]) for n in NAMES6)
+        rows = max(t.shape[1] for t in (gg["q_clean"], gg["q_noisy"]) if t is not None)
+        wsz = 2 * (w.batch * w.H * rows * 4 + 256)
+        if not w.packed:
+            wsz = max(wsz, binding.bdlm_workspace_bytes(binding.make_params(w.batch, w.L, M, w.H, w.H_kv, w.d),
+                                                        binding.BDLM_WS_BWD))
+        return fo, gr, torch.empty(wsz, dtype=torch.uint8, device="cuda")
+
+    def run_fwd(gg, fo):
+        if w.packed:
+            binding.bdlm_attn_fwd_packed(*[gg[n] for n in NAMES6], M, block_prefix=gg["block_prefix"], out=fo,
+                                         impl=impl, window=w.window)
+        else:
+            binding.bdlm_attn_fwd(*[gg[n] for n in NAMES6], M, out=fo, impl=impl, window=w.window)
+
+    def run_bwd(gg, fo, gr, wsb, passes=0):
+        if w.packed:
+            binding.bdlm_attn_bwd_packed(*[gg[n] for n in NAMES6], fo[0], fo[1], fo[2], fo[3], gg["do_clean"],
+                                         gg["do_noisy"], M, block_prefix=gg["block_prefix"], out=gr, workspace=wsb,
+                                         impl=impl, passes=passes, window=w.window)
+        else:
+            binding.bdlm_attn_bwd(*[gg[n] for n in NAMES6], fo[0], fo[1], fo[2], fo[3], gg["do_clean"],
+                                  gg["do_noisy"], M, out=gr, workspace=wsb, impl=impl, passes=passes,
+                                  window=w.window)
+
+    fwd_out, grads, ws = make_buffers(g)
+
     def fwd():
-        binding.bdlm_attn_fwd(*[g[n] for n in NAMES6], M, out=fwd_out, impl=impl, window=w.window)
+        run_fwd(g, fwd_out)
 
     def bwd(passes=0):
-        binding.bdlm_attn_bwd(*[g[n] for n in NAMES6], fwd_out[0], fwd_out[1], fwd_out[2], fwd_out[3],
-                              g["do_clean"], g["do_noisy"], M, out=grads, workspace=ws, impl=impl, passes=passes,
-                              window=w.window)
+        run_bwd(g, fwd_out, grads, ws, passes)
 
     for _ in range(args.warmup):
         fwd()
@@ -295,19 +332,18 @@ def run_ours(args, w):
     # ---- end to end through the public call with HOST buffers (pinned), copies inside ---------
     e2e = None
     if rank == 0 or world > 1:
-        host_in = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True).copy_(v) for k, v in g.items()}
-        host_out = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in fwd_out + grads]
+        host_in = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True).copy_(v) for k, v in g.items()
+                   if v is not None}
+        host_out = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in fwd_out + grads if t is not None]
         h2d = sum(t.numel() * t.element_size() for t in host_in.values())
         d2h = sum(t.numel() * t.element_size() for t in host_out)
 
         # Three streams and two sets of device buffers: the copies of step k+1 (host to device) and of step
         # k-1 (device to host) run under the kernels of step k.  Every step still copies all of its inputs in
         # and all of its results out inside the timed region; pipeline fill and drain are part of it too.
-        sets = [{"g": g, "fwd": fwd_out, "grads": grads, "ws": ws}]
-        sets.append({"g": {k_: torch.empty_like(v) for k_, v in g.items()},
-                     "fwd": tuple(torch.empty_like(t) for t in fwd_out),
-                     "grads": tuple(torch.empty_like(t) for t in grads),
-                     "ws": torch.empty_like(ws)})
+        g2 = {k_: like(v) for k_, v in g.items()}
+        fo2, gr2, ws2 = make_buffers(g2)
+        sets = [{"g": g, "fwd": fwd_out, "grads": grads, "ws": ws}, {"g": g2, "fwd": fo2, "grads": gr2, "ws": ws2}]
         s_comp = torch.cuda.current_stream()
         s_h2d, s_d2h = torch.cuda.Stream(), torch.cuda.Stream()
 
@@ -325,17 +361,14 @@ def run_ours(args, w):
                 s_comp.wait_event(h2d_done)
                 if k >= 2:
                     s_comp.wait_event(d2h_done[k - 2])          # the set's outputs have been read out
-                gg, fo = st["g"], st["fwd"]
-                binding.bdlm_attn_fwd(*[gg[n_] for n_ in NAMES6], M, out=fo, impl=impl, window=w.window)
-                binding.bdlm_attn_bwd(*[gg[n_] for n_ in NAMES6], fo[0], fo[1], fo[2], fo[3], gg["do_clean"],
-                                      gg["do_noisy"], M, out=st["grads"], workspace=st["ws"], impl=impl,
-                                      window=w.window)
+                run_fwd(st["g"], st["fwd"])
+                run_bwd(st["g"], st["fwd"], st["grads"], st["ws"])
                 ev_c = torch.cuda.Event()
                 ev_c.record(s_comp)
                 comp_done.append(ev_c)
                 with torch.cuda.stream(s_d2h):
                     s_d2h.wait_event(ev_c)
-                    for dst, src in zip(host_out, st["fwd"] + st["grads"]):
+                    for dst, src in zip(host_out, [t for t in st["fwd"] + st["grads"] if t is not None]):
                         dst.copy_(src, non_blocking=True)
                     ev_d = torch.cuda.Event()
                     ev_d.record(s_d2h)
@@ -393,7 +426,7 @@ def run_ours(args, w):
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": w.name, "batch": w.batch, "H": w.H, "H_kv": w.H_kv, "d": w.d, "L": w.L,
-                       "block_size": w.block_size, "window": w.window, "rope_theta": w.rope_theta, "parallelism": "replicas only",
+                       "block_size": w.block_size, "window": w.window, "n_blocks": w.n_blocks, "rope_theta": w.rope_theta, "parallelism": "replicas only",
                        "l2": "inputs larger than L2 (q/k/v/dO of one step exceed 126 MB)",
                        "kernel_impl": {0: "auto", 1: "portable", 2: "tcgen05"}[impl]},
             "pct_of_bf16_peak": {"measured_burst": 100 * value / world / peaks["bf16_tflops"],

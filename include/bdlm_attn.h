@@ -126,6 +126,59 @@ int bdlm_lse_merge(int32_t n_partials, int32_t batch, int32_t L, int32_t H, int3
                    int32_t partial_dtype,
                    void* o_out, float* lse_out, void* cuda_stream);
 
+/*
+ * Packed form: what one rank of the CSBP schedule launches (Algorithm 1 and Algorithm 2 of the paper), and
+ * DFlash2-style blocks (appendix E, Eq. dflash2-block-attention).
+ *
+ *   - Clean K/V are complete and addressed by position: k_clean, v_clean, dk_clean, dv_clean are
+ *     [batch, L, H_kv, d] with L = p->L (L need not be a multiple of block_size here).
+ *   - Clean queries are one run of consecutive positions: q_clean, o_clean, do_clean, dq_clean are
+ *     [batch, Lq_clean, H, d], lse_clean [batch, H, Lq_clean]; row i is the clean token at position
+ *     clean_q_pos0 + i and sees clean keys 0 .. clean_q_pos0 + i (one piece of the rank's context shard).
+ *   - Corrupted blocks are packed one after the other: every noisy tensor has n_blocks * block_size rows
+ *     (queries [batch, n_blocks*block_size, H, d], K/V [batch, n_blocks*block_size, H_kv, d], lse_noisy
+ *     [batch, H, n_blocks*block_size]).  Packed block b sees its own block_size noisy keys (bidirectional) and
+ *     the clean keys at positions j < block_prefix[b]: block_prefix[b] = (block index) * block_size for a
+ *     block of the BDLM layer, the anchor position a_b for a DFlash2 block.  block_prefix is a DEVICE array
+ *     of n_blocks int32 shared by all batch elements; it must be non-decreasing (sort the blocks); NULL means
+ *     b * block_size.  Row i of packed block b stands at position block_prefix[b] + i for the sliding
+ *     window; with window > 0 the blocks must not overlap in position (block_prefix[b+1] >= block_prefix[b]
+ *     + block_size).  Values are not validated by the library (it never reads device memory on the host).
+ *   - A query stream is left out by passing its q pointer as NULL; in the backward every tensor of that
+ *     stream (for the noisy stream also K/V and dK/dV) may then be NULL.
+ *   - Backward: dq_* and dk_noisy/dv_noisy are complete for the rows of this call; dk_clean/dv_clean
+ *     [batch, L, H_kv, d] are THIS CALL'S contribution for every clean key (overwritten, zero where no query
+ *     of the call sees the key): the reduce-scatter of Algorithm 2 adds them over the ranks' calls.
+ *   - Everything else (checks, statuses, layouts, stream semantics, reproducibility) is as for
+ *     bdlm_attn_fwd / bdlm_attn_bwd; kv_begin/kv_end select a clean shard in the forward; bwd_single_pass is
+ *     ignored.  Workspace of the backward: bdlm_workspace_bytes_packed(p, g, BDLM_WS_BWD).
+ */
+typedef struct {
+  int32_t Lq_clean;             /* rows of the clean query tensors (ignored when q_clean is NULL) */
+  int32_t clean_q_pos0;         /* position of clean query row 0; clean_q_pos0 + Lq_clean <= L */
+  int32_t n_blocks;             /* packed corrupted blocks (ignored when q_noisy is NULL) */
+  int32_t reserved;
+  const int32_t* block_prefix;  /* device, [n_blocks], non-decreasing; NULL = b * block_size */
+} bdlm_packed_geometry;
+
+size_t bdlm_workspace_bytes_packed(const bdlm_params* p, const bdlm_packed_geometry* g, int32_t which);
+
+int bdlm_attn_fwd_packed(const bdlm_params* p, const bdlm_packed_geometry* g,
+                         const void* q_clean, const void* k_clean, const void* v_clean,
+                         const void* q_noisy, const void* k_noisy, const void* v_noisy,
+                         void* o_clean, void* o_noisy, float* lse_clean, float* lse_noisy,
+                         void* cuda_stream);
+
+int bdlm_attn_bwd_packed(const bdlm_params* p, const bdlm_packed_geometry* g,
+                         const void* q_clean, const void* k_clean, const void* v_clean,
+                         const void* q_noisy, const void* k_noisy, const void* v_noisy,
+                         const void* o_clean, const void* o_noisy,
+                         const float* lse_clean, const float* lse_noisy,
+                         const void* do_clean, const void* do_noisy,
+                         void* dq_clean, void* dk_clean, void* dv_clean,
+                         void* dq_noisy, void* dk_noisy, void* dv_noisy,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Human-readable name of a status code (static storage). */
 const char* bdlm_status_string(int status);
 

@@ -20,7 +20,8 @@ PASS_DSUM, PASS_DKDV, PASS_DQ = 1, 2, 4
 
 EXPORTS = ("bdlm_workspace_bytes", "bdlm_attn_fwd", "bdlm_attn_bwd", "bdlm_lse_merge",
            "bdlm_status_string", "bdlm_get_device_status", "bdlm_set_trace_buffer",
-           "bdlm_attn_bwd_static_scratch")
+           "bdlm_attn_bwd_static_scratch", "bdlm_workspace_bytes_packed", "bdlm_attn_fwd_packed",
+           "bdlm_attn_bwd_packed")
 STATIC_SCRATCH_ROWS = 1 << 20
 TRACE_SLOTS = 256
 
@@ -39,6 +40,11 @@ class BdlmParams(ctypes.Structure):
                 ("kv_range_set", ctypes.c_int32), ("include_noisy_diag", ctypes.c_int32),
                 ("impl", ctypes.c_int32), ("bwd_passes", ctypes.c_int32), ("bwd_single_pass", ctypes.c_int32),
                 ("window", ctypes.c_int32), ("reserved", ctypes.c_int32 * 2)]
+
+
+class BdlmPackedGeometry(ctypes.Structure):
+    _fields_ = [("Lq_clean", ctypes.c_int32), ("clean_q_pos0", ctypes.c_int32), ("n_blocks", ctypes.c_int32),
+                ("reserved", ctypes.c_int32), ("block_prefix", ctypes.c_void_p)]
 
 
 _lib = None
@@ -70,6 +76,13 @@ def lib():
         L.bdlm_attn_bwd_static_scratch.argtypes = [pp] + [vp] * 18 + [vp]
         L.bdlm_set_trace_buffer.restype = ctypes.c_int
         L.bdlm_set_trace_buffer.argtypes = [vp, ctypes.c_size_t]
+        gp = ctypes.POINTER(BdlmPackedGeometry)
+        L.bdlm_workspace_bytes_packed.restype = ctypes.c_size_t
+        L.bdlm_workspace_bytes_packed.argtypes = [pp, gp, ctypes.c_int32]
+        L.bdlm_attn_fwd_packed.restype = ctypes.c_int
+        L.bdlm_attn_fwd_packed.argtypes = [pp, gp] + [vp] * 10 + [vp]
+        L.bdlm_attn_bwd_packed.restype = ctypes.c_int
+        L.bdlm_attn_bwd_packed.argtypes = [pp, gp] + [vp] * 18 + [vp, ctypes.c_size_t, vp]
         _lib = L
     return _lib
 
@@ -181,6 +194,90 @@ def bdlm_attn_bwd_static_scratch(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_
         _ptr(dq_c), _ptr(dk_c), _ptr(dv_c), _ptr(dq_n), _ptr(dk_n), _ptr(dv_n), _stream())
     if rc != 0:
         raise BdlmError(rc, "bdlm_attn_bwd_static_scratch")
+    return out
+
+
+def _packed_setup(q_clean, k_clean, q_noisy, block_size, block_prefix, clean_q_pos0, window, **kw):
+    """Parameters and geometry of a packed call.  `block_prefix` is an int32 CUDA tensor [n_blocks] (or None
+    for b * block_size); its ordering rules are checked here on a host copy because the C library never reads
+    device memory on the host."""
+    batch, L, H_kv, d = k_clean.shape
+    qref = q_clean if q_clean is not None else q_noisy
+    H = qref.shape[2]
+    p = make_params(batch, L, block_size, H, H_kv, d, window=window, **kw)
+    g = BdlmPackedGeometry()
+    g.Lq_clean = 0 if q_clean is None else q_clean.shape[1]
+    g.clean_q_pos0 = int(clean_q_pos0)
+    g.n_blocks = 0
+    g.block_prefix = None
+    if q_noisy is not None:
+        if q_noisy.shape[1] % block_size != 0:
+            raise ValueError("packed noisy rows must be a whole number of blocks")
+        g.n_blocks = q_noisy.shape[1] // block_size
+        if block_prefix is not None:
+            assert block_prefix.is_cuda and block_prefix.dtype == torch.int32 and block_prefix.is_contiguous()
+            if block_prefix.numel() != g.n_blocks:
+                raise ValueError("block_prefix needs one entry per packed block")
+            host = block_prefix.cpu()
+            step = host[1:] - host[:-1]
+            if host.numel() and (int(host.min()) < 0 or int(host.max()) > L):
+                raise ValueError("block_prefix entries must lie in [0, L]")
+            if step.numel() and int(step.min()) < 0:
+                raise ValueError("block_prefix must be non-decreasing (sort the packed blocks)")
+            if window > 0 and step.numel() and int(step.min()) < block_size:
+                raise ValueError("with a sliding window the packed blocks must not overlap in position")
+            g.block_prefix = block_prefix.data_ptr()
+    return p, g
+
+
+def bdlm_attn_fwd_packed(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, block_size, *,
+                         block_prefix=None, clean_q_pos0=0, out=None, scale=0.0, clean_mask_mode=0,
+                         kv_range=None, include_noisy_diag=True, impl=IMPL_AUTO, window=0):
+    """Forward of the packed form (one rank's launch of the CSBP schedule; DFlash2-style blocks).
+    q_clean [batch, Lq, H, d] or None: clean queries at positions clean_q_pos0 .. ; q_noisy
+    [batch, n_blocks*block_size, H, d] or None with k_noisy/v_noisy packed alike; k_clean/v_clean
+    [batch, L, H_kv, d] complete.  Returns (o_clean, lse_clean, o_noisy, lse_noisy)."""
+    p, g = _packed_setup(q_clean, k_clean, q_noisy, block_size, block_prefix, clean_q_pos0, window, scale=scale,
+                         clean_mask_mode=clean_mask_mode, kv_range=kv_range,
+                         include_noisy_diag=include_noisy_diag, impl=impl)
+    dev = k_clean.device
+    if out is None:
+        mk_o = lambda q: None if q is None else torch.empty_like(q)
+        mk_l = lambda q: None if q is None else torch.empty(p.batch, p.H, q.shape[1], dtype=torch.float32, device=dev)
+        out = (mk_o(q_clean), mk_l(q_clean), mk_o(q_noisy), mk_l(q_noisy))
+    o_c, l_c, o_n, l_n = out
+    rc = lib().bdlm_attn_fwd_packed(ctypes.byref(p), ctypes.byref(g), _ptr(q_clean), _ptr(k_clean), _ptr(v_clean),
+                                    _ptr(q_noisy), _ptr(k_noisy), _ptr(v_noisy),
+                                    _ptr(o_c), _ptr(o_n), _ptr(l_c), _ptr(l_n), _stream())
+    if rc != 0:
+        raise BdlmError(rc, "bdlm_attn_fwd_packed")
+    return o_c, l_c, o_n, l_n
+
+
+def bdlm_attn_bwd_packed(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, o_clean, lse_clean,
+                         o_noisy, lse_noisy, do_clean, do_noisy, block_size, *, block_prefix=None,
+                         clean_q_pos0=0, out=None, workspace=None, scale=0.0, clean_mask_mode=0,
+                         impl=IMPL_AUTO, passes=0, window=0):
+    """Backward of the packed form.  Returns (dq_clean, dk_clean, dv_clean, dq_noisy, dk_noisy, dv_noisy);
+    entries of a stream that was left out are None.  dk_clean/dv_clean are this call's contribution for
+    every clean key."""
+    p, g = _packed_setup(q_clean, k_clean, q_noisy, block_size, block_prefix, clean_q_pos0, window, scale=scale,
+                         clean_mask_mode=clean_mask_mode, impl=impl, bwd_passes=passes)
+    if out is None:
+        e = lambda t: None if t is None else torch.empty_like(t)
+        out = (e(q_clean), torch.empty_like(k_clean), torch.empty_like(v_clean), e(q_noisy),
+               e(k_noisy if q_noisy is not None else None), e(v_noisy if q_noisy is not None else None))
+    need = int(lib().bdlm_workspace_bytes_packed(ctypes.byref(p), ctypes.byref(g), BDLM_WS_BWD))
+    if workspace is None:
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=k_clean.device)
+    dq_c, dk_c, dv_c, dq_n, dk_n, dv_n = out
+    rc = lib().bdlm_attn_bwd_packed(ctypes.byref(p), ctypes.byref(g), _ptr(q_clean), _ptr(k_clean), _ptr(v_clean),
+                                    _ptr(q_noisy), _ptr(k_noisy), _ptr(v_noisy), _ptr(o_clean), _ptr(o_noisy),
+                                    _ptr(lse_clean), _ptr(lse_noisy), _ptr(do_clean), _ptr(do_noisy),
+                                    _ptr(dq_c), _ptr(dk_c), _ptr(dv_c), _ptr(dq_n), _ptr(dk_n), _ptr(dv_n),
+                                    _ptr(workspace), workspace.numel(), _stream())
+    if rc != 0:
+        raise BdlmError(rc, "bdlm_attn_bwd_packed")
     return out
 
 

@@ -14,10 +14,18 @@ unsigned long long* g_trace = nullptr;   // host-side copy of the trace buffer p
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-int check_params(const bdlm_params* p) {
+int check_params(const bdlm_params* p, const bdlm_packed_geometry* g = nullptr) {
   if (p == nullptr) return BDLM_ERR_INVALID_ARG;
   if (p->batch <= 0 || p->L <= 0 || p->block_size <= 0 || p->H <= 0 || p->H_kv <= 0) return BDLM_ERR_INVALID_ARG;
-  if (p->H % p->H_kv != 0 || p->L % p->block_size != 0) return BDLM_ERR_INVALID_ARG;
+  if (p->H % p->H_kv != 0) return BDLM_ERR_INVALID_ARG;
+  if (g == nullptr) {
+    if (p->L % p->block_size != 0) return BDLM_ERR_INVALID_ARG;
+  } else {
+    if (g->Lq_clean < 0 || g->clean_q_pos0 < 0 || g->n_blocks < 0) return BDLM_ERR_INVALID_ARG;
+    if ((int64_t)g->clean_q_pos0 + g->Lq_clean > p->L) return BDLM_ERR_INVALID_ARG;
+    if ((int64_t)g->n_blocks * p->block_size > (int64_t)1 << 30) return BDLM_ERR_INVALID_ARG;
+    if (g->block_prefix != nullptr && (reinterpret_cast<uintptr_t>(g->block_prefix) & 3u)) return BDLM_ERR_INVALID_ARG;
+  }
   if (p->clean_mask_mode != 0 && p->clean_mask_mode != 1) return BDLM_ERR_INVALID_ARG;
   if (p->impl < 0 || p->impl > 2) return BDLM_ERR_INVALID_ARG;
   if (p->bwd_passes < 0 || p->bwd_passes > 7) return BDLM_ERR_INVALID_ARG;
@@ -32,9 +40,15 @@ int check_params(const bdlm_params* p) {
   return BDLM_OK;
 }
 
-void fill(KArgs& a, const bdlm_params* p) {
+void fill(KArgs& a, const bdlm_params* p, const bdlm_packed_geometry* g) {
   a.batch = p->batch; a.L = p->L; a.M = p->block_size; a.H = p->H; a.Hkv = p->H_kv;
   a.G = p->H / p->H_kv; a.d = p->d;
+  if (g == nullptr) {
+    a.Lqc = p->L; a.cq_pos0 = 0; a.Ln = p->L; a.nb = p->L / p->block_size; a.prefix = nullptr;
+  } else {
+    a.Lqc = g->Lq_clean; a.cq_pos0 = g->clean_q_pos0; a.nb = g->n_blocks; a.Ln = g->n_blocks * p->block_size;
+    a.prefix = g->block_prefix;
+  }
   a.scale = p->scale > 0.f ? p->scale : 1.0f / sqrtf((float)p->d);
   a.scale_log2 = a.scale * LOG2E;
   a.mode = p->clean_mask_mode;
@@ -58,8 +72,10 @@ bool is_sm100() {
   return major == 10;
 }
 
-size_t dsum_bytes(const bdlm_params* p) {
-  size_t one = (size_t)p->batch * p->H * p->L * sizeof(float);
+size_t dsum_bytes(const bdlm_params* p, const bdlm_packed_geometry* g = nullptr) {
+  const size_t rows = g == nullptr ? (size_t)p->L
+                                   : (size_t)(g->Lq_clean > g->n_blocks * p->block_size ? g->Lq_clean : g->n_blocks * p->block_size);
+  size_t one = (size_t)p->batch * p->H * (rows > 0 ? rows : 1) * sizeof(float);
   return (one + 255) / 256 * 256;
 }
 
@@ -83,14 +99,13 @@ size_t bdlm_workspace_bytes(const bdlm_params* p, int32_t which) {
   return 0;
 }
 
-int bdlm_attn_fwd(const bdlm_params* p,
-                  const void* q_clean, const void* k_clean, const void* v_clean,
-                  const void* q_noisy, const void* k_noisy, const void* v_noisy,
-                  void* o_clean, void* o_noisy, float* lse_clean, float* lse_noisy,
-                  void* workspace, size_t workspace_bytes, void* cuda_stream) {
-  (void)workspace; (void)workspace_bytes;
-  int rc = check_params(p);
+static int fwd_impl(const bdlm_params* p, const bdlm_packed_geometry* g,
+                    const void* q_clean, const void* k_clean, const void* v_clean,
+                    const void* q_noisy, const void* k_noisy, const void* v_noisy,
+                    void* o_clean, void* o_noisy, float* lse_clean, float* lse_noisy, void* cuda_stream) {
+  int rc = check_params(p, g);
   if (rc != BDLM_OK) return rc;
+  if (g != nullptr && ((q_clean != nullptr && g->Lq_clean == 0) || (q_noisy != nullptr && g->n_blocks == 0))) return BDLM_ERR_INVALID_ARG;
   if (q_clean == nullptr && q_noisy == nullptr) return BDLM_ERR_INVALID_ARG;
   if (k_clean == nullptr || v_clean == nullptr) return BDLM_ERR_INVALID_ARG;
   if (q_clean != nullptr && (o_clean == nullptr || lse_clean == nullptr)) return BDLM_ERR_INVALID_ARG;
@@ -101,7 +116,7 @@ int bdlm_attn_fwd(const bdlm_params* p,
   if (!is_sm100()) return BDLM_ERR_UNSUPPORTED;
 
   KArgs a;
-  fill(a, p);
+  fill(a, p, g);
   using bf = __nv_bfloat16;
   a.q[CLEAN] = (const bf*)q_clean; a.q[NOISY] = (const bf*)q_noisy;
   a.k[CLEAN] = (const bf*)k_clean; a.k[NOISY] = (const bf*)(k_noisy ? k_noisy : k_clean);
@@ -118,6 +133,91 @@ int bdlm_attn_fwd(const bdlm_params* p,
   return e == cudaSuccess ? BDLM_OK : BDLM_ERR_CUDA;
 }
 
+static int bwd_impl(const bdlm_params* p, const bdlm_packed_geometry* g,
+                    const void* q_clean, const void* k_clean, const void* v_clean,
+                    const void* q_noisy, const void* k_noisy, const void* v_noisy,
+                    const void* o_clean, const void* o_noisy,
+                    const float* lse_clean, const float* lse_noisy,
+                    const void* do_clean, const void* do_noisy,
+                    void* dq_clean, void* dk_clean, void* dv_clean,
+                    void* dq_noisy, void* dk_noisy, void* dv_noisy,
+                    void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  int rc = check_params(p, g);
+  if (rc != BDLM_OK) return rc;
+  // the plain layer needs every tensor; a packed call may leave out one query stream with all that belongs to it
+  const bool has_c = (g == nullptr) || q_clean != nullptr;
+  const bool has_n = (g == nullptr) || q_noisy != nullptr;
+  if (!has_c && !has_n) return BDLM_ERR_INVALID_ARG;
+  if (g != nullptr && ((has_c && g->Lq_clean == 0) || (has_n && g->n_blocks == 0))) return BDLM_ERR_INVALID_ARG;
+  const void* always[] = {k_clean, v_clean, dk_clean, dv_clean, workspace};
+  for (const void* x : always) if (x == nullptr || !aligned16(x)) return BDLM_ERR_INVALID_ARG;
+  if (has_c) {
+    const void* need[] = {q_clean, o_clean, lse_clean, do_clean, dq_clean};
+    for (const void* x : need) if (x == nullptr || !aligned16(x)) return BDLM_ERR_INVALID_ARG;
+  }
+  if (has_n) {
+    const void* need[] = {q_noisy, k_noisy, v_noisy, o_noisy, lse_noisy, do_noisy, dq_noisy, dk_noisy, dv_noisy};
+    for (const void* x : need) if (x == nullptr || !aligned16(x)) return BDLM_ERR_INVALID_ARG;
+  }
+  if (p->kv_range_set && (p->kv_begin != 0 || p->kv_end != p->L)) return BDLM_ERR_UNSUPPORTED;
+  if (!p->include_noisy_diag) return BDLM_ERR_UNSUPPORTED;
+  const size_t need_ws = 2 * dsum_bytes(p, g) + (g == nullptr ? tc_bwd_extra_workspace(p) : 0);
+  if (workspace_bytes < need_ws) return BDLM_ERR_WORKSPACE_TOO_SMALL;
+  if (!is_sm100()) return BDLM_ERR_UNSUPPORTED;
+
+  KArgs a;
+  fill(a, p, g);
+  using bf = __nv_bfloat16;
+  a.q[CLEAN] = has_c ? (const bf*)q_clean : nullptr; a.q[NOISY] = has_n ? (const bf*)q_noisy : nullptr;
+  a.k[CLEAN] = (const bf*)k_clean; a.k[NOISY] = has_n ? (const bf*)k_noisy : nullptr;
+  a.v[CLEAN] = (const bf*)v_clean; a.v[NOISY] = has_n ? (const bf*)v_noisy : nullptr;
+  a.o[CLEAN] = (bf*)const_cast<void*>(o_clean); a.o[NOISY] = (bf*)const_cast<void*>(o_noisy);
+  a.lse[CLEAN] = const_cast<float*>(lse_clean); a.lse[NOISY] = const_cast<float*>(lse_noisy);
+  a.dout[CLEAN] = (const bf*)do_clean; a.dout[NOISY] = (const bf*)do_noisy;
+  float* ds_c = static_cast<float*>(workspace);
+  float* ds_n = reinterpret_cast<float*>(static_cast<char*>(workspace) + dsum_bytes(p, g));
+  a.dsum[CLEAN] = ds_c; a.dsum[NOISY] = ds_n;
+  a.dq[CLEAN] = (bf*)dq_clean; a.dq[NOISY] = (bf*)dq_noisy;
+  a.dk[CLEAN] = (bf*)dk_clean; a.dk[NOISY] = has_n ? (bf*)dk_noisy : nullptr;
+  a.dv[CLEAN] = (bf*)dv_clean; a.dv[NOISY] = has_n ? (bf*)dv_noisy : nullptr;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+
+  const bool tc_ok = tc_bwd_supported(a);
+  if (p->impl == 2 && !tc_ok) return BDLM_ERR_UNSUPPORTED;
+  a.single_pass = (p->bwd_single_pass && tc_ok && p->impl != 1 && g == nullptr) ? 1 : 0;
+  const int passes = p->bwd_passes ? p->bwd_passes : 7;
+  cudaError_t e = cudaSuccess;
+  if (passes & BDLM_BWD_PASS_DSUM) e = launch_dsum(a, ds_c, ds_n, st);
+  if (e != cudaSuccess) return BDLM_ERR_CUDA;
+  if (tc_ok && p->impl != 1) {
+    void* extra = static_cast<char*>(workspace) + 2 * dsum_bytes(p, g);
+    e = launch_tc_bwd(a, extra, passes, st);
+  } else {
+    e = launch_portable_bwd(a, passes, st);
+  }
+  return e == cudaSuccess ? BDLM_OK : BDLM_ERR_CUDA;
+}
+
+int bdlm_attn_fwd(const bdlm_params* p,
+                  const void* q_clean, const void* k_clean, const void* v_clean,
+                  const void* q_noisy, const void* k_noisy, const void* v_noisy,
+                  void* o_clean, void* o_noisy, float* lse_clean, float* lse_noisy,
+                  void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  (void)workspace; (void)workspace_bytes;
+  return fwd_impl(p, nullptr, q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, o_clean, o_noisy,
+                  lse_clean, lse_noisy, cuda_stream);
+}
+
+int bdlm_attn_fwd_packed(const bdlm_params* p, const bdlm_packed_geometry* g,
+                         const void* q_clean, const void* k_clean, const void* v_clean,
+                         const void* q_noisy, const void* k_noisy, const void* v_noisy,
+                         void* o_clean, void* o_noisy, float* lse_clean, float* lse_noisy,
+                         void* cuda_stream) {
+  if (g == nullptr) return BDLM_ERR_INVALID_ARG;
+  return fwd_impl(p, g, q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, o_clean, o_noisy,
+                  lse_clean, lse_noisy, cuda_stream);
+}
+
 int bdlm_attn_bwd(const bdlm_params* p,
                   const void* q_clean, const void* k_clean, const void* v_clean,
                   const void* q_noisy, const void* k_noisy, const void* v_noisy,
@@ -127,48 +227,30 @@ int bdlm_attn_bwd(const bdlm_params* p,
                   void* dq_clean, void* dk_clean, void* dv_clean,
                   void* dq_noisy, void* dk_noisy, void* dv_noisy,
                   void* workspace, size_t workspace_bytes, void* cuda_stream) {
-  int rc = check_params(p);
-  if (rc != BDLM_OK) return rc;
-  const void* ptrs[] = {q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, o_clean, o_noisy,
-                        lse_clean, lse_noisy, do_clean, do_noisy, dq_clean, dk_clean, dv_clean,
-                        dq_noisy, dk_noisy, dv_noisy, workspace};
-  for (const void* x : ptrs) if (x == nullptr || !aligned16(x)) return BDLM_ERR_INVALID_ARG;
-  if (p->kv_range_set && (p->kv_begin != 0 || p->kv_end != p->L)) return BDLM_ERR_UNSUPPORTED;
-  if (!p->include_noisy_diag) return BDLM_ERR_UNSUPPORTED;
-  if (workspace_bytes < bdlm_workspace_bytes(p, BDLM_WS_BWD)) return BDLM_ERR_WORKSPACE_TOO_SMALL;
-  if (!is_sm100()) return BDLM_ERR_UNSUPPORTED;
+  return bwd_impl(p, nullptr, q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, o_clean, o_noisy, lse_clean,
+                  lse_noisy, do_clean, do_noisy, dq_clean, dk_clean, dv_clean, dq_noisy, dk_noisy, dv_noisy,
+                  workspace, workspace_bytes, cuda_stream);
+}
 
-  KArgs a;
-  fill(a, p);
-  using bf = __nv_bfloat16;
-  a.q[CLEAN] = (const bf*)q_clean; a.q[NOISY] = (const bf*)q_noisy;
-  a.k[CLEAN] = (const bf*)k_clean; a.k[NOISY] = (const bf*)k_noisy;
-  a.v[CLEAN] = (const bf*)v_clean; a.v[NOISY] = (const bf*)v_noisy;
-  a.o[CLEAN] = (bf*)const_cast<void*>(o_clean); a.o[NOISY] = (bf*)const_cast<void*>(o_noisy);
-  a.lse[CLEAN] = const_cast<float*>(lse_clean); a.lse[NOISY] = const_cast<float*>(lse_noisy);
-  a.dout[CLEAN] = (const bf*)do_clean; a.dout[NOISY] = (const bf*)do_noisy;
-  float* ds_c = static_cast<float*>(workspace);
-  float* ds_n = reinterpret_cast<float*>(static_cast<char*>(workspace) + dsum_bytes(p));
-  a.dsum[CLEAN] = ds_c; a.dsum[NOISY] = ds_n;
-  a.dq[CLEAN] = (bf*)dq_clean; a.dq[NOISY] = (bf*)dq_noisy;
-  a.dk[CLEAN] = (bf*)dk_clean; a.dk[NOISY] = (bf*)dk_noisy;
-  a.dv[CLEAN] = (bf*)dv_clean; a.dv[NOISY] = (bf*)dv_noisy;
-  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+int bdlm_attn_bwd_packed(const bdlm_params* p, const bdlm_packed_geometry* g,
+                         const void* q_clean, const void* k_clean, const void* v_clean,
+                         const void* q_noisy, const void* k_noisy, const void* v_noisy,
+                         const void* o_clean, const void* o_noisy,
+                         const float* lse_clean, const float* lse_noisy,
+                         const void* do_clean, const void* do_noisy,
+                         void* dq_clean, void* dk_clean, void* dv_clean,
+                         void* dq_noisy, void* dk_noisy, void* dv_noisy,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (g == nullptr) return BDLM_ERR_INVALID_ARG;
+  return bwd_impl(p, g, q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, o_clean, o_noisy, lse_clean,
+                  lse_noisy, do_clean, do_noisy, dq_clean, dk_clean, dv_clean, dq_noisy, dk_noisy, dv_noisy,
+                  workspace, workspace_bytes, cuda_stream);
+}
 
-  const bool tc_ok = tc_bwd_supported(a);
-  if (p->impl == 2 && !tc_ok) return BDLM_ERR_UNSUPPORTED;
-  a.single_pass = (p->bwd_single_pass && tc_ok && p->impl != 1) ? 1 : 0;
-  const int passes = p->bwd_passes ? p->bwd_passes : 7;
-  cudaError_t e = cudaSuccess;
-  if (passes & BDLM_BWD_PASS_DSUM) e = launch_dsum(a, ds_c, ds_n, st);
-  if (e != cudaSuccess) return BDLM_ERR_CUDA;
-  if (tc_ok && p->impl != 1) {
-    void* extra = static_cast<char*>(workspace) + 2 * dsum_bytes(p);
-    e = launch_tc_bwd(a, extra, passes, st);
-  } else {
-    e = launch_portable_bwd(a, passes, st);
-  }
-  return e == cudaSuccess ? BDLM_OK : BDLM_ERR_CUDA;
+size_t bdlm_workspace_bytes_packed(const bdlm_params* p, const bdlm_packed_geometry* g, int32_t which) {
+  if (g == nullptr || check_params(p, g) != BDLM_OK) return 0;
+  if (which == BDLM_WS_BWD) return 2 * dsum_bytes(p, g);
+  return 0;
 }
 
 int bdlm_lse_merge(int32_t n_partials, int32_t batch, int32_t L, int32_t H, int32_t d,

@@ -14,8 +14,17 @@ constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
 
 // Kernel-side copy of the call: sizes, the resolved clean-key range, pointers per stream.
+//
+// Row counts.  L is the number of clean K/V rows (= clean token positions).  The clean query tensors
+// (q, o, dO, dQ, LSE, D) have Lqc rows standing at positions cq_pos0 .. cq_pos0 + Lqc - 1; every noisy
+// tensor (queries and keys) has Ln = nb * M rows, nb packed blocks.  The plain layer is Lqc = Ln = L,
+// cq_pos0 = 0, prefix = nullptr; one rank's launch of the CSBP schedule (Algorithms 1, 2) and
+// DFlash2-style blocks (appendix E) set them otherwise.
 struct KArgs {
   int batch, L, M, H, Hkv, G, d;
+  int Lqc, cq_pos0;   // clean query rows and the position of the first one
+  int Ln, nb;         // noisy rows (= nb * M) and packed blocks
+  const int* prefix;  // device [nb], non-decreasing: clean keys j < prefix[b] are visible to block b; nullptr = b * M
   float scale;        // q.k multiplier (1/sqrt(d) by default)
   float scale_log2;   // scale * log2(e): scores are exponentiated with exp2
   int mode;           // clean_mask_mode
@@ -29,38 +38,74 @@ struct KArgs {
   float* lse[2];
   // backward only
   const __nv_bfloat16* dout[2];
-  const float* dsum[2];   // D_i = sum_d dO*O, [batch, H, L]
+  const float* dsum[2];   // D_i = sum_d dO*O, [batch, H, rows of the stream's queries]
   __nv_bfloat16* dq[2];
   __nv_bfloat16* dk[2];
   __nv_bfloat16* dv[2];
   unsigned long long* trace;   // optional cycle counters (bdlm_set_trace_buffer), else nullptr
   int single_pass;             // backward: dQ accumulated in the dK/dV kernel through fp32 atomics
-  float* dq32[2];              // fp32 dQ accumulators [batch, L, H, d] (single-pass backward), else nullptr
+  float* dq32[2];              // fp32 dQ accumulators [batch, rows, H, d] (single-pass backward), else nullptr
 };
 
+__host__ __device__ __forceinline__ int rows_q(const KArgs& a, int qs) { return qs == CLEAN ? a.Lqc : a.Ln; }
+__host__ __device__ __forceinline__ int rows_k(const KArgs& a, int ks) { return ks == CLEAN ? a.L : a.Ln; }
+
+// Clean-prefix length of packed noisy block b.
+__device__ __forceinline__ int block_prefix(const KArgs& a, int b) {
+  return a.prefix != nullptr ? __ldg(a.prefix + b) : b * a.M;
+}
+// Smallest packed block index in [0, nb] whose prefix exceeds x (nb if none); the table is non-decreasing.
+__device__ __forceinline__ int first_block_prefix_gt(const KArgs& a, int x) {
+  if (a.prefix == nullptr) return min(a.nb, x < 0 ? 0 : x / a.M + 1);
+  int lo = 0, hi = a.nb;
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if (__ldg(a.prefix + mid) > x) hi = mid; else lo = mid + 1;
+  }
+  return lo;
+}
+
 // Visible key interval [lo, hi) of query row i (stream qs) inside key stream ks
-// (section 3.2: clean row -> clean keys 0..i; noisy row -> clean keys of earlier blocks and
-// the noisy keys of its own block).  Every row's visible set per key stream is one interval.
-__device__ __forceinline__ void visible_interval(int qs, int ks, int i, int M, int mode,
-                                                 int kv_begin, int kv_end, int diag,
-                                                 int& lo, int& hi, int window) {
-  // sliding-window layers: a clean key j is visible to position i only if i - j < window (0 = no window)
-  if (ks == CLEAN && window > 0) kv_begin = max(kv_begin, i - window + 1);
+// (section 3.2: clean row -> clean keys 0..position; noisy row -> the clean keys before its block's
+// prefix and the noisy keys of its own block).  Every row's visible set per key stream is one interval.
+// Sliding-window layers: a clean key j is visible to a token at position p only if p - j < window.
+__device__ __forceinline__ void visible_interval(const KArgs& a, int qs, int ks, int i, int& lo, int& hi) {
+  const int M = a.M;
+  if (ks == NOISY) {
+    if (qs == CLEAN || !a.diag) { lo = 0; hi = 0; }
+    else { lo = (i / M) * M; hi = lo + M; }
+    return;
+  }
+  int pos, lim;
   if (qs == CLEAN) {
-    if (ks == CLEAN) {
-      lo = kv_begin;
-      int lim = (mode == 0) ? (i + 1) : ((i / M + 1) * M);
-      hi = min(kv_end, lim);
-    } else {
-      lo = 0; hi = 0;
-    }
+    pos = a.cq_pos0 + i;
+    lim = (a.mode == 0) ? (pos + 1) : ((pos / M + 1) * M);
   } else {
-    if (ks == CLEAN) {
-      lo = kv_begin;
-      hi = min(kv_end, (i / M) * M);
-    } else {
-      lo = diag ? (i / M) * M : 0;
-      hi = diag ? lo + M : 0;
+    const int bi = i / M;
+    lim = block_prefix(a, bi);
+    pos = lim + (i - bi * M);
+  }
+  lo = a.kv_begin;
+  if (a.window > 0) lo = max(lo, pos - a.window + 1);
+  hi = min(a.kv_end, lim);
+}
+
+// Query rows [lo, hi) of stream qs (row indices of that stream's tensors) that see clean key j.
+// Needs token positions to be non-decreasing along the packed rows when a window is set.
+__device__ __forceinline__ void visible_queries_of_clean_key(const KArgs& a, int qs, int j, int& lo, int& hi) {
+  const int M = a.M, W = a.window;
+  if (qs == CLEAN) {
+    const int p_lo = (a.mode == 0) ? j : (j / M) * M;
+    lo = max(0, p_lo - a.cq_pos0);
+    hi = (W > 0) ? min(a.Lqc, j + W - a.cq_pos0) : a.Lqc;
+    hi = max(hi, 0);
+  } else {
+    lo = first_block_prefix_gt(a, j) * M;
+    hi = a.Ln;
+    if (W > 0) {
+      // first block that is not seen in full: prefix + M - 1 - j >= W
+      const int b1 = first_block_prefix_gt(a, j + W - M);
+      hi = (b1 >= a.nb) ? a.Ln : b1 * M + min(M, max(0, W + j - block_prefix(a, b1)));
     }
   }
 }

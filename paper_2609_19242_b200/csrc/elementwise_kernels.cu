@@ -127,14 +127,17 @@ cudaError_t launch_merge(int n, int batch, int L, int H, int d, const void* cons
 }
 
 cudaError_t launch_dsum(const KArgs& a, float* dsum_clean, float* dsum_noisy, cudaStream_t st) {
-  const int64_t nrows = (int64_t)a.batch * a.L * a.H;
-  const int blocks = (int)((nrows * 32 + 255) / 256);
   float* out[2] = {dsum_clean, dsum_noisy};
   for (int s = 0; s < 2; ++s) {
+    if (a.q[s] == nullptr) continue;   // a stream without queries has no D rows
+    const int rows = rows_q(a, s);
+    const int64_t nrows = (int64_t)a.batch * rows * a.H;
+    const int blocks = (int)((nrows * 32 + 255) / 256);
+    if (blocks == 0) continue;
     if (a.d == 128)
-      dsum_kernel<128><<<blocks, 256, 0, st>>>(a.dout[s], a.o[s], out[s], nrows, a.L, a.H);
+      dsum_kernel<128><<<blocks, 256, 0, st>>>(a.dout[s], a.o[s], out[s], nrows, rows, a.H);
     else
-      dsum_kernel<64><<<blocks, 256, 0, st>>>(a.dout[s], a.o[s], out[s], nrows, a.L, a.H);
+      dsum_kernel<64><<<blocks, 256, 0, st>>>(a.dout[s], a.o[s], out[s], nrows, rows, a.H);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }

@@ -70,7 +70,8 @@ __global__ void __launch_bounds__(NTHREADS) portable_fwd_kernel(const KArgs a) {
   bf16* Ks = reinterpret_cast<bf16*>(smem_raw);
   bf16* Vs = Ks + BK * LD;
 
-  const int L = a.L;
+  const int L = rows_q(a, qs);   // rows of this stream's query tensors
+  if (q0 >= L) return;
   const int r0 = q0 + warp * 16 + g, r1 = r0 + 8;
   const int64_t qld = (int64_t)a.H * D;
   const int64_t kld = (int64_t)a.Hkv * D;
@@ -93,14 +94,14 @@ __global__ void __launch_bounds__(NTHREADS) portable_fwd_kernel(const KArgs a) {
 
   for (int ks = 0; ks < 2; ++ks) {
     int seg_lo, seg_hi, tmp;
-    visible_interval(qs, ks, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, seg_lo, tmp, a.window);
-    visible_interval(qs, ks, last_row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, tmp, seg_hi, a.window);
+    visible_interval(a, qs, ks, q0, seg_lo, tmp);
+    visible_interval(a, qs, ks, last_row, tmp, seg_hi);
     if (seg_hi <= seg_lo) continue;
     int rlo0 = 0, rhi0 = 0, rlo1 = 0, rhi1 = 0;
-    if (r0 < L) visible_interval(qs, ks, r0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo0, rhi0, a.window);
-    if (r1 < L) visible_interval(qs, ks, r1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo1, rhi1, a.window);
-    const bf16* kbase = a.k[ks] + ((int64_t)b * L * a.Hkv + hk) * D;
-    const bf16* vbase = a.v[ks] + ((int64_t)b * L * a.Hkv + hk) * D;
+    if (r0 < L) visible_interval(a, qs, ks, r0, rlo0, rhi0);
+    if (r1 < L) visible_interval(a, qs, ks, r1, rlo1, rhi1);
+    const bf16* kbase = a.k[ks] + ((int64_t)b * rows_k(a, ks) * a.Hkv + hk) * D;
+    const bf16* vbase = a.v[ks] + ((int64_t)b * rows_k(a, ks) * a.Hkv + hk) * D;
 
     for (int k0 = seg_lo; k0 < seg_hi; k0 += BK) {
       __syncthreads();
@@ -207,7 +208,9 @@ __global__ void __launch_bounds__(NTHREADS) portable_dq_kernel(const KArgs a) {
   bf16* Ks = dOs + BQ * LD;
   bf16* Vs = Ks + BK * LD;
 
-  const int L = a.L;
+  if (a.q[qs] == nullptr) return;
+  const int L = rows_q(a, qs);   // rows of this stream's query tensors
+  if (q0 >= L) return;
   const int r0 = q0 + warp * 16 + g, r1 = r0 + 8;
   const int64_t qld = (int64_t)a.H * D;
   const int64_t kld = (int64_t)a.Hkv * D;
@@ -229,14 +232,14 @@ __global__ void __launch_bounds__(NTHREADS) portable_dq_kernel(const KArgs a) {
 
   for (int ks = 0; ks < 2; ++ks) {
     int seg_lo, seg_hi, tmp;
-    visible_interval(qs, ks, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, seg_lo, tmp, a.window);
-    visible_interval(qs, ks, last_row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, tmp, seg_hi, a.window);
+    visible_interval(a, qs, ks, q0, seg_lo, tmp);
+    visible_interval(a, qs, ks, last_row, tmp, seg_hi);
     if (seg_hi <= seg_lo) continue;
     int rlo0 = 0, rhi0 = 0, rlo1 = 0, rhi1 = 0;
-    if (r0 < L) visible_interval(qs, ks, r0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo0, rhi0, a.window);
-    if (r1 < L) visible_interval(qs, ks, r1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo1, rhi1, a.window);
-    const bf16* kbase = a.k[ks] + ((int64_t)b * L * a.Hkv + hk) * D;
-    const bf16* vbase = a.v[ks] + ((int64_t)b * L * a.Hkv + hk) * D;
+    if (r0 < L) visible_interval(a, qs, ks, r0, rlo0, rhi0);
+    if (r1 < L) visible_interval(a, qs, ks, r1, rlo1, rhi1);
+    const bf16* kbase = a.k[ks] + ((int64_t)b * rows_k(a, ks) * a.Hkv + hk) * D;
+    const bf16* vbase = a.v[ks] + ((int64_t)b * rows_k(a, ks) * a.Hkv + hk) * D;
 
     for (int k0 = seg_lo; k0 < seg_hi; k0 += BK) {
       __syncthreads();
@@ -321,7 +324,8 @@ __global__ void __launch_bounds__(NTHREADS) portable_dkdv_kernel(const KArgs a) 
   int* vlo_s = reinterpret_cast<int*>(d_s + BQ2);
   int* vhi_s = vlo_s + BQ2;
 
-  const int L = a.L, M = a.M;
+  const int L = rows_k(a, ks), M = a.M;   // rows of this stream's K/V tensors
+  if (k0 >= L || a.dk[ks] == nullptr) return;
   const int64_t qld = (int64_t)a.H * D;
   const int64_t kld = (int64_t)a.Hkv * D;
   const int64_t koff = ((int64_t)b * L * a.Hkv + hk) * D;
@@ -340,22 +344,23 @@ __global__ void __launch_bounds__(NTHREADS) portable_dkdv_kernel(const KArgs a) 
   for (int qs = 0; qs < 2; ++qs) {
     // query rows of stream qs that can see some key of this tile
     int q_lo, q_hi;
-    if (qs == CLEAN) {
-      if (ks == NOISY) continue;
-      q_lo = (a.mode == 0) ? k0 : (k0 / M) * M;
-      q_hi = (a.window > 0) ? min(L, k_last + a.window) : L;
-    } else if (ks == CLEAN) {
-      q_lo = (k0 / M + 1) * M;
-      q_hi = (a.window > 0) ? min(L, k_last + a.window) : L;
+    if (a.q[qs] == nullptr) continue;
+    if (ks == CLEAN) {
+      // the visible-query interval moves up with the key: first key's lower end, last key's upper end
+      int tmp;
+      visible_queries_of_clean_key(a, qs, k0, q_lo, tmp);
+      visible_queries_of_clean_key(a, qs, k_last, tmp, q_hi);
     } else {
+      if (qs == CLEAN) continue;
       q_lo = (k0 / M) * M;
       q_hi = min(L, (k_last / M + 1) * M);
     }
+    const int Lq = rows_q(a, qs);
     for (int hh = 0; hh < a.G; ++hh) {
       const int h = hk * a.G + hh;
-      const int64_t qoff = ((int64_t)b * L * a.H + h) * D;
-      const float* lsep = a.lse[qs] + ((int64_t)b * a.H + h) * L;
-      const float* dsp = a.dsum[qs] + ((int64_t)b * a.H + h) * L;
+      const int64_t qoff = ((int64_t)b * Lq * a.H + h) * D;
+      const float* lsep = a.lse[qs] + ((int64_t)b * a.H + h) * Lq;
+      const float* dsp = a.dsum[qs] + ((int64_t)b * a.H + h) * Lq;
       for (int qq = q_lo; qq < q_hi; qq += BQ2) {
         __syncthreads();
         load_tile<D, BQ2>(Qs, a.q[qs] + qoff + (int64_t)qq * qld, qld, q_hi - qq);
@@ -368,7 +373,7 @@ __global__ void __launch_bounds__(NTHREADS) portable_dkdv_kernel(const KArgs a) 
             float zz = lsep[i];
             z = isfinite(zz) ? zz * LOG2E : INFINITY;
             dd = dsp[i];
-            visible_interval(qs, ks, i, M, a.mode, a.kv_begin, a.kv_end, a.diag, lo, hi, a.window);
+            visible_interval(a, qs, ks, i, lo, hi);
           }
           lse_s[threadIdx.x] = z; d_s[threadIdx.x] = dd;
           vlo_s[threadIdx.x] = lo; vhi_s[threadIdx.x] = hi;
@@ -448,6 +453,10 @@ __global__ void __launch_bounds__(NTHREADS) portable_dkdv_kernel(const KArgs a) 
   }
 }
 
+int max_query_rows(const KArgs& a) {
+  return max(a.q[CLEAN] != nullptr ? a.Lqc : 0, a.q[NOISY] != nullptr ? a.Ln : 0);
+}
+
 template <typename K>
 cudaError_t set_smem(K kernel, size_t bytes) {
   return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
@@ -456,7 +465,7 @@ cudaError_t set_smem(K kernel, size_t bytes) {
 }  // namespace
 
 cudaError_t launch_portable_fwd(const KArgs& a, cudaStream_t st) {
-  dim3 grid((a.L + BQ - 1) / BQ, a.H, a.batch * 2);
+  dim3 grid((max_query_rows(a) + BQ - 1) / BQ, a.H, a.batch * 2);
   size_t smem = (size_t)2 * BK * (a.d + PAD) * sizeof(bf16);
   cudaError_t e;
   if (a.d == 128) {
@@ -472,7 +481,7 @@ cudaError_t launch_portable_fwd(const KArgs& a, cudaStream_t st) {
 cudaError_t launch_portable_bwd(const KArgs& a, int passes, cudaStream_t st) {
   cudaError_t e = cudaSuccess;
   if (passes & BDLM_BWD_PASS_DKDV) {
-    dim3 grid((a.L + BQ - 1) / BQ, a.Hkv, a.batch * 2);
+    dim3 grid((max(a.L, a.Ln) + BQ - 1) / BQ, a.Hkv, a.batch * 2);
     size_t smem = (size_t)(2 * BQ + 2 * BQ2) * (a.d + PAD) * sizeof(bf16) + 4 * BQ2 * sizeof(float);
     if (a.d == 128) {
       if ((e = set_smem(portable_dkdv_kernel<128>, smem)) != cudaSuccess) return e;
@@ -484,7 +493,7 @@ cudaError_t launch_portable_bwd(const KArgs& a, int passes, cudaStream_t st) {
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
   if (passes & BDLM_BWD_PASS_DQ) {
-    dim3 grid((a.L + BQ - 1) / BQ, a.H, a.batch * 2);
+    dim3 grid((max_query_rows(a) + BQ - 1) / BQ, a.H, a.batch * 2);
     size_t smem = (size_t)(2 * BQ + 2 * BK) * (a.d + PAD) * sizeof(bf16);
     if (a.d == 128) {
       if ((e = set_smem(portable_dq_kernel<128>, smem)) != cudaSuccess) return e;

@@ -99,17 +99,25 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
   const int ks = blockIdx.z & 1, b = blockIdx.z >> 1, hk = blockIdx.y;
   const int k0 = blockIdx.x * TILE;   // key tile 0 has the most query tiles: scheduled first
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int L = a.L, M = a.M, NT = L / TILE;
+  const int L = rows_k(a, ks), M = a.M;   // rows of this stream's K/V tensors
+  if (k0 >= L || a.dk[ks] == nullptr) return;
 
-  // query tiles that see this key tile: segment A then segment B, for each head of the group
-  int tA0, nA, tB0 = 0, nB = 0;
+  // query tiles that see this key tile: segment A (clean queries; noisy ones for a noisy key tile), then
+  // segment B (noisy queries of a clean key tile), for each head of the group.  The visible-query interval of
+  // a key moves up with the key: the tile's first key gives the lower end, its last key the upper end.
+  int tA0 = 0, nA = 0, tB0 = 0, nB = 0;
   if (ks == CLEAN) {
-    const int qa_lo = (a.mode == 0) ? k0 : (k0 / M) * M;
-    // with a sliding window the last query row that sees a key of this tile is k0 + TILE - 1 + window - 1
-    const int t_end = (a.window > 0) ? min(NT, (min(L, k0 + TILE - 1 + a.window) + TILE - 1) / TILE) : NT;
-    tA0 = qa_lo / TILE; nA = t_end - tA0;
-    const int qb_lo = (k0 / M + 1) * M;
-    if (qb_lo < L) { tB0 = qb_lo / TILE; nB = max(0, t_end - tB0); }
+    int lo, hi, tmp;
+    if (a.q[CLEAN] != nullptr) {
+      visible_queries_of_clean_key(a, CLEAN, k0, lo, tmp);
+      visible_queries_of_clean_key(a, CLEAN, k0 + TILE - 1, tmp, hi);
+      if (hi > lo) { tA0 = lo / TILE; nA = (hi + TILE - 1) / TILE - tA0; }
+    }
+    if (a.q[NOISY] != nullptr) {
+      visible_queries_of_clean_key(a, NOISY, k0, lo, tmp);
+      visible_queries_of_clean_key(a, NOISY, k0 + TILE - 1, tmp, hi);
+      if (hi > lo) { tB0 = lo / TILE; nB = (hi + TILE - 1) / TILE - tB0; }
+    }
   } else {
     const int lo = (k0 / M) * M, hi = min(L, ((k0 + TILE - 1) / M + 1) * M);
     tA0 = lo / TILE; nA = (hi + TILE - 1) / TILE - tA0;
@@ -175,8 +183,8 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
         mbar_expect_tx(bar_do_full + 8 * sd, TILE_BYTES);   // one arrival of two; the LSE/D rows follow
         tma_tile(sdO0 + sd * TILE_BYTES, &maps.dout[st.qs], bar_do_full + 8 * sd, st.h * 128, st.q0, b);
       }
-      const float* lsep = a.lse[st.qs] + ((int64_t)b * a.H + st.h) * L + st.q0;
-      const float* dsp = a.dsum[st.qs] + ((int64_t)b * a.H + st.h) * L + st.q0;
+      const float* lsep = a.lse[st.qs] + ((int64_t)b * a.H + st.h) * rows_q(a, st.qs) + st.q0;
+      const float* dsp = a.dsum[st.qs] + ((int64_t)b * a.H + st.h) * rows_q(a, st.qs) + st.q0;
       {
         const float4 z = reinterpret_cast<const float4*>(lsep)[lane];
         const float4 dd = reinterpret_cast<const float4*>(dsp)[lane];
@@ -259,29 +267,27 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
     const int c0 = w * CW;
     uint8_t* prow = sm + DKDV_P + (c0 >> 6) * PANEL_BYTES + r * 128;   // this thread's row of the P^T tile (panel of its columns)
     const int pch0 = (c0 & 63) >> 3;                           // its first 16-byte chunk in that row
-    // query rows that see key j, per query stream (section 3.2 read from the key's side)
-    int vq_lo[2], vq_hi[2];
+    // query rows that see key j, per query stream (section 3.2 read from the key's side), and the bounds inside
+    // which a query tile needs no masking: every key row of this tile sees all of it.  The visible-query
+    // interval is monotone in the key, so the last key's lower end and the first key's upper end decide.
+    int vqc_lo = 0, vqc_hi = 0, vqn_lo, vqn_hi, fullc_lo = 0, fullc_hi = 0, fulln_lo, fulln_hi;
     if (ks == CLEAN) {
-      const int q_end = (a.window > 0) ? min(L, j + a.window) : L;
-      vq_lo[CLEAN] = (a.mode == 0) ? j : (j / M) * M; vq_hi[CLEAN] = q_end;
-      vq_lo[NOISY] = (j / M + 1) * M; vq_hi[NOISY] = q_end;
-    } else {
-      vq_lo[CLEAN] = 0; vq_hi[CLEAN] = 0;
-      vq_lo[NOISY] = (j / M) * M; vq_hi[NOISY] = vq_lo[NOISY] + M;
-    }
-    const int vqc_lo = vq_lo[CLEAN], vqc_hi = vq_hi[CLEAN], vqn_lo = vq_lo[NOISY], vqn_hi = vq_hi[NOISY];
-    // a query tile [q0, q0+128) needs no masking iff every key row of this tile sees all of it: the visible-query
-    // interval is monotone in the key, so the last key's lower bound and the first key's upper bound decide
-    int fullc_lo, fullc_hi, fulln_lo, fulln_hi;
-    {
-      const int jl = k0 + TILE - 1;
-      if (ks == CLEAN) {
-        fullc_lo = (a.mode == 0) ? jl : (jl / M) * M; fullc_hi = (a.window > 0) ? min(L, k0 + a.window) : L;
-        fulln_lo = (jl / M + 1) * M; fulln_hi = fullc_hi;
-      } else {
-        fullc_lo = 0; fullc_hi = 0;
-        fulln_lo = (jl / M) * M; fulln_hi = (k0 / M) * M + M;
+      int tmp;
+      if (a.q[CLEAN] != nullptr) {
+        visible_queries_of_clean_key(a, CLEAN, j, vqc_lo, vqc_hi);
+        visible_queries_of_clean_key(a, CLEAN, k0 + TILE - 1, fullc_lo, tmp);
+        visible_queries_of_clean_key(a, CLEAN, k0, tmp, fullc_hi);
       }
+      if (a.q[NOISY] != nullptr) {
+        visible_queries_of_clean_key(a, NOISY, j, vqn_lo, vqn_hi);
+        visible_queries_of_clean_key(a, NOISY, k0 + TILE - 1, fulln_lo, tmp);
+        visible_queries_of_clean_key(a, NOISY, k0, tmp, fulln_hi);
+      } else {
+        vqn_lo = vqn_hi = fulln_lo = fulln_hi = 0;
+      }
+    } else {
+      vqn_lo = (j / M) * M; vqn_hi = vqn_lo + M;
+      fulln_lo = ((k0 + TILE - 1) / M) * M; fulln_hi = (k0 / M) * M + M;
     }
     bool ok = true;
     long long w_st = 0, w_dpt = 0, w_pf = 0, c_exp = 0, c_ds = 0, c_ld = 0, c_math = 0;
@@ -472,17 +478,19 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
   const int qs = blockIdx.z & 1, b = blockIdx.z >> 1, h = blockIdx.y, hk = h / a.G;
   const int q0 = (gridDim.x - 1 - blockIdx.x) * TILE;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int L = a.L;
+  if (a.q[qs] == nullptr) return;
+  const int L = rows_q(a, qs);   // rows of this stream's query tensors
+  if (q0 >= L) return;
 
   // key tiles visible from this query tile: clean segment, then noisy segment
   int lo0, lo1, nt0, nt1, lo_last0, lo_last1, hi_first0, hi_first1;
   {
     int lo_f, hi_f, lo_l, hi_l;
-    visible_interval(qs, 0, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_f, hi_f, a.window);
-    visible_interval(qs, 0, q0 + TILE - 1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_l, hi_l, a.window);
+    visible_interval(a, qs, 0, q0, lo_f, hi_f);
+    visible_interval(a, qs, 0, q0 + TILE - 1, lo_l, hi_l);
     lo0 = lo_f; lo_last0 = lo_l; hi_first0 = hi_f; nt0 = hi_l > lo_f ? (hi_l - lo_f + TILE - 1) / TILE : 0;
-    visible_interval(qs, 1, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_f, hi_f, a.window);
-    visible_interval(qs, 1, q0 + TILE - 1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_l, hi_l, a.window);
+    visible_interval(a, qs, 1, q0, lo_f, hi_f);
+    visible_interval(a, qs, 1, q0 + TILE - 1, lo_l, hi_l);
     lo1 = lo_f; lo_last1 = lo_l; hi_first1 = hi_f; nt1 = hi_l > lo_f ? (hi_l - lo_f + TILE - 1) / TILE : 0;
   }
   const int nsteps = nt0 + nt1;
@@ -602,8 +610,8 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
       dsum = a.dsum[qs][((int64_t)b * a.H + h) * L + row];
     }
     int rlo0, rhi0, rlo1, rhi1;
-    visible_interval(qs, 0, row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo0, rhi0, a.window);
-    visible_interval(qs, 1, row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo1, rhi1, a.window);
+    visible_interval(a, qs, 0, row, rlo0, rhi0);
+    visible_interval(a, qs, 1, row, rlo1, rhi1);
     bool ok = true;
     long long w_s = 0, w_dp = 0, c_ld = 0, c_exp = 0, c_ds = 0;
     Stopwatch<TR> sw;
@@ -921,8 +929,8 @@ tc_bwd1p_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __rest
       const int sd = i & 1;
       const QStep st = step_of(i);
       int lo_a, hi_a, lo_b, hi_b;
-      visible_interval(st.qs, ks, st.q0, M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_a, hi_a, a.window);
-      visible_interval(st.qs, ks, st.q0 + TILE - 1, M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_b, hi_b, a.window);
+      visible_interval(a, st.qs, ks, st.q0, lo_a, hi_a);
+      visible_interval(a, st.qs, ks, st.q0 + TILE - 1, lo_b, hi_b);
       const bool need_mask = (lo_b > k0) || (hi_a < k0 + TILE);
       ok = mbar_wait_timed<TR>(bar_do_full + 8 * sd, (i >> 1) & 1, abort_flag, w_st);
       ok = ok && mbar_wait_timed<TR>(bar_st, i & 1, abort_flag, w_st);
@@ -1055,7 +1063,7 @@ __global__ void __launch_bounds__(256) dq_convert_kernel(const float* __restrict
 }  // namespace
 
 bool tc_bwd_supported(const KArgs& a) {
-  return a.d == 128 && a.L % TILE == 0 && tc_encoder_available();
+  return a.d == 128 && tc_rows_ok(a) && tc_encoder_available();
 }
 // fp32 dQ accumulators of the single-pass backward: one [batch, L, H, 128] tensor per stream
 size_t tc_bwd_extra_workspace(const bdlm_params* p) {
@@ -1072,10 +1080,13 @@ cudaError_t launch_tc_bwd(const KArgs& a_in, void* extra_ws, int passes, cudaStr
   }
   BwdMaps maps;
   for (int s = 0; s < 2; ++s) {
-    if (!tc_make_map(&maps.q[s], a.q[s], a.H, a.L, a.batch, TILE)) return cudaErrorInvalidValue;
-    if (!tc_make_map(&maps.dout[s], a.dout[s], a.H, a.L, a.batch, TILE)) return cudaErrorInvalidValue;
-    if (!tc_make_map(&maps.k[s], a.k[s], a.Hkv, a.L, a.batch, TILE)) return cudaErrorInvalidValue;
-    if (!tc_make_map(&maps.v[s], a.v[s], a.Hkv, a.L, a.batch, TILE)) return cudaErrorInvalidValue;
+    // a stream that is left out gets the other stream's tensors as placeholders: its maps are never used
+    const int sq = a.q[s] != nullptr ? s : 1 - s;
+    const int sk = a.k[s] != nullptr ? s : CLEAN;
+    if (!tc_make_map(&maps.q[s], a.q[sq], a.H, rows_q(a, sq), a.batch, TILE)) return cudaErrorInvalidValue;
+    if (!tc_make_map(&maps.dout[s], a.dout[sq], a.H, rows_q(a, sq), a.batch, TILE)) return cudaErrorInvalidValue;
+    if (!tc_make_map(&maps.k[s], a.k[sk], a.Hkv, rows_k(a, sk), a.batch, TILE)) return cudaErrorInvalidValue;
+    if (!tc_make_map(&maps.v[s], a.v[sk], a.Hkv, rows_k(a, sk), a.batch, TILE)) return cudaErrorInvalidValue;
   }
   int* status = device_status_ptr();
   if (status == nullptr) return cudaErrorUnknown;
@@ -1099,14 +1110,14 @@ cudaError_t launch_tc_bwd(const KArgs& a_in, void* extra_ws, int passes, cudaStr
   if (passes & BDLM_BWD_PASS_DKDV) {
     auto kern = a.trace ? tc_dkdv_kernel<true> : tc_dkdv_kernel<false>;
     if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, DKDV_SMEM)) != cudaSuccess) return e;
-    dim3 grid(a.L / TILE, a.Hkv, a.batch * 2);
+    dim3 grid(max(a.L, a.k[NOISY] != nullptr ? a.Ln : 0) / TILE, a.Hkv, a.batch * 2);
     kern<<<grid, DKDV_THREADS, DKDV_SMEM, st>>>(maps, a, status);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
   if (passes & BDLM_BWD_PASS_DQ) {
     auto kern = a.trace ? tc_dq_kernel<true> : tc_dq_kernel<false>;
     if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, DQ_SMEM)) != cudaSuccess) return e;
-    dim3 grid(a.L / TILE, a.H, a.batch * 2);
+    dim3 grid(max(a.q[CLEAN] != nullptr ? a.Lqc : 0, a.q[NOISY] != nullptr ? a.Ln : 0) / TILE, a.H, a.batch * 2);
     kern<<<grid, BWD_THREADS, DQ_SMEM, st>>>(maps, a, status);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }

@@ -77,6 +77,8 @@ tc_fwd_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restri
   if (a.q[qs] == nullptr) return;
   const int h = blockIdx.y, hk = h / a.G;
   const int q0 = (gridDim.x - 1 - blockIdx.x) * TILE;
+  const int Lq = rows_q(a, qs);
+  if (q0 >= Lq) return;
   const int tid = threadIdx.x, warp = tid >> 5;
   const int row = q0 + tid;
 
@@ -99,11 +101,11 @@ tc_fwd_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restri
 #pragma unroll
   for (int ks = 0; ks < 2; ++ks) {
     int lo_f, hi_f, lo_l, hi_l;
-    visible_interval(qs, ks, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_f, hi_f, a.window);
-    visible_interval(qs, ks, q0 + TILE - 1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_l, hi_l, a.window);
+    visible_interval(a, qs, ks, q0, lo_f, hi_f);
+    visible_interval(a, qs, ks, q0 + TILE - 1, lo_l, hi_l);
     seg_lo[ks] = lo_f; seg_hi[ks] = hi_l; lo_last[ks] = lo_l; hi_first[ks] = hi_f;
     ntile[ks] = seg_hi[ks] > seg_lo[ks] ? (seg_hi[ks] - seg_lo[ks] + TILE - 1) / TILE : 0;
-    visible_interval(qs, ks, row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo[ks], rhi[ks], a.window);
+    visible_interval(a, qs, ks, row, rlo[ks], rhi[ks]);
   }
   const int nt = ntile[0] + ntile[1];
 
@@ -235,7 +237,7 @@ tc_fwd_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restri
   // ---- epilogue: O / l -> bf16, LSE ------------------------------------------------------------
   if (!fail) {
     const float inv = l > 0.f ? 1.f / l : 0.f;
-    bf16* orow = a.o[qs] + (((int64_t)b * a.L + row) * a.H + h) * 128;
+    bf16* orow = a.o[qs] + (((int64_t)b * Lq + row) * a.H + h) * 128;
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
       uint32_t o[32];
@@ -253,7 +255,7 @@ tc_fwd_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restri
         *reinterpret_cast<uint4*>(orow + c * 32 + e8 * 8) = v;
       }
     }
-    a.lse[qs][((int64_t)b * a.H + h) * a.L + row] = l > 0.f ? (m + log2f(l)) * LN2 : -INFINITY;
+    a.lse[qs][((int64_t)b * a.H + h) * Lq + row] = l > 0.f ? (m + log2f(l)) * LN2 : -INFINITY;
   } else if (tid == 0) {
     atomicExch(status, (int)BDLM_ERR_DEVICE_TIMEOUT);
   }
@@ -269,11 +271,11 @@ struct TileSched {
   int lo0, lo1, nt0, nt1, lo_last0, lo_last1, hi_first0, hi_first1;
   __device__ __forceinline__ void init(int qs, int q0, const KArgs& a) {
     int lo_f, hi_f, lo_l, hi_l;
-    visible_interval(qs, 0, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_f, hi_f, a.window);
-    visible_interval(qs, 0, q0 + TILE - 1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_l, hi_l, a.window);
+    visible_interval(a, qs, 0, q0, lo_f, hi_f);
+    visible_interval(a, qs, 0, q0 + TILE - 1, lo_l, hi_l);
     lo0 = lo_f; lo_last0 = lo_l; hi_first0 = hi_f; nt0 = hi_l > lo_f ? (hi_l - lo_f + TILE - 1) / TILE : 0;
-    visible_interval(qs, 1, q0, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_f, hi_f, a.window);
-    visible_interval(qs, 1, q0 + TILE - 1, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, lo_l, hi_l, a.window);
+    visible_interval(a, qs, 1, q0, lo_f, hi_f);
+    visible_interval(a, qs, 1, q0 + TILE - 1, lo_l, hi_l);
     lo1 = lo_f; lo_last1 = lo_l; hi_first1 = hi_f; nt1 = hi_l > lo_f ? (hi_l - lo_f + TILE - 1) / TILE : 0;
   }
   // a tile needs per-element masking unless every row of the query tile sees all of its 128 keys
@@ -316,6 +318,8 @@ tc_fwd2h_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __rest
   if (a.q[qs] == nullptr) return;
   const int h0 = blockIdx.y * 2, hk = h0 / a.G;
   const int q0 = (gridDim.x - 1 - blockIdx.x) * TILE;
+  const int Lq = rows_q(a, qs);
+  if (q0 >= Lq) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   TileSched sch;
@@ -416,8 +420,8 @@ tc_fwd2h_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __rest
     const uint32_t tS = tmem + lane_base + w * 128 + hc * 64;          // this thread's 64 score columns
     const uint32_t tO = tmem + lane_base + 256 + w * 128 + hc * 64;    // and its 64 output columns
     int rlo0, rhi0, rlo1, rhi1;
-    visible_interval(qs, 0, row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo0, rhi0, a.window);
-    visible_interval(qs, 1, row, a.M, a.mode, a.kv_begin, a.kv_end, a.diag, rlo1, rhi1, a.window);
+    visible_interval(a, qs, 0, row, rlo0, rhi0);
+    visible_interval(a, qs, 1, row, rlo1, rhi1);
     float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
     long long w_s = 0;
@@ -533,7 +537,7 @@ tc_fwd2h_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __rest
     if (ok) {
       tc_fence_after();
       const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
-      bf16* orow = a.o[qs] + (((int64_t)b * a.L + row) * a.H + h) * 128 + hc * 64;
+      bf16* orow = a.o[qs] + (((int64_t)b * Lq + row) * a.H + h) * 128 + hc * 64;
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
         uint32_t o[32];
@@ -551,7 +555,7 @@ tc_fwd2h_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __rest
           *reinterpret_cast<uint4*>(orow + c * 32 + e8 * 8) = v;
         }
       }
-      if (hc == 0) a.lse[qs][((int64_t)b * a.H + h) * a.L + row] = l_tot > 0.f ? (m_ref + log2f(l_tot)) * LN2 : -INFINITY;
+      if (hc == 0) a.lse[qs][((int64_t)b * a.H + h) * Lq + row] = l_tot > 0.f ? (m_ref + log2f(l_tot)) * LN2 : -INFINITY;
     }
   }
   tc_fence_before();
@@ -562,18 +566,29 @@ tc_fwd2h_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __rest
 
 }  // namespace
 
+// every tensor a tensor-core kernel touches must have a multiple of 128 rows
+bool tc_rows_ok(const KArgs& a) {
+  if (a.L % TILE != 0) return false;
+  if (a.q[CLEAN] != nullptr && (a.Lqc % TILE != 0 || a.Lqc == 0)) return false;
+  if (a.q[NOISY] != nullptr && (a.Ln % TILE != 0 || a.Ln == 0)) return false;
+  return true;
+}
+
 bool tc_fwd_supported(const KArgs& a) {
-  return a.d == 128 && a.L % TILE == 0 && encode_fn() != nullptr;
+  return a.d == 128 && tc_rows_ok(a) && encode_fn() != nullptr;
 }
 
 cudaError_t launch_tc_fwd(const KArgs& a, cudaStream_t st) {
   FwdMaps maps;
   for (int s = 0; s < 2; ++s) {
-    const void* q = a.q[s] ? (const void*)a.q[s] : (const void*)a.q[1 - s];
-    if (!tc_make_map(&maps.q[s], q, a.H, a.L, a.batch, TILE)) return cudaErrorInvalidValue;
-    if (!tc_make_map(&maps.k[s], a.k[s], a.Hkv, a.L, a.batch, TILE)) return cudaErrorInvalidValue;
-    if (!tc_make_map(&maps.v[s], a.v[s], a.Hkv, a.L, a.batch, TILE)) return cudaErrorInvalidValue;
+    // a stream that is left out gets the other stream's tensors as placeholders: its maps are never used
+    const int sq = a.q[s] ? s : 1 - s;
+    if (!tc_make_map(&maps.q[s], a.q[sq], a.H, rows_q(a, sq), a.batch, TILE)) return cudaErrorInvalidValue;
+    const int sk = (s == NOISY && (a.q[NOISY] == nullptr || a.Ln == 0 || !a.diag)) ? CLEAN : s;
+    if (!tc_make_map(&maps.k[s], a.k[sk], a.Hkv, rows_k(a, sk), a.batch, TILE)) return cudaErrorInvalidValue;
+    if (!tc_make_map(&maps.v[s], a.v[sk], a.Hkv, rows_k(a, sk), a.batch, TILE)) return cudaErrorInvalidValue;
   }
+  const int qrows = max(a.q[CLEAN] != nullptr ? a.Lqc : 0, a.q[NOISY] != nullptr ? a.Ln : 0);
   int* status = device_status_ptr();
   if (status == nullptr) return cudaErrorUnknown;
   cudaError_t e = cudaFuncSetAttribute(tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM);
@@ -582,11 +597,11 @@ cudaError_t launch_tc_fwd(const KArgs& a, cudaStream_t st) {
     auto kern = a.trace ? tc_fwd2h_kernel<true> : tc_fwd2h_kernel<false>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD2H_SMEM);
     if (e != cudaSuccess) return e;
-    dim3 grid4(a.L / TILE, a.H / 2, a.batch * 2);
+    dim3 grid4(qrows / TILE, a.H / 2, a.batch * 2);
     kern<<<grid4, FWD2H_THREADS, FWD2H_SMEM, st>>>(maps, a, status);
     return cudaGetLastError();
   }
-  dim3 grid(a.L / TILE, a.H, a.batch * 2);
+  dim3 grid(qrows / TILE, a.H, a.batch * 2);
   tc_fwd_kernel<<<grid, 128, FWD_SMEM, st>>>(maps, a, status);
   return cudaGetLastError();
 }

@@ -13,6 +13,7 @@ bool tc_encoder_available();
 // Tensor map over a [batch, L, heads, 128] bf16 tensor, box = 64 columns x `rows` rows, 128-byte swizzle.
 bool tc_make_map(CUtensorMap* m, const void* ptr, int heads, int L, int batch, int rows);
 
+bool tc_rows_ok(const KArgs& a);
 bool tc_fwd_supported(const KArgs& a);
 bool tc_bwd_supported(const KArgs& a);
 size_t tc_bwd_extra_workspace(const bdlm_params* p);

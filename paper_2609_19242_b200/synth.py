@@ -30,12 +30,25 @@ class Workload:
     kv_shards: int = 1        # > 1: forward is also run as that many clean-K/V shard partials
     seed: int = 0
     window: int = 0           # > 0: sliding-window layer, clean key j visible only if i - j < window
+    n_blocks: int = 0         # > 0: DFlash2-style packed form -- no clean queries, n_blocks sampled blocks whose
+                              # anchors (clean-prefix lengths) are drawn uniformly from [0, L] and sorted
+
+    @property
+    def packed(self):
+        return self.n_blocks > 0
+
+    def anchors(self):
+        """Sorted anchor positions of the sampled blocks (packed workloads), int64 numpy."""
+        rng = np.random.default_rng(self.seed + 7919)
+        return np.sort(rng.integers(0, self.L + 1, size=self.n_blocks)).astype(np.int64)
 
     def pairs_per_head(self):
         """Unmasked (query, key) pairs per (batch, query head): clean L(L+1)/2 and noisy
         L(L+M)/2 (appendix B, Eq. aligned-rank-work with P = 1); with a sliding window the
         clean keys of row i are cut to the last `window` positions up to i."""
         L, M, W = self.L, self.block_size, self.window
+        if self.packed:
+            return 0, int((M * (M + self.anchors())).sum())
         if W <= 0:
             return L * (L + 1) // 2, L * (L + M) // 2
         i = np.arange(L, dtype=np.int64)
@@ -60,6 +73,8 @@ WORKLOADS = {
     "32k_m256": Workload("32k_m256", 1, 32, 8, 128, 32768, 256, rope_theta=5e5),
     # sliding-window layer of a hybrid model (appendix K: 1,024-token windows); not a BASELINE config
     "32k_w1024": Workload("32k_w1024", 1, 32, 8, 128, 32768, 64, rope_theta=5e5, window=1024),
+    # DFlash2-shaped drafter layer (appendix E): 32K target-feature keys, 2048 sampled blocks of 16 tokens
+    "dflash32k": Workload("dflash32k", 1, 32, 8, 128, 32768, 16, n_blocks=2048),
 }
 
 
@@ -83,17 +98,20 @@ def _rope(x: torch.Tensor, theta: float) -> torch.Tensor:
 def make_inputs(w: Workload, device="cpu", with_grad=True):
     """Dict of bf16 tensors: q_clean,k_clean,v_clean,q_noisy,k_noisy,v_noisy and (optionally)
     do_clean, do_noisy.  The same seed on the same device type gives the same bits; callers
-    that compare two implementations hand both the SAME tensors."""
+    that compare two implementations hand both the SAME tensors.  A packed (DFlash2-style)
+    workload has no clean queries (q_clean, do_clean are None), noisy tensors of
+    n_blocks*block_size rows and an int32 `block_prefix` tensor with the sorted anchors."""
     g = torch.Generator(device=device)
     g.manual_seed(w.seed)
     out = {}
 
-    def draw(heads, sigma):
-        return torch.randn(w.batch, w.L, heads, w.d, generator=g, device=device,
+    def draw(rows, heads, sigma):
+        return torch.randn(w.batch, rows, heads, w.d, generator=g, device=device,
                            dtype=torch.float32) * sigma
 
     for stream in ("clean", "noisy"):
-        q, k, v = draw(w.H, 0.5), draw(w.H_kv, 0.5), draw(w.H_kv, 0.5)
+        rows = w.n_blocks * w.block_size if (w.packed and stream == "noisy") else w.L
+        q, k, v = draw(rows, w.H, 0.5), draw(rows, w.H_kv, 0.5), draw(rows, w.H_kv, 0.5)
         if w.rope_theta > 0:
             q, k = _rope(q, w.rope_theta), _rope(k, w.rope_theta)
         out[f"q_{stream}"] = q.to(torch.bfloat16)
@@ -102,7 +120,13 @@ def make_inputs(w: Workload, device="cpu", with_grad=True):
         del q, k, v
     if with_grad:
         for stream in ("clean", "noisy"):
-            out[f"do_{stream}"] = draw(w.H, 1.0).to(torch.bfloat16)
+            rows = w.n_blocks * w.block_size if (w.packed and stream == "noisy") else w.L
+            out[f"do_{stream}"] = draw(rows, w.H, 1.0).to(torch.bfloat16)
+    if w.packed:
+        out["q_clean"] = None
+        if with_grad:
+            out["do_clean"] = None
+        out["block_prefix"] = torch.from_numpy(w.anchors()).to(torch.int32).to(device)
     return out
 
 

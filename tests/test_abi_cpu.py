@@ -79,3 +79,27 @@ def test_workspace_size_formula():
     need = binding.bdlm_workspace_bytes(p, binding.BDLM_WS_BWD)
     assert need >= 2 * 2 * 8 * 512 * 4
     assert binding.bdlm_workspace_bytes(p, binding.BDLM_WS_FWD) == 0
+
+
+def test_packed_geometry_is_checked_without_a_device():
+    """Bad packed geometries are rejected before any pointer is used."""
+    L = binding.lib()
+    p = binding.make_params(1, 256, 16, 4, 2, 64)
+    fake = ctypes.c_void_p(0x1000)
+    for kw, code in [(dict(Lq_clean=-1), -1), (dict(Lq_clean=200, clean_q_pos0=100), -1),
+                     (dict(n_blocks=-2), -1), (dict(n_blocks=4, block_prefix=0x1002), -1)]:
+        g = binding.BdlmPackedGeometry()
+        g.Lq_clean, g.clean_q_pos0, g.n_blocks, g.block_prefix = 128, 0, 8, None
+        for k, v in kw.items():
+            setattr(g, k, v)
+        rc = L.bdlm_attn_fwd_packed(ctypes.byref(p), ctypes.byref(g), *([fake] * 10), None)
+        assert rc == code, kw
+        assert L.bdlm_workspace_bytes_packed(ctypes.byref(p), ctypes.byref(g), binding.BDLM_WS_BWD) == 0
+    g = binding.BdlmPackedGeometry()
+    g.Lq_clean, g.clean_q_pos0, g.n_blocks, g.block_prefix = 128, 64, 8, None
+    assert L.bdlm_workspace_bytes_packed(ctypes.byref(p), ctypes.byref(g), binding.BDLM_WS_BWD) >= 2 * 4 * 128 * 4
+    assert L.bdlm_attn_fwd_packed(ctypes.byref(p), None, *([fake] * 10), None) == -1
+    # a clean length that is not a multiple of the block size is fine in the packed form only
+    p2 = binding.make_params(1, 250, 16, 4, 2, 64)
+    assert L.bdlm_workspace_bytes_packed(ctypes.byref(p2), ctypes.byref(g), binding.BDLM_WS_BWD) > 0
+    assert binding.bdlm_workspace_bytes(p2, binding.BDLM_WS_BWD) == 0
