@@ -141,3 +141,62 @@ def check_sampled(w, impl, n_rows=256, g=None, fwd_out=None, check_bwd=True, rep
     if check_bwd:
         assert worst["dq"] <= TOL_GRAD and worst["dk"] <= TOL_GRAD and worst["dv"] <= TOL_GRAD, worst
     return worst
+
+
+def check_sampled_packed(w, impl, n_rows=256):
+    """Sampled-row parity of a packed (DFlash2-style) workload: O, LSE and dQ at sampled packed rows of
+    every (batch, head); dK/dV of the clean and the packed noisy keys through a second backward whose dO is
+    zero outside the sampled rows (dK/dV are linear in dO)."""
+    M = w.block_size
+    g = synth.make_inputs(w, "cuda")
+    pfx = g["block_prefix"]
+    anchors = w.anchors()
+    args = [g[n] for n in NAMES6]
+    out = binding.bdlm_attn_fwd_packed(*args, M, block_prefix=pfx, impl=impl)
+    grads = binding.bdlm_attn_bwd_packed(*args, out[0], out[1], out[2], out[3], None, g["do_noisy"], M,
+                                         block_prefix=pfx, impl=impl)
+    Ln = w.n_blocks * M
+    G = w.H // w.H_kv
+    rng = np.random.default_rng(17)
+    rows_of = {}
+    do_sp = torch.zeros_like(g["do_noisy"])
+    for b in range(w.batch):
+        for h in range(w.H):
+            fixed = [0, M - 1, M, Ln - M, Ln - 1, 127, 128]
+            rest = rng.choice(Ln, size=n_rows, replace=False)
+            rows = np.unique(np.concatenate([np.asarray(fixed), rest]))[:n_rows]
+            rows_of[(b, h)] = rows
+            r = torch.from_numpy(rows).cuda()
+            do_sp[b, r, h] = g["do_noisy"][b, r, h]
+    grads_sp = binding.bdlm_attn_bwd_packed(*args, out[0], out[1], out[2], out[3], None, do_sp, M,
+                                            block_prefix=pfx, impl=impl)
+    torch.cuda.synchronize()
+    assert binding.bdlm_get_device_status() == 0
+    worst = {"o": 0.0, "lse": 0.0, "dq": 0.0, "dk": 0.0, "dv": 0.0}
+    for b in range(w.batch):
+        for hk in range(w.H_kv):
+            kv = {n: synth.to_f64(g[n][b, :, hk]) for n in ("k_clean", "v_clean", "k_noisy", "v_noisy")}
+            acc = {"dk_clean": np.zeros((w.L, w.d)), "dv_clean": np.zeros((w.L, w.d)),
+                   "dk_noisy": np.zeros((Ln, w.d)), "dv_noisy": np.zeros((Ln, w.d))}
+            num = den = 0.0
+            for h in range(hk * G, (hk + 1) * G):
+                rows = rows_of[(b, h)]
+                rt = torch.from_numpy(rows).cuda()
+                ref = orc.attn_rows_packed(1, rows, synth.to_f64(g["q_noisy"][b, rt, h]), kv["k_clean"], kv["v_clean"],
+                                           kv["k_noisy"], kv["v_noisy"], M,
+                                           do_rows=synth.to_f64(g["do_noisy"][b, rt, h]), block_prefix=anchors)
+                worst["o"] = max(worst["o"], float(np.abs(synth.to_f64(out[2][b, rt, h]) - ref["o"]).max()))
+                worst["lse"] = max(worst["lse"], float(np.abs(synth.to_f64(out[3][b, h, rt]) - ref["lse"]).max()))
+                num += float(((synth.to_f64(grads[3][b, rt, h]) - ref["dq"]) ** 2).sum())
+                den += float((ref["dq"] ** 2).sum())
+                for n in acc:
+                    acc[n] += ref[n]
+            worst["dq"] = max(worst["dq"], (num / max(den, 1e-300)) ** 0.5)
+            idx = {"dk_clean": 1, "dv_clean": 2, "dk_noisy": 4, "dv_noisy": 5}
+            for n, want in acc.items():
+                got = synth.to_f64(grads_sp[idx[n]][b, :, hk])
+                assert np.isfinite(got).all(), n
+                worst[n[:2]] = max(worst[n[:2]], rel_l2(got, want))
+    assert worst["o"] <= TOL_O and worst["lse"] <= TOL_LSE, worst
+    assert worst["dq"] <= TOL_GRAD and worst["dk"] <= TOL_GRAD and worst["dv"] <= TOL_GRAD, worst
+    return worst

@@ -19,6 +19,12 @@ def test_sampled_rows_full_size(name):
     print(name, worst)
 
 
+def test_dflash32k_sampled_rows():
+    """DFlash2-shaped packed workload at the size bench.py runs it (2048 sampled blocks over 32K clean keys)."""
+    worst = pu.check_sampled_packed(WORKLOADS["dflash32k"], binding.IMPL_AUTO)
+    print("dflash32k", worst)
+
+
 def test_csbp128k_shards_merge_and_oracle():
     """CSBP rank-local emulation: 8 contiguous clean-K/V shards, each partial computed on its
     own, merged with bdlm_lse_merge, compared with the unsharded kernel and the oracle."""
