@@ -477,7 +477,7 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
 
   const int qs = blockIdx.z & 1, b = blockIdx.z >> 1, h = blockIdx.y, hk = h / a.G;
   const int q0 = (gridDim.x - 1 - blockIdx.x) * TILE;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;   // warp index, provably uniform
   if (a.q[qs] == nullptr) return;
   const int L = rows_q(a, qs);   // rows of this stream's query tensors
   if (q0 >= L) return;
@@ -510,7 +510,7 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = *tmem_slot;
+  const uint32_t tmem = __shfl_sync(0xffffffffu, *tmem_slot, 0);   // broadcast: provably warp-uniform
   const bool bad_base = (*abort_flag != 0);
   // TMEM columns: [0,64) Q (bf16 pairs)  [64,128) dO (bf16 pairs)  [128,256) S  [256,384) dP / dS  [384,512) dQ
   constexpr uint32_t C_Q = 0, C_DO = 64, C_S = 128, C_DP = 256, C_DQ = 384;
@@ -540,7 +540,9 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
       trace_add(a.trace, 32 + 12, tick<TR>() - t_begin); trace_add(a.trace, 32 + 13, w_empty);
     }
   } else if (warp == 9) {
-    if (lane == 0 && nsteps > 0) {
+    // the whole warp walks the loop; one elected lane issues (see elect_one)
+    if (nsteps > 0) {
+      const uint32_t el = elect_one();
       long long w_kv = 0, w_ds = 0, w_sf = 0, t_issue = 0;
       const long long t_begin = tick<TR>();
       const uint32_t kk_lo0 = desc_lo_k(sK0), km_lo0 = desc_lo_mn(sK0);   // K ring as K-major B (S) / MN-major B (dQ)
@@ -549,15 +551,15 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
       ok = ok && mbar_wait_abortable(bar_k_full, 0, abort_flag);
       if (ok) {
         tc_fence_after();
-        gemm_ts(tmem + C_S, tmem + C_Q, kk_lo0, IDESC_KK, 0u);
-        mma_commit(bar_s);
+        gemm_ts_e(tmem + C_S, tmem + C_Q, kk_lo0, IDESC_KK, 0u, el);
+        mma_commit_e(bar_s, el);
       }
       ok = ok && mbar_wait_abortable(bar_v_full, 0, abort_flag);
       if (ok) {
         tc_fence_after();
-        gemm_ts(tmem + C_DP, tmem + C_DO, vk_lo0, IDESC_KK, 0u);
-        mma_commit(bar_dp);
-        mma_commit(bar_v_empty);
+        gemm_ts_e(tmem + C_DP, tmem + C_DO, vk_lo0, IDESC_KK, 0u, el);
+        mma_commit_e(bar_dp, el);
+        mma_commit_e(bar_v_empty, el);
       }
       int sk = 0;   // i % 3
       for (int i = 0; i < nsteps && ok; ++i) {
@@ -568,8 +570,8 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
           if (!ok) break;
           tc_fence_after();
           const long long g0 = tick<TR>();
-          gemm_ts(tmem + C_S, tmem + C_Q, kk_lo0 + nk * TILE_LO, IDESC_KK, 0u);
-          mma_commit(bar_s);
+          gemm_ts_e(tmem + C_S, tmem + C_Q, kk_lo0 + nk * TILE_LO, IDESC_KK, 0u, el);
+          mma_commit_e(bar_s, el);
           t_issue += tick<TR>() - g0;
         }
         // dQ += dS_i K_i   (dS: bf16 pairs at columns [0,32) and [64,96) of the dP region)
@@ -577,8 +579,8 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
         if (!ok) break;
         tc_fence_after();
         const long long g1 = tick<TR>();
-        gemm_ts_mn<true>(tmem + C_DQ, tmem + C_DP, km_lo0 + sk * TILE_LO, IDESC_KM, i > 0 ? 1u : 0u);
-        mma_commit(bar_k_empty + 8 * sk);
+        gemm_ts_mn_cw_e<64>(tmem + C_DQ, tmem + C_DP, km_lo0 + sk * TILE_LO, IDESC_KM, i > 0 ? 1u : 0u, el);
+        mma_commit_e(bar_k_empty + 8 * sk, el);
         t_issue += tick<TR>() - g1;
         if (i + 1 < nsteps) {
           const int nv = (i + 1) & 1;
@@ -586,16 +588,18 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
           if (!ok) break;
           tc_fence_after();
           const long long g2 = tick<TR>();
-          gemm_ts(tmem + C_DP, tmem + C_DO, vk_lo0 + nv * TILE_LO, IDESC_KK, 0u);
-          mma_commit(bar_dp);
-          mma_commit(bar_v_empty + 8 * nv);
+          gemm_ts_e(tmem + C_DP, tmem + C_DO, vk_lo0 + nv * TILE_LO, IDESC_KK, 0u, el);
+          mma_commit_e(bar_dp, el);
+          mma_commit_e(bar_v_empty + 8 * nv, el);
           t_issue += tick<TR>() - g2;
         }
         sk = nk;
       }
-      mma_commit(bar_done);
+      mma_commit_e(bar_done, el);
+      if (lane == 0) {
       trace_add(a.trace, 32 + 8, tick<TR>() - t_begin); trace_add(a.trace, 32 + 9, w_kv); trace_add(a.trace, 32 + 10, w_ds);
       trace_add(a.trace, 32 + 11, w_sf); trace_add(a.trace, 32 + 14, t_issue);
+      }
     }
   } else {
     const int w = warp >> 2;

@@ -151,6 +151,41 @@ __device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
+// Warp-uniform issue.  When a whole warp walks the MMA loop (waits, descriptor arithmetic) and only the
+// instruction itself is predicated on one elected lane, the loop stays convergent and the compiler can keep
+// the descriptors in the uniform datapath; with the loop inside `if (lane == 0)` every operand is moved over
+// from a vector register per instruction, and issuing one MMA costs more than the 64 clocks it runs.
+__device__ __forceinline__ uint32_t elect_one() {   // 1 in exactly one lane of the (converged) warp, 0 elsewhere
+  uint32_t r;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void mma_ss_e(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate,
+                                         uint32_t elected) {
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "setp.ne.b32 q, %5, 0;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(elected) : "memory");
+}
+__device__ __forceinline__ void mma_ts_e(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate,
+                                         uint32_t elected) {
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "setp.ne.b32 q, %5, 0;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(elected) : "memory");
+}
+__device__ __forceinline__ void mma_commit_e(uint32_t bar, uint32_t elected) {
+  asm volatile(
+      "{\n\t.reg .pred q;\n\t"
+      "setp.ne.b32 q, %1, 0;\n\t"
+      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+      ::"r"(bar), "r"(elected) : "memory");
+}
+
 // 32 lanes x 32 consecutive fp32 columns: thread t of the warp gets lane (taddr.lane + t).
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
@@ -244,6 +279,26 @@ __device__ __forceinline__ void gemm_ts_mn(uint32_t d, uint32_t a_tmem, uint32_t
 #pragma unroll
   for (int kk = 0; kk < 8; ++kk)
     mma_ts(d, a_tmem + (SPLIT ? (kk < 4 ? kk * 8 : 64 + (kk - 4) * 8) : kk * 8), desc64(b_lo + moff(kk)), idesc, kk == 0 ? acc_first : 1u);
+}
+
+// The same GEMMs issued by the elected lane of a converged warp (see elect_one).
+__device__ __forceinline__ void gemm_ss_e(uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t acc_first, uint32_t el) {
+#pragma unroll
+  for (int kk = 0; kk < 8; ++kk) mma_ss_e(d, desc64(a_lo + koff(kk)), desc64(b_lo + koff(kk)), idesc, kk == 0 ? acc_first : 1u, el);
+}
+__device__ __forceinline__ void gemm_ts_e(uint32_t d, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc, uint32_t acc_first, uint32_t el) {
+#pragma unroll
+  for (int kk = 0; kk < 8; ++kk) mma_ts_e(d, a_tmem + kk * 8, desc64(b_lo + koff(kk)), idesc, kk == 0 ? acc_first : 1u, el);
+}
+template <int CW>
+__device__ __forceinline__ void gemm_ts_mn_cw_e(uint32_t d, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc, uint32_t acc_first, uint32_t el) {
+#pragma unroll
+  for (int kk = 0; kk < 8; ++kk)
+    mma_ts_e(d, a_tmem + ((kk * 16) / CW) * CW + ((kk * 16) % CW) / 2, desc64(b_lo + moff(kk)), idesc, kk == 0 ? acc_first : 1u, el);
+}
+__device__ __forceinline__ void gemm_ss_km_e(uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t acc_first, uint32_t el) {
+#pragma unroll
+  for (int kk = 0; kk < 8; ++kk) mma_ss_e(d, desc64(a_lo + koff(kk)), desc64(b_lo + moff(kk)), idesc, kk == 0 ? acc_first : 1u, el);
 }
 
 // A K-major tile and B MN-major tile, both in shared memory.
