@@ -98,7 +98,7 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
 
   const int ks = blockIdx.z & 1, b = blockIdx.z >> 1, hk = blockIdx.y;
   const int k0 = blockIdx.x * TILE;   // key tile 0 has the most query tiles: scheduled first
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;   // warp index, provably uniform
   const int L = rows_k(a, ks), M = a.M;   // rows of this stream's K/V tensors
   if (k0 >= L || a.dk[ks] == nullptr) return;
 
@@ -149,7 +149,7 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = *tmem_slot;
+  const uint32_t tmem = __shfl_sync(0xffffffffu, *tmem_slot, 0);   // broadcast: provably warp-uniform
   const bool bad_base = (*abort_flag != 0);
   // TMEM columns: [0,128) S^T   [128,256) dP^T / dS^T   [256,384) dV   [384,512) dK
 
@@ -199,8 +199,10 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
     }
     if (lane == 0) { trace_add(a.trace, 16 + 12, tick<TR>() - t_begin); trace_add(a.trace, 16 + 13, w_empty); }
   } else if (warp == DKDV_ISSUER) {
-    // ------------------------------------------------------------------ MMA issuer (one thread)
-    if (lane == 0 && nsteps > 0) {
+    // ------------------------------------------------------------------ MMA issuer: the whole warp walks the loop,
+    // one elected lane issues (see elect_one)
+    if (nsteps > 0) {
+      const uint32_t el = elect_one();
       long long w_pt = 0, w_sf = 0, w_dst = 0;
       const long long t_begin = tick<TR>();
       const uint32_t k_lo = desc_lo_k(sK), v_lo = desc_lo_k(sV), p_lo = desc_lo_k(sP);
@@ -210,14 +212,14 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       ok = ok && mbar_wait_abortable(bar_q_full, 0, abort_flag);
       if (ok) {
         tc_fence_after();
-        gemm_ss(tmem, k_lo, qk_lo0, IDESC_KK, 0u);
-        mma_commit(bar_st);
+        gemm_ss_e(tmem, k_lo, qk_lo0, IDESC_KK, 0u, el);
+        mma_commit_e(bar_st, el);
       }
       ok = ok && mbar_wait_abortable(bar_do_full, 0, abort_flag);
       if (ok) {
         tc_fence_after();
-        gemm_ss(tmem + 128, v_lo, dok_lo0, IDESC_KK, 0u);
-        mma_commit(bar_dpt);
+        gemm_ss_e(tmem + 128, v_lo, dok_lo0, IDESC_KK, 0u, el);
+        mma_commit_e(bar_dpt, el);
       }
       for (int i = 0; i < nsteps && ok; ++i) {
         const int sd = i & 1, sn = sd ^ 1;
@@ -228,34 +230,36 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
           ok = ok && mbar_wait_lean(bar_q_full + 8 * sn, ((i + 1) >> 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          gemm_ss(tmem, k_lo, qk_lo0 + sn * TILE_LO, IDESC_KK, 0u);
-          mma_commit(bar_st);
+          gemm_ss_e(tmem, k_lo, qk_lo0 + sn * TILE_LO, IDESC_KK, 0u, el);
+          mma_commit_e(bar_st, el);
         }
         // dV += P^T dO_i   (P^T from shared memory, K-major: row = key, contraction = query)
         ok = mbar_wait_timed<TR>(bar_pt, i & 1, abort_flag, w_pt);
         if (!ok) break;
         tc_fence_after();
-        gemm_ss_km(tmem + 256, p_lo, dom_lo0 + sd * TILE_LO, IDESC_KM, acc);
-        mma_commit(bar_do_empty + 8 * sd);
-        mma_commit(bar_pfree);
+        gemm_ss_km_e(tmem + 256, p_lo, dom_lo0 + sd * TILE_LO, IDESC_KM, acc, el);
+        mma_commit_e(bar_do_empty + 8 * sd, el);
+        mma_commit_e(bar_pfree, el);
         // dK += dS^T Q_i   (dS^T: bf16 pairs, each warpgroup's share at the start of its own dP^T columns)
         ok = mbar_wait_timed<TR>(bar_dst, i & 1, abort_flag, w_dst);
         if (!ok) break;
         tc_fence_after();
-        gemm_ts_mn_cw<DKDV_CW>(tmem + 384, tmem + 128, qm_lo0 + sd * TILE_LO, IDESC_KM, acc);
-        mma_commit(bar_q_empty + 8 * sd);
+        gemm_ts_mn_cw_e<DKDV_CW>(tmem + 384, tmem + 128, qm_lo0 + sd * TILE_LO, IDESC_KM, acc, el);
+        mma_commit_e(bar_q_empty + 8 * sd, el);
         // dP^T of the next step follows dK in the pipe, so it cannot overwrite dS^T(i) early
         if (i + 1 < nsteps) {
           ok = mbar_wait_lean(bar_do_full + 8 * sn, ((i + 1) >> 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          gemm_ss(tmem + 128, v_lo, dok_lo0 + sn * TILE_LO, IDESC_KK, 0u);
-          mma_commit(bar_dpt);
+          gemm_ss_e(tmem + 128, v_lo, dok_lo0 + sn * TILE_LO, IDESC_KK, 0u, el);
+          mma_commit_e(bar_dpt, el);
         }
       }
-      mma_commit(bar_done);
-      trace_add(a.trace, 16 + 8, tick<TR>() - t_begin); trace_add(a.trace, 16 + 9, w_pt);
-      trace_add(a.trace, 16 + 10, w_sf); trace_add(a.trace, 16 + 11, w_dst);
+      mma_commit_e(bar_done, el);
+      if (lane == 0) {
+        trace_add(a.trace, 16 + 8, tick<TR>() - t_begin); trace_add(a.trace, 16 + 9, w_pt);
+        trace_add(a.trace, 16 + 10, w_sf); trace_add(a.trace, 16 + 11, w_dst);
+      }
     }
   } else {
     // ------------------------------------------------------------------ compute warpgroups

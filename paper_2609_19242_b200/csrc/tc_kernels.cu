@@ -320,7 +320,7 @@ tc_fwd2h_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __rest
   const int q0 = (gridDim.x - 1 - blockIdx.x) * TILE;
   const int Lq = rows_q(a, qs);
   if (q0 >= Lq) return;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;   // warp index, provably uniform
 
   TileSched sch;
   sch.init(qs, q0, a);
@@ -341,7 +341,7 @@ tc_fwd2h_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __rest
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = *tmem_slot;
+  const uint32_t tmem = __shfl_sync(0xffffffffu, *tmem_slot, 0);   // broadcast: provably warp-uniform
   // TMEM columns: [0,128) S/P head A   [128,256) S/P head B   [256,384) O head A   [384,512) O head B
 
   if (warp == 16) {
@@ -367,17 +367,19 @@ tc_fwd2h_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __rest
       }
     }
   } else if (warp == 17) {
-    if (lane == 0 && nt > 0) {
+    // the whole warp walks the MMA loop; one elected lane issues (see elect_one)
+    if (nt > 0) {
+      const uint32_t el = elect_one();
       const uint32_t qa_lo = desc_lo_k(sQ), qb_lo = qa_lo + TILE_LO;
       const uint32_t k_lo0 = desc_lo_k(sK0), v_lo0 = desc_lo_mn(sK0 + TILE_BYTES);
       bool ok = mbar_wait_abortable(bar_q, 0, abort_flag);
       ok = ok && mbar_wait_abortable(bar_k_full, 0, abort_flag);
       if (ok) {
         tc_fence_after();
-        gemm_ss(tmem, qa_lo, k_lo0, IDESC_QK, 0u);
-        mma_commit(bar_s);
-        gemm_ss(tmem + 128, qb_lo, k_lo0, IDESC_QK, 0u);
-        mma_commit(bar_s + 8);
+        gemm_ss_e(tmem, qa_lo, k_lo0, IDESC_QK, 0u, el);
+        mma_commit_e(bar_s, el);
+        gemm_ss_e(tmem + 128, qb_lo, k_lo0, IDESC_QK, 0u, el);
+        mma_commit_e(bar_s + 8, el);
       }
       for (int t = 0; t < nt && ok; ++t) {
         const int s = t & 1;
@@ -389,25 +391,25 @@ tc_fwd2h_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __rest
         ok = ok && mbar_wait_lean(bar_v_full + 8 * s, (t >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        gemm_ts_mn<true>(tmem + 256, tmem, cv_lo, IDESC_PV, acc);
-        mma_commit(bar_o);
+        gemm_ts_mn_cw_e<64>(tmem + 256, tmem, cv_lo, IDESC_PV, acc, el);
+        mma_commit_e(bar_o, el);
         if (t + 1 < nt) {
           ok = mbar_wait_lean(bar_k_full + 8 * (s ^ 1), ((t + 1) >> 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          gemm_ss(tmem, qa_lo, nk_lo, IDESC_QK, 0u);
-          mma_commit(bar_s);
+          gemm_ss_e(tmem, qa_lo, nk_lo, IDESC_QK, 0u, el);
+          mma_commit_e(bar_s, el);
         }
         // head B
         ok = mbar_wait_lean(bar_p + 8, t & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        gemm_ts_mn<true>(tmem + 384, tmem + 128, cv_lo, IDESC_PV, acc);
-        mma_commit(bar_o + 8);
-        mma_commit(bar_kv_empty + 8 * s);
+        gemm_ts_mn_cw_e<64>(tmem + 384, tmem + 128, cv_lo, IDESC_PV, acc, el);
+        mma_commit_e(bar_o + 8, el);
+        mma_commit_e(bar_kv_empty + 8 * s, el);
         if (t + 1 < nt) {
-          gemm_ss(tmem + 128, qb_lo, nk_lo, IDESC_QK, 0u);
-          mma_commit(bar_s + 8);
+          gemm_ss_e(tmem + 128, qb_lo, nk_lo, IDESC_QK, 0u, el);
+          mma_commit_e(bar_s + 8, el);
         }
       }
     }
