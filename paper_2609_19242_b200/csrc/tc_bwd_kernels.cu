@@ -765,7 +765,7 @@ tc_bwd1p_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __rest
 
   const int ks = blockIdx.z & 1, b = blockIdx.z >> 1, hk = blockIdx.y;
   const int k0 = blockIdx.x * TILE;   // key tile 0 has the most query tiles: scheduled first
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;   // warp index, provably uniform
   const int L = a.L, M = a.M, NT = L / TILE;
 
   int tA0, nA, tB0 = 0, nB = 0;
@@ -806,7 +806,7 @@ tc_bwd1p_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __rest
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = *tmem_slot;
+  const uint32_t tmem = __shfl_sync(0xffffffffu, *tmem_slot, 0);   // broadcast: provably warp-uniform
   const bool bad_base = (*abort_flag != 0);
   // TMEM columns: [0,128) S^T / P^T   [128,256) dP^T, then dQ^T   [256,384) dV   [384,512) dK
 
@@ -856,7 +856,9 @@ tc_bwd1p_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __rest
     if (lane == 0) { trace_add(a.trace, 16 + 12, tick<TR>() - t_begin); trace_add(a.trace, 16 + 13, w_empty); }
   } else if (warp == 9) {
     // ------------------------------------------------------------------ MMA issuer (one thread)
-    if (lane == 0 && nsteps > 0) {
+    // the whole warp walks the MMA loop; one elected lane issues (see elect_one)
+    if (nsteps > 0) {
+      const uint32_t el = elect_one();
       const long long t_begin = tick<TR>();
       const uint32_t k_lo = desc_lo_k(sK), v_lo = desc_lo_k(sV), kt_lo = desc_lo_mn(sK);
       const uint32_t qk_lo0 = desc_lo_k(sQ0), qm_lo0 = desc_lo_mn(sQ0);
@@ -866,14 +868,14 @@ tc_bwd1p_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __rest
       ok = ok && mbar_wait_abortable(bar_q_full, 0, abort_flag);
       if (ok) {
         tc_fence_after();
-        gemm_ss(tmem, k_lo, qk_lo0, IDESC_KK, 0u);
-        mma_commit(bar_st);
+        gemm_ss_e(tmem, k_lo, qk_lo0, IDESC_KK, 0u, el);
+        mma_commit_e(bar_st, el);
       }
       ok = ok && mbar_wait_abortable(bar_do_full, 0, abort_flag);
       if (ok) {
         tc_fence_after();
-        gemm_ss(tmem + 128, v_lo, dok_lo0, IDESC_KK, 0u);
-        mma_commit(bar_dpt);
+        gemm_ss_e(tmem + 128, v_lo, dok_lo0, IDESC_KK, 0u, el);
+        mma_commit_e(bar_dpt, el);
       }
       for (int i = 0; i < nsteps && ok; ++i) {
         const int sd = i & 1;
@@ -882,34 +884,34 @@ tc_bwd1p_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __rest
         ok = mbar_wait_lean(bar_pt, i & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        gemm_ts_mn<true>(tmem + 256, tmem, dom_lo0 + sd * TILE_LO, IDESC_KM, acc);
-        mma_commit(bar_do_empty + 8 * sd);
+        gemm_ts_mn_cw_e<64>(tmem + 256, tmem, dom_lo0 + sd * TILE_LO, IDESC_KM, acc, el);
+        mma_commit_e(bar_do_empty + 8 * sd, el);
         if (i + 1 < nsteps) {   // S^T of the next step
           ok = mbar_wait_lean(bar_q_full + 8 * (sd ^ 1), ((i + 1) >> 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          gemm_ss(tmem, k_lo, qk_lo0 + (sd ^ 1) * TILE_LO, IDESC_KK, 0u);
-          mma_commit(bar_st);
+          gemm_ss_e(tmem, k_lo, qk_lo0 + (sd ^ 1) * TILE_LO, IDESC_KK, 0u, el);
+          mma_commit_e(bar_st, el);
         }
         // dS^T(i) is in shared memory: dQ^T = K^T dS^T into the columns dP^T(i) occupied, then dK += dS^T Q_i
         ok = mbar_wait_lean(bar_dst, i & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        gemm_ss_mm(tmem + 128, kt_lo, dsm_lo, IDESC_MM, 0u);
-        mma_commit(bar_dqf);
-        gemm_ss_km(tmem + 384, dsk_lo, qm_lo0 + sd * TILE_LO, IDESC_KM, acc);
-        mma_commit(bar_q_empty + 8 * sd);
+        gemm_ss_mm_e(tmem + 128, kt_lo, dsm_lo, IDESC_MM, 0u, el);
+        mma_commit_e(bar_dqf, el);
+        gemm_ss_km_e(tmem + 384, dsk_lo, qm_lo0 + sd * TILE_LO, IDESC_KM, acc, el);
+        mma_commit_e(bar_q_empty + 8 * sd, el);
         if (i + 1 < nsteps) {   // dP^T of the next step, once dQ^T(i) has been read out of those columns
           ok = mbar_wait_lean(bar_dqr, i & 1, abort_flag);
           ok = ok && mbar_wait_lean(bar_do_full + 8 * (sd ^ 1), ((i + 1) >> 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          gemm_ss(tmem + 128, v_lo, dok_lo0 + (sd ^ 1) * TILE_LO, IDESC_KK, 0u);
-          mma_commit(bar_dpt);
+          gemm_ss_e(tmem + 128, v_lo, dok_lo0 + (sd ^ 1) * TILE_LO, IDESC_KK, 0u, el);
+          mma_commit_e(bar_dpt, el);
         }
       }
-      mma_commit(bar_done);
-      trace_add(a.trace, 16 + 8, tick<TR>() - t_begin);
+      mma_commit_e(bar_done, el);
+      if (lane == 0) trace_add(a.trace, 16 + 8, tick<TR>() - t_begin);
     }
   } else {
     // ------------------------------------------------------------------ compute warpgroups

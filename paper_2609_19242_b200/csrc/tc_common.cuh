@@ -301,6 +301,11 @@ __device__ __forceinline__ void gemm_ss_km_e(uint32_t d, uint32_t a_lo, uint32_t
   for (int kk = 0; kk < 8; ++kk) mma_ss_e(d, desc64(a_lo + koff(kk)), desc64(b_lo + moff(kk)), idesc, kk == 0 ? acc_first : 1u, el);
 }
 
+__device__ __forceinline__ void gemm_ss_mm_e(uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t acc_first, uint32_t el) {
+#pragma unroll
+  for (int kk = 0; kk < 8; ++kk) mma_ss_e(d, desc64(a_lo + moff(kk)), desc64(b_lo + moff(kk)), idesc, kk == 0 ? acc_first : 1u, el);
+}
+
 // A K-major tile and B MN-major tile, both in shared memory.
 __device__ __forceinline__ void gemm_ss_km(uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t acc_first) {
 #pragma unroll
