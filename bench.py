@@ -36,9 +36,9 @@ NAMES6 = ["q_clean", "k_clean", "v_clean", "q_noisy", "k_noisy", "v_noisy"]
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant
 # kernel, from the ncu captures summarised under profiles/ ; keyed by (workload, kernel).
 NCU_TRAFFIC_BYTES = {
-    ("8k", "fwd"): 210109184 + 107100160,
-    ("8k", "bwd_dkdv"): 417515776 + 56512256,
-    ("8k", "bwd_dq"): 366033408 + 115696640,
+    ("8k", "fwd"): 212907520 + 109731328,
+    ("8k", "bwd_dkdv"): 417905664 + 55102208,
+    ("8k", "bwd_dq"): 365878272 + 115059200,
 }
 TRAFFIC_NOTE = ("ncu DRAM bytes were captured on the 8k workload only (profiles/tc_kernels_8k_ncu_full.md); "
                 "DRAM traffic of these L2-resident, tensor-bound kernels does not grow in proportion to the "
