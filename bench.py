@@ -39,10 +39,13 @@ NCU_TRAFFIC_BYTES = {
     ("8k", "fwd"): 212907520 + 109731328,
     ("8k", "bwd_dkdv"): 417905664 + 55102208,
     ("8k", "bwd_dq"): 365878272 + 115059200,
+    ("32k", "fwd"): 978337792 + 541234176,
+    ("32k", "bwd_dkdv"): 2465860864 + 249322752,
+    ("32k", "bwd_dq"): 1540940288 + 519113216,
 }
-TRAFFIC_NOTE = ("ncu DRAM bytes were captured on the 8k workload only (profiles/tc_kernels_8k_ncu_full.md); "
-                "DRAM traffic of these L2-resident, tensor-bound kernels does not grow in proportion to the "
-                "units processed, so no figure is extrapolated to other workloads")
+TRAFFIC_NOTE = ("dram__bytes_read.sum + dram__bytes_write.sum per launch from ncu captures of the 8k and the 32k "
+                "workload (profiles/tc_kernels_8k_ncu_full.md, profiles/tc_kernels_32k_dram_traffic.md; the two "
+                "counters take one pass); other workloads have no capture and report null")
 
 
 def load_peaks():
