@@ -10,10 +10,11 @@
 //               the CTA walks its visible key tiles and accumulates dQ += dS K
 //               (Eq. correctness-query-gradient).
 //
-// Both are warp-specialised: warp 8 issues TMA loads, warp 9 issues tcgen05.mma, warps 0-7
-// (two warpgroups, each owning half of the 128 score columns of every TMEM lane) recompute
-// P = exp(S - LSE) and dS = P * (dP - D) and hand them back to the tensor core as TMEM-resident
-// A operands.  Every wait is bounded and abortable.
+// Both are warp-specialised: warp 8 issues TMA loads, warp 9 issues tcgen05.mma (the whole warp walks the
+// loop convergently, one elected lane issues), warps 0-7 (two warpgroups, each owning half of the 128
+// score columns of every TMEM lane) recompute P = exp(S - LSE) and dS = P * (dP - D) and hand them back
+// to the tensor core (dS as a TMEM-resident A operand; P^T of the dK/dV pass through a shared-memory tile).
+// Every wait is bounded and abortable.
 #include "tc_common.cuh"
 #include "tc_launch.h"
 
@@ -31,15 +32,6 @@ constexpr int BWD_THREADS = 320;
 constexpr int TILE_BYTES = 2 * PANEL_BYTES;
 constexpr uint32_t IDESC_KK = make_idesc(128, 128, false, false);   // A, B both K-major
 constexpr uint32_t IDESC_KM = make_idesc(128, 128, false, true);    // B MN-major (a [k][n] tile as loaded)
-
-// K-major operand tile (two 64-column panels): descriptor of the kk-th 16-wide slice of the contraction dim
-__device__ __forceinline__ uint64_t kmajor_desc(uint32_t tile, int kk) {
-  return smem_desc(tile + (kk >> 2) * PANEL_BYTES + (kk & 3) * 32, 16, 1024);
-}
-// MN-major operand: the tile is stored [contraction row][128 columns]; slice kk = rows 16kk..16kk+15
-__device__ __forceinline__ uint64_t mnmajor_desc(uint32_t tile, int kk) {
-  return smem_desc(tile + kk * 2048, PANEL_BYTES, 1024);
-}
 
 __device__ __forceinline__ void tma_tile(uint32_t dst, const CUtensorMap* map, uint32_t bar, int col0, int row0, int b) {
   tma_load_3d(dst, map, bar, col0, row0, b);

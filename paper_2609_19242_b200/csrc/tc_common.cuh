@@ -254,34 +254,9 @@ __host__ __device__ constexpr uint32_t koff(int kk) { return (kk >> 2) * (PANEL_
 __host__ __device__ constexpr uint32_t moff(int kk) { return kk * 128; }                                        // MN-major slice (16 rows)
 constexpr uint32_t TILE_LO = (2 * PANEL_BYTES) >> 4;   // low-word stride between consecutive 32 KB tiles
 
-// D (+)= A B^T, A and B both K-major tiles in shared memory (8 k-slices of 16).
-__device__ __forceinline__ void gemm_ss(uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t acc_first) {
-#pragma unroll
-  for (int kk = 0; kk < 8; ++kk) mma_ss(d, desc64(a_lo + koff(kk)), desc64(b_lo + koff(kk)), idesc, kk == 0 ? acc_first : 1u);
-}
-// A = 64 contiguous TMEM columns of bf16 pairs, B K-major tile in shared memory.
-__device__ __forceinline__ void gemm_ts(uint32_t d, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc, uint32_t acc_first) {
-#pragma unroll
-  for (int kk = 0; kk < 8; ++kk) mma_ts(d, a_tmem + kk * 8, desc64(b_lo + koff(kk)), idesc, kk == 0 ? acc_first : 1u);
-}
-// A = bf16 pairs in TMEM, B MN-major tile ([contraction row][128 columns]) in shared memory.  `split`: the A
-// pairs of contraction indices 64..127 sit 64 columns after those of 0..63 (two warpgroups wrote them).
-// A = bf16 pairs in TMEM written by warpgroups that each own CW of the 128 contraction indices: the pairs of
-// index c sit at column (c / CW) * CW + (c % CW) / 2.  B MN-major tile in shared memory.
-template <int CW>
-__device__ __forceinline__ void gemm_ts_mn_cw(uint32_t d, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc, uint32_t acc_first) {
-#pragma unroll
-  for (int kk = 0; kk < 8; ++kk)
-    mma_ts(d, a_tmem + ((kk * 16) / CW) * CW + ((kk * 16) % CW) / 2, desc64(b_lo + moff(kk)), idesc, kk == 0 ? acc_first : 1u);
-}
-template <bool SPLIT>
-__device__ __forceinline__ void gemm_ts_mn(uint32_t d, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc, uint32_t acc_first) {
-#pragma unroll
-  for (int kk = 0; kk < 8; ++kk)
-    mma_ts(d, a_tmem + (SPLIT ? (kk < 4 ? kk * 8 : 64 + (kk - 4) * 8) : kk * 8), desc64(b_lo + moff(kk)), idesc, kk == 0 ? acc_first : 1u);
-}
-
-// The same GEMMs issued by the elected lane of a converged warp (see elect_one).
+// GEMMs over a 128-deep contraction (8 k-slices of 16), issued by the elected lane of a converged warp (see
+// elect_one).  Suffixes: ss = both operands in shared memory, ts = A as bf16 pairs in tensor memory; operands
+// are K-major unless the name says mn/km/mm (B MN-major; A K-major and B MN-major; both MN-major).
 __device__ __forceinline__ void gemm_ss_e(uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t acc_first, uint32_t el) {
 #pragma unroll
   for (int kk = 0; kk < 8; ++kk) mma_ss_e(d, desc64(a_lo + koff(kk)), desc64(b_lo + koff(kk)), idesc, kk == 0 ? acc_first : 1u, el);
@@ -304,17 +279,6 @@ __device__ __forceinline__ void gemm_ss_km_e(uint32_t d, uint32_t a_lo, uint32_t
 __device__ __forceinline__ void gemm_ss_mm_e(uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t acc_first, uint32_t el) {
 #pragma unroll
   for (int kk = 0; kk < 8; ++kk) mma_ss_e(d, desc64(a_lo + moff(kk)), desc64(b_lo + moff(kk)), idesc, kk == 0 ? acc_first : 1u, el);
-}
-
-// A K-major tile and B MN-major tile, both in shared memory.
-__device__ __forceinline__ void gemm_ss_km(uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t acc_first) {
-#pragma unroll
-  for (int kk = 0; kk < 8; ++kk) mma_ss(d, desc64(a_lo + koff(kk)), desc64(b_lo + moff(kk)), idesc, kk == 0 ? acc_first : 1u);
-}
-// A and B both MN-major tiles ([contraction row][128 columns]) in shared memory: D = A^T-tile x B-tile.
-__device__ __forceinline__ void gemm_ss_mm(uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t acc_first) {
-#pragma unroll
-  for (int kk = 0; kk < 8; ++kk) mma_ss(d, desc64(a_lo + moff(kk)), desc64(b_lo + moff(kk)), idesc, kk == 0 ? acc_first : 1u);
 }
 
 // Byte offset of element (row, col) inside a [128 x 128] bf16 tile stored as two swizzled panels
