@@ -177,3 +177,18 @@ def test_single_pass_backward_matches_oracle_and_two_pass(w):
         assert torch.equal(one[i], two[i])
     p = binding.make_params(w.batch, w.L, M, w.H, w.H_kv, w.d, bwd_single_pass=True)
     assert binding.bdlm_workspace_bytes(p, binding.BDLM_WS_BWD) >= 2 * w.batch * w.L * w.H * w.d * 4
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_large_logits(impl):
+    """Scores with a standard deviation of about 10 nats (q and k six times larger than in the workloads):
+    sharply peaked rows, row maxima that keep growing along the keys -- the running-maximum bookkeeping of
+    the forward (rescale only after a growth of 2^8) and the exp(S - LSE) recomputation of the backward."""
+    w = Workload("peaked", 1, 4, 2, 128, 640, 32)
+    inp = synth.make_inputs(w, "cpu")
+    for n in ("q_clean", "k_clean", "q_noisy", "k_noisy"):
+        inp[n] = (inp[n].float() * 6.0).to(torch.bfloat16)
+    # make the clean keys' scores drift upwards along the sequence for some rows: every later tile raises the maximum
+    ramp = torch.linspace(0.0, 3.0, w.L).view(1, w.L, 1, 1)
+    inp["k_clean"] = (inp["k_clean"].float() + ramp * inp["q_clean"].float().mean(dim=(1, 2), keepdim=True).sign()).to(torch.bfloat16)
+    pu.check_full(w, impl, inp=inp)
