@@ -144,6 +144,14 @@ int bdlm_lse_merge(int32_t n_partials, int32_t batch, int32_t L, int32_t H, int3
  *     b * block_size.  Row i of packed block b stands at position block_prefix[b] + i for the sliding
  *     window; with window > 0 the blocks must not overlap in position (block_prefix[b+1] >= block_prefix[b]
  *     + block_size).  Values are not validated by the library (it never reads device memory on the host).
+ *   - Clean K/V in gathered order (the all-gather output of Algorithm 1 used "directly without a reordering
+ *     copy": each key keeps its original position).  With kv_chunk_len > 0 the clean K/V tensors (and dK/dV)
+ *     are a sequence of chunks of kv_chunk_len rows; memory chunk m holds the keys at positions
+ *     kv_chunk_pos[m] .. kv_chunk_pos[m] + kv_chunk_len - 1 (for zigzag shards gathered rank by rank: chunks
+ *     r and 2P-1-r of rank r, one after the other).  kv_pos_chunk is the inverse permutation.  Requirements:
+ *     kv_chunk_len a multiple of 128 that divides L, chunk positions multiples of kv_chunk_len, window = 0,
+ *     kv_begin a multiple of 128; otherwise BDLM_ERR_UNSUPPORTED / BDLM_ERR_INVALID_ARG.  Masks, block_prefix,
+ *     clean_q_pos0 and kv_begin/kv_end are always in positions.
  *   - A query stream is left out by passing its q pointer as NULL; in the backward every tensor of that
  *     stream (for the noisy stream also K/V and dK/dV) may then be NULL.
  *   - Backward: dq_* and dk_noisy/dv_noisy are complete for the rows of this call; dk_clean/dv_clean
@@ -157,8 +165,10 @@ typedef struct {
   int32_t Lq_clean;             /* rows of the clean query tensors (ignored when q_clean is NULL) */
   int32_t clean_q_pos0;         /* position of clean query row 0; clean_q_pos0 + Lq_clean <= L */
   int32_t n_blocks;             /* packed corrupted blocks (ignored when q_noisy is NULL) */
-  int32_t reserved;
+  int32_t kv_chunk_len;         /* 0: clean K/V stored by position; > 0: stored as chunks of this many rows (see above) */
   const int32_t* block_prefix;  /* device, [n_blocks], non-decreasing; NULL = b * block_size */
+  const int32_t* kv_chunk_pos;  /* device, [L / kv_chunk_len]: position of the first key of memory chunk m */
+  const int32_t* kv_pos_chunk;  /* device, [L / kv_chunk_len]: memory chunk that holds positions c*kv_chunk_len .. (the inverse) */
 } bdlm_packed_geometry;
 
 size_t bdlm_workspace_bytes_packed(const bdlm_params* p, const bdlm_packed_geometry* g, int32_t which);

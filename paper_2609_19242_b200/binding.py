@@ -44,7 +44,8 @@ class BdlmParams(ctypes.Structure):
 
 class BdlmPackedGeometry(ctypes.Structure):
     _fields_ = [("Lq_clean", ctypes.c_int32), ("clean_q_pos0", ctypes.c_int32), ("n_blocks", ctypes.c_int32),
-                ("reserved", ctypes.c_int32), ("block_prefix", ctypes.c_void_p)]
+                ("kv_chunk_len", ctypes.c_int32), ("block_prefix", ctypes.c_void_p),
+                ("kv_chunk_pos", ctypes.c_void_p), ("kv_pos_chunk", ctypes.c_void_p)]
 
 
 _lib = None
@@ -197,7 +198,7 @@ def bdlm_attn_bwd_static_scratch(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_
     return out
 
 
-def _packed_setup(q_clean, k_clean, q_noisy, block_size, block_prefix, clean_q_pos0, window, **kw):
+def _packed_setup(q_clean, k_clean, q_noisy, block_size, block_prefix, clean_q_pos0, window, kv_chunks=None, **kw):
     """Parameters and geometry of a packed call.  `block_prefix` is an int32 CUDA tensor [n_blocks] (or None
     for b * block_size); its ordering rules are checked here on a host copy because the C library never reads
     device memory on the host."""
@@ -210,6 +211,23 @@ def _packed_setup(q_clean, k_clean, q_noisy, block_size, block_prefix, clean_q_p
     g.clean_q_pos0 = int(clean_q_pos0)
     g.n_blocks = 0
     g.block_prefix = None
+    g.kv_chunk_len, g.kv_chunk_pos, g.kv_pos_chunk = 0, None, None
+    keep = []   # device tables must outlive the launch call
+    if kv_chunks is not None:
+        # kv_chunks = (chunk_len, positions): memory chunk m of the clean K/V holds positions[m] .. + chunk_len - 1
+        chunk_len, positions = int(kv_chunks[0]), [int(x) for x in kv_chunks[1]]
+        n = L // chunk_len if chunk_len > 0 else 0
+        if chunk_len <= 0 or L % chunk_len != 0 or len(positions) != n:
+            raise ValueError("kv_chunks: chunk_len must divide L and there must be L / chunk_len positions")
+        if sorted(positions) != [c * chunk_len for c in range(n)]:
+            raise ValueError("kv_chunks: positions must be a permutation of the multiples of chunk_len")
+        inv = [0] * n
+        for m, pos in enumerate(positions):
+            inv[pos // chunk_len] = m
+        t_pos = torch.tensor(positions, dtype=torch.int32, device=k_clean.device)
+        t_inv = torch.tensor(inv, dtype=torch.int32, device=k_clean.device)
+        keep += [t_pos, t_inv]
+        g.kv_chunk_len, g.kv_chunk_pos, g.kv_pos_chunk = chunk_len, t_pos.data_ptr(), t_inv.data_ptr()
     if q_noisy is not None:
         if q_noisy.shape[1] % block_size != 0:
             raise ValueError("packed noisy rows must be a whole number of blocks")
@@ -227,18 +245,19 @@ def _packed_setup(q_clean, k_clean, q_noisy, block_size, block_prefix, clean_q_p
             if window > 0 and step.numel() and int(step.min()) < block_size:
                 raise ValueError("with a sliding window the packed blocks must not overlap in position")
             g.block_prefix = block_prefix.data_ptr()
+    g._keep = keep
     return p, g
 
 
 def bdlm_attn_fwd_packed(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, block_size, *,
                          block_prefix=None, clean_q_pos0=0, out=None, scale=0.0, clean_mask_mode=0,
-                         kv_range=None, include_noisy_diag=True, impl=IMPL_AUTO, window=0):
+                         kv_range=None, include_noisy_diag=True, impl=IMPL_AUTO, window=0, kv_chunks=None):
     """Forward of the packed form (one rank's launch of the CSBP schedule; DFlash2-style blocks).
     q_clean [batch, Lq, H, d] or None: clean queries at positions clean_q_pos0 .. ; q_noisy
     [batch, n_blocks*block_size, H, d] or None with k_noisy/v_noisy packed alike; k_clean/v_clean
     [batch, L, H_kv, d] complete.  Returns (o_clean, lse_clean, o_noisy, lse_noisy)."""
-    p, g = _packed_setup(q_clean, k_clean, q_noisy, block_size, block_prefix, clean_q_pos0, window, scale=scale,
-                         clean_mask_mode=clean_mask_mode, kv_range=kv_range,
+    p, g = _packed_setup(q_clean, k_clean, q_noisy, block_size, block_prefix, clean_q_pos0, window, kv_chunks,
+                         scale=scale, clean_mask_mode=clean_mask_mode, kv_range=kv_range,
                          include_noisy_diag=include_noisy_diag, impl=impl)
     dev = k_clean.device
     if out is None:
@@ -257,12 +276,12 @@ def bdlm_attn_fwd_packed(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, b
 def bdlm_attn_bwd_packed(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, o_clean, lse_clean,
                          o_noisy, lse_noisy, do_clean, do_noisy, block_size, *, block_prefix=None,
                          clean_q_pos0=0, out=None, workspace=None, scale=0.0, clean_mask_mode=0,
-                         impl=IMPL_AUTO, passes=0, window=0):
+                         impl=IMPL_AUTO, passes=0, window=0, kv_chunks=None):
     """Backward of the packed form.  Returns (dq_clean, dk_clean, dv_clean, dq_noisy, dk_noisy, dv_noisy);
     entries of a stream that was left out are None.  dk_clean/dv_clean are this call's contribution for
     every clean key."""
-    p, g = _packed_setup(q_clean, k_clean, q_noisy, block_size, block_prefix, clean_q_pos0, window, scale=scale,
-                         clean_mask_mode=clean_mask_mode, impl=impl, bwd_passes=passes)
+    p, g = _packed_setup(q_clean, k_clean, q_noisy, block_size, block_prefix, clean_q_pos0, window, kv_chunks,
+                         scale=scale, clean_mask_mode=clean_mask_mode, impl=impl, bwd_passes=passes)
     if out is None:
         e = lambda t: None if t is None else torch.empty_like(t)
         out = (e(q_clean), torch.empty_like(k_clean), torch.empty_like(v_clean), e(q_noisy),

@@ -25,6 +25,14 @@ int check_params(const bdlm_params* p, const bdlm_packed_geometry* g = nullptr) 
     if ((int64_t)g->clean_q_pos0 + g->Lq_clean > p->L) return BDLM_ERR_INVALID_ARG;
     if ((int64_t)g->n_blocks * p->block_size > (int64_t)1 << 30) return BDLM_ERR_INVALID_ARG;
     if (g->block_prefix != nullptr && (reinterpret_cast<uintptr_t>(g->block_prefix) & 3u)) return BDLM_ERR_INVALID_ARG;
+    if (g->kv_chunk_len < 0) return BDLM_ERR_INVALID_ARG;
+    if (g->kv_chunk_len > 0) {   // clean K/V in gathered order
+      if (g->kv_chunk_len % 128 != 0 || p->L % g->kv_chunk_len != 0) return BDLM_ERR_INVALID_ARG;
+      if (g->kv_chunk_pos == nullptr || g->kv_pos_chunk == nullptr) return BDLM_ERR_INVALID_ARG;
+      if ((reinterpret_cast<uintptr_t>(g->kv_chunk_pos) & 3u) || (reinterpret_cast<uintptr_t>(g->kv_pos_chunk) & 3u)) return BDLM_ERR_INVALID_ARG;
+      if (p->window > 0) return BDLM_ERR_UNSUPPORTED;
+      if (p->kv_range_set && p->kv_begin % 128 != 0) return BDLM_ERR_UNSUPPORTED;
+    }
   }
   if (p->clean_mask_mode != 0 && p->clean_mask_mode != 1) return BDLM_ERR_INVALID_ARG;
   if (p->impl < 0 || p->impl > 2) return BDLM_ERR_INVALID_ARG;
@@ -45,7 +53,9 @@ void fill(KArgs& a, const bdlm_params* p, const bdlm_packed_geometry* g) {
   a.G = p->H / p->H_kv; a.d = p->d;
   if (g == nullptr) {
     a.Lqc = p->L; a.cq_pos0 = 0; a.Ln = p->L; a.nb = p->L / p->block_size; a.prefix = nullptr;
+    a.kv_chunk_len = 0; a.kv_chunk_pos = nullptr; a.kv_pos_chunk = nullptr;
   } else {
+    a.kv_chunk_len = g->kv_chunk_len; a.kv_chunk_pos = g->kv_chunk_pos; a.kv_pos_chunk = g->kv_pos_chunk;
     a.Lqc = g->Lq_clean; a.cq_pos0 = g->clean_q_pos0; a.nb = g->n_blocks; a.Ln = g->n_blocks * p->block_size;
     a.prefix = g->block_prefix;
   }

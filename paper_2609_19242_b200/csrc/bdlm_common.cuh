@@ -25,6 +25,12 @@ struct KArgs {
   int Lqc, cq_pos0;   // clean query rows and the position of the first one
   int Ln, nb;         // noisy rows (= nb * M) and packed blocks
   const int* prefix;  // device [nb], non-decreasing: clean keys j < prefix[b] are visible to block b; nullptr = b * M
+  // Clean K/V in gathered order (Algorithm 1's all-gather output used without a reordering copy): memory is a
+  // sequence of chunks of kv_chunk_len rows, chunk m holds positions kv_chunk_pos[m] .. + kv_chunk_len - 1, and
+  // kv_pos_chunk is the inverse map (position chunk -> memory chunk).  kv_chunk_len = 0: stored by position.
+  int kv_chunk_len;
+  const int* kv_chunk_pos;
+  const int* kv_pos_chunk;
   float scale;        // q.k multiplier (1/sqrt(d) by default)
   float scale_log2;   // scale * log2(e): scores are exponentiated with exp2
   int mode;           // clean_mask_mode
@@ -49,6 +55,19 @@ struct KArgs {
 
 __host__ __device__ __forceinline__ int rows_q(const KArgs& a, int qs) { return qs == CLEAN ? a.Lqc : a.Ln; }
 __host__ __device__ __forceinline__ int rows_k(const KArgs& a, int ks) { return ks == CLEAN ? a.L : a.Ln; }
+
+// Memory row of the clean key at position `pos` (the first key of a tile; tiles never straddle a chunk).
+__device__ __forceinline__ int clean_key_row(const KArgs& a, int pos) {
+  if (a.kv_chunk_len == 0) return pos;
+  const int c = pos / a.kv_chunk_len;
+  return __ldg(a.kv_pos_chunk + c) * a.kv_chunk_len + (pos - c * a.kv_chunk_len);
+}
+// Position of the clean key stored at memory row `row`.
+__device__ __forceinline__ int clean_key_pos(const KArgs& a, int row) {
+  if (a.kv_chunk_len == 0) return row;
+  const int m = row / a.kv_chunk_len;
+  return __ldg(a.kv_chunk_pos + m) + (row - m * a.kv_chunk_len);
+}
 
 // Clean-prefix length of packed noisy block b.
 __device__ __forceinline__ int block_prefix(const KArgs& a, int b) {

@@ -105,8 +105,9 @@ __global__ void __launch_bounds__(NTHREADS) portable_fwd_kernel(const KArgs a) {
 
     for (int k0 = seg_lo; k0 < seg_hi; k0 += BK) {
       __syncthreads();
-      load_tile<D, BK>(Ks, kbase + (int64_t)k0 * kld, kld, seg_hi - k0);
-      load_tile<D, BK>(Vs, vbase + (int64_t)k0 * kld, kld, seg_hi - k0);
+      const int krow = ks == CLEAN ? clean_key_row(a, k0) : k0;   // where the tile's first key is stored
+      load_tile<D, BK>(Ks, kbase + (int64_t)krow * kld, kld, seg_hi - k0);
+      load_tile<D, BK>(Vs, vbase + (int64_t)krow * kld, kld, seg_hi - k0);
       __syncthreads();
 
       float s[BK / 8][4];
@@ -243,8 +244,9 @@ __global__ void __launch_bounds__(NTHREADS) portable_dq_kernel(const KArgs a) {
 
     for (int k0 = seg_lo; k0 < seg_hi; k0 += BK) {
       __syncthreads();
-      load_tile<D, BK>(Ks, kbase + (int64_t)k0 * kld, kld, seg_hi - k0);
-      load_tile<D, BK>(Vs, vbase + (int64_t)k0 * kld, kld, seg_hi - k0);
+      const int krow = ks == CLEAN ? clean_key_row(a, k0) : k0;   // where the tile's first key is stored
+      load_tile<D, BK>(Ks, kbase + (int64_t)krow * kld, kld, seg_hi - k0);
+      load_tile<D, BK>(Vs, vbase + (int64_t)krow * kld, kld, seg_hi - k0);
       __syncthreads();
 
       float s[BK / 8][4], dp[BK / 8][4];
@@ -312,7 +314,8 @@ __global__ void __launch_bounds__(NTHREADS) portable_dkdv_kernel(const KArgs a) 
   const int ks = blockIdx.z & 1;
   const int b = blockIdx.z >> 1;
   const int hk = blockIdx.y;
-  const int k0 = blockIdx.x * BQ;   // key tile 0 has the most queries: first
+  const int k0_row = blockIdx.x * BQ;   // the tile's first key in memory; key tile 0 has the most queries: first
+  const int k0 = ks == CLEAN ? clean_key_pos(a, k0_row) : k0_row;   // and its position
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   bf16* Ks = reinterpret_cast<bf16*>(smem_raw);
@@ -325,14 +328,14 @@ __global__ void __launch_bounds__(NTHREADS) portable_dkdv_kernel(const KArgs a) 
   int* vhi_s = vlo_s + BQ2;
 
   const int L = rows_k(a, ks), M = a.M;   // rows of this stream's K/V tensors
-  if (k0 >= L || a.dk[ks] == nullptr) return;
+  if (k0_row >= L || a.dk[ks] == nullptr) return;
   const int64_t qld = (int64_t)a.H * D;
   const int64_t kld = (int64_t)a.Hkv * D;
   const int64_t koff = ((int64_t)b * L * a.Hkv + hk) * D;
-  load_tile<D, BQ>(Ks, a.k[ks] + koff + (int64_t)k0 * kld, kld, L - k0);
-  load_tile<D, BQ>(Vs, a.v[ks] + koff + (int64_t)k0 * kld, kld, L - k0);
+  load_tile<D, BQ>(Ks, a.k[ks] + koff + (int64_t)k0_row * kld, kld, L - k0_row);
+  load_tile<D, BQ>(Vs, a.v[ks] + koff + (int64_t)k0_row * kld, kld, L - k0_row);
   const int j0 = k0 + warp * 16 + g, j1 = j0 + 8;
-  const int k_last = min(k0 + BQ, L) - 1;
+  const int k_last = k0 + min(BQ, L - k0_row) - 1;   // position of the tile's last key
 
   float dk[D / 8][4], dv[D / 8][4];
 #pragma unroll
@@ -442,13 +445,14 @@ __global__ void __launch_bounds__(NTHREADS) portable_dkdv_kernel(const KArgs a) 
   bf16* dvb = a.dv[ks] + koff;
 #pragma unroll
   for (int nt = 0; nt < D / 8; ++nt) {
-    if (j0 < L) {
-      *reinterpret_cast<uint32_t*>(dkb + j0 * kld + nt * 8 + 2 * t) = pack_bf16(dk[nt][0] * a.scale, dk[nt][1] * a.scale);
-      *reinterpret_cast<uint32_t*>(dvb + j0 * kld + nt * 8 + 2 * t) = pack_bf16(dv[nt][0], dv[nt][1]);
+    const int row0 = k0_row + (j0 - k0), row1 = row0 + 8;   // where the keys are stored
+    if (row0 < L) {
+      *reinterpret_cast<uint32_t*>(dkb + row0 * kld + nt * 8 + 2 * t) = pack_bf16(dk[nt][0] * a.scale, dk[nt][1] * a.scale);
+      *reinterpret_cast<uint32_t*>(dvb + row0 * kld + nt * 8 + 2 * t) = pack_bf16(dv[nt][0], dv[nt][1]);
     }
-    if (j1 < L) {
-      *reinterpret_cast<uint32_t*>(dkb + j1 * kld + nt * 8 + 2 * t) = pack_bf16(dk[nt][2] * a.scale, dk[nt][3] * a.scale);
-      *reinterpret_cast<uint32_t*>(dvb + j1 * kld + nt * 8 + 2 * t) = pack_bf16(dv[nt][2], dv[nt][3]);
+    if (row1 < L) {
+      *reinterpret_cast<uint32_t*>(dkb + row1 * kld + nt * 8 + 2 * t) = pack_bf16(dk[nt][2] * a.scale, dk[nt][3] * a.scale);
+      *reinterpret_cast<uint32_t*>(dvb + row1 * kld + nt * 8 + 2 * t) = pack_bf16(dv[nt][2], dv[nt][3]);
     }
   }
 }

@@ -89,10 +89,11 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + DKDV_BARS + 136);
 
   const int ks = blockIdx.z & 1, b = blockIdx.z >> 1, hk = blockIdx.y;
-  const int k0 = blockIdx.x * TILE;   // key tile 0 has the most query tiles: scheduled first
+  const int k0_row = blockIdx.x * TILE;   // the tile's first key in memory; key tile 0 has the most query tiles: scheduled first
+  const int k0 = ks == CLEAN ? clean_key_pos(a, k0_row) : k0_row;   // and its position
   const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;   // warp index, provably uniform
   const int L = rows_k(a, ks), M = a.M;   // rows of this stream's K/V tensors
-  if (k0 >= L || a.dk[ks] == nullptr) return;
+  if (k0_row >= L || a.dk[ks] == nullptr) return;
 
   // query tiles that see this key tile: segment A (clean queries; noisy ones for a noisy key tile), then
   // segment B (noisy queries of a clean key tile), for each head of the group.  The visible-query interval of
@@ -151,8 +152,8 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
     // ------------------------------------------------------------------ producer
     if (lane == 0) {
       mbar_expect_tx(bar_kv, 2 * TILE_BYTES);
-      tma_tile(sK, &maps.k[ks], bar_kv, hk * 128, k0, b);
-      tma_tile(sV, &maps.v[ks], bar_kv, hk * 128, k0, b);
+      tma_tile(sK, &maps.k[ks], bar_kv, hk * 128, k0_row, b);
+      tma_tile(sV, &maps.v[ks], bar_kv, hk * 128, k0_row, b);
     }
     bool ok = true;
     long long w_empty = 0;
@@ -411,7 +412,7 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       constexpr int EW = 256 / DKDV_NWG;                       // accumulator columns per thread
       const int acol = w * EW;                                 // first of them, in [0, 256)
       const bool is_dk = acol >= 128;
-      bf16* dst = (is_dk ? a.dk[ks] : a.dv[ks]) + (((int64_t)b * L + j) * a.Hkv + hk) * 128 + (acol & 127);
+      bf16* dst = (is_dk ? a.dk[ks] : a.dv[ks]) + (((int64_t)b * L + k0_row + r) * a.Hkv + hk) * 128 + (acol & 127);
       const float sc = is_dk ? a.scale : 1.f;
 #pragma unroll
       for (int c = 0; c < EW / 32; ++c) {
@@ -527,11 +528,12 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
         if (i >= 3) ok = mbar_wait_timed<TR>(bar_k_empty + 8 * sk, ((i / 3) - 1) & 1, abort_flag, w_empty);
         if (!ok) break;
         mbar_expect_tx(bar_k_full + 8 * sk, TILE_BYTES);
-        tma_tile(sK0 + sk * TILE_BYTES, &maps.k[ks], bar_k_full + 8 * sk, hk * 128, k0, b);
+        const int krow = ks == CLEAN ? clean_key_row(a, k0) : k0;   // where the tile's first key is stored
+        tma_tile(sK0 + sk * TILE_BYTES, &maps.k[ks], bar_k_full + 8 * sk, hk * 128, krow, b);
         if (i >= 2) ok = mbar_wait_timed<TR>(bar_v_empty + 8 * sv, ((i >> 1) - 1) & 1, abort_flag, w_empty);
         if (!ok) break;
         mbar_expect_tx(bar_v_full + 8 * sv, TILE_BYTES);
-        tma_tile(sV0 + sv * TILE_BYTES, &maps.v[ks], bar_v_full + 8 * sv, hk * 128, k0, b);
+        tma_tile(sV0 + sv * TILE_BYTES, &maps.v[ks], bar_v_full + 8 * sv, hk * 128, krow, b);
       }
       trace_add(a.trace, 32 + 12, tick<TR>() - t_begin); trace_add(a.trace, 32 + 13, w_empty);
     }

@@ -115,10 +115,11 @@ tc_fwd_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restri
     const uint32_t bar = bar_kv0 + 8 * (t & 1);
     const uint32_t dK = sKV + (t & 1) * 2 * TILE_BYTES, dV = dK + TILE_BYTES;
     mbar_expect_tx(bar, 2 * TILE_BYTES);
-    tma_load_3d(dK, &maps.k[ks], bar, hk * 128, k0, b);
-    tma_load_3d(dK + PANEL_BYTES, &maps.k[ks], bar, hk * 128 + 64, k0, b);
-    tma_load_3d(dV, &maps.v[ks], bar, hk * 128, k0, b);
-    tma_load_3d(dV + PANEL_BYTES, &maps.v[ks], bar, hk * 128 + 64, k0, b);
+    const int krow = ks == CLEAN ? clean_key_row(a, k0) : k0;   // where the tile's first key is stored
+    tma_load_3d(dK, &maps.k[ks], bar, hk * 128, krow, b);
+    tma_load_3d(dK + PANEL_BYTES, &maps.k[ks], bar, hk * 128 + 64, krow, b);
+    tma_load_3d(dV, &maps.v[ks], bar, hk * 128, krow, b);
+    tma_load_3d(dV + PANEL_BYTES, &maps.v[ks], bar, hk * 128 + 64, krow, b);
   };
 
   if (tid == 0 && nt > 0) {
@@ -359,11 +360,12 @@ tc_fwd2h_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __rest
         const int ks = tile_ks(t), k0 = tile_k0(t);
         const uint32_t dK = sK0 + s * 2 * TILE_BYTES, dV = dK + TILE_BYTES;
         mbar_expect_tx(bar_k_full + 8 * s, TILE_BYTES);
-        tma_load_3d(dK, &maps.k[ks], bar_k_full + 8 * s, hk * 128, k0, b);
-        tma_load_3d(dK + PANEL_BYTES, &maps.k[ks], bar_k_full + 8 * s, hk * 128 + 64, k0, b);
+        const int krow = ks == CLEAN ? clean_key_row(a, k0) : k0;   // where the tile's first key is stored
+        tma_load_3d(dK, &maps.k[ks], bar_k_full + 8 * s, hk * 128, krow, b);
+        tma_load_3d(dK + PANEL_BYTES, &maps.k[ks], bar_k_full + 8 * s, hk * 128 + 64, krow, b);
         mbar_expect_tx(bar_v_full + 8 * s, TILE_BYTES);
-        tma_load_3d(dV, &maps.v[ks], bar_v_full + 8 * s, hk * 128, k0, b);
-        tma_load_3d(dV + PANEL_BYTES, &maps.v[ks], bar_v_full + 8 * s, hk * 128 + 64, k0, b);
+        tma_load_3d(dV, &maps.v[ks], bar_v_full + 8 * s, hk * 128, krow, b);
+        tma_load_3d(dV + PANEL_BYTES, &maps.v[ks], bar_v_full + 8 * s, hk * 128 + 64, krow, b);
       }
     }
   } else if (warp == 17) {

@@ -188,3 +188,60 @@ def test_binding_rejects_bad_prefix_tables():
         binding.bdlm_attn_fwd_packed(*args, block_prefix=mk([0, 16, 64, 128]), window=64)   # overlapping blocks
     with pytest.raises(ValueError):
         binding.bdlm_attn_fwd_packed(*args, block_prefix=mk([0, 64, 128]))            # wrong length
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("P", [2, 4])
+def test_clean_kv_in_gathered_order(P, impl):
+    """The all-gathered clean K/V used without a reordering copy: ranks' zigzag shards one after the other in
+    memory, every key addressed by its original position.  Same tiles, same arithmetic: results are bitwise
+    those of the position-ordered call (dK/dV come back in the gathered order)."""
+    w = synth.Workload("gathered", 1, 4, 2, 128, 2048, 64)
+    g = pu.to_cuda(synth.make_inputs(w, "cpu"))
+    M, L = w.block_size, w.L
+    Lc = L // (2 * P)
+    order = [c for r in range(P) for c in (r, 2 * P - 1 - r)]           # memory chunk m holds position chunk order[m]
+    positions = [c * Lc for c in order]
+    gather = torch.cat([torch.arange(c * Lc, (c + 1) * Lc) for c in order]).cuda()
+    kg, vg = g["k_clean"][:, gather].contiguous(), g["v_clean"][:, gather].contiguous()
+    plan = schedule.csbp_plan(L, M, P)[P - 1]
+    rows = torch.cat([torch.arange(b * M, (b + 1) * M) for b in plan.blocks]).cuda()
+    pfx = torch.tensor(plan.block_prefix, dtype=torch.int32, device="cuda")
+    sub = {n: g[n][:, rows].contiguous() for n in ("q_noisy", "k_noisy", "v_noisy", "do_noisy")}
+    p0, p1 = plan.clean_ranges[1]
+    qc, doc = g["q_clean"][:, p0:p1].contiguous(), g["do_clean"][:, p0:p1].contiguous()
+    res = {}
+    for name, (kc, vc, kw) in {"by_position": (g["k_clean"], g["v_clean"], {}),
+                               "gathered": (kg, vg, {"kv_chunks": (Lc, positions)})}.items():
+        o = binding.bdlm_attn_fwd_packed(qc, kc, vc, sub["q_noisy"], sub["k_noisy"], sub["v_noisy"], M,
+                                         block_prefix=pfx, clean_q_pos0=p0, impl=impl, **kw)
+        gr = binding.bdlm_attn_bwd_packed(qc, kc, vc, sub["q_noisy"], sub["k_noisy"], sub["v_noisy"], o[0], o[1], o[2],
+                                          o[3], doc, sub["do_noisy"], M, block_prefix=pfx, clean_q_pos0=p0, impl=impl, **kw)
+        res[name] = (o, gr)
+    torch.cuda.synchronize()
+    assert binding.bdlm_get_device_status() == 0
+    (o_a, g_a), (o_b, g_b) = res["by_position"], res["gathered"]
+    for x, y in zip(o_a, o_b):
+        assert torch.equal(x, y)
+    for i in (0, 3, 4, 5):
+        assert torch.equal(g_a[i], g_b[i])
+    assert torch.equal(g_a[1][:, gather], g_b[1]) and torch.equal(g_a[2][:, gather], g_b[2])
+    # a shard of the gathered keys by position range, forward only
+    o_s = binding.bdlm_attn_fwd_packed(qc, kg, vg, None, None, None, M, clean_q_pos0=p0, impl=impl,
+                                       kv_range=(256, 1024), include_noisy_diag=False, kv_chunks=(Lc, positions))
+    o_r = binding.bdlm_attn_fwd_packed(qc, g["k_clean"], g["v_clean"], None, None, None, M, clean_q_pos0=p0, impl=impl,
+                                       kv_range=(256, 1024), include_noisy_diag=False)
+    assert torch.equal(o_s[0], o_r[0]) and torch.equal(o_s[1], o_r[1])
+
+
+def test_gathered_order_is_validated():
+    t = _cuda(_draw(17, 1, 512, 128, 0, 2, 1, 128))
+    args = (t["q_clean"], t["k_clean"], t["v_clean"], None, None, None, 32)
+    with pytest.raises(ValueError):
+        binding.bdlm_attn_fwd_packed(*args, kv_chunks=(128, [0, 128, 128, 384]))     # not a permutation
+    with pytest.raises(ValueError):
+        binding.bdlm_attn_fwd_packed(*args, kv_chunks=(100, [0, 100, 200, 300, 400]))   # does not divide L
+    with pytest.raises(binding.BdlmError):
+        binding.bdlm_attn_fwd_packed(*args, kv_chunks=(64, [c * 64 for c in range(8)]))  # chunks must be multiples of 128
+    with pytest.raises(binding.BdlmError):
+        binding.bdlm_attn_fwd_packed(*args, kv_chunks=(128, [0, 128, 256, 384]), window=64)  # no window with chunks
