@@ -287,33 +287,31 @@ struct TileSched {
 
 // ---------------------------------------------------------------- forward, warp-specialised
 // One CTA = one 128-row query tile of TWO query heads of the same KV group (same stream, same rows, so
-// the same key tiles and the same masks).  Warp 16 loads Q of both heads once and streams K/V tiles through
-// a 2-stage ring; warp 17 issues tcgen05.mma (QK^T from shared memory, PV with P as a TMEM operand);
-// warps 0-15 run the online softmax, two warpgroups per head, each owning one half of the 128 score
-// columns of every row (with one warpgroup per head a single warp per scheduler runs the whole row, about
-// 2300 clocks per tile; two bring it close to the exponential unit's floor).  The halves exchange their
-// partial row maximum through shared memory once per tile and add their partial row sums once at the end.
-// P (bf16) overwrites the S columns it was computed from; O is rescaled only when the running maximum
-// grew by more than 2^8 (the stale maximum is exact in the final LSE and normalisation).
-constexpr int FWD2H_THREADS = 576;                          // 16 softmax warps, producer warp, MMA warp
-constexpr int FWD2H_MX = 6 * TILE_BYTES;                    // mx_s[2][2][2][128] floats, then ls_s[2][2][128]
-constexpr int FWD2H_BARS = FWD2H_MX + 4096 + 2048;
-constexpr int FWD2H_SMEM = FWD2H_BARS + 256 + 1024;
+// the same key tiles and the same masks).  Warp 8 loads Q of both heads once and streams K/V tiles through
+// a 2-stage ring; warp 9 issues tcgen05.mma (QK^T from shared memory, PV with P as a TMEM operand: the whole
+// warp walks the loop, one elected lane issues); warps 0-7 run the online softmax, one warpgroup per head and
+// one thread per query row: the thread holds the tile's 128 scores in registers (one pass over S, no exchange
+// between threads; 320 threads leave it up to 200 registers).  While one head's warpgroup is in its
+// exponentials the tensor core runs the other head's P V and next Q K^T.  P (bf16) overwrites the first 64 of
+// the S columns it was computed from; O is rescaled only when the running maximum grew by more than 2^8 (the
+// stale maximum is exact in the final LSE and normalisation).
+// TMEM columns: [0,128) S/P head A   [128,256) S/P head B   [256,384) O head A   [384,512) O head B
+constexpr int FWDR_THREADS = 320;                            // 8 softmax warps, producer warp, MMA warp
+constexpr int FWDR_BARS = 6 * TILE_BYTES;                    // after Q (2 tiles) and the K/V ring (2 stages x 2 tiles)
+constexpr int FWDR_SMEM = FWDR_BARS + 256 + 1024;
 
 template <bool TR>
-__global__ void __launch_bounds__(FWD2H_THREADS, 1)
-tc_fwd2h_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restrict__ status) {
+__global__ void __launch_bounds__(FWDR_THREADS, 1)
+tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t sQ = base, sK0 = base + 2 * TILE_BYTES;   // stage s: K at sK0 + s*2*TILE, V after it
-  float* mx_s = reinterpret_cast<float*>(sm + FWD2H_MX);    // [tile parity][head][half][row]
-  float* ls_s = mx_s + 1024;                               // [head][half][row]
-  const uint32_t bars = base + FWD2H_BARS;
+  const uint32_t bars = base + FWDR_BARS;
   const uint32_t bar_q = bars, bar_k_full = bars + 8 /*[2]*/, bar_v_full = bars + 24 /*[2]*/, bar_kv_empty = bars + 40 /*[2]*/,
                  bar_s = bars + 56 /*[2]*/, bar_p = bars + 72 /*[2]*/, bar_o = bars + 88 /*[2]*/;
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + FWD2H_BARS + 128);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + FWD2H_BARS + 136);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + FWDR_BARS + 128);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + FWDR_BARS + 136);
 
   const int qs = blockIdx.z & 1, b = blockIdx.z >> 1;
   if (a.q[qs] == nullptr) return;
@@ -333,19 +331,19 @@ tc_fwd2h_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __rest
     mbar_init(bar_q, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar_k_full + 8 * i, 1); mbar_init(bar_v_full + 8 * i, 1); mbar_init(bar_kv_empty + 8 * i, 1);
-      mbar_init(bar_s + 8 * i, 1); mbar_init(bar_p + 8 * i, 256); mbar_init(bar_o + 8 * i, 1);
+      mbar_init(bar_s + 8 * i, 1); mbar_init(bar_p + 8 * i, 128); mbar_init(bar_o + 8 * i, 1);
     }
     *abort_flag = 0;
     fence_mbar_init();
   }
-  if (warp == 16) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
+  if (warp == 8) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = __shfl_sync(0xffffffffu, *tmem_slot, 0);   // broadcast: provably warp-uniform
   // TMEM columns: [0,128) S/P head A   [128,256) S/P head B   [256,384) O head A   [384,512) O head B
 
-  if (warp == 16) {
+  if (warp == 8) {
     if (lane == 0 && nt > 0) {
       mbar_expect_tx(bar_q, 2 * TILE_BYTES);
       tma_load_3d(sQ, &maps.q[qs], bar_q, h0 * 128, q0, b);
@@ -368,7 +366,7 @@ tc_fwd2h_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __rest
         tma_load_3d(dV + PANEL_BYTES, &maps.v[ks], bar_v_full + 8 * s, hk * 128 + 64, krow, b);
       }
     }
-  } else if (warp == 17) {
+  } else if (warp == 9) {
     // the whole warp walks the MMA loop; one elected lane issues (see elect_one)
     if (nt > 0) {
       const uint32_t el = elect_one();
@@ -393,7 +391,7 @@ tc_fwd2h_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __rest
         ok = ok && mbar_wait_lean(bar_v_full + 8 * s, (t >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        gemm_ts_mn_cw_e<64>(tmem + 256, tmem, cv_lo, IDESC_PV, acc, el);
+        gemm_ts_mn_cw_e<128>(tmem + 256, tmem, cv_lo, IDESC_PV, acc, el);
         mma_commit_e(bar_o, el);
         if (t + 1 < nt) {
           ok = mbar_wait_lean(bar_k_full + 8 * (s ^ 1), ((t + 1) >> 1) & 1, abort_flag);
@@ -406,7 +404,7 @@ tc_fwd2h_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __rest
         ok = mbar_wait_lean(bar_p + 8, t & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        gemm_ts_mn_cw_e<64>(tmem + 384, tmem + 128, cv_lo, IDESC_PV, acc, el);
+        gemm_ts_mn_cw_e<128>(tmem + 384, tmem + 128, cv_lo, IDESC_PV, acc, el);
         mma_commit_e(bar_o + 8, el);
         mma_commit_e(bar_kv_empty + 8 * s, el);
         if (t + 1 < nt) {
@@ -416,13 +414,13 @@ tc_fwd2h_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __rest
       }
     }
   } else {
-    const int g = warp >> 2, w = g >> 1, hc = g & 1;      // head, column half
+    const int w = warp >> 2;                               // head: one warpgroup per head, one thread per query row
     const int r = (warp & 3) * 32 + lane;
     const int row = q0 + r;
     const int h = h0 + w;
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t tS = tmem + lane_base + w * 128 + hc * 64;          // this thread's 64 score columns
-    const uint32_t tO = tmem + lane_base + 256 + w * 128 + hc * 64;    // and its 64 output columns
+    const uint32_t tS = tmem + lane_base + w * 128;          // this row's 128 score columns
+    const uint32_t tO = tmem + lane_base + 256 + w * 128;    // and its 128 output columns
     int rlo0, rhi0, rlo1, rhi1;
     visible_interval(a, qs, 0, row, rlo0, rhi0);
     visible_interval(a, qs, 1, row, rlo1, rhi1);
@@ -430,43 +428,35 @@ tc_fwd2h_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __rest
     bool ok = true;
     long long w_s = 0;
     const long long t_begin = tick<TR>();
-    for (int t = 0; t < nt; ++t) {
+    for (int t = 0; t < nt && ok; ++t) {
       const int ks = tile_ks(t), k0 = tile_k0(t);
-      // After a failed (timed-out) wait this warpgroup keeps walking the loop without touching tensor memory,
-      // so that it still meets its partner at every named barrier: the failure path must end, never hang.
-      if (ok) {
-        ok = mbar_wait_timed<TR>(bar_s + 8 * w, t & 1, abort_flag, w_s);
-        ok = __all_sync(0xffffffffu, ok);
-      }
+      ok = mbar_wait_timed<TR>(bar_s + 8 * w, t & 1, abort_flag, w_s);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
       tc_fence_after();
       const bool need_mask = sch.need_mask(ks, k0);
-      const int vlo = (ks == 0 ? rlo0 : rlo1) - k0 - hc * 64, vhi = (ks == 0 ? rhi0 : rhi1) - k0 - hc * 64;
-      // pass 1: maximum of this half row, exchanged with the other half
-      float mx = -INFINITY;
-      if (ok) {
-        uint32_t v0[32], v1[32];
-        tmem_ld32(tS, v0); tmem_ld32(tS + 32, v1);
+      const int vlo = (ks == 0 ? rlo0 : rlo1) - k0, vhi = (ks == 0 ? rhi0 : rhi1) - k0;
+      // the whole row of the tile in registers: one pass over S
+      uint32_t v[128];
+      {
+        uint32_t (*c)[32] = reinterpret_cast<uint32_t (*)[32]>(v);
+        tmem_ld32(tS, c[0]); tmem_ld32(tS + 32, c[1]); tmem_ld32(tS + 64, c[2]); tmem_ld32(tS + 96, c[3]);
         tmem_wait_ld();
-        if (need_mask) {
-#pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            mx = fmaxf(mx, (e >= vlo && e < vhi) ? __uint_as_float(v0[e]) : -INFINITY);
-            mx = fmaxf(mx, (e + 32 >= vlo && e + 32 < vhi) ? __uint_as_float(v1[e]) : -INFINITY);
-          }
-        } else {
-#pragma unroll
-          for (int e = 0; e < 32; ++e) mx = fmaxf(mx, fmaxf(__uint_as_float(v0[e]), __uint_as_float(v1[e])));
-        }
       }
-      mx *= a.scale_log2;
-      float* slot = mx_s + (((t & 1) * 2 + w) * 2) * 128;
-      slot[hc * 128 + r] = mx;
-      asm volatile("bar.sync %0, %1;" ::"r"(1 + w), "r"(256) : "memory");
-      mx = fmaxf(mx, slot[(hc ^ 1) * 128 + r]);
-      if (!ok) continue;
+      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+      if (need_mask) {
+#pragma unroll
+        for (int e = 0; e < 128; ++e) v[e] = (e >= vlo && e < vhi) ? v[e] : 0xff800000u;   // -inf on hidden keys
+      }
+#pragma unroll
+      for (int e = 0; e < 32; ++e) {
+        mx0 = fmaxf(mx0, __uint_as_float(v[e])); mx1 = fmaxf(mx1, __uint_as_float(v[32 + e]));
+        mx2 = fmaxf(mx2, __uint_as_float(v[64 + e])); mx3 = fmaxf(mx3, __uint_as_float(v[96 + e]));
+      }
+      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * a.scale_log2;
       const float m_new = fmaxf(m_ref, mx);
       const bool grow = m_new > m_ref + 8.0f;
-      if (__any_sync(0xffffffffu, grow)) {   // same decision in both halves: same rows, same m_ref, same m_new
+      if (__any_sync(0xffffffffu, grow)) {
         const float mb_new = (m_new == -INFINITY) ? 0.f : m_new;
         const float corr = exp2f(m_ref - mb_new);
         m_ref = m_new;
@@ -474,10 +464,10 @@ tc_fwd2h_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __rest
         if (t > 0) {
           ok = mbar_wait_abortable(bar_o + 8 * w, (t - 1) & 1, abort_flag);
           ok = __all_sync(0xffffffffu, ok);
-          if (!ok) continue;
+          if (!ok) break;
           tc_fence_after();
-#pragma unroll
-          for (int c = 0; c < 2; ++c) {
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
             uint32_t o[32];
             tmem_ld32(tO + c * 32, o);
             tmem_wait_ld();
@@ -488,84 +478,62 @@ tc_fwd2h_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __rest
         }
       }
       const float mb = (m_ref == -INFINITY) ? 0.f : m_ref;
-      // pass 2: p = exp2(s * scale - m) for this half row; bf16 pairs over its own first 32 columns
-      float psum = 0.f;
-      {
-        uint32_t v0[32], v1[32], pk[32];
-        tmem_ld32(tS, v0); tmem_ld32(tS + 32, v1);
-        tmem_wait_ld();
-        if (!need_mask) {
+      // p = exp2(s * scale - m) (exp2(-inf) = 0 on hidden keys); bf16 pairs over the first 64 columns
+      float ps0 = 0.f, ps1 = 0.f, ps2 = 0.f, ps3 = 0.f;
 #pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            const float p0 = exp2f(fmaf(__uint_as_float(v0[2 * e]), a.scale_log2, -mb));
-            const float p1 = exp2f(fmaf(__uint_as_float(v0[2 * e + 1]), a.scale_log2, -mb));
-            const float p2 = exp2f(fmaf(__uint_as_float(v1[2 * e]), a.scale_log2, -mb));
-            const float p3 = exp2f(fmaf(__uint_as_float(v1[2 * e + 1]), a.scale_log2, -mb));
-            psum += (p0 + p1) + (p2 + p3);
-            pk[e] = pack_bf16(p0, p1);
-            pk[16 + e] = pack_bf16(p2, p3);
-          }
-        } else {
+      for (int half = 0; half < 2; ++half) {
+        uint32_t pk[32];
 #pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            const int j = 2 * e;
-            float p0 = exp2f(fmaf(__uint_as_float(v0[2 * e]), a.scale_log2, -mb));
-            float p1 = exp2f(fmaf(__uint_as_float(v0[2 * e + 1]), a.scale_log2, -mb));
-            float p2 = exp2f(fmaf(__uint_as_float(v1[2 * e]), a.scale_log2, -mb));
-            float p3 = exp2f(fmaf(__uint_as_float(v1[2 * e + 1]), a.scale_log2, -mb));
-            p0 = (j >= vlo && j < vhi) ? p0 : 0.f;
-            p1 = (j + 1 >= vlo && j + 1 < vhi) ? p1 : 0.f;
-            p2 = (j + 32 >= vlo && j + 32 < vhi) ? p2 : 0.f;
-            p3 = (j + 33 >= vlo && j + 33 < vhi) ? p3 : 0.f;
-            psum += (p0 + p1) + (p2 + p3);
-            pk[e] = pack_bf16(p0, p1);
-            pk[16 + e] = pack_bf16(p2, p3);
-          }
+        for (int e = 0; e < 16; ++e) {
+          const int c = 64 * half + 4 * e;
+          const float p0 = exp2f(fmaf(__uint_as_float(v[c]), a.scale_log2, -mb));
+          const float p1 = exp2f(fmaf(__uint_as_float(v[c + 1]), a.scale_log2, -mb));
+          const float p2 = exp2f(fmaf(__uint_as_float(v[c + 2]), a.scale_log2, -mb));
+          const float p3 = exp2f(fmaf(__uint_as_float(v[c + 3]), a.scale_log2, -mb));
+          ps0 += p0; ps1 += p1; ps2 += p2; ps3 += p3;
+          pk[2 * e] = pack_bf16(p0, p1);
+          pk[2 * e + 1] = pack_bf16(p2, p3);
         }
-        tmem_st32(tS, pk);
+        tmem_st32(tS + 32 * half, pk);
       }
-      l += psum;
+      l += (ps0 + ps1) + (ps2 + ps3);
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(bar_p + 8 * w);
     }
     if (warp == 0 && lane == 0) { trace_add(a.trace, 0, nt); trace_add(a.trace, 1, w_s); trace_add(a.trace, 6, tick<TR>() - t_begin); }
-    // total row sum = sum of the two halves (both kept the same reference maximum)
-    ls_s[(w * 2 + hc) * 128 + r] = l;
-    asm volatile("bar.sync %0, %1;" ::"r"(1 + w), "r"(256) : "memory");
-    const float l_tot = l + ls_s[(w * 2 + (hc ^ 1)) * 128 + r];
     if (ok && nt > 0) {
       ok = mbar_wait_abortable(bar_o + 8 * w, (nt - 1) & 1, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
     }
     if (ok) {
       tc_fence_after();
-      const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
-      bf16* orow = a.o[qs] + (((int64_t)b * Lq + row) * a.H + h) * 128 + hc * 64;
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
+      const float inv = l > 0.f ? 1.f / l : 0.f;
+      bf16* orow = a.o[qs] + (((int64_t)b * Lq + row) * a.H + h) * 128;
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
         uint32_t o[32];
         if (nt > 0) { tmem_ld32(tO + c * 32, o); tmem_wait_ld(); }
 #pragma unroll
         for (int e8 = 0; e8 < 4; ++e8) {
-          uint4 v;
-          uint32_t* pv = reinterpret_cast<uint32_t*>(&v);
+          uint4 vv;
+          uint32_t* pv = reinterpret_cast<uint32_t*>(&vv);
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const float x0 = nt > 0 ? __uint_as_float(o[e8 * 8 + 2 * e]) * inv : 0.f;
             const float x1 = nt > 0 ? __uint_as_float(o[e8 * 8 + 2 * e + 1]) * inv : 0.f;
             pv[e] = pack_bf16(x0, x1);
           }
-          *reinterpret_cast<uint4*>(orow + c * 32 + e8 * 8) = v;
+          *reinterpret_cast<uint4*>(orow + c * 32 + e8 * 8) = vv;
         }
       }
-      if (hc == 0) a.lse[qs][((int64_t)b * a.H + h) * Lq + row] = l_tot > 0.f ? (m_ref + log2f(l_tot)) * LN2 : -INFINITY;
+      a.lse[qs][((int64_t)b * a.H + h) * Lq + row] = l > 0.f ? (m_ref + log2f(l)) * LN2 : -INFINITY;
     }
   }
   tc_fence_before();
   __syncthreads();
   if (threadIdx.x == 0 && *abort_flag) atomicExch(status, (int)BDLM_ERR_DEVICE_TIMEOUT);
-  if (warp == 16) tmem_dealloc(tmem, 512);
+  if (warp == 8) tmem_dealloc(tmem, 512);
 }
 
 }  // namespace
@@ -597,12 +565,12 @@ cudaError_t launch_tc_fwd(const KArgs& a, cudaStream_t st) {
   if (status == nullptr) return cudaErrorUnknown;
   cudaError_t e = cudaFuncSetAttribute(tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM);
   if (e != cudaSuccess) return e;
-  if (a.G % 2 == 0) {   // two heads of one KV group per CTA, four softmax warpgroups
-    auto kern = a.trace ? tc_fwd2h_kernel<true> : tc_fwd2h_kernel<false>;
-    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD2H_SMEM);
+  if (a.G % 2 == 0) {   // two heads of one KV group per CTA, one softmax warpgroup per head
+    auto kern = a.trace ? tc_fwdr_kernel<true> : tc_fwdr_kernel<false>;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, FWDR_SMEM);
     if (e != cudaSuccess) return e;
     dim3 grid4(qrows / TILE, a.H / 2, a.batch * 2);
-    kern<<<grid4, FWD2H_THREADS, FWD2H_SMEM, st>>>(maps, a, status);
+    kern<<<grid4, FWDR_THREADS, FWDR_SMEM, st>>>(maps, a, status);
     return cudaGetLastError();
   }
   dim3 grid(qrows / TILE, a.H, a.batch * 2);
