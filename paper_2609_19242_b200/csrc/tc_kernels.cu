@@ -309,7 +309,7 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
   const uint32_t sQ = base, sK0 = base + 2 * TILE_BYTES;   // stage s: K at sK0 + s*2*TILE, V after it
   const uint32_t bars = base + FWDR_BARS;
   const uint32_t bar_q = bars, bar_k_full = bars + 8 /*[2]*/, bar_v_full = bars + 24 /*[2]*/, bar_kv_empty = bars + 40 /*[2]*/,
-                 bar_s = bars + 56 /*[2]*/, bar_p = bars + 72 /*[2]*/, bar_o = bars + 88 /*[2]*/;
+                 bar_s = bars + 56 /*[2]*/, bar_o = bars + 72 /*[2]*/, bar_p = bars + 88 /*[head][key half]*/;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + FWDR_BARS + 128);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + FWDR_BARS + 136);
 
@@ -331,7 +331,8 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
     mbar_init(bar_q, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar_k_full + 8 * i, 1); mbar_init(bar_v_full + 8 * i, 1); mbar_init(bar_kv_empty + 8 * i, 1);
-      mbar_init(bar_s + 8 * i, 1); mbar_init(bar_p + 8 * i, 128); mbar_init(bar_o + 8 * i, 1);
+      mbar_init(bar_s + 8 * i, 1); mbar_init(bar_o + 8 * i, 1);
+      mbar_init(bar_p + 16 * i, 128); mbar_init(bar_p + 16 * i + 8, 128);
     }
     *abort_flag = 0;
     fence_mbar_init();
@@ -381,17 +382,28 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
         gemm_ss_e(tmem + 128, qb_lo, k_lo0, IDESC_QK, 0u, el);
         mma_commit_e(bar_s + 8, el);
       }
+      // O += P V over key half j of the tile: four k-slices of 16 keys
+      auto pv_half = [&](uint32_t d, uint32_t p_tmem, uint32_t v_lo, int j, uint32_t acc_first) {
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+          mma_ts_e(d, p_tmem + (4 * j + kk) * 8, desc64(v_lo + moff(4 * j + kk)), IDESC_PV, kk == 0 ? acc_first : 1u, el);
+      };
       for (int t = 0; t < nt && ok; ++t) {
         const int s = t & 1;
         const uint32_t cv_lo = v_lo0 + s * 2 * TILE_LO;
         const uint32_t nk_lo = k_lo0 + (s ^ 1) * 2 * TILE_LO;
         const uint32_t acc = t > 0 ? 1u : 0u;
-        // head A   (P: bf16 pairs at columns [0,32) and [64,96) of the head's S region)
+        // head A: P arrives in two halves of the keys (bf16 pairs at columns [0,32) and [32,64) of the head's S
+        // region), so P V over the first 64 keys runs while the softmax is still in the exponentials of the rest
         ok = mbar_wait_lean(bar_p, t & 1, abort_flag);
         ok = ok && mbar_wait_lean(bar_v_full + 8 * s, (t >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        gemm_ts_mn_cw_e<128>(tmem + 256, tmem, cv_lo, IDESC_PV, acc, el);
+        pv_half(tmem + 256, tmem, cv_lo, 0, acc);
+        ok = mbar_wait_lean(bar_p + 8, t & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        pv_half(tmem + 256, tmem, cv_lo, 1, 1u);
         mma_commit_e(bar_o, el);
         if (t + 1 < nt) {
           ok = mbar_wait_lean(bar_k_full + 8 * (s ^ 1), ((t + 1) >> 1) & 1, abort_flag);
@@ -401,10 +413,14 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
           mma_commit_e(bar_s, el);
         }
         // head B
-        ok = mbar_wait_lean(bar_p + 8, t & 1, abort_flag);
+        ok = mbar_wait_lean(bar_p + 16, t & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        gemm_ts_mn_cw_e<128>(tmem + 384, tmem + 128, cv_lo, IDESC_PV, acc, el);
+        pv_half(tmem + 384, tmem + 128, cv_lo, 0, acc);
+        ok = mbar_wait_lean(bar_p + 24, t & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        pv_half(tmem + 384, tmem + 128, cv_lo, 1, 1u);
         mma_commit_e(bar_o + 8, el);
         mma_commit_e(bar_kv_empty + 8 * s, el);
         if (t + 1 < nt) {
@@ -426,7 +442,7 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
     visible_interval(a, qs, 1, row, rlo1, rhi1);
     float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
-    long long w_s = 0;
+    long long w_s = 0, c_ld = 0, c_max = 0, c_exp = 0;
     const long long t_begin = tick<TR>();
     for (int t = 0; t < nt && ok; ++t) {
       const int ks = tile_ks(t), k0 = tile_k0(t);
@@ -437,12 +453,14 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
       const bool need_mask = sch.need_mask(ks, k0);
       const int vlo = (ks == 0 ? rlo0 : rlo1) - k0, vhi = (ks == 0 ? rhi0 : rhi1) - k0;
       // the whole row of the tile in registers: one pass over S
+      const long long tp0 = tick<TR>();
       uint32_t v[128];
       {
         uint32_t (*c)[32] = reinterpret_cast<uint32_t (*)[32]>(v);
         tmem_ld32(tS, c[0]); tmem_ld32(tS + 32, c[1]); tmem_ld32(tS + 64, c[2]); tmem_ld32(tS + 96, c[3]);
         tmem_wait_ld();
       }
+      const long long tp1 = tick<TR>();
       float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
       if (need_mask) {
 #pragma unroll
@@ -478,6 +496,7 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
         }
       }
       const float mb = (m_ref == -INFINITY) ? 0.f : m_ref;
+      const long long tp2 = tick<TR>();
       // p = exp2(s * scale - m) (exp2(-inf) = 0 on hidden keys); bf16 pairs over the first 64 columns
       float ps0 = 0.f, ps1 = 0.f, ps2 = 0.f, ps3 = 0.f;
 #pragma unroll
@@ -485,6 +504,11 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
         uint32_t pk[32];
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
+          if (half == 1 && e == 4) {   // the first half's store has landed by now: hand it over without stalling for it
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(bar_p + 16 * w);
+          }
           const int c = 64 * half + 4 * e;
           const float p0 = exp2f(fmaf(__uint_as_float(v[c]), a.scale_log2, -mb));
           const float p1 = exp2f(fmaf(__uint_as_float(v[c + 1]), a.scale_log2, -mb));
@@ -496,12 +520,14 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
         }
         tmem_st32(tS + 32 * half, pk);
       }
-      l += (ps0 + ps1) + (ps2 + ps3);
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(bar_p + 8 * w);
+      mbar_arrive(bar_p + 16 * w + 8);
+      l += (ps0 + ps1) + (ps2 + ps3);
+      c_ld += tp1 - tp0; c_max += tp2 - tp1; c_exp += tick<TR>() - tp2;
     }
-    if (warp == 0 && lane == 0) { trace_add(a.trace, 0, nt); trace_add(a.trace, 1, w_s); trace_add(a.trace, 6, tick<TR>() - t_begin); }
+    if (warp == 0 && lane == 0) { trace_add(a.trace, 0, nt); trace_add(a.trace, 1, w_s); trace_add(a.trace, 6, tick<TR>() - t_begin);
+      trace_add(a.trace, 3, c_ld); trace_add(a.trace, 4, c_max); trace_add(a.trace, 5, c_exp); }
     if (ok && nt > 0) {
       ok = mbar_wait_abortable(bar_o + 8 * w, (nt - 1) & 1, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
