@@ -61,10 +61,11 @@ typedef struct {
                                   (lets a caller time the passes separately; each pass needs the earlier ones'
                                   results from a previous call with the same workspace) */
   int32_t bwd_single_pass;     /* backward only: 0 = dK/dV pass + dQ pass, fixed summation order, bitwise reproducible;
-                                  1 = one pass: dQ is accumulated by the dK/dV kernel with fp32 atomic adds (5 GEMMs per
-                                  tile pair instead of 7; dQ is then reproducible only up to fp32 summation order).
-                                  Needs the larger workspace bdlm_workspace_bytes reports for this setting; falls back to
-                                  the two-pass path when the tensor-core kernels do not take the shape. */
+                                  1 = fused: one kernel produces dK, dV and dQ (5 GEMMs per tile pair instead of 7).  Each
+                                  CTA adds its dQ tiles into an fp32 accumulator in the workspace (bulk add-reductions), so
+                                  dQ is reproducible only up to fp32 summation order; dK and dV are as in the two-pass path.
+                                  Needs the larger workspace bdlm_workspace_bytes[_packed] reports for this setting; falls
+                                  back to the two-pass path when the tensor-core kernels do not take the shape. */
   int32_t window;              /* sliding-window layers: > 0 = a clean key j is visible to the query at position i (of either
                                   stream) only if additionally i - j < window; the noisy own block is unaffected.  0 = none. */
   int32_t reserved[2];

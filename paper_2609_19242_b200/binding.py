@@ -160,8 +160,8 @@ def bdlm_attn_bwd(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, o_clean,
                   o_noisy, lse_noisy, do_clean, do_noisy, block_size, *, out=None, workspace=None,
                   scale=0.0, clean_mask_mode=0, impl=IMPL_AUTO, passes=0, single_pass=False, window=0):
     """Backward of the layer.  Returns (dq_clean, dk_clean, dv_clean, dq_noisy, dk_noisy, dv_noisy).
-    `single_pass=True` selects the one-kernel backward (dQ by fp32 atomics: faster, dQ not bitwise
-    reproducible)."""
+    `single_pass=True` selects the fused one-kernel backward (dQ through fp32 add-reductions into a
+    workspace accumulator: faster, dQ reproducible only up to fp32 summation order)."""
     p = _shape_params(q_clean, k_clean, block_size, scale=scale, clean_mask_mode=clean_mask_mode, impl=impl,
                       bwd_passes=passes, bwd_single_pass=single_pass, window=window)
     if out is None:
@@ -276,12 +276,13 @@ def bdlm_attn_fwd_packed(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, b
 def bdlm_attn_bwd_packed(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, o_clean, lse_clean,
                          o_noisy, lse_noisy, do_clean, do_noisy, block_size, *, block_prefix=None,
                          clean_q_pos0=0, out=None, workspace=None, scale=0.0, clean_mask_mode=0,
-                         impl=IMPL_AUTO, passes=0, window=0, kv_chunks=None):
+                         impl=IMPL_AUTO, passes=0, single_pass=False, window=0, kv_chunks=None):
     """Backward of the packed form.  Returns (dq_clean, dk_clean, dv_clean, dq_noisy, dk_noisy, dv_noisy);
     entries of a stream that was left out are None.  dk_clean/dv_clean are this call's contribution for
-    every clean key."""
+    every clean key.  `single_pass` as in bdlm_attn_bwd."""
     p, g = _packed_setup(q_clean, k_clean, q_noisy, block_size, block_prefix, clean_q_pos0, window, kv_chunks,
-                         scale=scale, clean_mask_mode=clean_mask_mode, impl=impl, bwd_passes=passes)
+                         scale=scale, clean_mask_mode=clean_mask_mode, impl=impl, bwd_passes=passes,
+                         bwd_single_pass=single_pass)
     if out is None:
         e = lambda t: None if t is None else torch.empty_like(t)
         out = (e(q_clean), torch.empty_like(k_clean), torch.empty_like(v_clean), e(q_noisy),

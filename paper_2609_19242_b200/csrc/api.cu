@@ -105,7 +105,7 @@ extern "C" {
 
 size_t bdlm_workspace_bytes(const bdlm_params* p, int32_t which) {
   if (check_params(p) != BDLM_OK) return 0;
-  if (which == BDLM_WS_BWD) return 2 * dsum_bytes(p) + tc_bwd_extra_workspace(p);
+  if (which == BDLM_WS_BWD) return 2 * dsum_bytes(p) + tc_bwd_extra_workspace(p, nullptr);
   return 0;
 }
 
@@ -171,7 +171,7 @@ static int bwd_impl(const bdlm_params* p, const bdlm_packed_geometry* g,
   }
   if (p->kv_range_set && (p->kv_begin != 0 || p->kv_end != p->L)) return BDLM_ERR_UNSUPPORTED;
   if (!p->include_noisy_diag) return BDLM_ERR_UNSUPPORTED;
-  const size_t need_ws = 2 * dsum_bytes(p, g) + (g == nullptr ? tc_bwd_extra_workspace(p) : 0);
+  const size_t need_ws = 2 * dsum_bytes(p, g) + tc_bwd_extra_workspace(p, g);
   if (workspace_bytes < need_ws) return BDLM_ERR_WORKSPACE_TOO_SMALL;
   if (!is_sm100()) return BDLM_ERR_UNSUPPORTED;
 
@@ -194,7 +194,7 @@ static int bwd_impl(const bdlm_params* p, const bdlm_packed_geometry* g,
 
   const bool tc_ok = tc_bwd_supported(a);
   if (p->impl == 2 && !tc_ok) return BDLM_ERR_UNSUPPORTED;
-  a.single_pass = (p->bwd_single_pass && tc_ok && p->impl != 1 && g == nullptr) ? 1 : 0;
+  a.single_pass = (p->bwd_single_pass && tc_ok && p->impl != 1) ? 1 : 0;
   const int passes = p->bwd_passes ? p->bwd_passes : 7;
   cudaError_t e = cudaSuccess;
   if (passes & BDLM_BWD_PASS_DSUM) e = launch_dsum(a, ds_c, ds_n, st);
@@ -259,7 +259,7 @@ int bdlm_attn_bwd_packed(const bdlm_params* p, const bdlm_packed_geometry* g,
 
 size_t bdlm_workspace_bytes_packed(const bdlm_params* p, const bdlm_packed_geometry* g, int32_t which) {
   if (g == nullptr || check_params(p, g) != BDLM_OK) return 0;
-  if (which == BDLM_WS_BWD) return 2 * dsum_bytes(p, g);
+  if (which == BDLM_WS_BWD) return 2 * dsum_bytes(p, g) + tc_bwd_extra_workspace(p, g);
   return 0;
 }
 

@@ -723,77 +723,109 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
 
 
 // =============================================================================================
-// single-pass backward: the dK/dV kernel also produces dQ
+// fused backward: one kernel produces dK, dV and dQ
 // =============================================================================================
-// Same CTA unit and S^T / P^T / dV pipeline as tc_dkdv_kernel, but dS^T goes to a shared-memory tile
-// instead of tensor memory.  There it is the K-major A operand of dK += dS^T Q and the MN-major B
-// operand of dQ^T = K^T dS^T (K, resident, is the MN-major A operand), whose 128x128 fp32 result
-// lands in the tensor-memory columns dP^T has just vacated.  The compute warps add that tile to an
-// fp32 dQ buffer with red.global.add (a warp's 32 lanes are 32 consecutive head-dim elements of one
-// query row: one 128-byte atomic per instruction).  5 GEMMs and one exp phase per tile pair instead of
-// the 7 + 2 of the two-pass backward; dQ depends on the order the key tiles' atomics arrive in.
-// Shared memory: K, V, Q ring x2, dO ring x2 (+ LSE, D rows), dS^T.
-constexpr int P1_Q0 = 2 * TILE_BYTES;
-constexpr int P1_DO0 = 4 * TILE_BYTES;
-constexpr int P1_DS = 6 * TILE_BYTES;
-constexpr int P1_ARR = 7 * TILE_BYTES;            // lse_s[2][128], d_s[2][128]
-constexpr int P1_BARS = P1_ARR + 2048;
-constexpr int P1_SMEM = P1_BARS + 160;
-constexpr uint32_t IDESC_MM = make_idesc(128, 128, true, true);   // A and B both MN-major
+// Same CTA unit as tc_dkdv_kernel (one 128-key tile of one KV head, K and V resident), but a step is the
+// key tile against 64 query rows, so that tensor memory also holds a dQ^T tile and shared memory a staging
+// area for it: 5 GEMMs and one exp phase per (key tile, query rows) pair instead of the 7 + 2 of the
+// two-pass backward.
+//   tensor memory  [0,64) [64,128) S^T / P^T, two buffers   [128,192) dP^T   [192,256) dQ^T
+//                  [256,384) dV   [384,512) dK
+//   per step       S^T = K Q^T and dP^T = V dO^T (N = 64); P^T overwrites its own S^T columns as bf16 pairs
+//                  and is the TMEM-resident A operand of dV += P^T dO; dS^T goes to a shared-memory tile
+//                  (row = key, 64 queries = 128 bytes), the K-major A operand of dK += dS^T Q and the
+//                  MN-major B operand of dQ^T = K^T dS^T (K, resident, is the MN-major A operand).
+//   dQ             a fourth warpgroup copies each dQ^T tile (lane = head-dim index, column = query) into a
+//                  [64 query x 128] fp32 staging tile, and one of its threads hands it to the TMA engine as
+//                  a bulk add-reduction into the fp32 dQ accumulator [batch, H, rows, 128] (32 KB
+//                  contiguous).  The compute warps never touch dQ; the reduction runs behind the GEMMs.
+// dQ depends on the order in which the key tiles' reductions arrive (fp32 rounding only).
+// Shared memory: K, V, a 4-stage Q ring and a 3-stage dO ring of 64-row tiles (+ LSE, D rows), dS^T,
+// 4 dQ staging tiles of 16 query rows.  A Q stage is released by the last GEMM of its step and needed by the
+// first GEMM issued for the step after next, so the rings are one stage deeper than the look-ahead.
+constexpr int HT = 64;                              // query rows per step
+constexpr int HPANEL_BYTES = HT * 128;              // one 64-row x 64-column bf16 panel
+constexpr int HT_BYTES = 2 * HPANEL_BYTES;          // a [64 x 128] bf16 tile
+constexpr int STG_ROWS = 16;                        // query rows per dQ staging tile
+constexpr int STG_BYTES = STG_ROWS * 128 * 4;       // a [16 x 128] fp32 staging tile
+constexpr int BF_Q0 = 2 * TILE_BYTES;
+constexpr int BF_DO0 = BF_Q0 + 4 * HT_BYTES;
+constexpr int BF_DS = BF_DO0 + 3 * HT_BYTES;
+constexpr int BF_STG = BF_DS + PANEL_BYTES;
+constexpr int BF_ARR = BF_STG + 4 * STG_BYTES;      // lse_s[3][64], d_s[3][64]
+constexpr int BF_BARS = BF_ARR + 1536;
+constexpr int BF_SMEM = BF_BARS + 256;
+constexpr int BF_THREADS = 448;                     // warps 0-7 compute, 8 producer, 9 MMA issue, 10-13 dQ read-out
+constexpr uint32_t IDESC_N64 = make_idesc(128, 64, false, false);   // S^T, dP^T: A, B K-major, N = 64
+constexpr uint32_t IDESC_DQT = make_idesc(128, 64, true, true);     // dQ^T: A, B MN-major, N = 64
+constexpr uint32_t HPANEL_LO = HPANEL_BYTES >> 4, HT_LO = HT_BYTES >> 4;
+__host__ __device__ constexpr uint32_t koff_h(int kk) { return (kk >> 2) * HPANEL_LO + (kk & 3) * 2; }   // K-major slice of a 64-row tile
+__device__ __forceinline__ uint32_t desc_lo_mn_h(uint32_t addr) { return ((addr & 0x3FFFFu) >> 4) | (HPANEL_LO << 16); }
 
 template <bool TR>
-__global__ void __launch_bounds__(BWD_THREADS, 1)
-tc_bwd1p_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restrict__ status) {
+__global__ void __launch_bounds__(BF_THREADS, 1)
+tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restrict__ status) {
   extern __shared__ __align__(1024) uint8_t sm[];
   const uint32_t base = smem_u32(sm);
-  const uint32_t sK = base, sV = base + TILE_BYTES, sQ0 = base + P1_Q0, sdO0 = base + P1_DO0, sDS = base + P1_DS;
-  float* lse_s = reinterpret_cast<float*>(sm + P1_ARR);            // [2][128], log2 units
-  float* d_s = lse_s + 256;                                        // [2][128]
-  const uint32_t bars = base + P1_BARS;
-  const uint32_t bar_kv = bars, bar_q_full = bars + 8 /*[2]*/, bar_q_empty = bars + 24 /*[2]*/,
-                 bar_do_full = bars + 40 /*[2]*/, bar_do_empty = bars + 56 /*[2]*/,
-                 bar_st = bars + 72, bar_dpt = bars + 80, bar_pt = bars + 88, bar_dst = bars + 96,
-                 bar_dqf = bars + 104, bar_dqr = bars + 112, bar_done = bars + 120;
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + P1_BARS + 128);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + P1_BARS + 136);
+  const uint32_t sK = base, sV = base + TILE_BYTES, sQ0 = base + BF_Q0, sdO0 = base + BF_DO0, sDS = base + BF_DS,
+                 sSTG = base + BF_STG;
+  float* lse_s = reinterpret_cast<float*>(sm + BF_ARR);            // [3][64], log2 units
+  float* d_s = lse_s + 192;                                        // [3][64]
+  const uint32_t bars = base + BF_BARS;
+  const uint32_t bar_kv = bars, bar_q_full = bars + 8 /*[4]*/, bar_q_empty = bars + 40 /*[4]*/,
+                 bar_do_full = bars + 72 /*[3]*/, bar_do_empty = bars + 96 /*[3]*/,
+                 bar_st = bars + 120 /*[2]*/, bar_pt = bars + 136 /*[2]*/, bar_dpt = bars + 152, bar_dpfree = bars + 160,
+                 bar_dst = bars + 168, bar_dsfree = bars + 176, bar_dqf = bars + 184, bar_dqr = bars + 192,
+                 bar_done = bars + 200;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + BF_BARS + 208);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + BF_BARS + 216);
 
   const int ks = blockIdx.z & 1, b = blockIdx.z >> 1, hk = blockIdx.y;
-  const int k0 = blockIdx.x * TILE;   // key tile 0 has the most query tiles: scheduled first
+  const int k0_row = blockIdx.x * TILE;   // the tile's first key in memory; key tile 0 has the most query tiles: scheduled first
+  const int k0 = ks == CLEAN ? clean_key_pos(a, k0_row) : k0_row;   // and its position
   const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;   // warp index, provably uniform
-  const int L = a.L, M = a.M, NT = L / TILE;
+  const int L = rows_k(a, ks), M = a.M;
+  if (k0_row >= L || a.dk[ks] == nullptr) return;
 
-  int tA0, nA, tB0 = 0, nB = 0;
+  // 64-row query tiles that see this key tile: segment A (clean queries; noisy ones for a noisy key tile),
+  // then segment B (noisy queries of a clean key tile), for each head of the group
+  int tA0 = 0, nA = 0, tB0 = 0, nB = 0;
   if (ks == CLEAN) {
-    const int qa_lo = (a.mode == 0) ? k0 : (k0 / M) * M;
-    // with a sliding window the last query row that sees a key of this tile is k0 + TILE - 1 + window - 1
-    const int t_end = (a.window > 0) ? min(NT, (min(L, k0 + TILE - 1 + a.window) + TILE - 1) / TILE) : NT;
-    tA0 = qa_lo / TILE; nA = t_end - tA0;
-    const int qb_lo = (k0 / M + 1) * M;
-    if (qb_lo < L) { tB0 = qb_lo / TILE; nB = max(0, t_end - tB0); }
+    int lo, hi, tmp;
+    if (a.q[CLEAN] != nullptr) {
+      visible_queries_of_clean_key(a, CLEAN, k0, lo, tmp);
+      visible_queries_of_clean_key(a, CLEAN, k0 + TILE - 1, tmp, hi);
+      if (hi > lo) { tA0 = lo / HT; nA = (hi + HT - 1) / HT - tA0; }
+    }
+    if (a.q[NOISY] != nullptr) {
+      visible_queries_of_clean_key(a, NOISY, k0, lo, tmp);
+      visible_queries_of_clean_key(a, NOISY, k0 + TILE - 1, tmp, hi);
+      if (hi > lo) { tB0 = lo / HT; nB = (hi + HT - 1) / HT - tB0; }
+    }
   } else {
     const int lo = (k0 / M) * M, hi = min(L, ((k0 + TILE - 1) / M + 1) * M);
-    tA0 = lo / TILE; nA = (hi + TILE - 1) / TILE - tA0;
+    tA0 = lo / HT; nA = (hi + HT - 1) / HT - tA0;
   }
   const int per_head = nA + nB;
   const int nsteps = per_head * a.G;
-  auto step_of = [&](int i) {
+  int it_r = 0, it_h = hk * a.G;
+  auto step_cur = [&]() {
     QStep s;
-    const int hh = i / per_head, r = i - hh * per_head;
-    s.h = hk * a.G + hh;
-    if (r < nA) { s.qs = (ks == NOISY) ? NOISY : CLEAN; s.q0 = (tA0 + r) * TILE; }
-    else { s.qs = NOISY; s.q0 = (tB0 + r - nA) * TILE; }
+    s.h = it_h;
+    if (it_r < nA) { s.qs = (ks == NOISY) ? NOISY : CLEAN; s.q0 = (tA0 + it_r) * HT; }
+    else { s.qs = NOISY; s.q0 = (tB0 + it_r - nA) * HT; }
     return s;
   };
+  auto step_next = [&]() { if (++it_r == per_head) { it_r = 0; ++it_h; } };
 
   if (threadIdx.x == 0) {
-    if (base & 1023u) *abort_flag = 1; else *abort_flag = 0;
+    if (base & 1023u) *abort_flag = 1; else *abort_flag = 0;   // swizzled tiles need a 1024-byte aligned base
     mbar_init(bar_kv, 1);
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(bar_q_full + 8 * i, 1); mbar_init(bar_q_empty + 8 * i, 1);
-      mbar_init(bar_do_full + 8 * i, 2); mbar_init(bar_do_empty + 8 * i, 9);   // empty: dV done + 8 warps done with the D rows
-    }
-    mbar_init(bar_st, 1); mbar_init(bar_dpt, 1); mbar_init(bar_pt, 256); mbar_init(bar_dst, 256);
-    mbar_init(bar_dqf, 1); mbar_init(bar_dqr, 256); mbar_init(bar_done, 1);
+    for (int i = 0; i < 4; ++i) { mbar_init(bar_q_full + 8 * i, 1); mbar_init(bar_q_empty + 8 * i, 1); }
+    for (int i = 0; i < 3; ++i) { mbar_init(bar_do_full + 8 * i, 2); mbar_init(bar_do_empty + 8 * i, 9); }   // full: TMA bytes + LSE/D rows; empty: dV done + 8 compute warps done with the D rows
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_st + 8 * i, 1); mbar_init(bar_pt + 8 * i, 256); }
+    mbar_init(bar_dpt, 1); mbar_init(bar_dpfree, 256); mbar_init(bar_dst, 256); mbar_init(bar_dsfree, 1);
+    mbar_init(bar_dqf, 1); mbar_init(bar_dqr, 128); mbar_init(bar_done, 1);
     fence_mbar_init();
   }
   if (warp == 8) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
@@ -802,7 +834,6 @@ tc_bwd1p_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __rest
   tc_fence_after();
   const uint32_t tmem = __shfl_sync(0xffffffffu, *tmem_slot, 0);   // broadcast: provably warp-uniform
   const bool bad_base = (*abort_flag != 0);
-  // TMEM columns: [0,128) S^T / P^T   [128,256) dP^T, then dQ^T   [256,384) dV   [384,512) dK
 
   if (bad_base) {
     // fall through to the common exit
@@ -810,225 +841,311 @@ tc_bwd1p_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __rest
     // ------------------------------------------------------------------ producer
     if (lane == 0) {
       mbar_expect_tx(bar_kv, 2 * TILE_BYTES);
-      tma_tile(sK, &maps.k[ks], bar_kv, hk * 128, k0, b);
-      tma_tile(sV, &maps.v[ks], bar_kv, hk * 128, k0, b);
+      tma_tile(sK, &maps.k[ks], bar_kv, hk * 128, k0_row, b);
+      tma_tile(sV, &maps.v[ks], bar_kv, hk * 128, k0_row, b);
     }
     bool ok = true;
     long long w_empty = 0;
     const long long t_begin = tick<TR>();
+    int sd = 0, kd = 0;   // dO ring stage of step i and how many times the ring has wrapped
     for (int i = 0; i < nsteps && ok; ++i) {
-      const int sd = i & 1;
-      const QStep st = step_of(i);
-      if (i >= 2) ok = mbar_wait_timed<TR>(bar_q_empty + 8 * sd, ((i >> 1) - 1) & 1, abort_flag, w_empty);
+      const int sq = i & 3;
+      const QStep st = step_cur();
+      step_next();
+      if (i >= 4) ok = mbar_wait_timed<TR>(bar_q_empty + 8 * sq, ((i >> 2) - 1) & 1, abort_flag, w_empty);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       if (lane == 0) {
-        mbar_expect_tx(bar_q_full + 8 * sd, TILE_BYTES);
-        tma_tile(sQ0 + sd * TILE_BYTES, &maps.q[st.qs], bar_q_full + 8 * sd, st.h * 128, st.q0, b);
+        const uint32_t dst = sQ0 + sq * HT_BYTES, bar = bar_q_full + 8 * sq;
+        mbar_expect_tx(bar, HT_BYTES);
+        tma_load_3d(dst, &maps.q[st.qs], bar, st.h * 128, st.q0, b);
+        tma_load_3d(dst + HPANEL_BYTES, &maps.q[st.qs], bar, st.h * 128 + 64, st.q0, b);
       }
-      if (i >= 2) ok = mbar_wait_timed<TR>(bar_do_empty + 8 * sd, ((i >> 1) - 1) & 1, abort_flag, w_empty);
+      if (kd >= 1) ok = mbar_wait_timed<TR>(bar_do_empty + 8 * sd, (kd - 1) & 1, abort_flag, w_empty);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       if (lane == 0) {
-        mbar_expect_tx(bar_do_full + 8 * sd, TILE_BYTES);   // one arrival of two; the LSE/D rows follow
-        tma_tile(sdO0 + sd * TILE_BYTES, &maps.dout[st.qs], bar_do_full + 8 * sd, st.h * 128, st.q0, b);
+        const uint32_t dst = sdO0 + sd * HT_BYTES, bar = bar_do_full + 8 * sd;
+        mbar_expect_tx(bar, HT_BYTES);   // one arrival of two; the LSE/D rows follow
+        tma_load_3d(dst, &maps.dout[st.qs], bar, st.h * 128, st.q0, b);
+        tma_load_3d(dst + HPANEL_BYTES, &maps.dout[st.qs], bar, st.h * 128 + 64, st.q0, b);
       }
-      const float* lsep = a.lse[st.qs] + ((int64_t)b * a.H + st.h) * L + st.q0;
-      const float* dsp = a.dsum[st.qs] + ((int64_t)b * a.H + st.h) * L + st.q0;
-      {
-        const float4 z = reinterpret_cast<const float4*>(lsep)[lane];
-        const float4 dd = reinterpret_cast<const float4*>(dsp)[lane];
+      const int64_t row0 = ((int64_t)b * a.H + st.h) * rows_q(a, st.qs) + st.q0;
+      if (lane < 16) {
+        const float4 z = reinterpret_cast<const float4*>(a.lse[st.qs] + row0)[lane];
         float4 z2;
         z2.x = isfinite(z.x) ? z.x * LOG2E : INFINITY; z2.y = isfinite(z.y) ? z.y * LOG2E : INFINITY;
         z2.z = isfinite(z.z) ? z.z * LOG2E : INFINITY; z2.w = isfinite(z.w) ? z.w * LOG2E : INFINITY;
-        reinterpret_cast<float4*>(lse_s + sd * 128)[lane] = z2;
-        reinterpret_cast<float4*>(d_s + sd * 128)[lane] = dd;
+        reinterpret_cast<float4*>(lse_s + sd * 64)[lane] = z2;
+      } else {
+        reinterpret_cast<float4*>(d_s + sd * 64)[lane - 16] = reinterpret_cast<const float4*>(a.dsum[st.qs] + row0)[lane - 16];
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_do_full + 8 * sd);
+      if (++sd == 3) { sd = 0; ++kd; }
     }
-    if (lane == 0) { trace_add(a.trace, 16 + 12, tick<TR>() - t_begin); trace_add(a.trace, 16 + 13, w_empty); }
+    if (lane == 0) trace_add(a.trace, 16 + 13, w_empty);
   } else if (warp == 9) {
-    // ------------------------------------------------------------------ MMA issuer (one thread)
-    // the whole warp walks the MMA loop; one elected lane issues (see elect_one)
+    // ------------------------------------------------------------------ MMA issuer: the whole warp walks the loop,
+    // one elected lane issues (see elect_one)
     if (nsteps > 0) {
       const uint32_t el = elect_one();
+      long long w_pt = 0, w_dpf = 0, w_dst = 0, w_q = 0, w_do = 0;
       const long long t_begin = tick<TR>();
       const uint32_t k_lo = desc_lo_k(sK), v_lo = desc_lo_k(sV), kt_lo = desc_lo_mn(sK);
-      const uint32_t qk_lo0 = desc_lo_k(sQ0), qm_lo0 = desc_lo_mn(sQ0);
-      const uint32_t dok_lo0 = desc_lo_k(sdO0), dom_lo0 = desc_lo_mn(sdO0);
-      const uint32_t dsk_lo = desc_lo_k(sDS), dsm_lo = desc_lo_mn(sDS);
+      const uint32_t qk_lo0 = desc_lo_k(sQ0), qm_lo0 = desc_lo_mn_h(sQ0);       // Q ring, as K-major B (S^T) / MN-major B (dK)
+      const uint32_t dok_lo0 = desc_lo_k(sdO0), dom_lo0 = desc_lo_mn_h(sdO0);   // dO ring, as K-major B (dP^T) / MN-major B (dV)
+      const uint32_t dsk_lo = desc_lo_k(sDS), dsm_lo = desc_lo_k(sDS);          // dS^T: K-major A (dK) / MN-major B with one 64-query group (dQ^T)
+      auto issue_st = [&](int buf, int sq) {     // S^T = K Q^T into S^T buffer `buf`
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk)
+          mma_ss_e(tmem + 64 * buf, desc64(k_lo + koff(kk)), desc64(qk_lo0 + sq * HT_LO + koff_h(kk)), IDESC_N64, kk == 0 ? 0u : 1u, el);
+        mma_commit_e(bar_st + 8 * buf, el);
+      };
+      auto issue_dpt = [&](int sd) {             // dP^T = V dO^T
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk)
+          mma_ss_e(tmem + 128, desc64(v_lo + koff(kk)), desc64(dok_lo0 + sd * HT_LO + koff_h(kk)), IDESC_N64, kk == 0 ? 0u : 1u, el);
+        mma_commit_e(bar_dpt, el);
+      };
       bool ok = mbar_wait_abortable(bar_kv, 0, abort_flag);
       ok = ok && mbar_wait_abortable(bar_q_full, 0, abort_flag);
-      if (ok) {
-        tc_fence_after();
-        gemm_ss_e(tmem, k_lo, qk_lo0, IDESC_KK, 0u, el);
-        mma_commit_e(bar_st, el);
-      }
+      if (ok) { tc_fence_after(); issue_st(0, 0); }
       ok = ok && mbar_wait_abortable(bar_do_full, 0, abort_flag);
-      if (ok) {
-        tc_fence_after();
-        gemm_ss_e(tmem + 128, v_lo, dok_lo0, IDESC_KK, 0u, el);
-        mma_commit_e(bar_dpt, el);
-      }
+      if (ok) { tc_fence_after(); issue_dpt(0); }
+      int sd = 0, sn = 1, kn = 0;   // dO ring stage of step i, of step i + 1, and that one's wrap count
       for (int i = 0; i < nsteps && ok; ++i) {
-        const int sd = i & 1;
+        const int sb = i & 1, sq = i & 3, sqn = (i + 1) & 3;
         const uint32_t acc = i > 0 ? 1u : 0u;
-        // dV += P^T dO_i
-        ok = mbar_wait_lean(bar_pt, i & 1, abort_flag);
+        // S^T of the next step into the other buffer (its last reader, dV of step i-1, is ahead in the pipe)
+        if (i + 1 < nsteps) {
+          ok = mbar_wait_timed<TR>(bar_q_full + 8 * sqn, ((i + 1) >> 2) & 1, abort_flag, w_q);
+          if (!ok) break;
+          tc_fence_after();
+          issue_st(sb ^ 1, sqn);
+        }
+        // dV += P^T dO_i   (P^T: bf16 pairs at the start of each warpgroup's 32 S^T columns)
+        ok = mbar_wait_timed<TR>(bar_pt + 8 * sb, (i >> 1) & 1, abort_flag, w_pt);
         if (!ok) break;
         tc_fence_after();
-        gemm_ts_mn_cw_e<64>(tmem + 256, tmem, dom_lo0 + sd * TILE_LO, IDESC_KM, acc, el);
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+          mma_ts_e(tmem + 256, tmem + 64 * sb + (kk >> 1) * 32 + (kk & 1) * 8, desc64(dom_lo0 + sd * HT_LO + moff(kk)), IDESC_KM,
+                   kk == 0 ? acc : 1u, el);
         mma_commit_e(bar_do_empty + 8 * sd, el);
-        if (i + 1 < nsteps) {   // S^T of the next step
-          ok = mbar_wait_lean(bar_q_full + 8 * (sd ^ 1), ((i + 1) >> 1) & 1, abort_flag);
+        // dP^T of the next step, once every compute thread holds dP^T(i) in registers
+        if (i + 1 < nsteps) {
+          ok = mbar_wait_timed<TR>(bar_dpfree, i & 1, abort_flag, w_dpf);
+          ok = ok && mbar_wait_timed<TR>(bar_do_full + 8 * sn, kn & 1, abort_flag, w_do);
           if (!ok) break;
           tc_fence_after();
-          gemm_ss_e(tmem, k_lo, qk_lo0 + (sd ^ 1) * TILE_LO, IDESC_KK, 0u, el);
-          mma_commit_e(bar_st, el);
+          issue_dpt(sn);
         }
-        // dS^T(i) is in shared memory: dQ^T = K^T dS^T into the columns dP^T(i) occupied, then dK += dS^T Q_i
-        ok = mbar_wait_lean(bar_dst, i & 1, abort_flag);
+        // dQ^T = K^T dS^T (once the read-out warps hold the previous dQ^T), then dK += dS^T Q_i
+        ok = mbar_wait_timed<TR>(bar_dst, i & 1, abort_flag, w_dst);
+        if (i > 0) ok = ok && mbar_wait_timed<TR>(bar_dqr, (i - 1) & 1, abort_flag, w_dst);
         if (!ok) break;
         tc_fence_after();
-        gemm_ss_mm_e(tmem + 128, kt_lo, dsm_lo, IDESC_MM, 0u, el);
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk)
+          mma_ss_e(tmem + 192, desc64(kt_lo + moff(kk)), desc64(dsm_lo + moff(kk)), IDESC_DQT, kk == 0 ? 0u : 1u, el);
         mma_commit_e(bar_dqf, el);
-        gemm_ss_km_e(tmem + 384, dsk_lo, qm_lo0 + sd * TILE_LO, IDESC_KM, acc, el);
-        mma_commit_e(bar_q_empty + 8 * sd, el);
-        if (i + 1 < nsteps) {   // dP^T of the next step, once dQ^T(i) has been read out of those columns
-          ok = mbar_wait_lean(bar_dqr, i & 1, abort_flag);
-          ok = ok && mbar_wait_lean(bar_do_full + 8 * (sd ^ 1), ((i + 1) >> 1) & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-          gemm_ss_e(tmem + 128, v_lo, dok_lo0 + (sd ^ 1) * TILE_LO, IDESC_KK, 0u, el);
-          mma_commit_e(bar_dpt, el);
-        }
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+          mma_ss_e(tmem + 384, desc64(dsk_lo + 2 * kk), desc64(qm_lo0 + sq * HT_LO + moff(kk)), IDESC_KM, kk == 0 ? acc : 1u, el);
+        mma_commit_e(bar_q_empty + 8 * sq, el);
+        mma_commit_e(bar_dsfree, el);
+        sd = sn;
+        if (++sn == 3) { sn = 0; ++kn; }
       }
       mma_commit_e(bar_done, el);
-      if (lane == 0) trace_add(a.trace, 16 + 8, tick<TR>() - t_begin);
+      if (lane == 0) {
+        trace_add(a.trace, 16 + 8, tick<TR>() - t_begin); trace_add(a.trace, 16 + 9, w_pt);
+        trace_add(a.trace, 16 + 10, w_dpf); trace_add(a.trace, 16 + 11, w_dst);
+        trace_add(a.trace, 16 + 7, w_q); trace_add(a.trace, 16 + 12, w_do);
+      }
+    }
+  } else if (warp >= 10) {
+    // ------------------------------------------------------------------ dQ read-out warpgroup
+    const int dd = (warp & 3) * 32 + lane;                      // TMEM lane = head-dim index
+    const uint32_t tl = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+    const bool leader = threadIdx.x == 320;
+    bool ok = true;
+    long long w_dqf = 0, c_ro = 0;
+    for (int i = 0; i < nsteps; ++i) {
+      const QStep st = step_cur();
+      step_next();
+      // after a failed wait the warp still meets the others at the named barrier, then all leave together
+      if (ok) {
+        ok = mbar_wait_timed<TR>(bar_dqf, i & 1, abort_flag, w_dqf);
+        ok = __all_sync(0xffffffffu, ok);
+      }
+      const long long t0 = tick<TR>();
+      if (ok) tc_fence_after();
+      float* dst = a.dq32[st.qs] + (((int64_t)b * a.H + st.h) * rows_q(a, st.qs) + st.q0) * 128;
+      bool stop = false;
+      uint32_t v[64];
+      if (ok) {   // the whole tile into registers first: the tensor core gets its columns back at once
+        uint32_t (*c)[32] = reinterpret_cast<uint32_t (*)[32]>(v);
+        tmem_ld32(tl + 192, c[0]); tmem_ld32(tl + 224, c[1]);
+        tmem_wait_ld();
+        tc_fence_before();
+        mbar_arrive(bar_dqr);
+      }
+#pragma unroll
+      for (int qt = 0; qt < 4; ++qt) {   // 16 query columns at a time through staging tile `qt`
+        if (ok) {
+          // the reduction that read this staging tile last was waited for before the previous barrier
+          float* sg = reinterpret_cast<float*>(sm + BF_STG + qt * STG_BYTES) + dd;
+#pragma unroll
+          for (int e = 0; e < 16; ++e) sg[e * 128] = __uint_as_float(v[16 * qt + e]) * a.scale;
+          fence_async_smem();
+        }
+        if (leader) bulk_wait_read2();   // at most two reductions still reading: the next staging tile is free
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (*abort_flag) { stop = true; break; }
+        if (leader) {
+          bulk_reduce_add_f32(dst + qt * STG_ROWS * 128, sSTG + qt * STG_BYTES, STG_BYTES);
+          bulk_commit();
+        }
+      }
+      if (stop) break;
+      c_ro += tick<TR>() - t0;
+    }
+    if (leader) {
+      bulk_wait_all();
+      trace_add(a.trace, 16 + 14, w_dqf); trace_add(a.trace, 16 + 15, c_ro);
     }
   } else {
     // ------------------------------------------------------------------ compute warpgroups
-    const int w = warp >> 2;                                   // column half: query columns [64w, 64w+64)
-    const int r = (warp & 3) * 32 + lane;                      // TMEM lane: key row of S^T/dP^T, head-dim index of dQ^T
+    const int w = warp >> 2;                                   // column share: query columns [32 w, 32 w + 32) of the step's 64
+    const int r = (warp & 3) * 32 + lane;                      // TMEM lane = key row of the tile
     const int j = k0 + r;
     const uint32_t tl = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-    const int c0 = w * 64;
-    int vqc_lo, vqc_hi, vqn_lo, vqn_hi;   // query rows that see key j, per query stream
+    const int c0 = w * 32;
+    uint8_t* dsrow = sm + BF_DS + r * 128;                     // this thread's row of the dS^T tile
+    // query rows that see key j, per query stream (section 3.2 read from the key's side), and the bounds inside
+    // which a step needs no masking: every key row of this tile sees all of its queries
+    int vqc_lo = 0, vqc_hi = 0, vqn_lo, vqn_hi, fullc_lo = 0, fullc_hi = 0, fulln_lo, fulln_hi;
     if (ks == CLEAN) {
-      const int q_end = (a.window > 0) ? min(L, j + a.window) : L;
-      vqc_lo = (a.mode == 0) ? j : (j / M) * M; vqc_hi = q_end;
-      vqn_lo = (j / M + 1) * M; vqn_hi = q_end;
+      int tmp;
+      if (a.q[CLEAN] != nullptr) {
+        visible_queries_of_clean_key(a, CLEAN, j, vqc_lo, vqc_hi);
+        visible_queries_of_clean_key(a, CLEAN, k0 + TILE - 1, fullc_lo, tmp);
+        visible_queries_of_clean_key(a, CLEAN, k0, tmp, fullc_hi);
+      }
+      if (a.q[NOISY] != nullptr) {
+        visible_queries_of_clean_key(a, NOISY, j, vqn_lo, vqn_hi);
+        visible_queries_of_clean_key(a, NOISY, k0 + TILE - 1, fulln_lo, tmp);
+        visible_queries_of_clean_key(a, NOISY, k0, tmp, fulln_hi);
+      } else {
+        vqn_lo = vqn_hi = fulln_lo = fulln_hi = 0;
+      }
     } else {
-      vqc_lo = 0; vqc_hi = 0;
       vqn_lo = (j / M) * M; vqn_hi = vqn_lo + M;
+      fulln_lo = ((k0 + TILE - 1) / M) * M; fulln_hi = (k0 / M) * M + M;
     }
     bool ok = true;
-    long long w_st = 0, w_dpt = 0, w_dqf = 0;
+    long long w_st = 0, w_dpt = 0, w_dsf = 0, c_exp = 0, c_ds = 0;
     const long long t_begin = tick<TR>();
-    uint32_t x[64];   // P^T of the step in flight (fp32), kept from phase 1 to phase 2
-
-    // phase 1 of step i: P^T = exp2(S^T * scale - LSE) on visible pairs, bf16 pairs back into the S^T columns
-    auto phase1 = [&](int i) {
-      const int sd = i & 1;
-      const QStep st = step_of(i);
-      int lo_a, hi_a, lo_b, hi_b;
-      visible_interval(a, st.qs, ks, st.q0, lo_a, hi_a);
-      visible_interval(a, st.qs, ks, st.q0 + TILE - 1, lo_b, hi_b);
-      const bool need_mask = (lo_b > k0) || (hi_a < k0 + TILE);
-      ok = mbar_wait_timed<TR>(bar_do_full + 8 * sd, (i >> 1) & 1, abort_flag, w_st);
-      ok = ok && mbar_wait_timed<TR>(bar_st, i & 1, abort_flag, w_st);
+    int sd = 0, kd = 0;   // dO ring stage of step i and its wrap count
+    for (int i = 0; i < nsteps; ++i) {
+      const int sb = i & 1;
+      const QStep st = step_cur();
+      step_next();
+      const bool need_mask = (st.qs == CLEAN) ? (st.q0 < fullc_lo || st.q0 + HT > fullc_hi)
+                                              : (st.q0 < fulln_lo || st.q0 + HT > fulln_hi);
+      ok = mbar_wait_timed<TR>(bar_do_full + 8 * sd, kd & 1, abort_flag, w_st);
+      ok = ok && mbar_wait_timed<TR>(bar_st + 8 * sb, (i >> 1) & 1, abort_flag, w_st);
       ok = __all_sync(0xffffffffu, ok);
-      if (!ok) return;
+      if (!ok) break;
       tc_fence_after();
-      {
-        uint32_t (*c)[32] = reinterpret_cast<uint32_t (*)[32]>(x);
-        tmem_ld32(tl + c0, c[0]); tmem_ld32(tl + c0 + 32, c[1]);
-        tmem_wait_ld();
-      }
-      const float* lz = lse_s + sd * 128 + c0;
+      const long long t0 = tick<TR>();
+      uint32_t x[32];
+      tmem_ld32(tl + 64 * sb + c0, x);
+      tmem_wait_ld();
+      const float4* lz4 = reinterpret_cast<const float4*>(lse_s + sd * 64 + c0);
       if (!need_mask) {
 #pragma unroll
-        for (int c = 0; c < 64; ++c) x[c] = __float_as_uint(exp2f(fmaf(__uint_as_float(x[c]), a.scale_log2, -lz[c])));
+        for (int c4 = 0; c4 < 8; ++c4) {
+          const float4 z = lz4[c4];
+          float* xf = reinterpret_cast<float*>(x) + 4 * c4;
+          xf[0] = exp2f(fmaf(xf[0], a.scale_log2, -z.x));
+          xf[1] = exp2f(fmaf(xf[1], a.scale_log2, -z.y));
+          xf[2] = exp2f(fmaf(xf[2], a.scale_log2, -z.z));
+          xf[3] = exp2f(fmaf(xf[3], a.scale_log2, -z.w));
+        }
       } else {
+        // visible columns of this thread's key row inside the step: [vlo, vhi)
         const int vlo = (st.qs == CLEAN ? vqc_lo : vqn_lo) - st.q0 - c0, vhi = (st.qs == CLEAN ? vqc_hi : vqn_hi) - st.q0 - c0;
 #pragma unroll
-        for (int c = 0; c < 64; ++c) {
-          const float p = exp2f(fmaf(__uint_as_float(x[c]), a.scale_log2, -lz[c]));
-          x[c] = __float_as_uint((c >= vlo && c < vhi) ? p : 0.f);
+        for (int c4 = 0; c4 < 8; ++c4) {
+          const float4 z = lz4[c4];
+          const float zz[4] = {z.x, z.y, z.z, z.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int c = 4 * c4 + e;
+            const float p = exp2f(fmaf(__uint_as_float(x[c]), a.scale_log2, -zz[e]));
+            x[c] = __float_as_uint((c >= vlo && c < vhi) ? p : 0.f);
+          }
         }
       }
-      uint32_t pk[32];
+      {
+        uint32_t pk[16];
 #pragma unroll
-      for (int e = 0; e < 32; ++e) pk[e] = pack_bf16(__uint_as_float(x[2 * e]), __uint_as_float(x[2 * e + 1]));
-      tmem_st32(tl + c0, pk);
-      tmem_wait_st();
+        for (int e = 0; e < 16; ++e) pk[e] = pack_bf16(__uint_as_float(x[2 * e]), __uint_as_float(x[2 * e + 1]));
+        tmem_st16(tl + 64 * sb + c0, pk);
+        tmem_wait_st();
+      }
       tc_fence_before();
-      mbar_arrive(bar_pt);
-    };
+      mbar_arrive(bar_pt + 8 * sb);
+      const long long t1 = tick<TR>();
+      c_exp += t1 - t0;
 
-    if (nsteps > 0) phase1(0);
-    for (int i = 0; i < nsteps && ok; ++i) {
-      const int sd = i & 1;
-      // phase 2: dS^T = P^T * (dP^T - D), bf16, into the shared-memory tile (row = key, this half's 64 query columns)
       ok = mbar_wait_timed<TR>(bar_dpt, i & 1, abort_flag, w_dpt);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
+      const long long t2 = tick<TR>();
+      uint32_t pk[16];
       {
-        uint32_t y[64];
-        uint32_t (*c)[32] = reinterpret_cast<uint32_t (*)[32]>(y);
-        tmem_ld32(tl + 128 + c0, c[0]); tmem_ld32(tl + 128 + c0 + 32, c[1]);
+        uint32_t y[32];
+        tmem_ld32(tl + 128 + c0, y);
         tmem_wait_ld();
-        const float* dz = d_s + sd * 128 + c0;
-        uint8_t* rowp = sm + P1_DS + w * PANEL_BYTES + r * 128;
+        tc_fence_before();
+        mbar_arrive(bar_dpfree);   // dP^T(i) is in registers: the tensor core may overwrite its columns
+        const float4* dz4 = reinterpret_cast<const float4*>(d_s + sd * 64 + c0);
 #pragma unroll
-        for (int c8 = 0; c8 < 8; ++c8) {
-          uint4 v;
-          uint32_t* pv = reinterpret_cast<uint32_t*>(&v);
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const int c = c8 * 8 + 2 * e;
-            const float d0 = __uint_as_float(x[c]) * (__uint_as_float(y[c]) - dz[c]);
-            const float d1 = __uint_as_float(x[c + 1]) * (__uint_as_float(y[c + 1]) - dz[c + 1]);
-            pv[e] = pack_bf16(d0, d1);
-          }
-          *reinterpret_cast<uint4*>(rowp + ((c8 ^ (r & 7)) << 4)) = v;
+        for (int c4 = 0; c4 < 8; ++c4) {
+          const float4 dz = dz4[c4];
+          const float d0 = __uint_as_float(x[4 * c4 + 0]) * (__uint_as_float(y[4 * c4 + 0]) - dz.x);
+          const float d1 = __uint_as_float(x[4 * c4 + 1]) * (__uint_as_float(y[4 * c4 + 1]) - dz.y);
+          const float d2 = __uint_as_float(x[4 * c4 + 2]) * (__uint_as_float(y[4 * c4 + 2]) - dz.z);
+          const float d3 = __uint_as_float(x[4 * c4 + 3]) * (__uint_as_float(y[4 * c4 + 3]) - dz.w);
+          pk[2 * c4] = pack_bf16(d0, d1);
+          pk[2 * c4 + 1] = pack_bf16(d2, d3);
         }
       }
-      tc_fence_before();
+      c_ds += tick<TR>() - t2;
+      // dS^T(i) into the shared-memory tile, once dK and dQ^T of step i-1 have read dS^T(i-1)
+      if (i > 0) {
+        ok = mbar_wait_timed<TR>(bar_dsfree, (i - 1) & 1, abort_flag, w_dsf);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+      }
+#pragma unroll
+      for (int c8 = 0; c8 < 4; ++c8)
+        *reinterpret_cast<uint4*>(dsrow + (((4 * w + c8) ^ (r & 7)) << 4)) = make_uint4(pk[4 * c8], pk[4 * c8 + 1], pk[4 * c8 + 2], pk[4 * c8 + 3]);
       fence_async_smem();
       mbar_arrive(bar_dst);
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_do_empty + 8 * sd);   // this warp is done with the stage's D rows
-
-      // phase 1 of the next step runs before this step's dQ^T read-out: dQ^T(i) is still being computed
-      if (i + 1 < nsteps) { phase1(i + 1); if (!ok) break; }
-
-      // read-out: dQ[q, h, d] += scale * dQ^T[d, q]; this thread is head-dim element d = r of the step's query rows
-      ok = mbar_wait_timed<TR>(bar_dqf, i & 1, abort_flag, w_dqf);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      tc_fence_after();
-      {
-        const QStep st = step_of(i);
-        float* dst = a.dq32[st.qs] + (((int64_t)b * L + st.q0 + c0) * a.H + st.h) * 128 + r;
-        const int64_t qstride = (int64_t)a.H * 128;
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t v[32];
-          tmem_ld32(tl + 128 + c0 + c * 32, v);
-          tmem_wait_ld();
-#pragma unroll
-          for (int e = 0; e < 32; ++e) atomicAdd(dst + (c * 32 + e) * qstride, __uint_as_float(v[e]) * a.scale);
-        }
-      }
-      tc_fence_before();
-      mbar_arrive(bar_dqr);
+      if (++sd == 3) { sd = 0; ++kd; }
     }
     if (warp == 0 && lane == 0) {
       trace_add(a.trace, 16 + 0, nsteps); trace_add(a.trace, 16 + 1, w_st); trace_add(a.trace, 16 + 2, w_dpt);
-      trace_add(a.trace, 16 + 3, w_dqf); trace_add(a.trace, 16 + 6, tick<TR>() - t_begin);
+      trace_add(a.trace, 16 + 3, w_dsf); trace_add(a.trace, 16 + 4, c_exp); trace_add(a.trace, 16 + 5, c_ds);
+      trace_add(a.trace, 16 + 6, tick<TR>() - t_begin);
     }
     // epilogue: warpgroup 0 writes dV, warpgroup 1 writes dK (scaled)
     if (ok && nsteps > 0) {
@@ -1037,13 +1154,16 @@ tc_bwd1p_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __rest
     }
     if (ok) {
       tc_fence_after();
-      bf16* dst = (w == 0 ? a.dv[ks] : a.dk[ks]) + (((int64_t)b * L + j) * a.Hkv + hk) * 128;
+      bf16* dst = (w == 0 ? a.dv[ks] : a.dk[ks]) + (((int64_t)b * L + k0_row + r) * a.Hkv + hk) * 128;
       const float sc = (w == 0) ? 1.f : a.scale;
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         uint32_t v[32];
-        tmem_ld32(tl + 256 + w * 128 + c * 32, v);
-        tmem_wait_ld();
+        if (nsteps > 0) { tmem_ld32(tl + 256 + w * 128 + c * 32, v); tmem_wait_ld(); }
+        else {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) v[e] = 0u;
+        }
         store_row_chunk(dst + c * 32, v, sc);
       }
     }
@@ -1054,13 +1174,18 @@ tc_bwd1p_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __rest
   if (warp == 8) tmem_dealloc(tmem, 512);
 }
 
-// fp32 dQ accumulator -> bf16 dQ
-__global__ void __launch_bounds__(256) dq_convert_kernel(const float* __restrict__ src, bf16* __restrict__ dst, int64_t n8) {
-  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += (int64_t)gridDim.x * blockDim.x) {
-    const float4 u = reinterpret_cast<const float4*>(src)[2 * i], v = reinterpret_cast<const float4*>(src)[2 * i + 1];
-    uint4 o;
-    o.x = pack_bf16(u.x, u.y); o.y = pack_bf16(u.z, u.w); o.z = pack_bf16(v.x, v.y); o.w = pack_bf16(v.z, v.w);
-    reinterpret_cast<uint4*>(dst)[i] = o;
+// fp32 dQ accumulator [batch, H, rows, 128] -> bf16 dQ [batch, rows, H, 128]; one warp per 128-element row
+__global__ void __launch_bounds__(256) dq_convert_kernel(const float* __restrict__ src, bf16* __restrict__ dst, int batch, int H, int rows) {
+  const int lane = threadIdx.x & 31;
+  const int64_t n = (int64_t)batch * rows * H;
+  for (int64_t o = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5); o < n; o += (int64_t)gridDim.x * 8) {
+    const int h = (int)(o % H);
+    const int64_t bl = o / H;
+    const int l = (int)(bl % rows), b = (int)(bl / rows);
+    const float4 u = reinterpret_cast<const float4*>(src + (((int64_t)b * H + h) * rows + l) * 128)[lane];
+    uint2 v;
+    v.x = pack_bf16(u.x, u.y); v.y = pack_bf16(u.z, u.w);
+    reinterpret_cast<uint2*>(dst + o * 128)[lane] = v;
   }
 }
 
@@ -1069,26 +1194,30 @@ __global__ void __launch_bounds__(256) dq_convert_kernel(const float* __restrict
 bool tc_bwd_supported(const KArgs& a) {
   return a.d == 128 && tc_rows_ok(a) && tc_encoder_available();
 }
-// fp32 dQ accumulators of the single-pass backward: one [batch, L, H, 128] tensor per stream
-size_t tc_bwd_extra_workspace(const bdlm_params* p) {
-  if (!p->bwd_single_pass || p->d != 128 || p->L % TILE != 0 || p->impl == 1) return 0;
-  return 2 * (size_t)p->batch * p->L * p->H * 128 * sizeof(float);
+// fp32 dQ accumulators of the fused backward: one [batch, H, rows, 128] tensor per query stream
+size_t tc_bwd_extra_workspace(const bdlm_params* p, const bdlm_packed_geometry* g) {
+  if (!p->bwd_single_pass || p->d != 128 || p->impl == 1) return 0;
+  const size_t rows_c = g != nullptr ? (size_t)g->Lq_clean : (size_t)p->L;
+  const size_t rows_n = g != nullptr ? (size_t)g->n_blocks * p->block_size : (size_t)p->L;
+  return (rows_c + rows_n) * p->batch * p->H * 128 * sizeof(float);
 }
 
 cudaError_t launch_tc_bwd(const KArgs& a_in, void* extra_ws, int passes, cudaStream_t st) {
   KArgs a = a_in;
-  const size_t dq32_elems = (size_t)a.batch * a.L * a.H * 128;
+  const size_t dq32_elems[2] = {a.q[CLEAN] != nullptr ? (size_t)a.batch * a.H * a.Lqc * 128 : 0,
+                                a.q[NOISY] != nullptr ? (size_t)a.batch * a.H * a.Ln * 128 : 0};
   if (a.single_pass) {
     a.dq32[0] = static_cast<float*>(extra_ws);
-    a.dq32[1] = a.dq32[0] + dq32_elems;
+    a.dq32[1] = a.dq32[0] + dq32_elems[0];
   }
   BwdMaps maps;
   for (int s = 0; s < 2; ++s) {
     // a stream that is left out gets the other stream's tensors as placeholders: its maps are never used
     const int sq = a.q[s] != nullptr ? s : 1 - s;
     const int sk = a.k[s] != nullptr ? s : CLEAN;
-    if (!tc_make_map(&maps.q[s], a.q[sq], a.H, rows_q(a, sq), a.batch, TILE)) return cudaErrorInvalidValue;
-    if (!tc_make_map(&maps.dout[s], a.dout[sq], a.H, rows_q(a, sq), a.batch, TILE)) return cudaErrorInvalidValue;
+    const int qbox = a.single_pass ? HT : TILE;   // the fused kernel loads 64 query rows per step
+    if (!tc_make_map(&maps.q[s], a.q[sq], a.H, rows_q(a, sq), a.batch, qbox)) return cudaErrorInvalidValue;
+    if (!tc_make_map(&maps.dout[s], a.dout[sq], a.H, rows_q(a, sq), a.batch, qbox)) return cudaErrorInvalidValue;
     if (!tc_make_map(&maps.k[s], a.k[sk], a.Hkv, rows_k(a, sk), a.batch, TILE)) return cudaErrorInvalidValue;
     if (!tc_make_map(&maps.v[s], a.v[sk], a.Hkv, rows_k(a, sk), a.batch, TILE)) return cudaErrorInvalidValue;
   }
@@ -1096,16 +1225,17 @@ cudaError_t launch_tc_bwd(const KArgs& a_in, void* extra_ws, int passes, cudaStr
   if (status == nullptr) return cudaErrorUnknown;
   cudaError_t e;
   if (a.single_pass) {
-    // one kernel produces dK, dV and (through fp32 atomics) dQ; it runs for the DKDV pass bit, the DQ bit is a no-op
+    // one kernel produces dK, dV and (through fp32 add-reductions) dQ; it runs for the DKDV pass bit, the DQ bit is a no-op
     if (passes & BDLM_BWD_PASS_DKDV) {
-      if ((e = cudaMemsetAsync(a.dq32[0], 0, 2 * dq32_elems * sizeof(float), st)) != cudaSuccess) return e;
-      auto kern = a.trace ? tc_bwd1p_kernel<true> : tc_bwd1p_kernel<false>;
-      if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, P1_SMEM)) != cudaSuccess) return e;
-      dim3 grid(a.L / TILE, a.Hkv, a.batch * 2);
-      kern<<<grid, BWD_THREADS, P1_SMEM, st>>>(maps, a, status);
+      if ((e = cudaMemsetAsync(a.dq32[0], 0, (dq32_elems[0] + dq32_elems[1]) * sizeof(float), st)) != cudaSuccess) return e;
+      auto kern = a.trace ? tc_bwdf_kernel<true> : tc_bwdf_kernel<false>;
+      if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, BF_SMEM)) != cudaSuccess) return e;
+      dim3 grid(max(a.L, a.k[NOISY] != nullptr ? a.Ln : 0) / TILE, a.Hkv, a.batch * 2);
+      kern<<<grid, BF_THREADS, BF_SMEM, st>>>(maps, a, status);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
       for (int s2 = 0; s2 < 2; ++s2) {
-        dq_convert_kernel<<<148 * 8, 256, 0, st>>>(a.dq32[s2], a.dq[s2], (int64_t)(dq32_elems / 8));
+        if (dq32_elems[s2] == 0) continue;
+        dq_convert_kernel<<<148 * 8, 256, 0, st>>>(a.dq32[s2], a.dq[s2], a.batch, a.H, rows_q(a, s2));
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
       }
     }

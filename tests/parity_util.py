@@ -42,7 +42,7 @@ def gpu_bwd(g, fwd_out, M, do_clean=None, do_noisy=None, **kw):
                                  g["do_noisy"] if do_noisy is None else do_noisy, M, **kw)
 
 
-def check_full(w, impl, mode=0, check_bwd=True, inp=None):
+def check_full(w, impl, mode=0, check_bwd=True, inp=None, single_pass=False):
     """Whole-tensor parity against the full oracle (small shapes)."""
     inp = synth.make_inputs(w, "cpu") if inp is None else inp
     g = to_cuda(inp)
@@ -58,7 +58,7 @@ def check_full(w, impl, mode=0, check_bwd=True, inp=None):
         assert err <= (TOL_LSE if "lse" in name else TOL_O), (name, err)
     if not check_bwd:
         return
-    grads = gpu_bwd(g, out, M, clean_mask_mode=mode, impl=impl, window=w.window)
+    grads = gpu_bwd(g, out, M, clean_mask_mode=mode, impl=impl, window=w.window, single_pass=single_pass)
     torch.cuda.synchronize()
     gref = orc.attn_backward(*[x[n] for n in NAMES6], x["do_clean"], x["do_noisy"], M, clean_mask_mode=mode,
                              window=w.window)
@@ -70,7 +70,7 @@ def check_full(w, impl, mode=0, check_bwd=True, inp=None):
     assert binding.bdlm_get_device_status() == 0
 
 
-def check_sampled(w, impl, n_rows=256, g=None, fwd_out=None, check_bwd=True, report=None):
+def check_sampled(w, impl, n_rows=256, g=None, fwd_out=None, check_bwd=True, report=None, single_pass=False):
     """Sampled-row parity for sizes the full oracle cannot do: per (batch, head, stream)
     `n_rows` stratified query rows are recomputed by the oracle.  O and LSE come from the
     full forward.  dQ at the sampled rows comes from the full backward (a row's dQ depends on
@@ -90,13 +90,14 @@ def check_sampled(w, impl, n_rows=256, g=None, fwd_out=None, check_bwd=True, rep
                 rows_of[(b, h, s)] = synth.sample_rows(w, n_rows, seed=1000 * b + 10 * h + s)
     grads = grads_sp = None
     if check_bwd:
-        grads = gpu_bwd(g, fwd_out, M, impl=impl, window=w.window)
+        grads = gpu_bwd(g, fwd_out, M, impl=impl, window=w.window, single_pass=single_pass)
         do_sp = [torch.zeros_like(g["do_clean"]), torch.zeros_like(g["do_noisy"])]
         for (b, h, s), rows in rows_of.items():
             r = torch.from_numpy(rows).cuda()
             src = g["do_clean"] if s == 0 else g["do_noisy"]
             do_sp[s][b, r, h] = src[b, r, h]
-        grads_sp = gpu_bwd(g, fwd_out, M, do_clean=do_sp[0], do_noisy=do_sp[1], impl=impl, window=w.window)
+        grads_sp = gpu_bwd(g, fwd_out, M, do_clean=do_sp[0], do_noisy=do_sp[1], impl=impl, window=w.window,
+                           single_pass=single_pass)
         torch.cuda.synchronize()
         assert binding.bdlm_get_device_status() == 0
     worst = {"o": 0.0, "lse": 0.0, "dq": 0.0, "dk": 0.0, "dv": 0.0}
@@ -143,7 +144,7 @@ def check_sampled(w, impl, n_rows=256, g=None, fwd_out=None, check_bwd=True, rep
     return worst
 
 
-def check_sampled_packed(w, impl, n_rows=256):
+def check_sampled_packed(w, impl, n_rows=256, single_pass=False):
     """Sampled-row parity of a packed (DFlash2-style) workload: O, LSE and dQ at sampled packed rows of
     every (batch, head); dK/dV of the clean and the packed noisy keys through a second backward whose dO is
     zero outside the sampled rows (dK/dV are linear in dO)."""
@@ -154,7 +155,7 @@ def check_sampled_packed(w, impl, n_rows=256):
     args = [g[n] for n in NAMES6]
     out = binding.bdlm_attn_fwd_packed(*args, M, block_prefix=pfx, impl=impl)
     grads = binding.bdlm_attn_bwd_packed(*args, out[0], out[1], out[2], out[3], None, g["do_noisy"], M,
-                                         block_prefix=pfx, impl=impl)
+                                         block_prefix=pfx, impl=impl, single_pass=single_pass)
     Ln = w.n_blocks * M
     G = w.H // w.H_kv
     rng = np.random.default_rng(17)
@@ -169,7 +170,7 @@ def check_sampled_packed(w, impl, n_rows=256):
             r = torch.from_numpy(rows).cuda()
             do_sp[b, r, h] = g["do_noisy"][b, r, h]
     grads_sp = binding.bdlm_attn_bwd_packed(*args, out[0], out[1], out[2], out[3], None, do_sp, M,
-                                            block_prefix=pfx, impl=impl)
+                                            block_prefix=pfx, impl=impl, single_pass=single_pass)
     torch.cuda.synchronize()
     assert binding.bdlm_get_device_status() == 0
     worst = {"o": 0.0, "lse": 0.0, "dq": 0.0, "dk": 0.0, "dv": 0.0}

@@ -41,6 +41,14 @@ def test_random_plain_configurations(case):
     pu.check_full(w, binding.IMPL_AUTO, mode=mode)
 
 
+@pytest.mark.parametrize("case", [c for c in _plain_cases(24, 2024) if c[0].d == 128 and c[0].L % 128 == 0],
+                         ids=lambda c: f"{c[0].name}-L{c[0].L}-M{c[0].block_size}-H{c[0].H}/{c[0].H_kv}-w{c[0].window}-m{c[1]}")
+def test_random_plain_configurations_fused_backward(case):
+    """The tensor-core shaped cases again through the fused one-kernel backward."""
+    w, mode = case
+    pu.check_full(w, binding.IMPL_AUTO, mode=mode, single_pass=True)
+
+
 def _packed_cases(n, seed):
     rng = np.random.default_rng(seed)
     cases = []
@@ -74,6 +82,9 @@ def _packed_cases(n, seed):
 def test_random_packed_configurations(c):
     t = _draw(c["seed"], 1, c["Lk"], c["Lq"], c["Ln"], c["H"], c["Hkv"], c["d"])
     _run_and_check(t, c["M"], binding.IMPL_AUTO, prefix=c["prefix"], pos0=c["pos0"], window=c["window"], mode=c["mode"])
+    if c["d"] == 128 and c["Lk"] % 128 == 0 and c["Lq"] % 128 == 0 and c["Ln"] % 128 == 0:   # tensor-core shaped: also the fused backward
+        _run_and_check(t, c["M"], binding.IMPL_AUTO, prefix=c["prefix"], pos0=c["pos0"], window=c["window"], mode=c["mode"],
+                       single_pass=True)
 
 
 @pytest.mark.parametrize("seed", range(6))

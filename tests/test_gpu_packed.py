@@ -34,7 +34,7 @@ def _f64(t):
     return {k: (None if v is None else synth.to_f64(v)) for k, v in t.items()}
 
 
-def _run_and_check(t, M, impl, prefix=None, pos0=0, window=0, mode=0):
+def _run_and_check(t, M, impl, prefix=None, pos0=0, window=0, mode=0, single_pass=False):
     g, x = _cuda(t), _f64(t)
     pfx_dev = None if prefix is None else torch.tensor(prefix, dtype=torch.int32, device="cuda")
     kw = dict(block_prefix=pfx_dev, clean_q_pos0=pos0, impl=impl, window=window, clean_mask_mode=mode)
@@ -42,7 +42,7 @@ def _run_and_check(t, M, impl, prefix=None, pos0=0, window=0, mode=0):
                                        g["v_noisy"], M, **kw)
     grads = binding.bdlm_attn_bwd_packed(g["q_clean"], g["k_clean"], g["v_clean"], g["q_noisy"], g["k_noisy"],
                                          g["v_noisy"], out[0], out[1], out[2], out[3], g["do_clean"],
-                                         g["do_noisy"], M, **kw)
+                                         g["do_noisy"], M, single_pass=single_pass, **kw)
     torch.cuda.synchronize()
     assert binding.bdlm_get_device_status() == 0
     kn = x["k_noisy"] if x["k_noisy"] is not None else np.zeros((x["k_clean"].shape[0], M) + x["k_clean"].shape[2:])
@@ -108,6 +108,22 @@ def test_packed_with_sliding_window(impl):
     prefix = [b * 64 for b in (1, 5, 8, 11)]
     _run_and_check(t, 64, impl, prefix=prefix, pos0=640, window=200)
     _run_and_check(t, 64, impl, prefix=prefix, pos0=0, window=33)
+
+
+def test_fused_backward_on_packed_forms():
+    """The fused one-kernel backward on the packed forms: sampled blocks alone, a clean run at an offset, both
+    streams with a prefix table (both mask modes), a sliding window."""
+    rng = np.random.default_rng(5)
+    t = _draw(21, 1, 512, 0, 16 * 16, 4, 2, 128)
+    _run_and_check(t, 16, binding.IMPL_AUTO, prefix=sorted(int(v) for v in rng.integers(0, 513, size=16)), single_pass=True)
+    t = _draw(22, 2, 512, 128, 0, 4, 2, 128)
+    _run_and_check(t, 32, binding.IMPL_AUTO, pos0=256, single_pass=True)
+    t = _draw(23, 1, 512, 256, 256, 2, 1, 128)
+    for mode in (0, 1):
+        _run_and_check(t, 32, binding.IMPL_AUTO, prefix=[b * 32 for b in (0, 3, 4, 9, 10, 12, 14, 15)], pos0=128, mode=mode,
+                       single_pass=True)
+    t = _draw(24, 1, 768, 128, 256, 2, 1, 128)
+    _run_and_check(t, 64, binding.IMPL_AUTO, prefix=[b * 64 for b in (1, 5, 8, 11)], pos0=640, window=200, single_pass=True)
 
 
 def test_portable_kernels_take_ragged_packed_shapes():

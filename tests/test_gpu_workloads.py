@@ -19,6 +19,19 @@ def test_sampled_rows_full_size(name):
     print(name, worst)
 
 
+@pytest.mark.parametrize("name", ["32k", "32k_w1024"])
+def test_sampled_rows_full_size_fused_backward(name):
+    """The same check with the fused one-kernel backward, the configuration bench.py times."""
+    w = WORKLOADS[name]
+    worst = pu.check_sampled(w, binding.IMPL_AUTO, single_pass=True)
+    print(name, "fused", worst)
+
+
+def test_dflash32k_sampled_rows_fused_backward():
+    worst = pu.check_sampled_packed(WORKLOADS["dflash32k"], binding.IMPL_AUTO, single_pass=True)
+    print("dflash32k fused", worst)
+
+
 def test_dflash32k_sampled_rows():
     """DFlash2-shaped packed workload at the size bench.py runs it (2048 sampled blocks over 32K clean keys)."""
     worst = pu.check_sampled_packed(WORKLOADS["dflash32k"], binding.IMPL_AUTO)
