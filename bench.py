@@ -248,6 +248,7 @@ def run_ours(args, w):
     M = w.block_size
     g = synth.make_inputs(synth.small(w, seed=w.seed + rank), "cuda")
     impl = args.kernel_impl
+    fused = args.bwd == "fused"
 
     def like(t):
         return None if t is None else torch.empty_like(t)
@@ -261,8 +262,11 @@ def run_ours(args, w):
         gr = tuple(like(gg[n]) for n in NAMES6)
         rows = max(t.shape[1] for t in (gg["q_clean"], gg["q_noisy"]) if t is not None)
         wsz = 2 * (w.batch * w.H * rows * 4 + 256)
+        if fused:   # fp32 dQ accumulators of the fused backward, one per query stream
+            wsz += sum(t.shape[1] for t in (gg["q_clean"], gg["q_noisy"]) if t is not None) * w.batch * w.H * w.d * 4
         if not w.packed:
-            wsz = max(wsz, binding.bdlm_workspace_bytes(binding.make_params(w.batch, w.L, M, w.H, w.H_kv, w.d),
+            wsz = max(wsz, binding.bdlm_workspace_bytes(binding.make_params(w.batch, w.L, M, w.H, w.H_kv, w.d,
+                                                                            bwd_single_pass=fused),
                                                         binding.BDLM_WS_BWD))
         return fo, gr, torch.empty(wsz, dtype=torch.uint8, device="cuda")
 
@@ -277,11 +281,11 @@ def run_ours(args, w):
         if w.packed:
             binding.bdlm_attn_bwd_packed(*[gg[n] for n in NAMES6], fo[0], fo[1], fo[2], fo[3], gg["do_clean"],
                                          gg["do_noisy"], M, block_prefix=gg["block_prefix"], out=gr, workspace=wsb,
-                                         impl=impl, passes=passes, window=w.window)
+                                         impl=impl, passes=passes, window=w.window, single_pass=fused)
         else:
             binding.bdlm_attn_bwd(*[gg[n] for n in NAMES6], fo[0], fo[1], fo[2], fo[3], gg["do_clean"],
                                   gg["do_noisy"], M, out=gr, workspace=wsb, impl=impl, passes=passes,
-                                  window=w.window)
+                                  window=w.window, single_pass=fused)
 
     fwd_out, grads, ws = make_buffers(g)
 
@@ -300,7 +304,9 @@ def run_ours(args, w):
 
     # ---- timed region: K steps, device time, events between the kernels of a step -------------
     K = args.steps
-    names = ["fwd", "bwd_dsum", "bwd_dkdv", "bwd_dq"]
+    # two-pass backward: dK/dV pass, then dQ pass; fused backward: one kernel for both (launched by the DKDV
+    # pass bit together with the zero-fill of the fp32 dQ accumulators and their conversion; the DQ bit is a no-op)
+    names = ["fwd", "bwd_dsum", "bwd_fused" if fused else "bwd_dkdv", "bwd_dq"]
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(len(names) + 1)] for _ in range(K)]
     sampler = ClockSampler(physical_gpu_index(local))
     if rank == 0:
@@ -401,8 +407,10 @@ def run_ours(args, w):
     # ---- roofline of the dominant kernel (tensor-bound: algorithmic FLOPs / device time) -------
     # The counted backward is 5 GEMMs per pair (S, dP, dV, dK, dQ = 10d FLOPs).  The dK/dV pass owns
     # four of them (8d); the dQ pass owns dQ (2d) -- its recomputation of S and dP is not counted.
-    algo_flops = {"fwd": f_fwd, "bwd_dkdv": f_bwd * 0.8, "bwd_dq": f_bwd * 0.2, "bwd_dsum": 0.0}
-    dom = max(("fwd", "bwd_dkdv", "bwd_dq"), key=lambda n: per_kernel_ms[n])
+    # The fused kernel owns all five.
+    algo_flops = {"fwd": f_fwd, "bwd_dkdv": f_bwd * 0.8, "bwd_dq": 0.0 if fused else f_bwd * 0.2, "bwd_dsum": 0.0,
+                  "bwd_fused": f_bwd}
+    dom = max((n for n in names if n != "bwd_dsum"), key=lambda n: per_kernel_ms[n])
     peak = peaks["bf16_tflops_sustained"] if ms_step * K > 1000.0 else peaks["bf16_tflops"]
     achieved = algo_flops[dom] / (per_kernel_ms[dom] * 1e-3) / 1e12
     roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
@@ -431,11 +439,12 @@ def run_ours(args, w):
             "config": {"workload": w.name, "batch": w.batch, "H": w.H, "H_kv": w.H_kv, "d": w.d, "L": w.L,
                        "block_size": w.block_size, "window": w.window, "n_blocks": w.n_blocks, "rope_theta": w.rope_theta, "parallelism": "replicas only",
                        "l2": "inputs larger than L2 (q/k/v/dO of one step exceed 126 MB)",
-                       "kernel_impl": {0: "auto", 1: "portable", 2: "tcgen05"}[impl]},
+                       "kernel_impl": {0: "auto", 1: "portable", 2: "tcgen05"}[impl],
+                       "backward": "fused (one kernel; dQ through fp32 add-reductions)" if fused else "two-pass (dK/dV, then dQ)"},
             "pct_of_bf16_peak": {"measured_burst": 100 * value / world / peaks["bf16_tflops"],
                                  "measured_sustained": 100 * value / world / peaks["bf16_tflops_sustained"],
                                  "nominal_2250": 100 * value / world / 2250.0, "source": peaks["source"]},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": 5 * K, "roofline": roofline, "cpu_baseline": cpu}
+            "clocks": clocks, "e2e": e2e, "gpu_launches": (6 if fused else 5) * K, "roofline": roofline, "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -450,6 +459,8 @@ def main():
     ap.add_argument("--workload", default="32k", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--kernel-impl", type=int, default=0, help="0 auto, 1 portable mma.sync, 2 tcgen05")
     ap.add_argument("--oracle-rows", type=int, default=0, help="rows per stream in the oracle sample; 0 = size it for ~15 s")
+    ap.add_argument("--bwd", default="fused", choices=["fused", "two_pass"],
+                    help="backward: one fused kernel (dQ through fp32 add-reductions) or the bitwise reproducible two-pass path")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     w = synth.WORKLOADS[args.workload]
