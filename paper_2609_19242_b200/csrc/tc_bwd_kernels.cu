@@ -741,18 +741,18 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
 //                  contiguous).  The compute warps never touch dQ; the reduction runs behind the GEMMs.
 // dQ depends on the order in which the key tiles' reductions arrive (fp32 rounding only).
 // Shared memory: K, V, a 4-stage Q ring and a 3-stage dO ring of 64-row tiles (+ LSE, D rows), dS^T,
-// 4 dQ staging tiles of 16 query rows.  A Q stage is released by the last GEMM of its step and needed by the
+// 2 dQ staging tiles of 32 query rows.  A Q stage is released by the last GEMM of its step and needed by the
 // first GEMM issued for the step after next, so the rings are one stage deeper than the look-ahead.
 constexpr int HT = 64;                              // query rows per step
 constexpr int HPANEL_BYTES = HT * 128;              // one 64-row x 64-column bf16 panel
 constexpr int HT_BYTES = 2 * HPANEL_BYTES;          // a [64 x 128] bf16 tile
-constexpr int STG_ROWS = 16;                        // query rows per dQ staging tile
-constexpr int STG_BYTES = STG_ROWS * 128 * 4;       // a [16 x 128] fp32 staging tile
+constexpr int STG_ROWS = 32;                        // query rows per dQ staging tile
+constexpr int STG_BYTES = STG_ROWS * 128 * 4;       // a [32 x 128] fp32 staging tile
 constexpr int BF_Q0 = 2 * TILE_BYTES;
 constexpr int BF_DO0 = BF_Q0 + 4 * HT_BYTES;
 constexpr int BF_DS = BF_DO0 + 3 * HT_BYTES;
 constexpr int BF_STG = BF_DS + PANEL_BYTES;
-constexpr int BF_ARR = BF_STG + 4 * STG_BYTES;      // lse_s[3][64], d_s[3][64]
+constexpr int BF_ARR = BF_STG + 2 * STG_BYTES;      // lse_s[3][64], d_s[3][64]
 constexpr int BF_BARS = BF_ARR + 1536;
 constexpr int BF_SMEM = BF_BARS + 256;
 constexpr int BF_THREADS = 448;                     // warps 0-7 compute, 8 producer, 9 MMA issue, 10-13 dQ read-out
@@ -993,15 +993,18 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
         mbar_arrive(bar_dqr);
       }
 #pragma unroll
-      for (int qt = 0; qt < 4; ++qt) {   // 16 query columns at a time through staging tile `qt`
+      for (int qt = 0; qt < 2; ++qt) {   // 32 query columns at a time through staging tile `qt`
+        // the reduction that read this staging tile last (one step ago) must have finished reading it; the one
+        // issued for the other tile stays in flight.  The engine takes a fixed few hundred clocks per reduction on
+        // top of about 25 bytes per clock, so the tiles are as large as shared memory allows.
+        if (leader) bulk_wait_read1();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
         if (ok) {
-          // the reduction that read this staging tile last was waited for before the previous barrier
           float* sg = reinterpret_cast<float*>(sm + BF_STG + qt * STG_BYTES) + dd;
 #pragma unroll
-          for (int e = 0; e < 16; ++e) sg[e * 128] = __uint_as_float(v[16 * qt + e]) * a.scale;
+          for (int e = 0; e < 32; ++e) sg[e * 128] = __uint_as_float(v[32 * qt + e]) * a.scale;
           fence_async_smem();
         }
-        if (leader) bulk_wait_read2();   // at most two reductions still reading: the next staging tile is free
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (*abort_flag) { stop = true; break; }
         if (leader) {

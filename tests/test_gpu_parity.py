@@ -159,8 +159,8 @@ def test_skipping_a_stream():
                                Workload("sp_m16", 1, 2, 2, 128, 512, 16),
                                Workload("sp_w200", 1, 2, 1, 128, 768, 32, window=200)], ids=lambda w: w.name)
 def test_single_pass_backward_matches_oracle_and_two_pass(w):
-    """The opt-in one-kernel backward (dQ through fp32 atomics): same tolerances against the oracle; dK and
-    dV come from the same fixed-order accumulation as the two-pass kernels, so they are bitwise equal."""
+    """The fused one-kernel backward (dQ through fp32 add-reductions): same tolerances against the oracle; dK
+    and dV come from the same fixed-order accumulation as in the two-pass kernels and are bitwise equal."""
     inp = synth.make_inputs(w, "cpu")
     g = pu.to_cuda(inp)
     x = pu.f64(inp)
@@ -173,7 +173,7 @@ def test_single_pass_backward_matches_oracle_and_two_pass(w):
     gref = orc.attn_backward(*[x[n] for n in pu.NAMES6], x["do_clean"], x["do_noisy"], M, window=w.window)
     for got, want in zip(one, gref):
         assert pu.rel_l2(synth.to_f64(got), want) <= pu.TOL_GRAD
-    for i in (1, 2, 4, 5):
+    for i in (1, 2, 4, 5):   # dK, dV: the same products accumulated in the same order
         assert torch.equal(one[i], two[i])
     p = binding.make_params(w.batch, w.L, M, w.H, w.H_kv, w.d, bwd_single_pass=True)
     assert binding.bdlm_workspace_bytes(p, binding.BDLM_WS_BWD) >= 2 * w.batch * w.L * w.H * w.d * 4
