@@ -729,9 +729,11 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
 // key tile against 64 query rows, so that tensor memory also holds a dQ^T tile and shared memory a staging
 // area for it: 5 GEMMs and one exp phase per (key tile, query rows) pair instead of the 7 + 2 of the
 // two-pass backward.
-//   tensor memory  [0,64) [64,128) S^T / P^T, two buffers   [128,192) dP^T   [192,256) dQ^T
+//   tensor memory  [0,64) S^T / P^T   [64,128) K as bf16 pairs   [128,192) dP^T   [192,256) dQ^T
 //                  [256,384) dV   [384,512) dK
-//   per step       S^T = K Q^T and dP^T = V dO^T (N = 64); P^T overwrites its own S^T columns as bf16 pairs
+//   per step       S^T = K Q^T and dP^T = V dO^T (N = 64).  An N = 64 MMA with both operands in shared memory
+//                  asks it for 6 KB per 32 clocks, half as much again as it delivers, so K is also kept in
+//                  tensor memory and S^T reads only Q from shared memory.  P^T overwrites its own S^T columns as bf16 pairs
 //                  and is the TMEM-resident A operand of dV += P^T dO; dS^T goes to a shared-memory tile
 //                  (row = key, 64 queries = 128 bytes), the K-major A operand of dK += dS^T Q and the
 //                  MN-major B operand of dQ^T = K^T dS^T (K, resident, is the MN-major A operand).
@@ -774,7 +776,7 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
   const uint32_t bars = base + BF_BARS;
   const uint32_t bar_kv = bars, bar_q_full = bars + 8 /*[4]*/, bar_q_empty = bars + 40 /*[4]*/,
                  bar_do_full = bars + 72 /*[3]*/, bar_do_empty = bars + 96 /*[3]*/,
-                 bar_st = bars + 120 /*[2]*/, bar_pt = bars + 136 /*[2]*/, bar_dpt = bars + 152, bar_dpfree = bars + 160,
+                 bar_st = bars + 120, bar_kready = bars + 128, bar_pt = bars + 136, bar_dpt = bars + 152, bar_dpfree = bars + 160,
                  bar_dst = bars + 168, bar_dsfree = bars + 176, bar_dqf = bars + 184, bar_dqr = bars + 192,
                  bar_done = bars + 200;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + BF_BARS + 208);
@@ -823,7 +825,7 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
     mbar_init(bar_kv, 1);
     for (int i = 0; i < 4; ++i) { mbar_init(bar_q_full + 8 * i, 1); mbar_init(bar_q_empty + 8 * i, 1); }
     for (int i = 0; i < 3; ++i) { mbar_init(bar_do_full + 8 * i, 2); mbar_init(bar_do_empty + 8 * i, 9); }   // full: TMA bytes + LSE/D rows; empty: dV done + 8 compute warps done with the D rows
-    for (int i = 0; i < 2; ++i) { mbar_init(bar_st + 8 * i, 1); mbar_init(bar_pt + 8 * i, 256); }
+    mbar_init(bar_st, 1); mbar_init(bar_pt, 256); mbar_init(bar_kready, 128);
     mbar_init(bar_dpt, 1); mbar_init(bar_dpfree, 256); mbar_init(bar_dst, 256); mbar_init(bar_dsfree, 1);
     mbar_init(bar_dqf, 1); mbar_init(bar_dqr, 128); mbar_init(bar_done, 1);
     fence_mbar_init();
@@ -896,11 +898,11 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       const uint32_t qk_lo0 = desc_lo_k(sQ0), qm_lo0 = desc_lo_mn_h(sQ0);       // Q ring, as K-major B (S^T) / MN-major B (dK)
       const uint32_t dok_lo0 = desc_lo_k(sdO0), dom_lo0 = desc_lo_mn_h(sdO0);   // dO ring, as K-major B (dP^T) / MN-major B (dV)
       const uint32_t dsk_lo = desc_lo_k(sDS), dsm_lo = desc_lo_k(sDS);          // dS^T: K-major A (dK) / MN-major B with one 64-query group (dQ^T)
-      auto issue_st = [&](int buf, int sq) {     // S^T = K Q^T into S^T buffer `buf`
+      auto issue_st = [&](int sq) {     // S^T = K Q^T, K from tensor memory
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)
-          mma_ss_e(tmem + 64 * buf, desc64(k_lo + koff(kk)), desc64(qk_lo0 + sq * HT_LO + koff_h(kk)), IDESC_N64, kk == 0 ? 0u : 1u, el);
-        mma_commit_e(bar_st + 8 * buf, el);
+          mma_ts_e(tmem, tmem + 64 + kk * 8, desc64(qk_lo0 + sq * HT_LO + koff_h(kk)), IDESC_N64, kk == 0 ? 0u : 1u, el);
+        mma_commit_e(bar_st, el);
       };
       auto issue_dpt = [&](int sd) {             // dP^T = V dO^T
 #pragma unroll
@@ -909,30 +911,31 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
         mma_commit_e(bar_dpt, el);
       };
       bool ok = mbar_wait_abortable(bar_kv, 0, abort_flag);
+      ok = ok && mbar_wait_abortable(bar_kready, 0, abort_flag);
       ok = ok && mbar_wait_abortable(bar_q_full, 0, abort_flag);
-      if (ok) { tc_fence_after(); issue_st(0, 0); }
+      if (ok) { tc_fence_after(); issue_st(0); }
       ok = ok && mbar_wait_abortable(bar_do_full, 0, abort_flag);
       if (ok) { tc_fence_after(); issue_dpt(0); }
       int sd = 0, sn = 1, kn = 0;   // dO ring stage of step i, of step i + 1, and that one's wrap count
       for (int i = 0; i < nsteps && ok; ++i) {
-        const int sb = i & 1, sq = i & 3, sqn = (i + 1) & 3;
+        const int sq = i & 3, sqn = (i + 1) & 3;
         const uint32_t acc = i > 0 ? 1u : 0u;
-        // S^T of the next step into the other buffer (its last reader, dV of step i-1, is ahead in the pipe)
-        if (i + 1 < nsteps) {
-          ok = mbar_wait_timed<TR>(bar_q_full + 8 * sqn, ((i + 1) >> 2) & 1, abort_flag, w_q);
-          if (!ok) break;
-          tc_fence_after();
-          issue_st(sb ^ 1, sqn);
-        }
         // dV += P^T dO_i   (P^T: bf16 pairs at the start of each warpgroup's 32 S^T columns)
-        ok = mbar_wait_timed<TR>(bar_pt + 8 * sb, (i >> 1) & 1, abort_flag, w_pt);
+        ok = mbar_wait_timed<TR>(bar_pt, i & 1, abort_flag, w_pt);
         if (!ok) break;
         tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk)
-          mma_ts_e(tmem + 256, tmem + 64 * sb + (kk >> 1) * 32 + (kk & 1) * 8, desc64(dom_lo0 + sd * HT_LO + moff(kk)), IDESC_KM,
+          mma_ts_e(tmem + 256, tmem + (kk >> 1) * 32 + (kk & 1) * 8, desc64(dom_lo0 + sd * HT_LO + moff(kk)), IDESC_KM,
                    kk == 0 ? acc : 1u, el);
         mma_commit_e(bar_do_empty + 8 * sd, el);
+        // S^T of the next step over P^T(i): its reader, dV(i), is ahead in the pipe
+        if (i + 1 < nsteps) {
+          ok = mbar_wait_timed<TR>(bar_q_full + 8 * sqn, ((i + 1) >> 2) & 1, abort_flag, w_q);
+          if (!ok) break;
+          tc_fence_after();
+          issue_st(sqn);
+        }
         // dP^T of the next step, once every compute thread holds dP^T(i) in registers
         if (i + 1 < nsteps) {
           ok = mbar_wait_timed<TR>(bar_dpfree, i & 1, abort_flag, w_dpf);
@@ -1051,21 +1054,30 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
     bool ok = true;
     long long w_st = 0, w_dpt = 0, w_dsf = 0, c_exp = 0, c_ds = 0;
     const long long t_begin = tick<TR>();
+    if (w == 0 && nsteps > 0) {   // warpgroup 0 copies K into tensor memory (one key row per lane)
+      ok = mbar_wait_abortable(bar_kv, 0, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (ok) {
+        row_smem_to_tmem(sm, r, tl + 64);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar_kready);
+      }
+    }
     int sd = 0, kd = 0;   // dO ring stage of step i and its wrap count
-    for (int i = 0; i < nsteps; ++i) {
-      const int sb = i & 1;
+    for (int i = 0; i < nsteps && ok; ++i) {
       const QStep st = step_cur();
       step_next();
       const bool need_mask = (st.qs == CLEAN) ? (st.q0 < fullc_lo || st.q0 + HT > fullc_hi)
                                               : (st.q0 < fulln_lo || st.q0 + HT > fulln_hi);
       ok = mbar_wait_timed<TR>(bar_do_full + 8 * sd, kd & 1, abort_flag, w_st);
-      ok = ok && mbar_wait_timed<TR>(bar_st + 8 * sb, (i >> 1) & 1, abort_flag, w_st);
+      ok = ok && mbar_wait_timed<TR>(bar_st, i & 1, abort_flag, w_st);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
       const long long t0 = tick<TR>();
       uint32_t x[32];
-      tmem_ld32(tl + 64 * sb + c0, x);
+      tmem_ld32(tl + c0, x);
       tmem_wait_ld();
       const float4* lz4 = reinterpret_cast<const float4*>(lse_s + sd * 64 + c0);
       if (!need_mask) {
@@ -1097,11 +1109,11 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
         uint32_t pk[16];
 #pragma unroll
         for (int e = 0; e < 16; ++e) pk[e] = pack_bf16(__uint_as_float(x[2 * e]), __uint_as_float(x[2 * e + 1]));
-        tmem_st16(tl + 64 * sb + c0, pk);
+        tmem_st16(tl + c0, pk);
         tmem_wait_st();
       }
       tc_fence_before();
-      mbar_arrive(bar_pt + 8 * sb);
+      mbar_arrive(bar_pt);
       const long long t1 = tick<TR>();
       c_exp += t1 - t0;
 
