@@ -36,10 +36,12 @@ NAMES6 = ["q_clean", "k_clean", "v_clean", "q_noisy", "k_noisy", "v_noisy"]
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant
 # kernel, from the ncu captures summarised under profiles/ ; keyed by (workload, kernel).
 NCU_TRAFFIC_BYTES = {
-    ("8k", "fwd"): 212907520 + 109731328,
+    ("8k", "fwd"): 209486848 + 106197248,
+    ("8k", "bwd_fused"): 1000546560 + 532201216,
     ("8k", "bwd_dkdv"): 417905664 + 55102208,
     ("8k", "bwd_dq"): 365878272 + 115059200,
-    ("32k", "fwd"): 978337792 + 541234176,
+    ("32k", "fwd"): 965603328 + 523699712,
+    ("32k", "bwd_fused"): 6375630848 + 3351806720,
     ("32k", "bwd_dkdv"): 2465860864 + 249322752,
     ("32k", "bwd_dq"): 1540940288 + 519113216,
 }
