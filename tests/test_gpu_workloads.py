@@ -60,7 +60,8 @@ def test_csbp128k_shards_merge_and_oracle():
     pu.check_sampled(w, binding.IMPL_AUTO, g=g, fwd_out=(o_c, l_c, o_n, l_n))
 
 
-def test_256k_sampled_rows():
+@pytest.mark.parametrize("fused", [False, True], ids=["two_pass", "fused"])
+def test_256k_sampled_rows(fused):
     w = WORKLOADS["256k"]
-    worst = pu.check_sampled(w, binding.IMPL_AUTO)
-    print("256k", worst)
+    worst = pu.check_sampled(w, binding.IMPL_AUTO, single_pass=fused)
+    print("256k", "fused" if fused else "two-pass", worst)
