@@ -9,8 +9,11 @@
 //   dQ pass     one CTA per 128-row query tile of one head; Q and dO stay in shared memory,
 //               the CTA walks its visible key tiles and accumulates dQ += dS K
 //               (Eq. correctness-query-gradient).
+//   fused       the dK/dV unit with 64-query steps: the same CTA also forms dQ^T = K^T dS^T per step and a
+//               fourth warpgroup adds it into an fp32 dQ accumulator through TMA bulk reductions
+//               (5 GEMMs per pair instead of 7; selected with bwd_single_pass).
 //
-// Both are warp-specialised: warp 8 issues TMA loads, warp 9 issues tcgen05.mma (the whole warp walks the
+// All are warp-specialised: warp 8 issues TMA loads, warp 9 issues tcgen05.mma (the whole warp walks the
 // loop convergently, one elected lane issues), warps 0-7 (two warpgroups, each owning half of the 128
 // score columns of every TMEM lane) recompute P = exp(S - LSE) and dS = P * (dP - D) and hand them back
 // to the tensor core (dS as a TMEM-resident A operand; P^T of the dK/dV pass through a shared-memory tile).
