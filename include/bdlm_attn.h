@@ -99,8 +99,11 @@ int bdlm_attn_fwd(const bdlm_params* p,
  * its saved O and LSE, and the upstream gradient dO of both streams.  dK/dV of a KV head are
  * summed over the query heads of its group; clean dK/dV are summed over clean and noisy
  * queries; noisy dK/dV only over the queries of the same block.  The summation order is
- * fixed, so results are bitwise reproducible.  Requires the full clean key range.
- * The workspace (bdlm_workspace_bytes(p, BDLM_WS_BWD)) holds D_i = sum_d dO_i,d * O_i,d.
+ * fixed, so results are bitwise reproducible (with bwd_single_pass = 1: dK and dV are, dQ is
+ * reproducible up to fp32 summation order).  Requires the full clean key range.
+ * The workspace (bdlm_workspace_bytes(p, BDLM_WS_BWD)) holds D_i = sum_d dO_i,d * O_i,d and, with
+ * bwd_single_pass = 1, an fp32 dQ accumulator [batch, H, rows, 128] per query stream; nothing in it
+ * has to be initialised or kept between calls.
  */
 int bdlm_attn_bwd(const bdlm_params* p,
                   const void* q_clean, const void* k_clean, const void* v_clean,
@@ -159,8 +162,8 @@ int bdlm_lse_merge(int32_t n_partials, int32_t batch, int32_t L, int32_t H, int3
  *     [batch, L, H_kv, d] are THIS CALL'S contribution for every clean key (overwritten, zero where no query
  *     of the call sees the key): the reduce-scatter of Algorithm 2 adds them over the ranks' calls.
  *   - Everything else (checks, statuses, layouts, stream semantics, reproducibility) is as for
- *     bdlm_attn_fwd / bdlm_attn_bwd; kv_begin/kv_end select a clean shard in the forward; bwd_single_pass is
- *     ignored.  Workspace of the backward: bdlm_workspace_bytes_packed(p, g, BDLM_WS_BWD).
+ *     bdlm_attn_fwd / bdlm_attn_bwd, bwd_single_pass included; kv_begin/kv_end select a clean shard in the
+ *     forward.  Workspace of the backward: bdlm_workspace_bytes_packed(p, g, BDLM_WS_BWD).
  */
 typedef struct {
   int32_t Lq_clean;             /* rows of the clean query tensors (ignored when q_clean is NULL) */
