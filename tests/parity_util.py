@@ -75,8 +75,11 @@ def check_sampled(w, impl, n_rows=256, g=None, fwd_out=None, check_bwd=True, rep
     `n_rows` stratified query rows are recomputed by the oracle.  O and LSE come from the
     full forward.  dQ at the sampled rows comes from the full backward (a row's dQ depends on
     that row's dO only).  dK/dV are linear in dO, so a second backward with dO zeroed outside
-    the sampled rows is compared, for every key, with the oracle's sum over those rows."""
+    the sampled rows is compared, for every key, with the oracle's sum over those rows.
+    `single_pass` selects the backward path; a tuple such as (False, True) checks several paths
+    against one evaluation of the oracle (the worst figure over the paths is reported)."""
     M = w.block_size
+    variants = tuple(single_pass) if isinstance(single_pass, (tuple, list)) else (single_pass,)
     if g is None:
         g = synth.make_inputs(w, "cuda")
     if fwd_out is None:
@@ -88,16 +91,17 @@ def check_sampled(w, impl, n_rows=256, g=None, fwd_out=None, check_bwd=True, rep
         for h in range(w.H):
             for s in (0, 1):
                 rows_of[(b, h, s)] = synth.sample_rows(w, n_rows, seed=1000 * b + 10 * h + s)
-    grads = grads_sp = None
+    grads, grads_sp = {}, {}
     if check_bwd:
-        grads = gpu_bwd(g, fwd_out, M, impl=impl, window=w.window, single_pass=single_pass)
         do_sp = [torch.zeros_like(g["do_clean"]), torch.zeros_like(g["do_noisy"])]
         for (b, h, s), rows in rows_of.items():
             r = torch.from_numpy(rows).cuda()
             src = g["do_clean"] if s == 0 else g["do_noisy"]
             do_sp[s][b, r, h] = src[b, r, h]
-        grads_sp = gpu_bwd(g, fwd_out, M, do_clean=do_sp[0], do_noisy=do_sp[1], impl=impl, window=w.window,
-                           single_pass=single_pass)
+        for sp in variants:
+            grads[sp] = [t.clone() for t in gpu_bwd(g, fwd_out, M, impl=impl, window=w.window, single_pass=sp)]
+            grads_sp[sp] = [t.clone() for t in gpu_bwd(g, fwd_out, M, do_clean=do_sp[0], do_noisy=do_sp[1], impl=impl,
+                                                       window=w.window, single_pass=sp)]
         torch.cuda.synchronize()
         assert binding.bdlm_get_device_status() == 0
     worst = {"o": 0.0, "lse": 0.0, "dq": 0.0, "dk": 0.0, "dv": 0.0}
@@ -107,7 +111,7 @@ def check_sampled(w, impl, n_rows=256, g=None, fwd_out=None, check_bwd=True, rep
         for hk in range(w.H_kv):
             kv = {n: synth.to_f64(g[n][b, :, hk]) for n in ("k_clean", "v_clean", "k_noisy", "v_noisy")}
             acc = {n: np.zeros((w.L, w.d)) for n in ("dk_clean", "dv_clean", "dk_noisy", "dv_noisy")}
-            dq_num = [0.0, 0.0]
+            dq_num = {sp: [0.0, 0.0] for sp in variants}
             dq_den = [0.0, 0.0]
             for h in range(hk * G, (hk + 1) * G):
                 for s in (0, 1):
@@ -122,19 +126,21 @@ def check_sampled(w, impl, n_rows=256, g=None, fwd_out=None, check_bwd=True, rep
                     worst["o"] = max(worst["o"], float(np.abs(o_got - ref["o"]).max()))
                     worst["lse"] = max(worst["lse"], float(np.abs(l_got - ref["lse"]).max()))
                     if check_bwd:
-                        dq_got = synth.to_f64(grads[3 * s][b, rt, h])
-                        dq_num[s] += float(((dq_got - ref["dq"]) ** 2).sum())
+                        for sp in variants:
+                            dq_got = synth.to_f64(grads[sp][3 * s][b, rt, h])
+                            dq_num[sp][s] += float(((dq_got - ref["dq"]) ** 2).sum())
                         dq_den[s] += float((ref["dq"] ** 2).sum())
                         for n in acc:
                             acc[n] += ref[n]
             if check_bwd:
-                for s in (0, 1):
-                    worst["dq"] = max(worst["dq"], (dq_num[s] / max(dq_den[s], 1e-300)) ** 0.5)
                 idx = {"dk_clean": 1, "dv_clean": 2, "dk_noisy": 4, "dv_noisy": 5}
-                for n, want in acc.items():
-                    got = synth.to_f64(grads_sp[idx[n]][b, :, hk])
-                    assert np.isfinite(got).all(), n
-                    worst[n[:2]] = max(worst[n[:2]], rel_l2(got, want))
+                for sp in variants:
+                    for s in (0, 1):
+                        worst["dq"] = max(worst["dq"], (dq_num[sp][s] / max(dq_den[s], 1e-300)) ** 0.5)
+                    for n, want in acc.items():
+                        got = synth.to_f64(grads_sp[sp][idx[n]][b, :, hk])
+                        assert np.isfinite(got).all(), n
+                        worst[n[:2]] = max(worst[n[:2]], rel_l2(got, want))
     if report is not None:
         report.update(worst)
     assert worst["o"] <= TOL_O, worst
