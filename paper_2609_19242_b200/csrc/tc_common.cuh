@@ -39,19 +39,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after ~2^31 clock ticks (about a second) and reports failure, so a
-// protocol slip ends the kernel with an error status instead of hanging the device.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > (1ll << 31)) return false;
-  }
-  return true;
-}
-
-// Wait used by the warp-specialised kernels: also gives up as soon as another role has raised the
-// CTA's abort flag, and raises it itself on a timeout, so every role leaves its loop.
+// Bounded wait of the warp-specialised kernels: gives up after ~2^31 clock ticks (about a second), so a
+// protocol slip ends the kernel with an error status instead of hanging the device; it also gives up as soon
+// as another role has raised the CTA's abort flag, and raises it itself on a timeout, so every role leaves its loop.
 __device__ __forceinline__ bool mbar_wait_abortable(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
@@ -140,28 +130,9 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {  
   asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
 }
 
-// D[tmem] (+)= A[smem] * B[smem], bf16 inputs, fp32 accumulate; issued by one thread.
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// mbarrier arrive once all MMAs issued so far by this thread have completed.
-__device__ __forceinline__ void mma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-// Warp-uniform issue.  When a whole warp walks the MMA loop (waits, descriptor arithmetic) and only the
+// tcgen05.mma: D[tmem] (+)= A * B, bf16 inputs, fp32 accumulate (ss: A and B from shared memory; ts: A from tensor
+// memory), and tcgen05.commit: mbarrier arrive once all MMAs issued so far by the thread have completed.
+// Warp-uniform issue: when a whole warp walks the MMA loop (waits, descriptor arithmetic) and only the
 // instruction itself is predicated on one elected lane, the loop stays convergent and the compiler can keep
 // the descriptors in the uniform datapath; with the loop inside `if (lane == 0)` every operand is moved over
 // from a vector register per instruction, and issuing one MMA costs more than the 64 clocks it runs.

@@ -58,228 +58,23 @@ namespace {
 constexpr uint32_t IDESC_QK = make_idesc(128, 128, false, false);
 constexpr uint32_t IDESC_PV = make_idesc(128, 128, false, true);
 constexpr int TILE_BYTES = 2 * PANEL_BYTES;   // 128 x 128 bf16
-#ifndef BDLM_P_IN_TMEM
-#define BDLM_P_IN_TMEM 1
-#endif
-constexpr int FWD_SMEM = 6 * TILE_BYTES + 128 + 1024;   // Q, 2x(K,V), P, barriers, alignment slack
 
-__global__ void __launch_bounds__(128, 1)
-tc_fwd_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restrict__ status) {
-  extern __shared__ uint8_t smem_raw[];
-  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t sQ = base, sKV = base + TILE_BYTES, sP = base + 5 * TILE_BYTES;
-  const uint32_t bars = base + 6 * TILE_BYTES;
-  const uint32_t bar_q = bars, bar_kv0 = bars + 8, bar_s = bars + 24, bar_o = bars + 32;
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + 6 * TILE_BYTES + 64);
-
-  const int qs = blockIdx.z & 1, b = blockIdx.z >> 1;
-  if (a.q[qs] == nullptr) return;
-  const int h = blockIdx.y, hk = h / a.G;
-  const int q0 = (gridDim.x - 1 - blockIdx.x) * TILE;
-  const int Lq = rows_q(a, qs);
-  if (q0 >= Lq) return;
-  const int tid = threadIdx.x, warp = tid >> 5;
-  const int row = q0 + tid;
-
-  if (tid == 0) {
-    mbar_init(bar_q, 1); mbar_init(bar_kv0, 1); mbar_init(bar_kv0 + 8, 1); mbar_init(bar_s, 1); mbar_init(bar_o, 1);
-    fence_mbar_init();
-    prefetch_tmap(&maps.q[qs]); prefetch_tmap(&maps.k[0]); prefetch_tmap(&maps.v[0]);
-  }
-  if (warp == 0) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 256);
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem = *tmem_slot;
-  const uint32_t tS = tmem + ((uint32_t)(warp * 32) << 16);   // columns 0..127: S
-  const uint32_t tO = tS + 128;                               // columns 128..255: O
-
-  // key segments visible from this query tile: clean keys first, then noisy keys
-  int seg_lo[2], seg_hi[2], lo_last[2], hi_first[2], ntile[2];
-  int rlo[2], rhi[2];
-#pragma unroll
-  for (int ks = 0; ks < 2; ++ks) {
-    int lo_f, hi_f, lo_l, hi_l;
-    visible_interval(a, qs, ks, q0, lo_f, hi_f);
-    visible_interval(a, qs, ks, q0 + TILE - 1, lo_l, hi_l);
-    seg_lo[ks] = lo_f; seg_hi[ks] = hi_l; lo_last[ks] = lo_l; hi_first[ks] = hi_f;
-    ntile[ks] = seg_hi[ks] > seg_lo[ks] ? (seg_hi[ks] - seg_lo[ks] + TILE - 1) / TILE : 0;
-    visible_interval(a, qs, ks, row, rlo[ks], rhi[ks]);
-  }
-  const int nt = ntile[0] + ntile[1];
-
-  auto issue_kv = [&](int t) {   // thread 0 only
-    const int ks = t < ntile[0] ? 0 : 1;
-    const int k0 = ks == 0 ? seg_lo[0] + t * TILE : seg_lo[1] + (t - ntile[0]) * TILE;
-    const uint32_t bar = bar_kv0 + 8 * (t & 1);
-    const uint32_t dK = sKV + (t & 1) * 2 * TILE_BYTES, dV = dK + TILE_BYTES;
-    mbar_expect_tx(bar, 2 * TILE_BYTES);
-    const int krow = ks == CLEAN ? clean_key_row(a, k0) : k0;   // where the tile's first key is stored
-    tma_load_3d(dK, &maps.k[ks], bar, hk * 128, krow, b);
-    tma_load_3d(dK + PANEL_BYTES, &maps.k[ks], bar, hk * 128 + 64, krow, b);
-    tma_load_3d(dV, &maps.v[ks], bar, hk * 128, krow, b);
-    tma_load_3d(dV + PANEL_BYTES, &maps.v[ks], bar, hk * 128 + 64, krow, b);
-  };
-
-  if (tid == 0 && nt > 0) {
-    mbar_expect_tx(bar_q, TILE_BYTES);
-    tma_load_3d(sQ, &maps.q[qs], bar_q, h * 128, q0, b);
-    tma_load_3d(sQ + PANEL_BYTES, &maps.q[qs], bar_q, h * 128 + 64, q0, b);
-    issue_kv(0);
-  }
-
-  float m = -INFINITY, l = 0.f;
-  bool fail = false;
-  for (int t = 0; t < nt; ++t) {
-    const int ks = t < ntile[0] ? 0 : 1;
-    const int k0 = ks == 0 ? seg_lo[0] + t * TILE : seg_lo[1] + (t - ntile[0]) * TILE;
-    const uint32_t sK = sKV + (t & 1) * 2 * TILE_BYTES, sV = sK + TILE_BYTES;
-    if (tid == 0 && t + 1 < nt) issue_kv(t + 1);   // stage (t+1)&1 was released by the PV MMA of tile t-1
-    if (t == 0) fail |= !mbar_wait(bar_q, 0);
-    fail |= !mbar_wait(bar_kv0 + 8 * (t & 1), (t >> 1) & 1);
-    if (tid == 0 && !fail) {
-      tc_fence_after();
-#pragma unroll
-      for (int kk = 0; kk < 8; ++kk) {
-        const uint32_t off = (kk >> 2) * PANEL_BYTES + (kk & 3) * 32;
-        mma_ss(tmem, smem_desc(sQ + off, 16, 1024), smem_desc(sK + off, 16, 1024), IDESC_QK, kk > 0);
-      }
-      mma_commit(bar_s);
-    }
-    fail |= !mbar_wait(bar_s, t & 1);
-    tc_fence_after();
-
-    // ---- softmax on this thread's row -----------------------------------------------------
-    uint32_t sr[128];
-    {
-      uint32_t (*c)[32] = reinterpret_cast<uint32_t (*)[32]>(sr);
-      tmem_ld32(tS, c[0]); tmem_ld32(tS + 32, c[1]); tmem_ld32(tS + 64, c[2]); tmem_ld32(tS + 96, c[3]);
-      tmem_wait_ld();
-    }
-    const bool need_mask = (k0 < lo_last[ks]) || (k0 + TILE > hi_first[ks]);
-    float mx = -INFINITY;
-#pragma unroll
-    for (int c = 0; c < 128; ++c) {
-      float x = __uint_as_float(sr[c]) * a.scale_log2;
-      if (need_mask) {
-        const int j = k0 + c;
-        x = (j >= rlo[ks] && j < rhi[ks]) ? x : -INFINITY;
-      }
-      sr[c] = __float_as_uint(x);
-      mx = fmaxf(mx, x);
-    }
-    const float m_new = fmaxf(m, mx);
-    const float mb = (m_new == -INFINITY) ? 0.f : m_new;
-    const float corr = exp2f(m - mb);
-    m = m_new;
-    float psum = 0.f;
-#if BDLM_P_IN_TMEM
-    // P (bf16 pairs) overwrites the first 64 columns of this row's S in tensor memory
-#pragma unroll
-    for (int c32 = 0; c32 < 2; ++c32) {
-      uint32_t pk[32];
-#pragma unroll
-      for (int e = 0; e < 32; ++e) {
-        const float p0 = exp2f(__uint_as_float(sr[c32 * 64 + 2 * e]) - mb);
-        const float p1 = exp2f(__uint_as_float(sr[c32 * 64 + 2 * e + 1]) - mb);
-        psum += p0 + p1;
-        pk[e] = pack_bf16(p0, p1);
-      }
-      tmem_st32(tS + c32 * 32, pk);
-    }
-#else
-    uint8_t* prow = sm + (sP - base);
-#pragma unroll
-    for (int c8 = 0; c8 < 16; ++c8) {
-      float p[8];
-#pragma unroll
-      for (int e = 0; e < 8; ++e) { p[e] = exp2f(__uint_as_float(sr[c8 * 8 + e]) - mb); psum += p[e]; }
-      uint4 v;
-      v.x = pack_bf16(p[0], p[1]); v.y = pack_bf16(p[2], p[3]); v.z = pack_bf16(p[4], p[5]); v.w = pack_bf16(p[6], p[7]);
-      *reinterpret_cast<uint4*>(prow + sw128_offset(tid, c8 * 8)) = v;
-    }
-#endif
-    l = l * corr + psum;
-    if (t > 0) {   // rescale the running output (the previous PV MMA has completed)
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t o[32];
-        tmem_ld32(tO + c * 32, o);
-        tmem_wait_ld();
-#pragma unroll
-        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * corr);
-        tmem_st32(tO + c * 32, o);
-      }
-    }
-    tmem_wait_st();
-    tc_fence_before();
-    fence_async_smem();
-    if (__syncthreads_or(fail)) { fail = true; break; }
-    if (tid == 0) {
-      tc_fence_after();
-#pragma unroll
-      for (int kk = 0; kk < 8; ++kk) {
-#if BDLM_P_IN_TMEM
-        mma_ts(tmem + 128, tmem + kk * 8, smem_desc(sV + kk * 2048, PANEL_BYTES, 1024), IDESC_PV,
-               (t > 0 || kk > 0) ? 1u : 0u);
-#else
-        const uint32_t aoff = (kk >> 2) * PANEL_BYTES + (kk & 3) * 32;
-        mma_ss(tmem + 128, smem_desc(sP + aoff, 16, 1024), smem_desc(sV + kk * 2048, PANEL_BYTES, 1024), IDESC_PV,
-               (t > 0 || kk > 0) ? 1u : 0u);
-#endif
-      }
-      mma_commit(bar_o);
-    }
-    fail |= !mbar_wait(bar_o, t & 1);
-    tc_fence_after();
-  }
-
-  // ---- epilogue: O / l -> bf16, LSE ------------------------------------------------------------
-  if (!fail) {
-    const float inv = l > 0.f ? 1.f / l : 0.f;
-    bf16* orow = a.o[qs] + (((int64_t)b * Lq + row) * a.H + h) * 128;
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      uint32_t o[32];
-      if (nt > 0) { tmem_ld32(tO + c * 32, o); tmem_wait_ld(); }
-#pragma unroll
-      for (int e8 = 0; e8 < 4; ++e8) {
-        uint4 v;
-        uint32_t* pv = reinterpret_cast<uint32_t*>(&v);
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          float x0 = nt > 0 ? __uint_as_float(o[e8 * 8 + 2 * e]) * inv : 0.f;
-          float x1 = nt > 0 ? __uint_as_float(o[e8 * 8 + 2 * e + 1]) * inv : 0.f;
-          pv[e] = pack_bf16(x0, x1);
-        }
-        *reinterpret_cast<uint4*>(orow + c * 32 + e8 * 8) = v;
-      }
-    }
-    a.lse[qs][((int64_t)b * a.H + h) * Lq + row] = l > 0.f ? (m + log2f(l)) * LN2 : -INFINITY;
-  } else if (tid == 0) {
-    atomicExch(status, (int)BDLM_ERR_DEVICE_TIMEOUT);
-  }
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem, 256);
-}
-
-
-// Key tiles visible from one 128-row query tile: a clean segment then a noisy segment, each a run
+// Key tiles visible from a run of query rows: a clean segment then a noisy segment, each a run
 // of 128-key tiles starting at the first visible key; scalars only (no indexed arrays).
 struct TileSched {
   int lo0, lo1, nt0, nt1, lo_last0, lo_last1, hi_first0, hi_first1;
-  __device__ __forceinline__ void init(int qs, int q0, const KArgs& a) {
+  // key tiles seen by the query rows [q0, q_last]: the visible interval of a row moves up with the row, so the
+  // first row gives the lower end and the last row the upper end
+  __device__ __forceinline__ void init(int qs, int q0, int q_last, const KArgs& a) {
     int lo_f, hi_f, lo_l, hi_l;
     visible_interval(a, qs, 0, q0, lo_f, hi_f);
-    visible_interval(a, qs, 0, q0 + TILE - 1, lo_l, hi_l);
+    visible_interval(a, qs, 0, q_last, lo_l, hi_l);
     lo0 = lo_f; lo_last0 = lo_l; hi_first0 = hi_f; nt0 = hi_l > lo_f ? (hi_l - lo_f + TILE - 1) / TILE : 0;
     visible_interval(a, qs, 1, q0, lo_f, hi_f);
-    visible_interval(a, qs, 1, q0 + TILE - 1, lo_l, hi_l);
+    visible_interval(a, qs, 1, q_last, lo_l, hi_l);
     lo1 = lo_f; lo_last1 = lo_l; hi_first1 = hi_f; nt1 = hi_l > lo_f ? (hi_l - lo_f + TILE - 1) / TILE : 0;
   }
-  // a tile needs per-element masking unless every row of the query tile sees all of its 128 keys
+  // a tile needs per-element masking unless every one of the query rows sees all of its 128 keys
   __device__ __forceinline__ bool need_mask(int ks, int k0) const {
     return ks == 0 ? (k0 < lo_last0 || k0 + TILE > hi_first0) : (k0 < lo_last1 || k0 + TILE > hi_first1);
   }
@@ -295,12 +90,16 @@ struct TileSched {
 // exponentials the tensor core runs the other head's P V and next Q K^T.  P (bf16) overwrites the first 64 of
 // the S columns it was computed from; O is rescaled only when the running maximum grew by more than 2^8 (the
 // stale maximum is exact in the final LSE and normalisation).
+// With an odd number of query heads per KV head (PAIRQ) the two warpgroups take two consecutive query tiles of
+// ONE head instead: the CTA walks the union of their key tiles (the later tile's list contains the earlier
+// one's except for noisy diagonal tiles), a tile that one of them does not see at all is masked out for it
+// like any other hidden key, and a second tile past the end of the tensor stays masked and is not written.
 // TMEM columns: [0,128) S/P head A   [128,256) S/P head B   [256,384) O head A   [384,512) O head B
 constexpr int FWDR_THREADS = 320;                            // 8 softmax warps, producer warp, MMA warp
 constexpr int FWDR_BARS = 6 * TILE_BYTES;                    // after Q (2 tiles) and the K/V ring (2 stages x 2 tiles)
 constexpr int FWDR_SMEM = FWDR_BARS + 256 + 1024;
 
-template <bool TR>
+template <bool TR, bool PAIRQ>
 __global__ void __launch_bounds__(FWDR_THREADS, 1)
 tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
@@ -315,14 +114,16 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
 
   const int qs = blockIdx.z & 1, b = blockIdx.z >> 1;
   if (a.q[qs] == nullptr) return;
-  const int h0 = blockIdx.y * 2, hk = h0 / a.G;
-  const int q0 = (gridDim.x - 1 - blockIdx.x) * TILE;
+  // warpgroup w works on head h0 + w * HSTEP, query rows q0 + w * QSTEP ...
+  constexpr int HSTEP = PAIRQ ? 0 : 1, QSTEP = PAIRQ ? TILE : 0, QROWS = PAIRQ ? 2 * TILE : TILE;
+  const int h0 = PAIRQ ? blockIdx.y : blockIdx.y * 2, hk = h0 / a.G;
+  const int q0 = (gridDim.x - 1 - blockIdx.x) * QROWS;
   const int Lq = rows_q(a, qs);
   if (q0 >= Lq) return;
   const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;   // warp index, provably uniform
 
   TileSched sch;
-  sch.init(qs, q0, a);
+  sch.init(qs, q0, min(q0 + QROWS, Lq) - 1, a);
   const int nt = sch.nt0 + sch.nt1;
   auto tile_ks = [&](int t) { return t < sch.nt0 ? 0 : 1; };
   auto tile_k0 = [&](int t) { return t < sch.nt0 ? sch.lo0 + t * TILE : sch.lo1 + (t - sch.nt0) * TILE; };
@@ -349,8 +150,9 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
       mbar_expect_tx(bar_q, 2 * TILE_BYTES);
       tma_load_3d(sQ, &maps.q[qs], bar_q, h0 * 128, q0, b);
       tma_load_3d(sQ + PANEL_BYTES, &maps.q[qs], bar_q, h0 * 128 + 64, q0, b);
-      tma_load_3d(sQ + TILE_BYTES, &maps.q[qs], bar_q, h0 * 128 + 128, q0, b);
-      tma_load_3d(sQ + TILE_BYTES + PANEL_BYTES, &maps.q[qs], bar_q, h0 * 128 + 192, q0, b);
+      // (rows past the end of the tensor are filled with zeros)
+      tma_load_3d(sQ + TILE_BYTES, &maps.q[qs], bar_q, (h0 + HSTEP) * 128, q0 + QSTEP, b);
+      tma_load_3d(sQ + TILE_BYTES + PANEL_BYTES, &maps.q[qs], bar_q, (h0 + HSTEP) * 128 + 64, q0 + QSTEP, b);
       bool ok = true;
       for (int t = 0; t < nt && ok; ++t) {
         const int s = t & 1;
@@ -432,14 +234,17 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
   } else {
     const int w = warp >> 2;                               // head: one warpgroup per head, one thread per query row
     const int r = (warp & 3) * 32 + lane;
-    const int row = q0 + r;
-    const int h = h0 + w;
+    const int row = q0 + w * QSTEP + r;
+    const int h = h0 + w * HSTEP;
+    const bool row_ok = row < Lq;                            // PAIRQ: the second tile may lie past the end
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t tS = tmem + lane_base + w * 128;          // this row's 128 score columns
     const uint32_t tO = tmem + lane_base + 256 + w * 128;    // and its 128 output columns
-    int rlo0, rhi0, rlo1, rhi1;
-    visible_interval(a, qs, 0, row, rlo0, rhi0);
-    visible_interval(a, qs, 1, row, rlo1, rhi1);
+    int rlo0 = 0, rhi0 = 0, rlo1 = 0, rhi1 = 0;
+    if (row_ok) {
+      visible_interval(a, qs, 0, row, rlo0, rhi0);
+      visible_interval(a, qs, 1, row, rlo1, rhi1);
+    }
     float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
     long long w_s = 0, c_ld = 0, c_max = 0, c_exp = 0;
@@ -450,7 +255,7 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const bool need_mask = sch.need_mask(ks, k0);
+      const bool need_mask = sch.need_mask(ks, k0) || (PAIRQ && q0 + QROWS > Lq);
       const int vlo = (ks == 0 ? rlo0 : rlo1) - k0, vhi = (ks == 0 ? rhi0 : rhi1) - k0;
       // the whole row of the tile in registers: one pass over S
       const long long tp0 = tick<TR>();
@@ -550,10 +355,10 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
             const float x1 = nt > 0 ? __uint_as_float(o[e8 * 8 + 2 * e + 1]) * inv : 0.f;
             pv[e] = pack_bf16(x0, x1);
           }
-          *reinterpret_cast<uint4*>(orow + c * 32 + e8 * 8) = vv;
+          if (row_ok) *reinterpret_cast<uint4*>(orow + c * 32 + e8 * 8) = vv;
         }
       }
-      a.lse[qs][((int64_t)b * a.H + h) * Lq + row] = l > 0.f ? (m_ref + log2f(l)) * LN2 : -INFINITY;
+      if (row_ok) a.lse[qs][((int64_t)b * a.H + h) * Lq + row] = l > 0.f ? (m_ref + log2f(l)) * LN2 : -INFINITY;
     }
   }
   tc_fence_before();
@@ -589,18 +394,21 @@ cudaError_t launch_tc_fwd(const KArgs& a, cudaStream_t st) {
   const int qrows = max(a.q[CLEAN] != nullptr ? a.Lqc : 0, a.q[NOISY] != nullptr ? a.Ln : 0);
   int* status = device_status_ptr();
   if (status == nullptr) return cudaErrorUnknown;
-  cudaError_t e = cudaFuncSetAttribute(tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM);
-  if (e != cudaSuccess) return e;
+  cudaError_t e;
   if (a.G % 2 == 0) {   // two heads of one KV group per CTA, one softmax warpgroup per head
-    auto kern = a.trace ? tc_fwdr_kernel<true> : tc_fwdr_kernel<false>;
+    auto kern = a.trace ? tc_fwdr_kernel<true, false> : tc_fwdr_kernel<false, false>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, FWDR_SMEM);
     if (e != cudaSuccess) return e;
-    dim3 grid4(qrows / TILE, a.H / 2, a.batch * 2);
-    kern<<<grid4, FWDR_THREADS, FWDR_SMEM, st>>>(maps, a, status);
+    dim3 grid(qrows / TILE, a.H / 2, a.batch * 2);
+    kern<<<grid, FWDR_THREADS, FWDR_SMEM, st>>>(maps, a, status);
     return cudaGetLastError();
   }
-  dim3 grid(qrows / TILE, a.H, a.batch * 2);
-  tc_fwd_kernel<<<grid, 128, FWD_SMEM, st>>>(maps, a, status);
+  // odd group size: two consecutive query tiles of one head per CTA
+  auto kern = a.trace ? tc_fwdr_kernel<true, true> : tc_fwdr_kernel<false, true>;
+  e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, FWDR_SMEM);
+  if (e != cudaSuccess) return e;
+  dim3 grid((qrows / TILE + 1) / 2, a.H, a.batch * 2);
+  kern<<<grid, FWDR_THREADS, FWDR_SMEM, st>>>(maps, a, status);
   return cudaGetLastError();
 }
 

@@ -126,6 +126,17 @@ def test_fused_backward_on_packed_forms():
     _run_and_check(t, 64, binding.IMPL_AUTO, prefix=[b * 64 for b in (1, 5, 8, 11)], pos0=640, window=200, single_pass=True)
 
 
+def test_packed_forms_with_odd_group_sizes():
+    """MHA and G = 3 on the packed forms: a single clean query tile (the forward's tile pair is half empty), three
+    tiles of sampled blocks, both streams."""
+    t = _draw(31, 1, 512, 128, 384, 3, 3, 128)
+    _run_and_check(t, 32, binding.IMPL_TCGEN05, prefix=[b * 32 for b in (0, 1, 2, 5, 6, 7, 9, 11, 12, 13, 14, 15)], pos0=256)
+    t = _draw(32, 1, 384, 0, 3 * 128, 3, 1, 128)
+    _run_and_check(t, 128, binding.IMPL_TCGEN05, prefix=[0, 130, 384], single_pass=True)
+    t = _draw(33, 2, 640, 384, 128, 2, 2, 128)
+    _run_and_check(t, 64, binding.IMPL_TCGEN05, prefix=[64, 500], pos0=128, window=150, single_pass=True)
+
+
 def test_portable_kernels_take_ragged_packed_shapes():
     """d = 64, a clean length that is no multiple of anything, a short clean run."""
     t = _draw(15, 1, 203, 37, 5 * 24, 2, 2, 64)

@@ -179,6 +179,18 @@ def test_single_pass_backward_matches_oracle_and_two_pass(w):
     assert binding.bdlm_workspace_bytes(p, binding.BDLM_WS_BWD) >= 2 * w.batch * w.L * w.H * w.d * 4
 
 
+@pytest.mark.parametrize("w,mode", [(Workload("mha_3tiles", 1, 2, 2, 128, 384, 32), 0),
+                                    (Workload("g3_5tiles", 2, 3, 1, 128, 640, 64), 0),
+                                    (Workload("mha_1tile", 1, 1, 1, 128, 128, 16), 1),
+                                    (Workload("g1_window", 1, 2, 2, 128, 768, 32, window=200), 0),
+                                    (Workload("g3_m256", 1, 3, 1, 128, 512, 256), 1)], ids=lambda x: x.name if hasattr(x, "name") else str(x))
+def test_odd_group_sizes(w, mode):
+    """An odd number of query heads per KV head (MHA included): the forward pairs two consecutive query tiles of
+    one head per CTA -- odd tile counts leave the last pair half empty -- and the backward kernels walk G heads."""
+    pu.check_full(w, binding.IMPL_TCGEN05, mode=mode)
+    pu.check_full(w, binding.IMPL_TCGEN05, mode=mode, single_pass=True)
+
+
 @pytest.mark.parametrize("impl", IMPLS)
 def test_large_logits(impl):
     """Scores with a standard deviation of about 10 nats (q and k six times larger than in the workloads):
