@@ -161,10 +161,21 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
     bool ok = true;
     long long w_empty = 0;
     const long long t_begin = tick<TR>();
+    // the LSE and D rows of a step are fetched one step ahead, so that the round trip to global memory lies under
+    // the waits for the ring stages instead of in front of the stage's full barrier
+    auto fetch_rows = [&](const QStep& s, float4& z, float4& dd) {
+      const int64_t row0 = ((int64_t)b * a.H + s.h) * rows_q(a, s.qs) + s.q0;
+      z = reinterpret_cast<const float4*>(a.lse[s.qs] + row0)[lane];
+      dd = reinterpret_cast<const float4*>(a.dsum[s.qs] + row0)[lane];
+    };
+    float4 z_next = make_float4(0.f, 0.f, 0.f, 0.f), d_next = z_next;
+    if (nsteps > 0) fetch_rows(step_cur(), z_next, d_next);
     for (int i = 0; i < nsteps && ok; ++i) {
       const int sd = i & 1;
       const QStep st = step_cur();
       step_next();
+      const float4 z = z_next, dd = d_next;
+      if (i + 1 < nsteps) fetch_rows(step_cur(), z_next, d_next);
       if (i >= 2) ok = mbar_wait_timed<TR>(bar_q_empty + 8 * sd, ((i >> 1) - 1) & 1, abort_flag, w_empty);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
@@ -179,11 +190,7 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
         mbar_expect_tx(bar_do_full + 8 * sd, TILE_BYTES);   // one arrival of two; the LSE/D rows follow
         tma_tile(sdO0 + sd * TILE_BYTES, &maps.dout[st.qs], bar_do_full + 8 * sd, st.h * 128, st.q0, b);
       }
-      const float* lsep = a.lse[st.qs] + ((int64_t)b * a.H + st.h) * rows_q(a, st.qs) + st.q0;
-      const float* dsp = a.dsum[st.qs] + ((int64_t)b * a.H + st.h) * rows_q(a, st.qs) + st.q0;
       {
-        const float4 z = reinterpret_cast<const float4*>(lsep)[lane];
-        const float4 dd = reinterpret_cast<const float4*>(dsp)[lane];
         float4 z2;
         z2.x = isfinite(z.x) ? z.x * LOG2E : INFINITY; z2.y = isfinite(z.y) ? z.y * LOG2E : INFINITY;
         z2.z = isfinite(z.z) ? z.z * LOG2E : INFINITY; z2.w = isfinite(z.w) ? z.w * LOG2E : INFINITY;
@@ -745,17 +752,19 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
 //                  a bulk add-reduction into the fp32 dQ accumulator [batch, H, rows, 128] (32 KB
 //                  contiguous).  The compute warps never touch dQ; the reduction runs behind the GEMMs.
 // dQ depends on the order in which the key tiles' reductions arrive (fp32 rounding only).
-// Shared memory: K, V, a 4-stage Q ring and a 3-stage dO ring of 64-row tiles (+ LSE, D rows), dS^T,
-// 2 dQ staging tiles of 32 query rows.  A Q stage is released by the last GEMM of its step and needed by the
-// first GEMM issued for the step after next, so the rings are one stage deeper than the look-ahead.
+// Shared memory: K, V, a 3-stage Q ring and a 2-stage dO ring of 64-row tiles (+ LSE, D rows, fetched one step
+// ahead by the producer), dS^T, 2 dQ staging tiles of 64 query rows: one reduction per step, the next step's tile
+// is written while it runs (the engine takes a fixed few hundred clocks per reduction on top of about 25 bytes per
+// clock, so one 32 KB operation beats two of 16 KB).
 constexpr int HT = 64;                              // query rows per step
 constexpr int HPANEL_BYTES = HT * 128;              // one 64-row x 64-column bf16 panel
 constexpr int HT_BYTES = 2 * HPANEL_BYTES;          // a [64 x 128] bf16 tile
-constexpr int STG_ROWS = 32;                        // query rows per dQ staging tile
-constexpr int STG_BYTES = STG_ROWS * 128 * 4;       // a [32 x 128] fp32 staging tile
+constexpr int BF_QS = 3;                            // Q ring stages
+constexpr int BF_DOS = 2;                           // dO ring stages
+constexpr int STG_BYTES = HT * 128 * 4;             // a [64 query x 128] fp32 staging tile
 constexpr int BF_Q0 = 2 * TILE_BYTES;
-constexpr int BF_DO0 = BF_Q0 + 4 * HT_BYTES;
-constexpr int BF_DS = BF_DO0 + 3 * HT_BYTES;
+constexpr int BF_DO0 = BF_Q0 + BF_QS * HT_BYTES;
+constexpr int BF_DS = BF_DO0 + BF_DOS * HT_BYTES;
 constexpr int BF_STG = BF_DS + PANEL_BYTES;
 constexpr int BF_ARR = BF_STG + 2 * STG_BYTES;      // lse_s[3][64], d_s[3][64]
 constexpr int BF_BARS = BF_ARR + 1536;
@@ -853,11 +862,22 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
     long long w_empty = 0;
     const long long t_begin = tick<TR>();
     int sd = 0, kd = 0;   // dO ring stage of step i and how many times the ring has wrapped
+    // the LSE (lanes 0-15) and D (lanes 16-31) rows of a step are fetched one step ahead, so that the round trip
+    // to global memory lies under the waits for the ring stages instead of in front of the stage's full barrier
+    auto fetch_rows = [&](const QStep& s) {
+      const int64_t row0 = ((int64_t)b * a.H + s.h) * rows_q(a, s.qs) + s.q0;
+      const float* src = (lane < 16 ? a.lse[s.qs] : a.dsum[s.qs]) + row0;
+      return reinterpret_cast<const float4*>(src)[lane & 15];
+    };
+    float4 rows_next = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (nsteps > 0) rows_next = fetch_rows(step_cur());
+    int sq = 0, kq = 0;   // Q ring stage of step i and its wrap count
     for (int i = 0; i < nsteps && ok; ++i) {
-      const int sq = i & 3;
       const QStep st = step_cur();
       step_next();
-      if (i >= 4) ok = mbar_wait_timed<TR>(bar_q_empty + 8 * sq, ((i >> 2) - 1) & 1, abort_flag, w_empty);
+      const float4 rows = rows_next;
+      if (i + 1 < nsteps) rows_next = fetch_rows(step_cur());
+      if (kq >= 1) ok = mbar_wait_timed<TR>(bar_q_empty + 8 * sq, (kq - 1) & 1, abort_flag, w_empty);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       if (lane == 0) {
@@ -875,19 +895,18 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
         tma_load_3d(dst, &maps.dout[st.qs], bar, st.h * 128, st.q0, b);
         tma_load_3d(dst + HPANEL_BYTES, &maps.dout[st.qs], bar, st.h * 128 + 64, st.q0, b);
       }
-      const int64_t row0 = ((int64_t)b * a.H + st.h) * rows_q(a, st.qs) + st.q0;
       if (lane < 16) {
-        const float4 z = reinterpret_cast<const float4*>(a.lse[st.qs] + row0)[lane];
         float4 z2;
-        z2.x = isfinite(z.x) ? z.x * LOG2E : INFINITY; z2.y = isfinite(z.y) ? z.y * LOG2E : INFINITY;
-        z2.z = isfinite(z.z) ? z.z * LOG2E : INFINITY; z2.w = isfinite(z.w) ? z.w * LOG2E : INFINITY;
+        z2.x = isfinite(rows.x) ? rows.x * LOG2E : INFINITY; z2.y = isfinite(rows.y) ? rows.y * LOG2E : INFINITY;
+        z2.z = isfinite(rows.z) ? rows.z * LOG2E : INFINITY; z2.w = isfinite(rows.w) ? rows.w * LOG2E : INFINITY;
         reinterpret_cast<float4*>(lse_s + sd * 64)[lane] = z2;
       } else {
-        reinterpret_cast<float4*>(d_s + sd * 64)[lane - 16] = reinterpret_cast<const float4*>(a.dsum[st.qs] + row0)[lane - 16];
+        reinterpret_cast<float4*>(d_s + sd * 64)[lane - 16] = rows;
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_do_full + 8 * sd);
-      if (++sd == 3) { sd = 0; ++kd; }
+      if (++sd == BF_DOS) { sd = 0; ++kd; }
+      if (++sq == BF_QS) { sq = 0; ++kq; }
     }
     if (lane == 0) trace_add(a.trace, 16 + 13, w_empty);
   } else if (warp == 9) {
@@ -919,9 +938,9 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       if (ok) { tc_fence_after(); issue_st(0); }
       ok = ok && mbar_wait_abortable(bar_do_full, 0, abort_flag);
       if (ok) { tc_fence_after(); issue_dpt(0); }
-      int sd = 0, sn = 1, kn = 0;   // dO ring stage of step i, of step i + 1, and that one's wrap count
+      int sd = 0, sn = 1 % BF_DOS, kn = 1 / BF_DOS;   // dO ring stage of step i, of step i + 1, and that one's wrap count
+      int sq = 0, sqn = 1 % BF_QS, kqn = 1 / BF_QS;   // Q ring stage of step i, of step i + 1, and that one's wrap count
       for (int i = 0; i < nsteps && ok; ++i) {
-        const int sq = i & 3, sqn = (i + 1) & 3;
         const uint32_t acc = i > 0 ? 1u : 0u;
         // dV += P^T dO_i   (P^T: bf16 pairs at the start of each warpgroup's 32 S^T columns)
         ok = mbar_wait_timed<TR>(bar_pt, i & 1, abort_flag, w_pt);
@@ -934,7 +953,7 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
         mma_commit_e(bar_do_empty + 8 * sd, el);
         // S^T of the next step over P^T(i): its reader, dV(i), is ahead in the pipe
         if (i + 1 < nsteps) {
-          ok = mbar_wait_timed<TR>(bar_q_full + 8 * sqn, ((i + 1) >> 2) & 1, abort_flag, w_q);
+          ok = mbar_wait_timed<TR>(bar_q_full + 8 * sqn, kqn & 1, abort_flag, w_q);
           if (!ok) break;
           tc_fence_after();
           issue_st(sqn);
@@ -962,7 +981,9 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
         mma_commit_e(bar_q_empty + 8 * sq, el);
         mma_commit_e(bar_dsfree, el);
         sd = sn;
-        if (++sn == 3) { sn = 0; ++kn; }
+        if (++sn == BF_DOS) { sn = 0; ++kn; }
+        sq = sqn;
+        if (++sqn == BF_QS) { sqn = 0; ++kqn; }
       }
       mma_commit_e(bar_done, el);
       if (lane == 0) {
@@ -989,7 +1010,6 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       const long long t0 = tick<TR>();
       if (ok) tc_fence_after();
       float* dst = a.dq32[st.qs] + (((int64_t)b * a.H + st.h) * rows_q(a, st.qs) + st.q0) * 128;
-      bool stop = false;
       uint32_t v[64];
       if (ok) {   // the whole tile into registers first: the tensor core gets its columns back at once
         uint32_t (*c)[32] = reinterpret_cast<uint32_t (*)[32]>(v);
@@ -998,27 +1018,22 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
         tc_fence_before();
         mbar_arrive(bar_dqr);
       }
+      // staging tile i & 1: the reduction that read it last (two steps ago) must have finished reading it; the one
+      // issued for the other tile stays in flight
+      if (leader) bulk_wait_read1();
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (ok) {
+        float* sg = reinterpret_cast<float*>(sm + BF_STG + (i & 1) * STG_BYTES) + dd;
 #pragma unroll
-      for (int qt = 0; qt < 2; ++qt) {   // 32 query columns at a time through staging tile `qt`
-        // the reduction that read this staging tile last (one step ago) must have finished reading it; the one
-        // issued for the other tile stays in flight.  The engine takes a fixed few hundred clocks per reduction on
-        // top of about 25 bytes per clock, so the tiles are as large as shared memory allows.
-        if (leader) bulk_wait_read1();
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (ok) {
-          float* sg = reinterpret_cast<float*>(sm + BF_STG + qt * STG_BYTES) + dd;
-#pragma unroll
-          for (int e = 0; e < 32; ++e) sg[e * 128] = __uint_as_float(v[32 * qt + e]) * a.scale;
-          fence_async_smem();
-        }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (*abort_flag) { stop = true; break; }
-        if (leader) {
-          bulk_reduce_add_f32(dst + qt * STG_ROWS * 128, sSTG + qt * STG_BYTES, STG_BYTES);
-          bulk_commit();
-        }
+        for (int e = 0; e < HT; ++e) sg[e * 128] = __uint_as_float(v[e]) * a.scale;
+        fence_async_smem();
       }
-      if (stop) break;
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (*abort_flag) break;
+      if (leader) {
+        bulk_reduce_add_f32(dst, sSTG + (i & 1) * STG_BYTES, STG_BYTES);
+        bulk_commit();
+      }
       c_ro += tick<TR>() - t0;
     }
     if (leader) {
@@ -1158,7 +1173,7 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       mbar_arrive(bar_dst);
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_do_empty + 8 * sd);   // this warp is done with the stage's D rows
-      if (++sd == 3) { sd = 0; ++kd; }
+      if (++sd == BF_DOS) { sd = 0; ++kd; }
     }
     if (warp == 0 && lane == 0) {
       trace_add(a.trace, 16 + 0, nsteps); trace_add(a.trace, 16 + 1, w_st); trace_add(a.trace, 16 + 2, w_dpt);
