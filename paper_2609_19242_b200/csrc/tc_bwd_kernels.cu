@@ -766,9 +766,9 @@ constexpr int BF_Q0 = 2 * TILE_BYTES;
 constexpr int BF_DO0 = BF_Q0 + BF_QS * HT_BYTES;
 constexpr int BF_DS = BF_DO0 + BF_DOS * HT_BYTES;
 constexpr int BF_STG = BF_DS + PANEL_BYTES;
-constexpr int BF_ARR = BF_STG + 2 * STG_BYTES;      // lse_s[3][64], d_s[3][64]
-constexpr int BF_BARS = BF_ARR + 1536;
-constexpr int BF_SMEM = BF_BARS + 256;
+constexpr int BF_ARR = BF_STG + 2 * STG_BYTES;      // lse_s[4][64], d_s[4][64]: the LSE / D rows have a ring of their own
+constexpr int BF_BARS = BF_ARR + 2048;
+constexpr int BF_SMEM = BF_BARS + 320;
 constexpr int BF_THREADS = 448;                     // warps 0-7 compute, 8 producer, 9 MMA issue, 10-13 dQ read-out
 constexpr uint32_t IDESC_N64 = make_idesc(128, 64, false, false);   // S^T, dP^T: A, B K-major, N = 64
 constexpr uint32_t IDESC_DQT = make_idesc(128, 64, true, true);     // dQ^T: A, B MN-major, N = 64
@@ -783,14 +783,14 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
   const uint32_t base = smem_u32(sm);
   const uint32_t sK = base, sV = base + TILE_BYTES, sQ0 = base + BF_Q0, sdO0 = base + BF_DO0, sDS = base + BF_DS,
                  sSTG = base + BF_STG;
-  float* lse_s = reinterpret_cast<float*>(sm + BF_ARR);            // [3][64], log2 units
-  float* d_s = lse_s + 192;                                        // [3][64]
+  float* lse_s = reinterpret_cast<float*>(sm + BF_ARR);            // [4][64], log2 units
+  float* d_s = lse_s + 256;                                        // [4][64]
   const uint32_t bars = base + BF_BARS;
   const uint32_t bar_kv = bars, bar_q_full = bars + 8 /*[4]*/, bar_q_empty = bars + 40 /*[4]*/,
                  bar_do_full = bars + 72 /*[3]*/, bar_do_empty = bars + 96 /*[3]*/,
                  bar_st = bars + 120, bar_kready = bars + 128, bar_pt = bars + 136, bar_dpt = bars + 152, bar_dpfree = bars + 160,
                  bar_dst = bars + 168, bar_dsfree = bars + 176, bar_dqf = bars + 184, bar_dqr = bars + 192,
-                 bar_done = bars + 200;
+                 bar_done = bars + 200, bar_rows_full = bars + 224 /*[4]*/, bar_rows_empty = bars + 256 /*[4]*/;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + BF_BARS + 208);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + BF_BARS + 216);
 
@@ -836,7 +836,8 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
     if (base & 1023u) *abort_flag = 1; else *abort_flag = 0;   // swizzled tiles need a 1024-byte aligned base
     mbar_init(bar_kv, 1);
     for (int i = 0; i < 4; ++i) { mbar_init(bar_q_full + 8 * i, 1); mbar_init(bar_q_empty + 8 * i, 1); }
-    for (int i = 0; i < 3; ++i) { mbar_init(bar_do_full + 8 * i, 2); mbar_init(bar_do_empty + 8 * i, 9); }   // full: TMA bytes + LSE/D rows; empty: dV done + 8 compute warps done with the D rows
+    for (int i = 0; i < 3; ++i) { mbar_init(bar_do_full + 8 * i, 1); mbar_init(bar_do_empty + 8 * i, 1); }   // empty: dV done
+    for (int i = 0; i < 4; ++i) { mbar_init(bar_rows_full + 8 * i, 1); mbar_init(bar_rows_empty + 8 * i, 8); }   // empty: the 8 compute warps are done with the stage's LSE / D rows
     mbar_init(bar_st, 1); mbar_init(bar_pt, 256); mbar_init(bar_kready, 128);
     mbar_init(bar_dpt, 1); mbar_init(bar_dpfree, 256); mbar_init(bar_dst, 256); mbar_init(bar_dsfree, 1);
     mbar_init(bar_dqf, 1); mbar_init(bar_dqr, 128); mbar_init(bar_done, 1);
@@ -891,20 +892,26 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       if (!ok) break;
       if (lane == 0) {
         const uint32_t dst = sdO0 + sd * HT_BYTES, bar = bar_do_full + 8 * sd;
-        mbar_expect_tx(bar, HT_BYTES);   // one arrival of two; the LSE/D rows follow
+        mbar_expect_tx(bar, HT_BYTES);
         tma_load_3d(dst, &maps.dout[st.qs], bar, st.h * 128, st.q0, b);
         tma_load_3d(dst + HPANEL_BYTES, &maps.dout[st.qs], bar, st.h * 128 + 64, st.q0, b);
       }
+      // the rows live in a ring of their own: the dO tile is free again as soon as dV has read it, the D rows
+      // only when the compute warps have formed dS
+      const int sr = i & 3;
+      if (i >= 4) ok = mbar_wait_timed<TR>(bar_rows_empty + 8 * sr, ((i >> 2) - 1) & 1, abort_flag, w_empty);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
       if (lane < 16) {
         float4 z2;
         z2.x = isfinite(rows.x) ? rows.x * LOG2E : INFINITY; z2.y = isfinite(rows.y) ? rows.y * LOG2E : INFINITY;
         z2.z = isfinite(rows.z) ? rows.z * LOG2E : INFINITY; z2.w = isfinite(rows.w) ? rows.w * LOG2E : INFINITY;
-        reinterpret_cast<float4*>(lse_s + sd * 64)[lane] = z2;
+        reinterpret_cast<float4*>(lse_s + sr * 64)[lane] = z2;
       } else {
-        reinterpret_cast<float4*>(d_s + sd * 64)[lane - 16] = rows;
+        reinterpret_cast<float4*>(d_s + sr * 64)[lane - 16] = rows;
       }
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_do_full + 8 * sd);
+      if (lane == 0) mbar_arrive(bar_rows_full + 8 * sr);
       if (++sd == BF_DOS) { sd = 0; ++kd; }
       if (++sq == BF_QS) { sq = 0; ++kq; }
     }
@@ -1082,13 +1089,13 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
         mbar_arrive(bar_kready);
       }
     }
-    int sd = 0, kd = 0;   // dO ring stage of step i and its wrap count
     for (int i = 0; i < nsteps && ok; ++i) {
       const QStep st = step_cur();
       step_next();
       const bool need_mask = (st.qs == CLEAN) ? (st.q0 < fullc_lo || st.q0 + HT > fullc_hi)
                                               : (st.q0 < fulln_lo || st.q0 + HT > fulln_hi);
-      ok = mbar_wait_timed<TR>(bar_do_full + 8 * sd, kd & 1, abort_flag, w_st);
+      const int sr = i & 3;
+      ok = mbar_wait_timed<TR>(bar_rows_full + 8 * sr, (i >> 2) & 1, abort_flag, w_st);
       ok = ok && mbar_wait_timed<TR>(bar_st, i & 1, abort_flag, w_st);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
@@ -1097,7 +1104,7 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       uint32_t x[32];
       tmem_ld32(tl + c0, x);
       tmem_wait_ld();
-      const float4* lz4 = reinterpret_cast<const float4*>(lse_s + sd * 64 + c0);
+      const float4* lz4 = reinterpret_cast<const float4*>(lse_s + sr * 64 + c0);
       if (!need_mask) {
 #pragma unroll
         for (int c4 = 0; c4 < 8; ++c4) {
@@ -1147,7 +1154,7 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
         tmem_wait_ld();
         tc_fence_before();
         mbar_arrive(bar_dpfree);   // dP^T(i) is in registers: the tensor core may overwrite its columns
-        const float4* dz4 = reinterpret_cast<const float4*>(d_s + sd * 64 + c0);
+        const float4* dz4 = reinterpret_cast<const float4*>(d_s + sr * 64 + c0);
 #pragma unroll
         for (int c4 = 0; c4 < 8; ++c4) {
           const float4 dz = dz4[c4];
@@ -1172,8 +1179,7 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       fence_async_smem();
       mbar_arrive(bar_dst);
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_do_empty + 8 * sd);   // this warp is done with the stage's D rows
-      if (++sd == BF_DOS) { sd = 0; ++kd; }
+      if (lane == 0) mbar_arrive(bar_rows_empty + 8 * sr);   // this warp is done with the stage's LSE / D rows
     }
     if (warp == 0 && lane == 0) {
       trace_add(a.trace, 16 + 0, nsteps); trace_add(a.trace, 16 + 1, w_st); trace_add(a.trace, 16 + 2, w_dpt);
