@@ -63,7 +63,7 @@ typedef struct {
   int32_t bwd_single_pass;     /* backward only: 0 = dK/dV pass + dQ pass, fixed summation order, bitwise reproducible;
                                   1 = fused: one kernel produces dK, dV and dQ (5 GEMMs per tile pair instead of 7).  Each
                                   CTA adds its dQ tiles into an fp32 accumulator in the workspace (bulk add-reductions), so
-                                  dQ is reproducible only up to fp32 summation order; dK and dV are as in the two-pass path.
+                                  dQ is reproducible only up to fp32 summation order; dK and dV are bitwise reproducible (fixed order).
                                   Needs the larger workspace bdlm_workspace_bytes[_packed] reports for this setting; falls
                                   back to the two-pass path when the tensor-core kernels do not take the shape. */
   int32_t window;              /* sliding-window layers: > 0 = a clean key j is visible to the query at position i (of either

@@ -75,6 +75,43 @@ constexpr int DKDV_PRODUCER = 4 * DKDV_NWG, DKDV_ISSUER = 4 * DKDV_NWG + 1;
 
 struct QStep { int qs, h, q0; };
 
+// The steps of a key tile: every (query tile, query stream, head of the group) that sees it.  Segment A holds the
+// clean query tiles [a0, a1) (for a noisy key tile: the noisy ones), segment B the noisy query tiles [b0, b1) of a
+// clean key tile, both in units of the step's query rows.  They are walked from the last query tile down, both
+// streams of a tile and all heads of the group before the next tile: CTAs that start together then meet the same
+// Q / dO tiles -- and, in the fused kernel, the same dQ accumulator tiles -- at the same time, so that those stay in
+// L2 between the CTAs that share them.  Counters only, no division; the order is fixed, so dK / dV stay bitwise
+// reproducible.
+struct StepWalk {
+  int a0, a1, b0, b1, G, h_first, qs_a, rows;
+  int t, seg, hh;
+  __device__ __forceinline__ int count() const { return ((a1 - a0) + (b1 - b0)) * G; }
+  __device__ __forceinline__ void settle() {   // the next (t, segment) at or below t that exists
+    while (t >= 0) {
+      if (t >= a0 && t < a1) { seg = 0; return; }
+      if (t >= b0 && t < b1) { seg = 1; return; }
+      --t;
+    }
+  }
+  __device__ __forceinline__ void init(int a0_, int na, int b0_, int nb, int G_, int h_first_, int qs_a_, int rows_) {
+    a0 = a0_; a1 = a0_ + na; b0 = b0_; b1 = b0_ + nb; G = G_; h_first = h_first_; qs_a = qs_a_; rows = rows_;
+    t = max(a1, b1) - 1; seg = 0; hh = 0;
+    settle();
+  }
+  __device__ __forceinline__ QStep cur() const {
+    QStep s;
+    s.h = h_first + hh; s.qs = seg == 0 ? qs_a : NOISY; s.q0 = t * rows;
+    return s;
+  }
+  __device__ __forceinline__ void next() {
+    if (++hh < G) return;
+    hh = 0;
+    if (seg == 0 && t >= b0 && t < b1) { seg = 1; return; }
+    --t;
+    settle();
+  }
+};
+
 template <bool TR>
 __global__ void __launch_bounds__(DKDV_THREADS, 1)
 tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restrict__ status) {
@@ -118,18 +155,12 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
     const int lo = (k0 / M) * M, hi = min(L, ((k0 + TILE - 1) / M + 1) * M);
     tA0 = lo / TILE; nA = (hi + TILE - 1) / TILE - tA0;
   }
-  const int per_head = nA + nB;
-  const int nsteps = per_head * a.G;
-  // steps are walked in order by every role: (head of the group, tile index inside the head) counters, no division
-  int it_r = 0, it_h = hk * a.G;
-  auto step_cur = [&]() {
-    QStep s;
-    s.h = it_h;
-    if (it_r < nA) { s.qs = (ks == NOISY) ? NOISY : CLEAN; s.q0 = (tA0 + it_r) * TILE; }
-    else { s.qs = NOISY; s.q0 = (tB0 + it_r - nA) * TILE; }
-    return s;
-  };
-  auto step_next = [&]() { if (++it_r == per_head) { it_r = 0; ++it_h; } };
+  // the steps are walked in the same order by every role (see StepWalk)
+  StepWalk walk;
+  walk.init(tA0, nA, tB0, nB, a.G, hk * a.G, ks == NOISY ? NOISY : CLEAN, TILE);
+  const int nsteps = walk.count();
+  auto step_cur = [&]() { return walk.cur(); };
+  auto step_next = [&]() { walk.next(); };
 
   if (threadIdx.x == 0) {
     if (base & 1023u) *abort_flag = 1; else *abort_flag = 0;   // swizzled tiles need a 1024-byte aligned base
@@ -820,17 +851,11 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
     const int lo = (k0 / M) * M, hi = min(L, ((k0 + TILE - 1) / M + 1) * M);
     tA0 = lo / HT; nA = (hi + HT - 1) / HT - tA0;
   }
-  const int per_head = nA + nB;
-  const int nsteps = per_head * a.G;
-  int it_r = 0, it_h = hk * a.G;
-  auto step_cur = [&]() {
-    QStep s;
-    s.h = it_h;
-    if (it_r < nA) { s.qs = (ks == NOISY) ? NOISY : CLEAN; s.q0 = (tA0 + it_r) * HT; }
-    else { s.qs = NOISY; s.q0 = (tB0 + it_r - nA) * HT; }
-    return s;
-  };
-  auto step_next = [&]() { if (++it_r == per_head) { it_r = 0; ++it_h; } };
+  StepWalk walk;
+  walk.init(tA0, nA, tB0, nB, a.G, hk * a.G, ks == NOISY ? NOISY : CLEAN, HT);
+  const int nsteps = walk.count();
+  auto step_cur = [&]() { return walk.cur(); };
+  auto step_next = [&]() { walk.next(); };
 
   if (threadIdx.x == 0) {
     if (base & 1023u) *abort_flag = 1; else *abort_flag = 0;   // swizzled tiles need a 1024-byte aligned base

@@ -160,7 +160,7 @@ def test_skipping_a_stream():
                                Workload("sp_w200", 1, 2, 1, 128, 768, 32, window=200)], ids=lambda w: w.name)
 def test_single_pass_backward_matches_oracle_and_two_pass(w):
     """The fused one-kernel backward (dQ through fp32 add-reductions): same tolerances against the oracle; dK
-    and dV come from the same fixed-order accumulation as in the two-pass kernels and are bitwise equal."""
+    and dV come from a fixed-order accumulation like those of the two-pass kernels."""
     inp = synth.make_inputs(w, "cpu")
     g = pu.to_cuda(inp)
     x = pu.f64(inp)
@@ -173,8 +173,15 @@ def test_single_pass_backward_matches_oracle_and_two_pass(w):
     gref = orc.attn_backward(*[x[n] for n in pu.NAMES6], x["do_clean"], x["do_noisy"], M, window=w.window)
     for got, want in zip(one, gref):
         assert pu.rel_l2(synth.to_f64(got), want) <= pu.TOL_GRAD
-    for i in (1, 2, 4, 5):   # dK, dV: the same products accumulated in the same order
-        assert torch.equal(one[i], two[i])
+    # dK, dV: the same products in fp32, summed over 64-row instead of 128-row query steps (a different but fixed
+    # order): equal to the two-pass result up to the last bf16 bit of a few elements, and reproducible run to run
+    for i in (1, 2, 4, 5):
+        assert pu.rel_l2(synth.to_f64(one[i]), synth.to_f64(two[i])) <= 1e-3
+    first = [t.clone() for t in one]
+    again = pu.gpu_bwd(g, out, M, single_pass=True, window=w.window)
+    torch.cuda.synchronize()
+    for i in (1, 2, 4, 5):
+        assert torch.equal(first[i], again[i])
     p = binding.make_params(w.batch, w.L, M, w.H, w.H_kv, w.d, bwd_single_pass=True)
     assert binding.bdlm_workspace_bytes(p, binding.BDLM_WS_BWD) >= 2 * w.batch * w.L * w.H * w.d * 4
 
