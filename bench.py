@@ -36,14 +36,14 @@ NAMES6 = ["q_clean", "k_clean", "v_clean", "q_noisy", "k_noisy", "v_noisy"]
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant
 # kernel, from the ncu captures summarised under profiles/ ; keyed by (workload, kernel).
 NCU_TRAFFIC_BYTES = {
-    ("8k", "fwd"): 209486848 + 106197248,
-    ("8k", "bwd_fused"): 1000546560 + 532201216,
-    ("8k", "bwd_dkdv"): 417905664 + 55102208,
-    ("8k", "bwd_dq"): 365878272 + 115059200,
-    ("32k", "fwd"): 965603328 + 523699712,
-    ("32k", "bwd_fused"): 6375630848 + 3351806720,
-    ("32k", "bwd_dkdv"): 2465860864 + 249322752,
-    ("32k", "bwd_dq"): 1540940288 + 519113216,
+    ("8k", "fwd"): 207913984 + 109006592,
+    ("8k", "bwd_fused"): 762043904 + 374662144,
+    ("8k", "bwd_dkdv"): 380482816 + 54774784,
+    ("8k", "bwd_dq"): 365881344 + 115298560,
+    ("32k", "fwd"): 964474368 + 522727680,
+    ("32k", "bwd_fused"): 5886429184 + 3367195136,
+    ("32k", "bwd_dkdv"): 2396964864 + 250488576,
+    ("32k", "bwd_dq"): 1545019136 + 518886400,
 }
 TRAFFIC_NOTE = ("dram__bytes_read.sum + dram__bytes_write.sum per launch from ncu captures of the 8k and the 32k "
                 "workload (profiles/tc_kernels_8k_ncu_full.md, profiles/tc_kernels_32k_dram_traffic.md; the two "
