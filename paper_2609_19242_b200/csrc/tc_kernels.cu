@@ -190,6 +190,8 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
         for (int kk = 0; kk < 4; ++kk)
           mma_ts_e(d, p_tmem + (4 * j + kk) * 8, desc64(v_lo + moff(4 * j + kk)), IDESC_PV, kk == 0 ? acc_first : 1u, el);
       };
+      long long w_p = 0, w_v = 0, w_k = 0;
+      const long long tm0 = tick<TR>();
       for (int t = 0; t < nt && ok; ++t) {
         const int s = t & 1;
         const uint32_t cv_lo = v_lo0 + s * 2 * TILE_LO;
@@ -197,29 +199,29 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
         const uint32_t acc = t > 0 ? 1u : 0u;
         // head A: P arrives in two halves of the keys (bf16 pairs at columns [0,32) and [32,64) of the head's S
         // region), so P V over the first 64 keys runs while the softmax is still in the exponentials of the rest
-        ok = mbar_wait_lean(bar_p, t & 1, abort_flag);
-        ok = ok && mbar_wait_lean(bar_v_full + 8 * s, (t >> 1) & 1, abort_flag);
+        ok = mbar_wait_timed<TR>(bar_p, t & 1, abort_flag, w_p);
+        ok = ok && mbar_wait_timed<TR>(bar_v_full + 8 * s, (t >> 1) & 1, abort_flag, w_v);
         if (!ok) break;
         tc_fence_after();
         pv_half(tmem + 256, tmem, cv_lo, 0, acc);
-        ok = mbar_wait_lean(bar_p + 8, t & 1, abort_flag);
+        ok = mbar_wait_timed<TR>(bar_p + 8, t & 1, abort_flag, w_p);
         if (!ok) break;
         tc_fence_after();
         pv_half(tmem + 256, tmem, cv_lo, 1, 1u);
         mma_commit_e(bar_o, el);
         if (t + 1 < nt) {
-          ok = mbar_wait_lean(bar_k_full + 8 * (s ^ 1), ((t + 1) >> 1) & 1, abort_flag);
+          ok = mbar_wait_timed<TR>(bar_k_full + 8 * (s ^ 1), ((t + 1) >> 1) & 1, abort_flag, w_k);
           if (!ok) break;
           tc_fence_after();
           gemm_ss_e(tmem, qa_lo, nk_lo, IDESC_QK, 0u, el);
           mma_commit_e(bar_s, el);
         }
         // head B
-        ok = mbar_wait_lean(bar_p + 16, t & 1, abort_flag);
+        ok = mbar_wait_timed<TR>(bar_p + 16, t & 1, abort_flag, w_p);
         if (!ok) break;
         tc_fence_after();
         pv_half(tmem + 384, tmem + 128, cv_lo, 0, acc);
-        ok = mbar_wait_lean(bar_p + 24, t & 1, abort_flag);
+        ok = mbar_wait_timed<TR>(bar_p + 24, t & 1, abort_flag, w_p);
         if (!ok) break;
         tc_fence_after();
         pv_half(tmem + 384, tmem + 128, cv_lo, 1, 1u);
@@ -229,6 +231,9 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
           gemm_ss_e(tmem + 128, qb_lo, nk_lo, IDESC_QK, 0u, el);
           mma_commit_e(bar_s + 8, el);
         }
+      }
+      if (lane == 0) {
+        trace_add(a.trace, 8, tick<TR>() - tm0); trace_add(a.trace, 9, w_p); trace_add(a.trace, 10, w_v); trace_add(a.trace, 11, w_k);
       }
     }
   } else {
