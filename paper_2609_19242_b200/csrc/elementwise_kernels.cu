@@ -69,39 +69,50 @@ __global__ void __launch_bounds__(256) merge_kernel(MergeArgs ma, int64_t total_
   }
 }
 
-// One warp per (batch, row, head): D = sum over d of dO * O, fp32.
+// D = sum over d of dO * O, fp32.  D / 8 lanes per (batch, row, head) with 16-byte loads, four rows per lane group in
+// flight (the kernel is a pure stream over dO and O: enough bytes in flight per thread to keep HBM busy).
 template <int D>
 __global__ void __launch_bounds__(256) dsum_kernel(const bf16* __restrict__ dout, const bf16* __restrict__ o,
                                                    float* __restrict__ dsum, int64_t nrows, int L, int H) {
-  const int lane = threadIdx.x & 31;
-  const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  if (w >= nrows) return;   // whole warp leaves together
-  constexpr int EPL = D / 32;   // elements per lane: 4 (d=128) or 2 (d=64)
-  const bf16* pa = dout + w * D + lane * EPL;
-  const bf16* pb = o + w * D + lane * EPL;
-  float acc = 0.f;
-  if (EPL == 4) {
-    uint2 ua = *reinterpret_cast<const uint2*>(pa), ub = *reinterpret_cast<const uint2*>(pb);
-    float2 a0 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&ua.x));
-    float2 a1 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&ua.y));
-    float2 b0 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&ub.x));
-    float2 b1 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&ub.y));
-    acc = a0.x * b0.x + a0.y * b0.y + a1.x * b1.x + a1.y * b1.y;
-  } else {
-    uint32_t ua = *reinterpret_cast<const uint32_t*>(pa), ub = *reinterpret_cast<const uint32_t*>(pb);
-    float2 a0 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&ua));
-    float2 b0 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&ub));
-    acc = a0.x * b0.x + a0.y * b0.y;
+  constexpr int LPR = D / 8;            // lanes per row: 16 (d = 128) or 8 (d = 64)
+  constexpr int RPW = 32 / LPR;         // rows per warp and pass
+  constexpr int UNROLL = 4;
+  const int lane = threadIdx.x & 31, sub = lane / LPR, c = lane % LPR;
+  const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int64_t base = warp * (RPW * UNROLL);
+  uint4 ua[UNROLL], ub[UNROLL];
+#pragma unroll
+  for (int j = 0; j < UNROLL; ++j) {
+    const int64_t w = base + j * RPW + sub;
+    if (w < nrows) {
+      ua[j] = *reinterpret_cast<const uint4*>(dout + w * D + c * 8);
+      ub[j] = *reinterpret_cast<const uint4*>(o + w * D + c * 8);
+    } else {
+      ua[j] = make_uint4(0u, 0u, 0u, 0u); ub[j] = ua[j];
+    }
   }
 #pragma unroll
-  for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
-  if (lane == 0) {
-    // w indexes [batch, L, H]; D is stored [batch, H, L]
-    const int h = (int)(w % H);
-    const int64_t row = w / H;
-    const int64_t bidx = row / L;
-    const int i = (int)(row % L);
-    dsum[(bidx * H + h) * L + i] = acc;
+  for (int j = 0; j < UNROLL; ++j) {
+    const uint32_t* pa = reinterpret_cast<const uint32_t*>(&ua[j]);
+    const uint32_t* pb = reinterpret_cast<const uint32_t*>(&ub[j]);
+    float acc = 0.f;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pa[e]));
+      const float2 y = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pb[e]));
+      acc = fmaf(x.x, y.x, fmaf(x.y, y.y, acc));
+    }
+#pragma unroll
+    for (int sft = LPR / 2; sft > 0; sft >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, sft);
+    const int64_t w = base + j * RPW + sub;
+    if (c == 0 && w < nrows) {
+      // w indexes [batch, L, H]; D is stored [batch, H, L]
+      const int h = (int)(w % H);
+      const int64_t row = w / H;
+      const int64_t bidx = row / L;
+      const int i = (int)(row % L);
+      dsum[(bidx * H + h) * L + i] = acc;
+    }
   }
 }
 
@@ -132,7 +143,8 @@ cudaError_t launch_dsum(const KArgs& a, float* dsum_clean, float* dsum_noisy, cu
     if (a.q[s] == nullptr) continue;   // a stream without queries has no D rows
     const int rows = rows_q(a, s);
     const int64_t nrows = (int64_t)a.batch * rows * a.H;
-    const int blocks = (int)((nrows * 32 + 255) / 256);
+    const int rows_per_block = 8 * (32 / (a.d / 8)) * 4;   // 8 warps, 32 / (d / 8) rows per warp and pass, 4 passes
+    const int blocks = (int)((nrows + rows_per_block - 1) / rows_per_block);
     if (blocks == 0) continue;
     if (a.d == 128)
       dsum_kernel<128><<<blocks, 256, 0, st>>>(a.dout[s], a.o[s], out[s], nrows, rows, a.H);
