@@ -94,7 +94,7 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
         self.thread.join(timeout=2)
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in self.rows:
             if len(r) < 7:
@@ -104,11 +104,15 @@ class ClockSampler:
                 mx.append(float(r[1]))
             except ValueError:
                 continue
+            try:
+                pw.append(float(r[2]))
+            except ValueError:
+                pass
             for n, v in zip(names, r[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "reasons": sorted(reasons), "power_w_max": max(pw) if pw else None}   # nvidia-smi averages power.draw over about a second: the maximum over the samples is the closest to the draw under load
 
 
 def physical_gpu_index(local):
