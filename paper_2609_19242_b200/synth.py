@@ -75,6 +75,8 @@ WORKLOADS = {
     "32k_w1024": Workload("32k_w1024", 1, 32, 8, 128, 32768, 64, rope_theta=5e5, window=1024),
     # DFlash2-shaped drafter layer (appendix E): 32K target-feature keys, 2048 sampled blocks of 16 tokens
     "dflash32k": Workload("dflash32k", 1, 32, 8, 128, 32768, 16, n_blocks=2048),
+    # multi-head attention without KV sharing (one query head per KV head); not a BASELINE config
+    "mha16k": Workload("mha16k", 1, 8, 8, 128, 16384, 32),
 }
 
 

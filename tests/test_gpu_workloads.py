@@ -27,6 +27,12 @@ def test_sampled_rows_full_size_fused_backward(name):
     print(name, "fused", worst)
 
 
+def test_mha16k_sampled_rows():
+    """One query head per KV head: the forward pairs consecutive query tiles of a head; both backward paths."""
+    worst = pu.check_sampled(WORKLOADS["mha16k"], binding.IMPL_AUTO, single_pass=(False, True))
+    print("mha16k", worst)
+
+
 def test_dflash32k_sampled_rows_fused_backward():
     worst = pu.check_sampled_packed(WORKLOADS["dflash32k"], binding.IMPL_AUTO, single_pass=True)
     print("dflash32k fused", worst)
