@@ -198,6 +198,38 @@ def test_odd_group_sizes(w, mode):
     pu.check_full(w, binding.IMPL_TCGEN05, mode=mode, single_pass=True)
 
 
+def test_trailing_padding_leaves_real_rows_unchanged():
+    """A length that is no multiple of 128 takes the mma.sync kernels; padded with trailing rows (dO = 0 there) to
+    a multiple of 128 it takes the tensor-core kernels, and nothing changes for the real rows: later positions are
+    invisible to every earlier row of either stream."""
+    w = Workload("ragged", 1, 4, 2, 128, 160, 32)
+    inp = synth.make_inputs(w, "cpu")
+    x = pu.f64(inp)
+    M, L, Lp = w.block_size, w.L, 256
+    pad = {}
+    gen = torch.Generator().manual_seed(7)
+    for n, t in inp.items():
+        extra = torch.randn((t.shape[0], Lp - L) + tuple(t.shape[2:]), generator=gen).to(t.dtype)
+        if n.startswith("do_"):
+            extra.zero_()
+        pad[n] = torch.cat([t, extra], dim=1).contiguous()
+    g = pu.to_cuda(pad)
+    out = pu.gpu_fwd(g, M, impl=binding.IMPL_TCGEN05)
+    ref = orc.attn_forward(*[x[n] for n in pu.NAMES6], M)
+    for got, want, tol, is_lse in ((out[0], ref[0], pu.TOL_O, False), (out[1], ref[1], pu.TOL_LSE, True),
+                                   (out[2], ref[2], pu.TOL_O, False), (out[3], ref[3], pu.TOL_LSE, True)):
+        gotn = synth.to_f64(got)
+        gotn = gotn[:, :, :L] if is_lse else gotn[:, :L]
+        assert np.abs(gotn - want).max() <= tol
+    gref = orc.attn_backward(*[x[n] for n in pu.NAMES6], x["do_clean"], x["do_noisy"], M)
+    for sp in (False, True):
+        grads = pu.gpu_bwd(g, out, M, impl=binding.IMPL_TCGEN05, single_pass=sp)
+        torch.cuda.synchronize()
+        assert binding.bdlm_get_device_status() == 0
+        for got, want in zip(grads, gref):
+            assert pu.rel_l2(synth.to_f64(got)[:, :L], want) <= pu.TOL_GRAD
+
+
 @pytest.mark.parametrize("impl", IMPLS)
 def test_large_logits(impl):
     """Scores with a standard deviation of about 10 nats (q and k six times larger than in the workloads):
