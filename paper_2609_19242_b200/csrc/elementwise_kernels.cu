@@ -15,13 +15,14 @@ struct MergeArgs {
   int n;
 };
 
-// One thread owns 8 consecutive head-dim elements of one (row, head).  The running state
+// One thread owns EPT (8 or 16) consecutive head-dim elements of one (row, head).  The running state
 // (numerator, m, normaliser) stays in fp32 registers until the final division, so no thread
 // reads state another thread has already overwritten.
-template <bool F32IN>
+template <bool F32IN, int EPT>
 __global__ void __launch_bounds__(256) merge_kernel(MergeArgs ma, int64_t total_chunks, int L, int H, int d,
                                                     bf16* __restrict__ o_out, float* __restrict__ lse_out) {
-  const int cpr = d / 8;   // chunks per (row, head)
+  constexpr int NV = F32IN ? EPT / 4 : EPT / 8;   // 16-byte vectors per thread and partial
+  const int cpr = d / EPT;   // chunks per (row, head)
   for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total_chunks;
        idx += (int64_t)gridDim.x * blockDim.x) {
     const int c = (int)(idx % cpr);
@@ -31,40 +32,61 @@ __global__ void __launch_bounds__(256) merge_kernel(MergeArgs ma, int64_t total_
     const int64_t bidx = row / L;
     const int i = (int)(row % L);
     const int64_t lidx = (bidx * H + h) * L + i;
-    float num[8];
+    float num[EPT];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) num[e] = 0.f;
+    for (int e = 0; e < EPT; ++e) num[e] = 0.f;
     float m = -INFINITY, norm = 0.f;
-    for (int j = 0; j < ma.n; ++j) {
-      const float z = ma.lse[j][lidx];
-      const float m_new = fmaxf(m, z);
-      const float w_acc = isfinite(m) ? expf(m - m_new) : 0.f;
-      const float w_j = isfinite(z) ? expf(z - m_new) : 0.f;
-      float x[8];
-      if (F32IN) {
-        const float4* p = reinterpret_cast<const float4*>(static_cast<const float*>(ma.o[j]) + idx * 8);
-        float4 u = p[0], v = p[1];
-        x[0] = u.x; x[1] = u.y; x[2] = u.z; x[3] = u.w; x[4] = v.x; x[5] = v.y; x[6] = v.z; x[7] = v.w;
-      } else {
-        uint4 u = *reinterpret_cast<const uint4*>(static_cast<const bf16*>(ma.o[j]) + idx * 8);
-        const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&u);
+    // four partials at a time: their loads are issued together (the kernel is a pure stream, it needs bytes in flight),
+    // then they are folded in left to right
+    for (int j0 = 0; j0 < ma.n; j0 += 4) {
+      float z4[4];
+      uint4 u4[4][NV];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          float2 f = __bfloat1622float2(p2[e]);
-          x[2 * e] = f.x; x[2 * e + 1] = f.y;
+      for (int jj = 0; jj < 4; ++jj) {
+        const int j = j0 + jj;
+        if (j < ma.n) {
+          z4[jj] = ma.lse[j][lidx];
+          const uint4* p = F32IN ? reinterpret_cast<const uint4*>(static_cast<const float*>(ma.o[j]) + idx * EPT)
+                                 : reinterpret_cast<const uint4*>(static_cast<const bf16*>(ma.o[j]) + idx * EPT);
+#pragma unroll
+          for (int v = 0; v < NV; ++v) u4[jj][v] = p[v];
         }
       }
 #pragma unroll
-      for (int e = 0; e < 8; ++e) num[e] = w_acc * num[e] + w_j * x[e];
-      norm = w_acc * norm + w_j;
-      m = m_new;
+      for (int jj = 0; jj < 4; ++jj) {
+        if (j0 + jj >= ma.n) break;
+        const float z = z4[jj];
+        const float m_new = fmaxf(m, z);
+        const float w_acc = isfinite(m) ? expf(m - m_new) : 0.f;
+        const float w_j = isfinite(z) ? expf(z - m_new) : 0.f;
+        float x[EPT];
+        if (F32IN) {
+          const float* pf = reinterpret_cast<const float*>(&u4[jj][0]);
+#pragma unroll
+          for (int e = 0; e < EPT; ++e) x[e] = pf[e];
+        } else {
+          const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&u4[jj][0]);
+#pragma unroll
+          for (int e = 0; e < EPT / 2; ++e) {
+            float2 f = __bfloat1622float2(p2[e]);
+            x[2 * e] = f.x; x[2 * e + 1] = f.y;
+          }
+        }
+#pragma unroll
+        for (int e = 0; e < EPT; ++e) num[e] = w_acc * num[e] + w_j * x[e];
+        norm = w_acc * norm + w_j;
+        m = m_new;
+      }
     }
     const float inv = norm > 0.f ? 1.f / norm : 0.f;
-    uint4 outv;
-    uint32_t* ow = reinterpret_cast<uint32_t*>(&outv);
 #pragma unroll
-    for (int e = 0; e < 4; ++e) ow[e] = pack_bf16(num[2 * e] * inv, num[2 * e + 1] * inv);
-    *reinterpret_cast<uint4*>(o_out + idx * 8) = outv;
+    for (int v = 0; v < EPT / 8; ++v) {
+      uint4 outv;
+      uint32_t* ow = reinterpret_cast<uint32_t*>(&outv);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) ow[e] = pack_bf16(num[8 * v + 2 * e] * inv, num[8 * v + 2 * e + 1] * inv);
+      reinterpret_cast<uint4*>(o_out + idx * EPT)[v] = outv;
+    }
     if (c == 0) lse_out[lidx] = norm > 0.f ? m + logf(norm) : -INFINITY;
   }
 }
@@ -127,13 +149,19 @@ cudaError_t launch_merge(int n, int batch, int L, int H, int d, const void* cons
     ma.o[j] = j < n ? o_parts[j] : nullptr;
     ma.lse[j] = j < n ? lse_parts[j] : nullptr;
   }
-  const int64_t total = (int64_t)batch * L * H * (d / 8);
+  // few partials: 16 elements per thread (more bytes in flight per thread); otherwise 8
+  const int ept = (d % 16 == 0 && n <= 3) ? 16 : 8;
+  const int64_t total = (int64_t)batch * L * H * (d / ept);
   int64_t want = (total + 255) / 256;
   int blocks = (int)(want < 148 * 16 ? (want > 0 ? want : 1) : 148 * 16);
-  if (dtype == 1)
-    merge_kernel<true><<<blocks, 256, 0, st>>>(ma, total, L, H, d, static_cast<bf16*>(o_out), lse_out);
-  else
-    merge_kernel<false><<<blocks, 256, 0, st>>>(ma, total, L, H, d, static_cast<bf16*>(o_out), lse_out);
+  bf16* oo = static_cast<bf16*>(o_out);
+  if (dtype == 1) {
+    if (ept == 16) merge_kernel<true, 16><<<blocks, 256, 0, st>>>(ma, total, L, H, d, oo, lse_out);
+    else merge_kernel<true, 8><<<blocks, 256, 0, st>>>(ma, total, L, H, d, oo, lse_out);
+  } else {
+    if (ept == 16) merge_kernel<false, 16><<<blocks, 256, 0, st>>>(ma, total, L, H, d, oo, lse_out);
+    else merge_kernel<false, 8><<<blocks, 256, 0, st>>>(ma, total, L, H, d, oo, lse_out);
+  }
   return cudaGetLastError();
 }
 
