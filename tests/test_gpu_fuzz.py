@@ -49,6 +49,26 @@ def test_random_plain_configurations_fused_backward(case):
     pu.check_full(w, binding.IMPL_AUTO, mode=mode, single_pass=True)
 
 
+def _larger_cases(n, seed):
+    rng = np.random.default_rng(seed)
+    cases = []
+    for i in range(n):
+        L = 128 * int(rng.integers(5, 15))
+        M = int(rng.choice([m for m in (8, 16, 24, 32, 48, 64, 96, 128, 192, 256, 384) if L % m == 0]))
+        Hkv, G = int(rng.choice([1, 2, 3])), int(rng.choice([1, 2, 3, 4, 5]))
+        cases.append((Workload(f"big{i}", int(rng.choice([1, 2])), Hkv * G, Hkv, 128, L, M,
+                               window=int(rng.choice([0, 0, 0, 130, 700])), seed=300 + i), int(rng.choice([0, 0, 1]))))
+    return cases
+
+
+@pytest.mark.parametrize("case", _larger_cases(6, 5), ids=lambda c: f"{c[0].name}-L{c[0].L}-M{c[0].block_size}-H{c[0].H}/{c[0].H_kv}-w{c[0].window}-m{c[1]}")
+def test_random_larger_configurations(case):
+    """Five to fourteen tiles per stream, group sizes 1 to 5, through the tensor-core kernels and both backward paths."""
+    w, mode = case
+    pu.check_full(w, binding.IMPL_TCGEN05, mode=mode)
+    pu.check_full(w, binding.IMPL_TCGEN05, mode=mode, single_pass=True, check_bwd=True)
+
+
 def _packed_cases(n, seed):
     rng = np.random.default_rng(seed)
     cases = []
