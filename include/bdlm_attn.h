@@ -65,7 +65,8 @@ typedef struct {
                                   CTA adds its dQ tiles into an fp32 accumulator in the workspace (bulk add-reductions), so
                                   dQ is reproducible only up to fp32 summation order; dK and dV are bitwise reproducible (fixed order).
                                   Needs the larger workspace bdlm_workspace_bytes[_packed] reports for this setting; falls
-                                  back to the two-pass path when the tensor-core kernels do not take the shape. */
+                                  back to the two-pass path when the tensor-core kernels do not take the shape.  With
+                                  bwd_passes the fused kernel runs under BDLM_BWD_PASS_DKDV; BDLM_BWD_PASS_DQ is then a no-op. */
   int32_t window;              /* sliding-window layers: > 0 = a clean key j is visible to the query at position i (of either
                                   stream) only if additionally i - j < window; the noisy own block is unaffected.  0 = none. */
   int32_t reserved[2];
