@@ -983,13 +983,13 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
           tc_fence_after();
           issue_st(sqn);
         }
-        // dP^T of the next step, once every compute thread holds dP^T(i) in registers
-        if (i + 1 < nsteps) {
-          ok = mbar_wait_timed<TR>(bar_dpfree, i & 1, abort_flag, w_dpf);
-          ok = ok && mbar_wait_timed<TR>(bar_do_full + 8 * sn, kn & 1, abort_flag, w_do);
-          if (!ok) break;
+        // dP^T of the next step, once every compute thread holds dP^T(i) in registers -- now, if its dO tile has
+        // landed; after dQ^T and dK otherwise (a late load does not hold up the GEMMs that are ready)
+        bool dpt_due = i + 1 < nsteps;
+        if (dpt_due && mbar_try_wait(bar_dpfree, i & 1) && mbar_try_wait(bar_do_full + 8 * sn, kn & 1)) {
           tc_fence_after();
           issue_dpt(sn);
+          dpt_due = false;
         }
         // dQ^T = K^T dS^T (once the read-out warps hold the previous dQ^T), then dK += dS^T Q_i
         ok = mbar_wait_timed<TR>(bar_dst, i & 1, abort_flag, w_dst);
@@ -1005,6 +1005,13 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
           mma_ss_e(tmem + 384, desc64(dsk_lo + 2 * kk), desc64(qm_lo0 + sq * HT_LO + moff(kk)), IDESC_KM, kk == 0 ? acc : 1u, el);
         mma_commit_e(bar_q_empty + 8 * sq, el);
         mma_commit_e(bar_dsfree, el);
+        if (dpt_due) {
+          ok = mbar_wait_timed<TR>(bar_dpfree, i & 1, abort_flag, w_dpf);
+          ok = ok && mbar_wait_timed<TR>(bar_do_full + 8 * sn, kn & 1, abort_flag, w_do);
+          if (!ok) break;
+          tc_fence_after();
+          issue_dpt(sn);
+        }
         sd = sn;
         if (++sn == BF_DOS) { sn = 0; ++kn; }
         sq = sqn;
