@@ -33,21 +33,18 @@ METRIC = "BDLM attn fwd+bwd TFLOP/s (unmasked FLOPs)"
 UNIT = "TFLOP/s"
 NAMES6 = ["q_clean", "k_clean", "v_clean", "q_noisy", "k_noisy", "v_noisy"]
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant
-# kernel, from the ncu captures summarised under profiles/ ; keyed by (workload, kernel).
-NCU_TRAFFIC_BYTES = {
-    ("8k", "fwd"): 207913984 + 109006592,
-    ("8k", "bwd_fused"): 762043904 + 374662144,
-    ("8k", "bwd_dkdv"): 380482816 + 54774784,
-    ("8k", "bwd_dq"): 365881344 + 115298560,
-    ("32k", "fwd"): 964474368 + 522727680,
-    ("32k", "bwd_fused"): 5886429184 + 3367195136,
-    ("32k", "bwd_dkdv"): 2396964864 + 250488576,
-    ("32k", "bwd_dq"): 1545019136 + 518886400,
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of a kernel from a one-pass ncu capture of
+# this command, keyed by (workload, kernel), each with the digest of the kernel sources it was captured on
+# (kernel_source_digest): a figure is reported only for the build it belongs to.
+_CAPTURED_ON = "unset"
+NCU_TRAFFIC = {
+    ("32k", "fwd"): {"bytes": 964474368 + 522727680, "kernel_source": _CAPTURED_ON},
+    ("32k", "bwd_fused"): {"bytes": 5886429184 + 3367195136, "kernel_source": _CAPTURED_ON},
+    ("32k", "bwd_dkdv"): {"bytes": 2396964864 + 250488576, "kernel_source": _CAPTURED_ON},
+    ("32k", "bwd_dq"): {"bytes": 1545019136 + 518886400, "kernel_source": _CAPTURED_ON},
 }
-TRAFFIC_NOTE = ("dram__bytes_read.sum + dram__bytes_write.sum per launch from ncu captures of the 8k and the 32k "
-                "workload (profiles/tc_kernels_8k_ncu_full.md, profiles/tc_kernels_32k_dram_traffic.md; the two "
-                "counters take one pass); other workloads have no capture and report null")
+TRAFFIC_NOTE = ("dram__bytes_read.sum + dram__bytes_write.sum per launch from a one-pass ncu capture of this command on "
+                "the 32k workload")
 
 
 def load_peaks():
@@ -234,6 +231,204 @@ def aggregate_tflops(flops_per_replica, ms_per_step, world):
 # ------------------------------------------------------------------------------------------
 # our arm
 # ------------------------------------------------------------------------------------------
+def kernel_source_digest():
+    """sha256 over the tensor-core kernel sources: an ncu traffic figure belongs to the build it was captured on."""
+    import hashlib
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2609_19242_b200", "csrc")
+    for f in ("bdlm_common.cuh", "tc_common.cuh", "tc_kernels.cu", "tc_bwd_kernels.cu"):
+        with open(os.path.join(csrc, f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+class LayerRun:
+    """Inputs, outputs and workspace of one workload on the current device, and the calls of one step."""
+
+    def __init__(self, w, binding, seed_offset, impl, fused):
+        self.w, self.binding, self.impl, self.fused = w, binding, impl, fused
+        self.M = w.block_size
+        self.g = synth.make_inputs(synth.small(w, seed=w.seed + seed_offset), "cuda")
+        self.fwd_out, self.grads, self.ws = self.make_buffers(self.g)
+
+    def like(self, t):
+        return None if t is None else torch.empty_like(t)
+
+    def lse_like(self, q):
+        w = self.w
+        return None if q is None else torch.empty(w.batch, w.H, q.shape[1], dtype=torch.float32, device="cuda")
+
+    def make_buffers(self, gg):
+        """Outputs, gradients and workspace of one step for the inputs `gg`."""
+        w, binding = self.w, self.binding
+        fo = (self.like(gg["q_clean"]), self.lse_like(gg["q_clean"]), self.like(gg["q_noisy"]), self.lse_like(gg["q_noisy"]))
+        gr = tuple(self.like(gg[n]) for n in NAMES6)
+        rows = max(t.shape[1] for t in (gg["q_clean"], gg["q_noisy"]) if t is not None)
+        wsz = 2 * (w.batch * w.H * rows * 4 + 256)
+        if self.fused:   # fp32 dQ accumulators of the fused backward, one per query stream
+            wsz += sum(t.shape[1] for t in (gg["q_clean"], gg["q_noisy"]) if t is not None) * w.batch * w.H * w.d * 4
+        if not w.packed:
+            wsz = max(wsz, binding.bdlm_workspace_bytes(
+                binding.make_params(w.batch, w.L, self.M, w.H, w.H_kv, w.d, bwd_single_pass=self.fused), binding.BDLM_WS_BWD))
+        return fo, gr, torch.empty(wsz, dtype=torch.uint8, device="cuda")
+
+    def run_fwd(self, gg=None, fo=None, **kw):
+        w, binding = self.w, self.binding
+        gg = self.g if gg is None else gg
+        fo = self.fwd_out if fo is None else fo
+        if w.packed:
+            binding.bdlm_attn_fwd_packed(*[gg[n] for n in NAMES6], self.M, block_prefix=gg["block_prefix"], out=fo,
+                                         impl=self.impl, window=w.window, **kw)
+        else:
+            binding.bdlm_attn_fwd(*[gg[n] for n in NAMES6], self.M, out=fo, impl=self.impl, window=w.window, **kw)
+
+    def run_bwd(self, gg=None, fo=None, gr=None, wsb=None, passes=0):
+        w, binding = self.w, self.binding
+        gg = self.g if gg is None else gg
+        fo = self.fwd_out if fo is None else fo
+        gr = self.grads if gr is None else gr
+        wsb = self.ws if wsb is None else wsb
+        if w.packed:
+            binding.bdlm_attn_bwd_packed(*[gg[n] for n in NAMES6], fo[0], fo[1], fo[2], fo[3], gg["do_clean"],
+                                         gg["do_noisy"], self.M, block_prefix=gg["block_prefix"], out=gr, workspace=wsb,
+                                         impl=self.impl, passes=passes, window=w.window, single_pass=self.fused)
+        else:
+            binding.bdlm_attn_bwd(*[gg[n] for n in NAMES6], fo[0], fo[1], fo[2], fo[3], gg["do_clean"],
+                                  gg["do_noisy"], self.M, out=gr, workspace=wsb, impl=self.impl, passes=passes,
+                                  window=w.window, single_pass=self.fused)
+
+    def kernel_names(self):
+        # two-pass backward: dK/dV pass, then dQ pass; fused backward: one kernel for both (launched by the DKDV
+        # pass bit together with the zero-fill of the fp32 dQ accumulators and their conversion; the DQ bit is a no-op)
+        return ["fwd", "bwd_dsum", "bwd_fused" if self.fused else "bwd_dkdv", "bwd_dq"]
+
+    def timed_steps(self, K, warmup, barrier, sampler=None):
+        """W warm-up steps, then K timed steps with events between the kernels of a step.  Returns the total time of
+        the K steps (ms, device clock), the per-step times and the mean time per kernel."""
+        binding = self.binding
+        for _ in range(warmup):
+            self.run_fwd()
+            self.run_bwd()
+        torch.cuda.synchronize()
+        if binding.bdlm_get_device_status() != 0:
+            raise RuntimeError("device-side wait timed out during warm-up")
+        names = self.kernel_names()
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(len(names) + 1)] for _ in range(K)]
+        if sampler is not None:
+            sampler.start()
+            time.sleep(0.25)
+        barrier()
+        e_start, e_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e_start.record()
+        for i in range(K):
+            ev[i][0].record()
+            self.run_fwd()
+            ev[i][1].record()
+            self.run_bwd(passes=binding.PASS_DSUM)
+            ev[i][2].record()
+            self.run_bwd(passes=binding.PASS_DKDV)
+            ev[i][3].record()
+            self.run_bwd(passes=binding.PASS_DQ)
+            ev[i][4].record()
+        e_stop.record()
+        barrier()
+        ms_total = e_start.elapsed_time(e_stop)
+        clocks = sampler.stop() if sampler is not None else None
+        if binding.bdlm_get_device_status() != 0:
+            raise RuntimeError("device-side wait timed out during the timed region")
+        per_step = [ev[i][0].elapsed_time(ev[i][len(names)]) for i in range(K)]
+        per_kernel = {n: float(np.mean([ev[i][j].elapsed_time(ev[i][j + 1]) for i in range(K)])) for j, n in enumerate(names)}
+        return ms_total, per_step, per_kernel, clocks
+
+
+def fractions(tflops, peaks):
+    return {"frac_burst": tflops / peaks["bf16_tflops"], "frac_sustained": tflops / peaks["bf16_tflops_sustained"],
+            "frac_nominal_2250": tflops / 2250.0}
+
+
+def sharded_forward_leg(run, peaks, steps, warmup):
+    """The CSBP rank-local emulation as its configuration states it: the forward as one partial per contiguous
+    clean-K/V shard (include_noisy_diag = 0) plus the noisy-diagonal partial (empty clean range), combined by
+    bdlm_lse_merge (Eq. csbp-lse-merge) -- one merge call per query stream.  Timed with events: the partial
+    launches, the two merges, and the whole."""
+    w, binding = run.w, run.binding
+    g, M, S = run.g, run.M, w.kv_shards
+    step = w.L // S
+    part_out = [(run.like(g["q_clean"]), run.lse_like(g["q_clean"]), run.like(g["q_noisy"]), run.lse_like(g["q_noisy"]))
+                for _ in range(S)]
+    diag_out = (None, None, run.like(g["q_noisy"]), run.lse_like(g["q_noisy"]))
+    merged = (run.like(g["q_clean"]), run.lse_like(g["q_clean"]), run.like(g["q_noisy"]), run.lse_like(g["q_noisy"]))
+
+    def partials():
+        for s in range(S):
+            run.run_fwd(fo=part_out[s], kv_range=(s * step, (s + 1) * step), include_noisy_diag=False)
+        binding.bdlm_attn_fwd(None, g["k_clean"], g["v_clean"], g["q_noisy"], g["k_noisy"], g["v_noisy"], M,
+                              out=diag_out, kv_range=(0, 0), impl=run.impl)
+
+    def merges():
+        binding.bdlm_lse_merge([p[0] for p in part_out], [p[1] for p in part_out], out=(merged[0], merged[1]))
+        binding.bdlm_lse_merge([p[2] for p in part_out] + [diag_out[2]], [p[3] for p in part_out] + [diag_out[3]],
+                               out=(merged[2], merged[3]))
+
+    for _ in range(warmup):
+        partials()
+        merges()
+    torch.cuda.synchronize()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+    for i in range(steps):
+        ev[i][0].record()
+        partials()
+        ev[i][1].record()
+        merges()
+        ev[i][2].record()
+    torch.cuda.synchronize()
+    if binding.bdlm_get_device_status() != 0:
+        raise RuntimeError("device-side wait timed out in the sharded forward")
+    ms_part = [ev[i][0].elapsed_time(ev[i][1]) for i in range(steps)]
+    ms_merge = [ev[i][1].elapsed_time(ev[i][2]) for i in range(steps)]
+    # bytes the two merges must move: every partial's O (bf16) and LSE (fp32) in, the merged O and LSE out
+    o_bytes = w.batch * w.L * w.H * w.d * 2
+    l_bytes = w.batch * w.H * w.L * 4
+    merge_bytes = (S + 1) * (o_bytes + l_bytes) + (S + 2) * (o_bytes + l_bytes)
+    f_fwd, _ = w.flops()
+    ms_m = float(np.mean(ms_merge))
+    ms_all = float(np.mean(ms_part)) + ms_m
+    # agreement with the unsharded forward of the same inputs (already in run.fwd_out from the timed steps)
+    diff = {"o_clean": float((merged[0].float() - run.fwd_out[0].float()).abs().max()),
+            "lse_clean": float((merged[1] - run.fwd_out[1]).abs().max()),
+            "o_noisy": float((merged[2].float() - run.fwd_out[2].float()).abs().max()),
+            "lse_noisy": float((merged[3] - run.fwd_out[3]).abs().max())}
+    return {"shards": S, "partials": f"{S} clean-K/V shard partials (both query streams) + 1 noisy-diagonal partial",
+            "steps": steps, "ms_partials": float(np.mean(ms_part)), "ms_merge": ms_m, "ms_total": ms_all,
+            "ms_total_min": float(np.min(np.add(ms_part, ms_merge))), "ms_total_median": float(np.median(np.add(ms_part, ms_merge))),
+            "fwd_tflops": f_fwd / (ms_all * 1e-3) / 1e12,
+            "merge": {"calls": 2, "n_partials": [S, S + 1], "algorithmic_bytes": merge_bytes,
+                      "achieved_gbs": merge_bytes / (ms_m * 1e-3) / 1e9, "peak_gbs": peaks["hbm_gbs"],
+                      "frac": merge_bytes / (ms_m * 1e-3) / 1e9 / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                      "ms_min": float(np.min(ms_merge)), "ms_median": float(np.median(ms_merge))},
+            "max_abs_diff_vs_unsharded_forward": diff}
+
+
+def other_config_line(name, binding, peaks, impl, fused, steps, warmup, local):
+    """One more workload on the same GPU, timed like the headline: value, per-kernel times, clocks."""
+    w = synth.WORKLOADS[name]
+    run = LayerRun(w, binding, 0, impl, fused)
+    sampler = ClockSampler(physical_gpu_index(local))
+    ms_total, per_step, per_kernel, clocks = run.timed_steps(steps, warmup, torch.cuda.synchronize, sampler)
+    f_fwd, f_bwd = w.flops()
+    ms_step = ms_total / steps
+    tf = (f_fwd + f_bwd) / (ms_step * 1e-3) / 1e12
+    out = {"workload": name, "L": w.L, "block_size": w.block_size, "steps": steps, "warmup": warmup,
+           "value": tf, "unit": UNIT, "ms_per_step": ms_step, "ms_per_step_min": float(np.min(per_step)),
+           "ms_per_step_median": float(np.median(per_step)), "per_kernel_ms": per_kernel, "clocks": clocks}
+    out.update(fractions(tf, peaks))
+    if w.kv_shards > 1:
+        out["sharded_fwd"] = sharded_forward_leg(run, peaks, steps, warmup)
+    del run
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_ours(args, w):
     from paper_2609_19242_b200 import binding
     import torch.distributed as dist
@@ -251,94 +446,18 @@ def run_ours(args, w):
         torch.cuda.synchronize()
 
     peaks = load_peaks()
-    M = w.block_size
-    g = synth.make_inputs(synth.small(w, seed=w.seed + rank), "cuda")
     impl = args.kernel_impl
     fused = args.bwd == "fused"
-
-    def like(t):
-        return None if t is None else torch.empty_like(t)
-
-    def lse_like(q):
-        return None if q is None else torch.empty(w.batch, w.H, q.shape[1], dtype=torch.float32, device="cuda")
-
-    def make_buffers(gg):
-        """Outputs, gradients and workspace of one step for the inputs `gg`."""
-        fo = (like(gg["q_clean"]), lse_like(gg["q_clean"]), like(gg["q_noisy"]), lse_like(gg["q_noisy"]))
-        gr = tuple(like(gg[n]) for n in NAMES6)
-        rows = max(t.shape[1] for t in (gg["q_clean"], gg["q_noisy"]) if t is not None)
-        wsz = 2 * (w.batch * w.H * rows * 4 + 256)
-        if fused:   # fp32 dQ accumulators of the fused backward, one per query stream
-            wsz += sum(t.shape[1] for t in (gg["q_clean"], gg["q_noisy"]) if t is not None) * w.batch * w.H * w.d * 4
-        if not w.packed:
-            wsz = max(wsz, binding.bdlm_workspace_bytes(binding.make_params(w.batch, w.L, M, w.H, w.H_kv, w.d,
-                                                                            bwd_single_pass=fused),
-                                                        binding.BDLM_WS_BWD))
-        return fo, gr, torch.empty(wsz, dtype=torch.uint8, device="cuda")
-
-    def run_fwd(gg, fo):
-        if w.packed:
-            binding.bdlm_attn_fwd_packed(*[gg[n] for n in NAMES6], M, block_prefix=gg["block_prefix"], out=fo,
-                                         impl=impl, window=w.window)
-        else:
-            binding.bdlm_attn_fwd(*[gg[n] for n in NAMES6], M, out=fo, impl=impl, window=w.window)
-
-    def run_bwd(gg, fo, gr, wsb, passes=0):
-        if w.packed:
-            binding.bdlm_attn_bwd_packed(*[gg[n] for n in NAMES6], fo[0], fo[1], fo[2], fo[3], gg["do_clean"],
-                                         gg["do_noisy"], M, block_prefix=gg["block_prefix"], out=gr, workspace=wsb,
-                                         impl=impl, passes=passes, window=w.window, single_pass=fused)
-        else:
-            binding.bdlm_attn_bwd(*[gg[n] for n in NAMES6], fo[0], fo[1], fo[2], fo[3], gg["do_clean"],
-                                  gg["do_noisy"], M, out=gr, workspace=wsb, impl=impl, passes=passes,
-                                  window=w.window, single_pass=fused)
-
-    fwd_out, grads, ws = make_buffers(g)
-
-    def fwd():
-        run_fwd(g, fwd_out)
-
-    def bwd(passes=0):
-        run_bwd(g, fwd_out, grads, ws, passes)
-
-    for _ in range(args.warmup):
-        fwd()
-        bwd()
-    torch.cuda.synchronize()
-    if binding.bdlm_get_device_status() != 0:
-        raise RuntimeError("device-side wait timed out during warm-up")
+    run = LayerRun(w, binding, rank, impl, fused)
+    g, fwd_out, grads, ws = run.g, run.fwd_out, run.grads, run.ws
+    like = run.like
 
     # ---- timed region: K steps, device time, events between the kernels of a step -------------
     K = args.steps
-    # two-pass backward: dK/dV pass, then dQ pass; fused backward: one kernel for both (launched by the DKDV
-    # pass bit together with the zero-fill of the fp32 dQ accumulators and their conversion; the DQ bit is a no-op)
-    names = ["fwd", "bwd_dsum", "bwd_fused" if fused else "bwd_dkdv", "bwd_dq"]
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(len(names) + 1)] for _ in range(K)]
-    sampler = ClockSampler(physical_gpu_index(local))
-    if rank == 0:
-        sampler.start()
-        time.sleep(0.25)
-    barrier()
-    e_start, e_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e_start.record()
-    for i in range(K):
-        ev[i][0].record()
-        fwd()
-        ev[i][1].record()
-        bwd(binding.PASS_DSUM)
-        ev[i][2].record()
-        bwd(binding.PASS_DKDV)
-        ev[i][3].record()
-        bwd(binding.PASS_DQ)
-        ev[i][4].record()
-    e_stop.record()
-    barrier()
-    ms_total = e_start.elapsed_time(e_stop)
-    clocks = sampler.stop() if rank == 0 else None
-    if binding.bdlm_get_device_status() != 0:
-        raise RuntimeError("device-side wait timed out during the timed region")
+    names = run.kernel_names()
+    sampler = ClockSampler(physical_gpu_index(local)) if rank == 0 else None
+    ms_total, per_step, per_kernel_ms, clocks = run.timed_steps(K, args.warmup, barrier, sampler)
     ms_total = max_over_ranks(ms_total, "cuda", world)
-    per_kernel_ms = {n: float(np.mean([ev[i][j].elapsed_time(ev[i][j + 1]) for i in range(K)])) for j, n in enumerate(names)}
 
     f_fwd, f_bwd = w.flops()
     ms_step = ms_total / K
@@ -357,7 +476,7 @@ def run_ours(args, w):
         # k-1 (device to host) run under the kernels of step k.  Every step still copies all of its inputs in
         # and all of its results out inside the timed region; pipeline fill and drain are part of it too.
         g2 = {k_: like(v) for k_, v in g.items()}
-        fo2, gr2, ws2 = make_buffers(g2)
+        fo2, gr2, ws2 = run.make_buffers(g2)
         sets = [{"g": g, "fwd": fwd_out, "grads": grads, "ws": ws}, {"g": g2, "fwd": fo2, "grads": gr2, "ws": ws2}]
         s_comp = torch.cuda.current_stream()
         s_h2d, s_d2h = torch.cuda.Stream(), torch.cuda.Stream()
@@ -376,8 +495,8 @@ def run_ours(args, w):
                 s_comp.wait_event(h2d_done)
                 if k >= 2:
                     s_comp.wait_event(d2h_done[k - 2])          # the set's outputs have been read out
-                run_fwd(st["g"], st["fwd"])
-                run_bwd(st["g"], st["fwd"], st["grads"], st["ws"])
+                run.run_fwd(st["g"], st["fwd"])
+                run.run_bwd(st["g"], st["fwd"], st["grads"], st["ws"])
                 ev_c = torch.cuda.Event()
                 ev_c.record(s_comp)
                 comp_done.append(ev_c)
@@ -403,7 +522,7 @@ def run_ours(args, w):
         e2e = {"value": aggregate_tflops(f_fwd + f_bwd, ms_e2e, world), "unit": UNIT,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e,
                "steps": n_e2e, "overlap": "copies of neighbouring steps run under the kernels (3 streams, 2 buffer sets)"}
-        del host_in, host_out, sets
+        del host_in, host_out, sets, g2, fo2, gr2, ws2
 
     if rank != 0:
         if world > 1:
@@ -419,12 +538,31 @@ def run_ours(args, w):
     dom = max((n for n in names if n != "bwd_dsum"), key=lambda n: per_kernel_ms[n])
     peak = peaks["bf16_tflops_sustained"] if ms_step * K > 1000.0 else peaks["bf16_tflops"]
     achieved = algo_flops[dom] / (per_kernel_ms[dom] * 1e-3) / 1e12
+    digest = kernel_source_digest()
+    cap = NCU_TRAFFIC.get((w.name, dom))
+    traffic = cap["bytes"] if cap is not None and cap["kernel_source"] == digest else None
+    if cap is None:
+        traffic_note = TRAFFIC_NOTE + "; this workload has no capture"
+    elif traffic is None:
+        traffic_note = TRAFFIC_NOTE + "; the capture on record predates the current kernel source, so none is reported"
+    else:
+        traffic_note = TRAFFIC_NOTE
     roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                 "frac": achieved / peak, "peak_source": peaks["source"] +
-                (" sustained" if peak == peaks["bf16_tflops_sustained"] else " burst"),
-                "traffic": NCU_TRAFFIC_BYTES.get((w.name, dom)), "traffic_note": TRAFFIC_NOTE,
+                (" sustained (timed region longer than 1 s)" if peak == peaks["bf16_tflops_sustained"] else " burst"),
+                "traffic": traffic, "traffic_note": traffic_note, "kernel_source": digest,
                 "per_kernel_ms": per_kernel_ms,
                 "per_kernel_tflops": {n: (algo_flops[n] / (per_kernel_ms[n] * 1e-3) / 1e12) for n in names}}
+    roofline.update(fractions(achieved, peaks))
+
+    # ---- the other single-GPU configurations the target is stated on, and the paper-range block sizes ------
+    others = None
+    if world == 1 and args.other_configs and w.name == "32k":
+        del run, g, fwd_out, grads, ws
+        torch.cuda.empty_cache()
+        others = {}
+        for name, st_, wu_ in (("csbp128k", 3, 3), ("256k", 3, 3), ("32k_m512", 5, 3), ("32k_m1024", 5, 3), ("8k", 10, 3)):
+            others[name] = other_config_line(name, binding, peaks, impl, fused, st_, wu_, local)
 
     # ---- CPU baseline: the oracle on a bounded sample, on this machine's host cores ---------------
     cpu = None
@@ -435,22 +573,24 @@ def run_ours(args, w):
             rows = args.oracle_rows
             t, f = oracle_sample(w, inp, rows, seed=0)
         else:
-            rows, t, f = timed_oracle_sample(w, inp, 40.0, w.L)
+            rows, t, f = timed_oracle_sample(w, inp, 20.0, w.L)
         cpu = {"value": f / t / 1e12, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                "sample": f"{rows} sampled query rows per stream of (batch 0, head 0), fwd+bwd, fp64, {t:.1f} s"}
 
+    pct = fractions(value / world, peaks)
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
-            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "ms_per_step": ms_step, "ms_per_step_min": float(np.min(per_step)), "ms_per_step_median": float(np.median(per_step)),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": w.name, "batch": w.batch, "H": w.H, "H_kv": w.H_kv, "d": w.d, "L": w.L,
                        "block_size": w.block_size, "window": w.window, "n_blocks": w.n_blocks, "rope_theta": w.rope_theta, "parallelism": "replicas only",
                        "l2": "inputs larger than L2 (q/k/v/dO of one step exceed 126 MB)",
                        "kernel_impl": {0: "auto", 1: "portable", 2: "tcgen05"}[impl],
                        "backward": "fused (one kernel; dQ through fp32 add-reductions)" if fused else "two-pass (dK/dV, then dQ)"},
-            "pct_of_bf16_peak": {"measured_burst": 100 * value / world / peaks["bf16_tflops"],
-                                 "measured_sustained": 100 * value / world / peaks["bf16_tflops_sustained"],
-                                 "nominal_2250": 100 * value / world / 2250.0, "source": peaks["source"]},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": (6 if fused else 5) * K, "roofline": roofline, "cpu_baseline": cpu}
+            "pct_of_bf16_peak": {"measured_burst": 100 * pct["frac_burst"], "measured_sustained": 100 * pct["frac_sustained"],
+                                 "nominal_2250": 100 * pct["frac_nominal_2250"], "source": peaks["source"]},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": (6 if fused else 5) * K, "roofline": roofline, "cpu_baseline": cpu,
+            "other_configs": others}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -468,6 +608,8 @@ def main():
     ap.add_argument("--bwd", default="fused", choices=["fused", "two_pass"],
                     help="backward: one fused kernel (dQ through fp32 add-reductions) or the bitwise reproducible two-pass path")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-other-configs", dest="other_configs", action="store_false",
+                    help="skip the csbp128k / 256k / block-size legs that the default 32k run appends")
     args = ap.parse_args()
     w = synth.WORKLOADS[args.workload]
     if args.impl == "reference":

@@ -60,19 +60,28 @@ typedef struct {
   int32_t bwd_passes;          /* backward only: 0 = all passes; otherwise a bit set of BDLM_BWD_PASS_* to run
                                   (lets a caller time the passes separately; each pass needs the earlier ones'
                                   results from a previous call with the same workspace) */
-  int32_t bwd_single_pass;     /* backward only: 0 = dK/dV pass + dQ pass, fixed summation order, bitwise reproducible;
-                                  1 = fused: one kernel produces dK, dV and dQ (5 GEMMs per tile pair instead of 7).  Each
-                                  CTA adds its dQ tiles into an fp32 accumulator in the workspace (bulk add-reductions), so
-                                  dQ is reproducible only up to fp32 summation order; dK and dV are bitwise reproducible (fixed order).
-                                  Needs the larger workspace bdlm_workspace_bytes[_packed] reports for this setting; falls
-                                  back to the two-pass path when the tensor-core kernels do not take the shape.  With
-                                  bwd_passes the fused kernel runs under BDLM_BWD_PASS_DKDV; BDLM_BWD_PASS_DQ is then a no-op. */
+  int32_t bwd_single_pass;     /* backward only: which kernels form the gradients (BDLM_BWD_AUTO / _FUSED / _TWO_PASS).
+                                  BDLM_BWD_FUSED (1): one kernel produces dK, dV and dQ (5 GEMMs per tile pair instead of 7).
+                                  Each CTA adds its dQ tiles into an fp32 accumulator in the workspace (bulk add-reductions),
+                                  so dQ is reproducible only up to fp32 summation order; dK and dV are bitwise reproducible
+                                  (fixed order).  Needs the workspace bdlm_workspace_bytes[_packed] reports for this setting
+                                  (BDLM_ERR_WORKSPACE_TOO_SMALL otherwise); shapes the tensor-core kernels do not take
+                                  (d = 64, rows not a multiple of 128, impl = 1) run the two-pass path.
+                                  BDLM_BWD_TWO_PASS (2): dK/dV pass + dQ pass, fixed summation order, every gradient
+                                  bitwise reproducible; needs only the D rows in the workspace.
+                                  BDLM_BWD_AUTO (0, the default of a zeroed struct): the fused kernel when the workspace
+                                  passed to the call is at least the size bdlm_workspace_bytes[_packed] reports for this
+                                  setting (the fused size), the two-pass path when it is smaller (it must still hold the
+                                  D rows: the size reported for BDLM_BWD_TWO_PASS).
+                                  With bwd_passes the fused kernel runs under BDLM_BWD_PASS_DKDV; BDLM_BWD_PASS_DQ is then
+                                  a no-op. */
   int32_t window;              /* sliding-window layers: > 0 = a clean key j is visible to the query at position i (of either
                                   stream) only if additionally i - j < window; the noisy own block is unaffected.  0 = none. */
   int32_t reserved[2];
 } bdlm_params;
 
 enum { BDLM_BWD_PASS_DSUM = 1, BDLM_BWD_PASS_DKDV = 2, BDLM_BWD_PASS_DQ = 4 };
+enum { BDLM_BWD_AUTO = 0, BDLM_BWD_FUSED = 1, BDLM_BWD_TWO_PASS = 2 };   /* values of bdlm_params.bwd_single_pass */
 
 enum { BDLM_WS_FWD = 0, BDLM_WS_BWD = 1 };
 
@@ -99,12 +108,15 @@ int bdlm_attn_fwd(const bdlm_params* p,
  * correctness-clean-gradient, correctness-query-gradient).  Inputs are the forward's inputs,
  * its saved O and LSE, and the upstream gradient dO of both streams.  dK/dV of a KV head are
  * summed over the query heads of its group; clean dK/dV are summed over clean and noisy
- * queries; noisy dK/dV only over the queries of the same block.  The summation order is
- * fixed, so results are bitwise reproducible (with bwd_single_pass = 1: dK and dV are, dQ is
- * reproducible up to fp32 summation order).  Requires the full clean key range.
- * The workspace (bdlm_workspace_bytes(p, BDLM_WS_BWD)) holds D_i = sum_d dO_i,d * O_i,d and, with
- * bwd_single_pass = 1, an fp32 dQ accumulator [batch, H, rows, 128] per query stream; nothing in it
- * has to be initialised or kept between calls.
+ * queries; noisy dK/dV only over the queries of the same block.  The summation order of dK and dV
+ * is fixed, so they are bitwise reproducible; dQ is too on the two-pass path, and reproducible up to
+ * fp32 summation order when the fused kernel runs (see bdlm_params.bwd_single_pass for which one
+ * does).  Requires the full clean key range.
+ * The workspace holds D_i = sum_d dO_i,d * O_i,d and, for the fused kernel, an fp32 dQ accumulator
+ * [batch, H, rows, 128] per query stream; nothing in it has to be initialised or kept between calls.
+ * bdlm_workspace_bytes(p, BDLM_WS_BWD) reports the size for p->bwd_single_pass; with the default
+ * (BDLM_BWD_AUTO) that is the fused kernel's size, and a call given less than that -- but at least
+ * the BDLM_BWD_TWO_PASS size -- runs the two-pass kernels.
  */
 int bdlm_attn_bwd(const bdlm_params* p,
                   const void* q_clean, const void* k_clean, const void* v_clean,
@@ -149,8 +161,8 @@ int bdlm_lse_merge(int32_t n_partials, int32_t batch, int32_t L, int32_t H, int3
  *     b * block_size.  Row i of packed block b stands at position block_prefix[b] + i for the sliding
  *     window; with window > 0 the blocks must not overlap in position (block_prefix[b+1] >= block_prefix[b]
  *     + block_size).  Values are not validated by the library (it never reads device memory on the host).
- *   - Clean K/V in gathered order (the all-gather output of Algorithm 1 used "directly without a reordering
- *     copy": each key keeps its original position).  With kv_chunk_len > 0 the clean K/V tensors (and dK/dV)
+ *   - Clean K/V in gathered order (Algorithm 1 and the paper's paragraph on its fused operator: the kernels read
+ *     the all-gather's output where it lies and mask every key by the position it came from).  With kv_chunk_len > 0 the clean K/V tensors (and dK/dV)
  *     are a sequence of chunks of kv_chunk_len rows; memory chunk m holds the keys at positions
  *     kv_chunk_pos[m] .. kv_chunk_pos[m] + kv_chunk_len - 1 (for zigzag shards gathered rank by rank: chunks
  *     r and 2P-1-r of rank r, one after the other).  kv_pos_chunk is the inverse permutation.  Requirements:
@@ -212,10 +224,17 @@ int bdlm_get_device_status(void* cuda_stream);
  * bdlm_attn_bwd; the D_i scratch lives in a fixed device array inside the library
  * (2 * BDLM_STATIC_SCRATCH_ROWS floats = 8 MiB, resident on every GPU that loads the library
  * until the process exits).  The call allocates and frees nothing.
+ *   - It always runs the two-pass kernels (as bdlm_attn_bwd with BDLM_BWD_TWO_PASS; p->bwd_single_pass
+ *     is ignored): the fused kernel's fp32 dQ accumulators would need 512 bytes per query row and head,
+ *     far more than a fixed array can reasonably hold.  Every gradient is therefore bitwise reproducible.
  *   - Limit: batch * H * L <= BDLM_STATIC_SCRATCH_ROWS, otherwise
- *     BDLM_ERR_STATIC_SCRATCH_TOO_SMALL is returned and nothing is launched.
+ *     BDLM_ERR_STATIC_SCRATCH_TOO_SMALL is returned and nothing is launched.  Other errors are
+ *     those of bdlm_attn_bwd (an unsupported head dimension is BDLM_ERR_UNSUPPORTED here too).
  *   - The first call on each device looks up the array's device address (with that device
- *     current); make that first call outside any stream capture.
+ *     current); make that first call outside any stream capture.  The address is remembered per
+ *     device ordinal for the life of the device's primary context: after cudaDeviceReset (or any
+ *     other teardown of that context) the library must be reloaded before this entry point is
+ *     used on that device again.
  *   - All calls on a device share the one array and it keeps the previous call's contents.
  *     Nothing in it has to start at zero (each call rewrites D in full before reading it), but
  *     two calls that overlap on the GPU -- different streams, or different host threads -- race
@@ -236,14 +255,31 @@ int bdlm_attn_bwd_static_scratch(const bdlm_params* p,
  * Tracing (no counterpart in the paper; the paper reports GPU spans in its appendix K only).
  * When a device buffer of at least BDLM_TRACE_SLOTS 64-bit counters is set, the tensor-core
  * kernels add, per CTA and role, the clock cycles spent waiting and computing:
- *   slot = kernel * 16 + counter, kernel 0 = forward, 1 = dK/dV pass, 2 = dQ pass;
+ *   slot = kernel * 16 + counter, kernel 0 = forward, 1 = dK/dV pass or the fused backward (whichever
+ *   runs), 2 = dQ pass;
  *   counters 0..7 belong to compute warp 0 (0 steps, 1..5 waits/compute phases in kernel order,
- *   6 total), 8..11 to the MMA thread (8 total, 9..11 waits), 12..13 to the producer (12 total,
- *   13 wait for a free stage).
- * Pass NULL to switch tracing off (the default).  The caller zeroes and reads the buffer.
+ *   6 total; 7 in the fused backward: the MMA warp's wait for Q tiles), 8..11 to the MMA warp (8 total,
+ *   9..11 waits), 12..13 to the producer (12 total or, fused, the MMA warp's wait for dO tiles; 13 wait
+ *   for a free stage), 14..15 kernel-specific (dK/dV pass: S^T load and exponent arithmetic; fused: the
+ *   read-out warpgroup's wait for dQ^T and its busy time).
+ * The buffer is set per device (the device current at the call) and applies to every later launch on
+ * that device from any thread.  Pass NULL to switch tracing off (the default).  The caller zeroes and
+ * reads the buffer.
  */
 enum { BDLM_TRACE_SLOTS = 256 };
 int bdlm_set_trace_buffer(void* device_counters, size_t bytes);
+
+/*
+ * Self-test of the bounded device-side waits (no counterpart in the paper).  Every wait inside the
+ * kernels gives up after a limit of clock ticks, raises its CTA's abort flag so that the other roles
+ * leave their loops too, and the kernel reports BDLM_ERR_DEVICE_TIMEOUT through the device status
+ * word instead of hanging the GPU.  This call launches a one-CTA kernel without any copy or
+ * tensor-core work in which one warp waits, with a limit of `limit_ticks` clock ticks (1 .. 2^31), on
+ * a barrier that nothing will ever complete, and a second warp waits on the same barrier with the
+ * kernels' regular limit (about a second) and leaves as soon as the first warp has raised the flag.  Afterwards bdlm_get_device_status returns
+ * BDLM_ERR_DEVICE_TIMEOUT once, and BDLM_OK on the next call.  The kernel always terminates.
+ */
+int bdlm_selftest_wait_timeout(int64_t limit_ticks, void* cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -17,11 +17,12 @@ LIB_PATH = os.path.join(_HERE, "libbdlm_attn.so")
 BDLM_WS_FWD, BDLM_WS_BWD = 0, 1
 IMPL_AUTO, IMPL_PORTABLE, IMPL_TCGEN05 = 0, 1, 2
 PASS_DSUM, PASS_DKDV, PASS_DQ = 1, 2, 4
+BWD_AUTO, BWD_FUSED, BWD_TWO_PASS = 0, 1, 2
 
 EXPORTS = ("bdlm_workspace_bytes", "bdlm_attn_fwd", "bdlm_attn_bwd", "bdlm_lse_merge",
            "bdlm_status_string", "bdlm_get_device_status", "bdlm_set_trace_buffer",
            "bdlm_attn_bwd_static_scratch", "bdlm_workspace_bytes_packed", "bdlm_attn_fwd_packed",
-           "bdlm_attn_bwd_packed")
+           "bdlm_attn_bwd_packed", "bdlm_selftest_wait_timeout")
 STATIC_SCRATCH_ROWS = 1 << 20
 TRACE_SLOTS = 256
 
@@ -84,6 +85,8 @@ def lib():
         L.bdlm_attn_fwd_packed.argtypes = [pp, gp] + [vp] * 10 + [vp]
         L.bdlm_attn_bwd_packed.restype = ctypes.c_int
         L.bdlm_attn_bwd_packed.argtypes = [pp, gp] + [vp] * 18 + [vp, ctypes.c_size_t, vp]
+        L.bdlm_selftest_wait_timeout.restype = ctypes.c_int
+        L.bdlm_selftest_wait_timeout.argtypes = [ctypes.c_int64, vp]
         _lib = L
     return _lib
 
@@ -96,7 +99,9 @@ bdlm_status_string = status_string
 
 
 def make_params(batch, L, block_size, H, H_kv, d, scale=0.0, clean_mask_mode=0, kv_range=None,
-                include_noisy_diag=True, impl=IMPL_AUTO, bwd_passes=0, bwd_single_pass=False, window=0) -> BdlmParams:
+                include_noisy_diag=True, impl=IMPL_AUTO, bwd_passes=0, bwd_single_pass=None, window=0) -> BdlmParams:
+    """`bwd_single_pass`: None = automatic (BDLM_BWD_AUTO: the fused kernel when the workspace has room for it),
+    True = the fused kernel (BDLM_BWD_FUSED), False = the two-pass kernels (BDLM_BWD_TWO_PASS)."""
     p = BdlmParams()
     p.batch, p.L, p.block_size, p.H, p.H_kv, p.d = batch, L, block_size, H, H_kv, d
     p.scale = float(scale)
@@ -108,7 +113,7 @@ def make_params(batch, L, block_size, H, H_kv, d, scale=0.0, clean_mask_mode=0, 
     p.include_noisy_diag = 1 if include_noisy_diag else 0
     p.impl = impl
     p.bwd_passes = bwd_passes
-    p.bwd_single_pass = 1 if bwd_single_pass else 0
+    p.bwd_single_pass = BWD_AUTO if bwd_single_pass is None else (BWD_FUSED if bwd_single_pass else BWD_TWO_PASS)
     p.window = int(window)
     return p
 
@@ -158,10 +163,12 @@ def bdlm_attn_fwd(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, block_si
 
 def bdlm_attn_bwd(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, o_clean, lse_clean,
                   o_noisy, lse_noisy, do_clean, do_noisy, block_size, *, out=None, workspace=None,
-                  scale=0.0, clean_mask_mode=0, impl=IMPL_AUTO, passes=0, single_pass=False, window=0):
+                  scale=0.0, clean_mask_mode=0, impl=IMPL_AUTO, passes=0, single_pass=None, window=0):
     """Backward of the layer.  Returns (dq_clean, dk_clean, dv_clean, dq_noisy, dk_noisy, dv_noisy).
     `single_pass=True` selects the fused one-kernel backward (dQ through fp32 add-reductions into a
-    workspace accumulator: faster, dQ reproducible only up to fp32 summation order)."""
+    workspace accumulator: faster, dQ reproducible only up to fp32 summation order), `False` the two-pass
+    kernels (every gradient bitwise reproducible); `None` (default) lets the library take the fused kernel
+    whenever the workspace it is given has room for it -- the workspace allocated here always has."""
     p = _shape_params(q_clean, k_clean, block_size, scale=scale, clean_mask_mode=clean_mask_mode, impl=impl,
                       bwd_passes=passes, bwd_single_pass=single_pass, window=window)
     if out is None:
@@ -276,7 +283,7 @@ def bdlm_attn_fwd_packed(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, b
 def bdlm_attn_bwd_packed(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, o_clean, lse_clean,
                          o_noisy, lse_noisy, do_clean, do_noisy, block_size, *, block_prefix=None,
                          clean_q_pos0=0, out=None, workspace=None, scale=0.0, clean_mask_mode=0,
-                         impl=IMPL_AUTO, passes=0, single_pass=False, window=0, kv_chunks=None):
+                         impl=IMPL_AUTO, passes=0, single_pass=None, window=0, kv_chunks=None):
     """Backward of the packed form.  Returns (dq_clean, dk_clean, dv_clean, dq_noisy, dk_noisy, dv_noisy);
     entries of a stream that was left out are None.  dk_clean/dv_clean are this call's contribution for
     every clean key.  `single_pass` as in bdlm_attn_bwd."""
@@ -323,6 +330,14 @@ def bdlm_lse_merge(o_partials, lse_partials, *, out=None):
 
 def bdlm_get_device_status() -> int:
     return int(lib().bdlm_get_device_status(_stream()))
+
+
+def bdlm_selftest_wait_timeout(limit_ticks: int) -> None:
+    """Launches the library's bounded-wait self-test kernel: a wait that runs out after `limit_ticks`
+    clock ticks; afterwards bdlm_get_device_status() reports BDLM_ERR_DEVICE_TIMEOUT once."""
+    rc = lib().bdlm_selftest_wait_timeout(int(limit_ticks), _stream())
+    if rc != 0:
+        raise BdlmError(rc, "bdlm_selftest_wait_timeout")
 
 
 def bdlm_set_trace_buffer(counters) -> None:

@@ -3,6 +3,8 @@
 // bdlm_get_device_status), no output on stdout/stderr.
 #include <math.h>
 
+#include <atomic>
+
 #include "bdlm_common.cuh"
 #include "tc_launch.h"
 
@@ -10,7 +12,15 @@ namespace bdlm {
 namespace {
 
 __device__ int g_device_status = 0;
-unsigned long long* g_trace = nullptr;   // host-side copy of the trace buffer pointer
+constexpr int kMaxDevices = 64;
+unsigned long long* g_trace[kMaxDevices] = {};   // trace buffer of each device ordinal (host-side copy of the pointer)
+std::atomic<int> g_sm_count[kMaxDevices] = {};
+
+int current_device() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+  return dev;
+}
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -37,7 +47,7 @@ int check_params(const bdlm_params* p, const bdlm_packed_geometry* g = nullptr) 
   if (p->clean_mask_mode != 0 && p->clean_mask_mode != 1) return BDLM_ERR_INVALID_ARG;
   if (p->impl < 0 || p->impl > 2) return BDLM_ERR_INVALID_ARG;
   if (p->bwd_passes < 0 || p->bwd_passes > 7) return BDLM_ERR_INVALID_ARG;
-  if (p->bwd_single_pass != 0 && p->bwd_single_pass != 1) return BDLM_ERR_INVALID_ARG;
+  if (p->bwd_single_pass < 0 || p->bwd_single_pass > 2) return BDLM_ERR_INVALID_ARG;
   if (p->window < 0) return BDLM_ERR_INVALID_ARG;
   if (!(p->scale >= 0.f) || isinf(p->scale)) return BDLM_ERR_INVALID_ARG;
   if (p->kv_range_set) {
@@ -70,7 +80,10 @@ void fill(KArgs& a, const bdlm_params* p, const bdlm_packed_geometry* g) {
     a.q[s] = a.k[s] = a.v[s] = nullptr; a.o[s] = nullptr; a.lse[s] = nullptr;
     a.dout[s] = nullptr; a.dsum[s] = nullptr; a.dq[s] = a.dk[s] = a.dv[s] = nullptr;
   }
-  a.trace = g_trace;
+  {
+    const int dev = current_device();
+    a.trace = dev >= 0 ? g_trace[dev] : nullptr;
+  }
   a.single_pass = 0; a.dq32[0] = a.dq32[1] = nullptr;
 }
 
@@ -91,6 +104,17 @@ size_t dsum_bytes(const bdlm_params* p, const bdlm_packed_geometry* g = nullptr)
 
 }  // namespace
 
+int device_sm_count() {
+  const int dev = current_device();
+  if (dev < 0) return 1;
+  int n = g_sm_count[dev].load(std::memory_order_relaxed);
+  if (n <= 0) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 1;
+    g_sm_count[dev].store(n, std::memory_order_relaxed);
+  }
+  return n;
+}
+
 int* device_status_ptr() {
   int* ptr = nullptr;
   if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_device_status) != cudaSuccess) return nullptr;
@@ -105,7 +129,8 @@ extern "C" {
 
 size_t bdlm_workspace_bytes(const bdlm_params* p, int32_t which) {
   if (check_params(p) != BDLM_OK) return 0;
-  if (which == BDLM_WS_BWD) return 2 * dsum_bytes(p) + tc_bwd_extra_workspace(p, nullptr);
+  if (which == BDLM_WS_BWD)
+    return 2 * dsum_bytes(p) + (p->bwd_single_pass != BDLM_BWD_TWO_PASS ? tc_bwd_fused_workspace(p, nullptr) : 0);
   return 0;
 }
 
@@ -171,8 +196,10 @@ static int bwd_impl(const bdlm_params* p, const bdlm_packed_geometry* g,
   }
   if (p->kv_range_set && (p->kv_begin != 0 || p->kv_end != p->L)) return BDLM_ERR_UNSUPPORTED;
   if (!p->include_noisy_diag) return BDLM_ERR_UNSUPPORTED;
-  const size_t need_ws = 2 * dsum_bytes(p, g) + tc_bwd_extra_workspace(p, g);
-  if (workspace_bytes < need_ws) return BDLM_ERR_WORKSPACE_TOO_SMALL;
+  // the D rows are always needed; the fp32 dQ accumulators of the fused kernel only when that kernel runs
+  const size_t need_min = 2 * dsum_bytes(p, g);
+  const size_t need_fused = need_min + tc_bwd_fused_workspace(p, g);
+  if (workspace_bytes < (p->bwd_single_pass == BDLM_BWD_FUSED ? need_fused : need_min)) return BDLM_ERR_WORKSPACE_TOO_SMALL;
   if (!is_sm100()) return BDLM_ERR_UNSUPPORTED;
 
   KArgs a;
@@ -194,7 +221,10 @@ static int bwd_impl(const bdlm_params* p, const bdlm_packed_geometry* g,
 
   const bool tc_ok = tc_bwd_supported(a);
   if (p->impl == 2 && !tc_ok) return BDLM_ERR_UNSUPPORTED;
-  a.single_pass = (p->bwd_single_pass && tc_ok && p->impl != 1) ? 1 : 0;
+  // automatic: the fused kernel whenever the tensor-core kernels take the shape and the workspace has room for its
+  // fp32 dQ accumulators; the two-pass path otherwise (and always when it is asked for)
+  a.single_pass = (p->bwd_single_pass != BDLM_BWD_TWO_PASS && tc_ok && p->impl != 1 && need_fused > need_min &&
+                   workspace_bytes >= need_fused) ? 1 : 0;
   const int passes = p->bwd_passes ? p->bwd_passes : 7;
   cudaError_t e = cudaSuccess;
   if (passes & BDLM_BWD_PASS_DSUM) e = launch_dsum(a, ds_c, ds_n, st);
@@ -259,7 +289,8 @@ int bdlm_attn_bwd_packed(const bdlm_params* p, const bdlm_packed_geometry* g,
 
 size_t bdlm_workspace_bytes_packed(const bdlm_params* p, const bdlm_packed_geometry* g, int32_t which) {
   if (g == nullptr || check_params(p, g) != BDLM_OK) return 0;
-  if (which == BDLM_WS_BWD) return 2 * dsum_bytes(p, g) + tc_bwd_extra_workspace(p, g);
+  if (which == BDLM_WS_BWD)
+    return 2 * dsum_bytes(p, g) + (p->bwd_single_pass != BDLM_BWD_TWO_PASS ? tc_bwd_fused_workspace(p, g) : 0);
   return 0;
 }
 
@@ -283,7 +314,9 @@ int bdlm_lse_merge(int32_t n_partials, int32_t batch, int32_t L, int32_t H, int3
 int bdlm_set_trace_buffer(void* device_counters, size_t bytes) {
   if (device_counters != nullptr && (bytes < BDLM_TRACE_SLOTS * sizeof(unsigned long long) || !aligned16(device_counters)))
     return BDLM_ERR_INVALID_ARG;
-  g_trace = static_cast<unsigned long long*>(device_counters);
+  const int dev = current_device();
+  if (dev < 0) return BDLM_ERR_CUDA;
+  g_trace[dev] = static_cast<unsigned long long*>(device_counters);
   return BDLM_OK;
 }
 

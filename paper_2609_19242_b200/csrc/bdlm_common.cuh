@@ -49,8 +49,8 @@ struct KArgs {
   __nv_bfloat16* dk[2];
   __nv_bfloat16* dv[2];
   unsigned long long* trace;   // optional cycle counters (bdlm_set_trace_buffer), else nullptr
-  int single_pass;             // backward: dQ accumulated in the dK/dV kernel through fp32 atomics
-  float* dq32[2];              // fp32 dQ accumulators [batch, rows, H, d] (single-pass backward), else nullptr
+  int single_pass;             // backward: the fused kernel forms dQ^T per step and adds it into dq32 by TMA bulk add-reductions
+  float* dq32[2];              // fp32 dQ accumulators [batch, H, rows, 128] (fused backward), else nullptr
 };
 
 __host__ __device__ __forceinline__ int rows_q(const KArgs& a, int qs) { return qs == CLEAN ? a.Lqc : a.Ln; }
@@ -133,6 +133,9 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
+
+// Number of SMs of the current device (cached per device ordinal; 1 if the query fails).
+int device_sm_count();
 
 // Launchers (host).  Each enqueues on `st` and returns the launch's cudaError_t.
 cudaError_t launch_portable_fwd(const KArgs& a, cudaStream_t st);

@@ -1,5 +1,5 @@
 // Bandwidth-bound kernels of the BDLM attention path: the LSE merge of partial outputs
-// (Eq. csbp-lse-merge, with the final division of Implementation 1 fused in) and the
+// (Eq. csbp-lse-merge over n partials, final division included) and the
 // backward preprocess D_i = sum_d dO_i,d * O_i,d.
 #include "bdlm_common.cuh"
 
@@ -15,9 +15,13 @@ struct MergeArgs {
   int n;
 };
 
-// One thread owns EPT (8 or 16) consecutive head-dim elements of one (row, head).  The running state
-// (numerator, m, normaliser) stays in fp32 registers until the final division, so no thread
-// reads state another thread has already overwritten.
+// Eq. csbp-lse-merge for n partials at once: with m = max_j z_j and w_j = exp(z_j - m),
+//   O = sum_j w_j O_j / sum_j w_j,   z = m + log sum_j w_j.
+// One thread owns EPT (8 or 16) consecutive head-dim elements of one (row, head).  It first reads the row's n LSEs
+// (n <= 16: they stay in registers), takes their maximum and turns them into normalised weights w_j / sum w; an empty
+// partial (z_j = -inf) gets weight 0, a row whose partials are all empty gets O = 0 and z = -inf.  Then the
+// partial outputs are streamed through once, four partials' loads in flight at a time, and added up with their
+// weights -- no running rescale and nothing another thread could overwrite.
 template <bool F32IN, int EPT>
 __global__ void __launch_bounds__(256) merge_kernel(MergeArgs ma, int64_t total_chunks, int L, int H, int d,
                                                     bf16* __restrict__ o_out, float* __restrict__ lse_out) {
@@ -32,22 +36,33 @@ __global__ void __launch_bounds__(256) merge_kernel(MergeArgs ma, int64_t total_
     const int64_t bidx = row / L;
     const int i = (int)(row % L);
     const int64_t lidx = (bidx * H + h) * L + i;
-    float num[EPT];
+    float wgt[MAX_PARTIALS];
+    float m = -INFINITY;
 #pragma unroll
-    for (int e = 0; e < EPT; ++e) num[e] = 0.f;
-    float m = -INFINITY, norm = 0.f;
-    // four partials at a time: their loads are issued together (the kernel is a pure stream, it needs bytes in flight),
-    // then they are folded in left to right
-    for (int j0 = 0; j0 < ma.n; j0 += 4) {
-      float z4[4];
+    for (int j = 0; j < MAX_PARTIALS; ++j) {
+      wgt[j] = j < ma.n ? ma.lse[j][lidx] : -INFINITY;
+      m = fmaxf(m, wgt[j]);
+    }
+    const float m_ref = (m == -INFINITY) ? 0.f : m;   // all empty: every weight becomes exp(-inf) = 0
+    float wsum = 0.f;
+#pragma unroll
+    for (int j = 0; j < MAX_PARTIALS; ++j) {
+      wgt[j] = (wgt[j] == -INFINITY) ? 0.f : expf(wgt[j] - m_ref);
+      wsum += wgt[j];
+    }
+    const float inv = wsum > 0.f ? 1.f / wsum : 0.f;
+    float acc[EPT];
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) acc[e] = 0.f;
+#pragma unroll
+    for (int j0 = 0; j0 < MAX_PARTIALS; j0 += 4) {
+      if (j0 >= ma.n) break;
       uint4 u4[4][NV];
 #pragma unroll
       for (int jj = 0; jj < 4; ++jj) {
-        const int j = j0 + jj;
-        if (j < ma.n) {
-          z4[jj] = ma.lse[j][lidx];
-          const uint4* p = F32IN ? reinterpret_cast<const uint4*>(static_cast<const float*>(ma.o[j]) + idx * EPT)
-                                 : reinterpret_cast<const uint4*>(static_cast<const bf16*>(ma.o[j]) + idx * EPT);
+        if (j0 + jj < ma.n) {
+          const uint4* p = F32IN ? reinterpret_cast<const uint4*>(static_cast<const float*>(ma.o[j0 + jj]) + idx * EPT)
+                                 : reinterpret_cast<const uint4*>(static_cast<const bf16*>(ma.o[j0 + jj]) + idx * EPT);
 #pragma unroll
           for (int v = 0; v < NV; ++v) u4[jj][v] = p[v];
         }
@@ -55,39 +70,31 @@ __global__ void __launch_bounds__(256) merge_kernel(MergeArgs ma, int64_t total_
 #pragma unroll
       for (int jj = 0; jj < 4; ++jj) {
         if (j0 + jj >= ma.n) break;
-        const float z = z4[jj];
-        const float m_new = fmaxf(m, z);
-        const float w_acc = isfinite(m) ? expf(m - m_new) : 0.f;
-        const float w_j = isfinite(z) ? expf(z - m_new) : 0.f;
-        float x[EPT];
+        const float wj = wgt[j0 + jj] * inv;
         if (F32IN) {
           const float* pf = reinterpret_cast<const float*>(&u4[jj][0]);
 #pragma unroll
-          for (int e = 0; e < EPT; ++e) x[e] = pf[e];
+          for (int e = 0; e < EPT; ++e) acc[e] = fmaf(wj, pf[e], acc[e]);
         } else {
           const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&u4[jj][0]);
 #pragma unroll
           for (int e = 0; e < EPT / 2; ++e) {
-            float2 f = __bfloat1622float2(p2[e]);
-            x[2 * e] = f.x; x[2 * e + 1] = f.y;
+            const float2 f = __bfloat1622float2(p2[e]);
+            acc[2 * e] = fmaf(wj, f.x, acc[2 * e]);
+            acc[2 * e + 1] = fmaf(wj, f.y, acc[2 * e + 1]);
           }
         }
-#pragma unroll
-        for (int e = 0; e < EPT; ++e) num[e] = w_acc * num[e] + w_j * x[e];
-        norm = w_acc * norm + w_j;
-        m = m_new;
       }
     }
-    const float inv = norm > 0.f ? 1.f / norm : 0.f;
 #pragma unroll
     for (int v = 0; v < EPT / 8; ++v) {
       uint4 outv;
       uint32_t* ow = reinterpret_cast<uint32_t*>(&outv);
 #pragma unroll
-      for (int e = 0; e < 4; ++e) ow[e] = pack_bf16(num[8 * v + 2 * e] * inv, num[8 * v + 2 * e + 1] * inv);
+      for (int e = 0; e < 4; ++e) ow[e] = pack_bf16(acc[8 * v + 2 * e], acc[8 * v + 2 * e + 1]);
       reinterpret_cast<uint4*>(o_out + idx * EPT)[v] = outv;
     }
-    if (c == 0) lse_out[lidx] = norm > 0.f ? m + logf(norm) : -INFINITY;
+    if (c == 0) lse_out[lidx] = wsum > 0.f ? m + logf(wsum) : -INFINITY;
   }
 }
 
@@ -153,7 +160,8 @@ cudaError_t launch_merge(int n, int batch, int L, int H, int d, const void* cons
   const int ept = (d % 16 == 0 && n <= 3) ? 16 : 8;
   const int64_t total = (int64_t)batch * L * H * (d / ept);
   int64_t want = (total + 255) / 256;
-  int blocks = (int)(want < 148 * 16 ? (want > 0 ? want : 1) : 148 * 16);
+  const int64_t cap = (int64_t)device_sm_count() * 16;
+  int blocks = (int)(want < cap ? (want > 0 ? want : 1) : cap);
   bf16* oo = static_cast<bf16*>(o_out);
   if (dtype == 1) {
     if (ept == 16) merge_kernel<true, 16><<<blocks, 256, 0, st>>>(ma, total, L, H, d, oo, lse_out);

@@ -22,7 +22,9 @@ float* g_scratch_ptr[kMaxDevices] = {};   // device address of g_static_dsum, pe
 std::mutex g_scratch_mutex;
 
 // The array's name is only a host-side handle; kernels need the device address, which differs
-// per device.  Looked up once per device, with that device current.
+// per device.  Looked up once per device, with that device current, and remembered per device
+// ordinal: the address belongs to the device's primary context and goes stale if that context is
+// torn down (cudaDeviceReset) -- the library has to be reloaded then.
 int scratch_for_current_device(float** out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return BDLM_ERR_CUDA;
@@ -51,16 +53,23 @@ extern "C" int bdlm_attn_bwd_static_scratch(const bdlm_params* p,
                                             void* dq_noisy, void* dk_noisy, void* dv_noisy,
                                             void* cuda_stream) {
   if (p == nullptr) return BDLM_ERR_INVALID_ARG;
-  const size_t need = bdlm_workspace_bytes(p, BDLM_WS_BWD);
-  if (need == 0) return BDLM_ERR_INVALID_ARG;                 // invalid parameters (the regular checks say which)
+  // Always the two-pass kernels: they need only the D rows.  (The fused kernel's fp32 dQ accumulators take 512 bytes
+  // per query row and head; no fixed array of a sensible size could hold them.)
+  bdlm_params q = *p;
+  q.bwd_single_pass = BDLM_BWD_TWO_PASS;
+  const size_t need = bdlm_workspace_bytes(&q, BDLM_WS_BWD);
+  if (need == 0)   // invalid or unsupported parameters: the regular entry point's checks say which, before they touch anything
+    return bdlm_attn_bwd(&q, q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, o_clean, o_noisy, lse_clean,
+                         lse_noisy, do_clean, do_noisy, dq_clean, dk_clean, dv_clean, dq_noisy, dk_noisy, dv_noisy,
+                         nullptr, 0, cuda_stream);
   const size_t have = sizeof(float) * 2 * (size_t)BDLM_STATIC_SCRATCH_ROWS;
-  if ((int64_t)p->batch * p->H * p->L > (int64_t)BDLM_STATIC_SCRATCH_ROWS || need > have)
+  if ((int64_t)q.batch * q.H * q.L > (int64_t)BDLM_STATIC_SCRATCH_ROWS || need > have)
     return BDLM_ERR_STATIC_SCRATCH_TOO_SMALL;
   float* scratch = nullptr;
   const int rc = scratch_for_current_device(&scratch);
   if (rc != BDLM_OK) return rc;
   // D is rewritten in full by every call before it is read, so nothing has to be cleared.
-  return bdlm_attn_bwd(p, q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, o_clean, o_noisy,
+  return bdlm_attn_bwd(&q, q_clean, k_clean, v_clean, q_noisy, k_noisy, v_noisy, o_clean, o_noisy,
                        lse_clean, lse_noisy, do_clean, do_noisy, dq_clean, dk_clean, dv_clean,
                        dq_noisy, dk_noisy, dv_noisy, scratch, have, cuda_stream);
 }

@@ -177,7 +177,7 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
     // fall through to the common exit
   } else if (warp == DKDV_PRODUCER) {
     // ------------------------------------------------------------------ producer
-    if (lane == 0) {
+    if (lane == 0 && nsteps > 0) {   // a key tile no query sees writes zeros and waits for nothing: it must not leave a copy in flight
       mbar_expect_tx(bar_kv, 2 * TILE_BYTES);
       tma_tile(sK, &maps.k[ks], bar_kv, hk * 128, k0_row, b);
       tma_tile(sV, &maps.v[ks], bar_kv, hk * 128, k0_row, b);
@@ -872,7 +872,7 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
     // fall through to the common exit
   } else if (warp == 8) {
     // ------------------------------------------------------------------ producer
-    if (lane == 0) {
+    if (lane == 0 && nsteps > 0) {   // a key tile no query sees writes zeros and waits for nothing: it must not leave a copy in flight
       mbar_expect_tx(bar_kv, 2 * TILE_BYTES);
       tma_tile(sK, &maps.k[ks], bar_kv, hk * 128, k0_row, b);
       tma_tile(sV, &maps.v[ks], bar_kv, hk * 128, k0_row, b);
@@ -1060,8 +1060,16 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
         for (int e = 0; e < HT; ++e) sg[e * 128] = __uint_as_float(v[e]) * a.scale;
         fence_async_smem();
       }
-      asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (*abort_flag) break;
+      // the second meeting also takes the decision to leave, for all 128 threads at once (a flag raised between two
+      // threads' reads must not send some of them to the exit and the rest to the next meeting)
+      uint32_t leave;
+      asm volatile(
+          "{\n\t.reg .pred p, q;\n\t"
+          "setp.ne.b32 q, %1, 0;\n\t"
+          "bar.red.or.pred p, 1, 128, q;\n\t"
+          "selp.u32 %0, 1, 0, p;\n\t}"
+          : "=r"(leave) : "r"(*abort_flag) : "memory");
+      if (leave) break;
       if (leader) {
         bulk_reduce_add_f32(dst, sSTG + (i & 1) * STG_BYTES, STG_BYTES);
         bulk_commit();
@@ -1259,10 +1267,11 @@ bool tc_bwd_supported(const KArgs& a) {
   return a.d == 128 && tc_rows_ok(a) && tc_encoder_available();
 }
 // fp32 dQ accumulators of the fused backward: one [batch, H, rows, 128] tensor per query stream
-size_t tc_bwd_extra_workspace(const bdlm_params* p, const bdlm_packed_geometry* g) {
-  if (!p->bwd_single_pass || p->d != 128 || p->impl == 1) return 0;
+size_t tc_bwd_fused_workspace(const bdlm_params* p, const bdlm_packed_geometry* g) {
+  if (p->d != 128 || p->impl == 1) return 0;
   const size_t rows_c = g != nullptr ? (size_t)g->Lq_clean : (size_t)p->L;
   const size_t rows_n = g != nullptr ? (size_t)g->n_blocks * p->block_size : (size_t)p->L;
+  if (p->L % TILE != 0 || rows_c % TILE != 0 || rows_n % TILE != 0) return 0;   // such shapes take the mma.sync kernels
   return (rows_c + rows_n) * p->batch * p->H * 128 * sizeof(float);
 }
 
@@ -1299,7 +1308,7 @@ cudaError_t launch_tc_bwd(const KArgs& a_in, void* extra_ws, int passes, cudaStr
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
       for (int s2 = 0; s2 < 2; ++s2) {
         if (dq32_elems[s2] == 0) continue;
-        dq_convert_kernel<<<148 * 8, 256, 0, st>>>(a.dq32[s2], a.dq[s2], a.batch, a.H, rows_q(a, s2));
+        dq_convert_kernel<<<device_sm_count() * 8, 256, 0, st>>>(a.dq32[s2], a.dq[s2], a.batch, a.H, rows_q(a, s2));
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
       }
     }

@@ -42,14 +42,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Bounded wait of the warp-specialised kernels: gives up after ~2^31 clock ticks (about a second), so a
 // protocol slip ends the kernel with an error status instead of hanging the device; it also gives up as soon
 // as another role has raised the CTA's abort flag, and raises it itself on a timeout, so every role leaves its loop.
-__device__ __forceinline__ bool mbar_wait_abortable(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+constexpr long long WAIT_LIMIT_TICKS = 1ll << 31;
+__device__ __forceinline__ bool mbar_wait_abortable(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                    long long limit_ticks = WAIT_LIMIT_TICKS) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   int spins = 0;
   while (!mbar_try_wait(bar, parity)) {
     if ((++spins & 63) == 0) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > (1ll << 31)) { *abort_flag = 1; return false; }
+      if (clock64() - t0 > limit_ticks) { *abort_flag = 1; return false; }
     }
   }
   return true;

@@ -40,9 +40,23 @@ EncodeTiledFn encode_fn() {
 bool tc_encoder_available() { return encode_fn() != nullptr; }
 
 // [batch, L, heads, 128] bf16 viewed as 3-D (heads*128, L, batch); box = 64 columns x `rows` rows.
+// Encoding a map costs the host a microsecond or two and a call needs six to eight of them, which shows at sizes
+// where a whole step takes a few milliseconds; a training loop passes the same tensors again and again, so each host
+// thread keeps the maps it encoded last in a small direct-mapped table keyed by (address, shape, box).  A map is a
+// plain 128-byte value that describes addresses and strides only, so a copy of it is as good as a fresh encode.
 bool tc_make_map(CUtensorMap* m, const void* ptr, int heads, int L, int batch, int rows) {
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr || ptr == nullptr) return false;
+  struct Entry { const void* ptr; int heads, L, batch, rows; bool valid; CUtensorMap map; };
+  constexpr int kEntries = 64;
+  thread_local Entry cache[kEntries] = {};
+  const uint64_t key = (reinterpret_cast<uint64_t>(ptr) >> 8) * 0x9E3779B97F4A7C15ull + (uint64_t)rows * 0x632BE59BD9B4E019ull +
+                       (uint64_t)L * 31 + (uint64_t)heads;
+  Entry& e = cache[(key >> 32) % kEntries];
+  if (e.valid && e.ptr == ptr && e.heads == heads && e.L == L && e.batch == batch && e.rows == rows) {
+    *m = e.map;
+    return true;
+  }
   cuuint64_t gdim[3] = {(cuuint64_t)heads * 128, (cuuint64_t)L, (cuuint64_t)batch};
   cuuint64_t gstride[2] = {(cuuint64_t)heads * 128 * 2, (cuuint64_t)L * heads * 128 * 2};
   cuuint32_t box[3] = {64, (cuuint32_t)rows, 1};
@@ -50,7 +64,9 @@ bool tc_make_map(CUtensorMap* m, const void* ptr, int heads, int L, int batch, i
   CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), gdim, gstride, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS;
+  if (r != CUDA_SUCCESS) return false;
+  e.ptr = ptr; e.heads = heads; e.L = L; e.batch = batch; e.rows = rows; e.map = *m; e.valid = true;
+  return true;
 }
 
 namespace {

@@ -16,7 +16,8 @@ bool tc_make_map(CUtensorMap* m, const void* ptr, int heads, int L, int batch, i
 bool tc_rows_ok(const KArgs& a);
 bool tc_fwd_supported(const KArgs& a);
 bool tc_bwd_supported(const KArgs& a);
-size_t tc_bwd_extra_workspace(const bdlm_params* p, const bdlm_packed_geometry* g);
+// Bytes of the fused backward's fp32 dQ accumulators for these sizes (0 when the fused kernel cannot take them).
+size_t tc_bwd_fused_workspace(const bdlm_params* p, const bdlm_packed_geometry* g);
 cudaError_t launch_tc_fwd(const KArgs& a, cudaStream_t st);
 cudaError_t launch_tc_bwd(const KArgs& a, void* extra_ws, int passes, cudaStream_t st);
 

@@ -71,6 +71,8 @@ WORKLOADS = {
     "256k": Workload("256k", 1, 32, 8, 128, 262144, 16),
     # paper-shaped block size (appendix J uses 128..1024, default 256); not a BASELINE config
     "32k_m256": Workload("32k_m256", 1, 32, 8, 128, 32768, 256, rope_theta=5e5),
+    "32k_m512": Workload("32k_m512", 1, 32, 8, 128, 32768, 512, rope_theta=5e5),
+    "32k_m1024": Workload("32k_m1024", 1, 32, 8, 128, 32768, 1024, rope_theta=5e5),
     # sliding-window layer of a hybrid model (appendix K: 1,024-token windows); not a BASELINE config
     "32k_w1024": Workload("32k_w1024", 1, 32, 8, 128, 32768, 64, rope_theta=5e5, window=1024),
     # DFlash2-shaped drafter layer (appendix E): 32K target-feature keys, 2048 sampled blocks of 16 tokens

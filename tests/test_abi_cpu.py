@@ -79,6 +79,27 @@ def test_workspace_size_formula():
     need = binding.bdlm_workspace_bytes(p, binding.BDLM_WS_BWD)
     assert need >= 2 * 2 * 8 * 512 * 4
     assert binding.bdlm_workspace_bytes(p, binding.BDLM_WS_FWD) == 0
+    # the backward modes: two-pass needs the D rows only; fused and automatic add the fp32 dQ accumulators
+    # (2 streams x batch x H x L x 128 floats) when the tensor-core kernels take the shape, nothing otherwise
+    mk = lambda sp, **kw: binding.bdlm_workspace_bytes(binding.make_params(2, 512, 32, 8, 2, 128, bwd_single_pass=sp, **kw),
+                                                      binding.BDLM_WS_BWD)
+    d_rows = 2 * 2 * 8 * 512 * 4
+    acc = 2 * 2 * 8 * 512 * 128 * 4
+    assert mk(False) == d_rows and mk(True) == d_rows + acc and mk(None) == d_rows + acc
+    assert mk(None, impl=binding.IMPL_PORTABLE) == d_rows
+    ragged = binding.make_params(1, 160, 32, 4, 2, 128, bwd_single_pass=True)
+    assert binding.bdlm_workspace_bytes(ragged, binding.BDLM_WS_BWD) < 2 * 160 * 4 * 128 * 4
+    d64 = binding.make_params(1, 256, 16, 4, 2, 64, bwd_single_pass=None)
+    assert binding.bdlm_workspace_bytes(d64, binding.BDLM_WS_BWD) == 2 * 4 * 256 * 4
+    # a forced fused backward refuses a workspace that holds only the D rows; the automatic mode accepts it
+    ok = ctypes.c_void_p(0x1000)
+    forced = binding.make_params(2, 512, 32, 8, 2, 128, bwd_single_pass=True)
+    assert binding.lib().bdlm_attn_bwd(ctypes.byref(forced), *([ok] * 18), ok, d_rows, None) == -3
+    bad_mode = binding.make_params(2, 512, 32, 8, 2, 128)
+    bad_mode.bwd_single_pass = 3
+    assert binding.lib().bdlm_attn_bwd(ctypes.byref(bad_mode), *([ok] * 18), ok, 1 << 30, None) == -1
+    assert binding.lib().bdlm_selftest_wait_timeout(0, None) == -1
+    assert binding.lib().bdlm_selftest_wait_timeout(1 << 40, None) == -1
 
 
 def test_packed_geometry_is_checked_without_a_device():

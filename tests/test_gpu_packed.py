@@ -243,7 +243,8 @@ def test_clean_kv_in_gathered_order(P, impl):
         o = binding.bdlm_attn_fwd_packed(qc, kc, vc, sub["q_noisy"], sub["k_noisy"], sub["v_noisy"], M,
                                          block_prefix=pfx, clean_q_pos0=p0, impl=impl, **kw)
         gr = binding.bdlm_attn_bwd_packed(qc, kc, vc, sub["q_noisy"], sub["k_noisy"], sub["v_noisy"], o[0], o[1], o[2],
-                                          o[3], doc, sub["do_noisy"], M, block_prefix=pfx, clean_q_pos0=p0, impl=impl, **kw)
+                                          o[3], doc, sub["do_noisy"], M, block_prefix=pfx, clean_q_pos0=p0, impl=impl,
+                                          single_pass=False, **kw)   # two-pass: dQ is compared bitwise below
         res[name] = (o, gr)
     torch.cuda.synchronize()
     assert binding.bdlm_get_device_status() == 0
@@ -272,3 +273,43 @@ def test_gathered_order_is_validated():
         binding.bdlm_attn_fwd_packed(*args, kv_chunks=(64, [c * 64 for c in range(8)]))  # chunks must be multiples of 128
     with pytest.raises(binding.BdlmError):
         binding.bdlm_attn_fwd_packed(*args, kv_chunks=(128, [0, 128, 256, 384]), window=64)  # no window with chunks
+
+
+@pytest.mark.parametrize("single_pass", [False, True])
+def test_clean_key_tiles_that_no_query_sees(single_pass):
+    """Sampled blocks with low anchors over a long clean sequence: most clean key tiles are seen by no query of the
+    call (their CTAs write zeros and must leave without a copy in flight), with seen tiles before and between
+    them.  dK/dV of the clean keys: zero beyond the last anchor, equal to the oracle, and -- for the keys that are
+    seen -- bitwise those of the same call on a clean sequence cut off after the last seen tile."""
+    M, L, H, Hkv = 32, 2048, 4, 2
+    prefix = [0, 40, 130, 130, 600, 610, 900, 1000]              # last seen clean key: 999 -> key tiles 8..15 unseen
+    nb = len(prefix)
+    t = _draw(23, 1, L, 0, nb * M, H, Hkv, 128)
+    g = _cuda(t)
+    pfx = torch.tensor(prefix, dtype=torch.int32, device="cuda")
+
+    def run(Lk):
+        kc, vc = g["k_clean"][:, :Lk].contiguous(), g["v_clean"][:, :Lk].contiguous()
+        o = binding.bdlm_attn_fwd_packed(None, kc, vc, g["q_noisy"], g["k_noisy"], g["v_noisy"], M, block_prefix=pfx,
+                                         impl=binding.IMPL_TCGEN05)
+        gr = binding.bdlm_attn_bwd_packed(None, kc, vc, g["q_noisy"], g["k_noisy"], g["v_noisy"], None, None, o[2], o[3],
+                                          None, g["do_noisy"], M, block_prefix=pfx, impl=binding.IMPL_TCGEN05,
+                                          single_pass=single_pass)
+        return o, gr
+
+    for rep in range(3):   # repeated: a copy left in flight by a retired CTA would land in its successor's tiles
+        o_full, g_full = run(L)
+        o_cut, g_cut = run(1024)
+        torch.cuda.synchronize()
+        assert binding.bdlm_get_device_status() == 0
+        assert torch.equal(o_full[2], o_cut[2]) and torch.equal(o_full[3], o_cut[3])
+        for i in (1, 2):
+            assert torch.equal(g_full[i][:, :1024], g_cut[i])
+            assert float(g_full[i][:, 1000:].float().abs().max()) == 0.0
+        for i in (4, 5):
+            assert torch.equal(g_full[i], g_cut[i])
+    x = {k: synth.to_f64(v) for k, v in t.items() if v is not None}
+    ref = orc.attn_packed(None, x["k_clean"], x["v_clean"], x["q_noisy"], x["k_noisy"], x["v_noisy"], M,
+                          do_noisy=x["do_noisy"], block_prefix=prefix)
+    for i, n in ((1, "dk_clean"), (2, "dv_clean"), (3, "dq_noisy"), (4, "dk_noisy"), (5, "dv_noisy")):
+        assert pu.rel_l2(synth.to_f64(g_full[i]), ref[n]) <= pu.TOL_GRAD, n

@@ -243,3 +243,51 @@ def test_large_logits(impl):
     ramp = torch.linspace(0.0, 3.0, w.L).view(1, w.L, 1, 1)
     inp["k_clean"] = (inp["k_clean"].float() + ramp * inp["q_clean"].float().mean(dim=(1, 2), keepdim=True).sign()).to(torch.bfloat16)
     pu.check_full(w, impl, inp=inp)
+
+
+def test_default_backward_takes_the_fused_kernel_when_the_workspace_has_room():
+    """bdlm_params zeroed (BDLM_BWD_AUTO): with the workspace bdlm_workspace_bytes recommends the fused kernel runs
+    (dK, dV bitwise those of the forced fused call), with only the D rows' worth of workspace the two-pass kernels
+    run (every gradient bitwise that of the forced two-pass call); a forced fused call refuses the small workspace."""
+    w = Workload("auto_bwd", 1, 4, 2, 128, 512, 32)
+    g = pu.to_cuda(synth.make_inputs(w, "cpu"))
+    M = w.block_size
+    out = pu.gpu_fwd(g, M)
+    mk = lambda sp: binding.make_params(w.batch, w.L, M, w.H, w.H_kv, w.d, bwd_single_pass=sp)
+    big = binding.bdlm_workspace_bytes(mk(None), binding.BDLM_WS_BWD)
+    small = binding.bdlm_workspace_bytes(mk(False), binding.BDLM_WS_BWD)
+    assert big == binding.bdlm_workspace_bytes(mk(True), binding.BDLM_WS_BWD)
+    assert big >= small + 2 * w.batch * w.L * w.H * 128 * 4 and small >= 2 * w.batch * w.H * w.L * 4
+    ws_big = torch.empty(big, dtype=torch.uint8, device="cuda")
+    ws_small = torch.empty(small, dtype=torch.uint8, device="cuda")
+    fused = [t.clone() for t in pu.gpu_bwd(g, out, M, single_pass=True, workspace=ws_big)]
+    two = [t.clone() for t in pu.gpu_bwd(g, out, M, single_pass=False, workspace=ws_small)]
+    auto_big = [t.clone() for t in pu.gpu_bwd(g, out, M, single_pass=None, workspace=ws_big)]
+    auto_small = [t.clone() for t in pu.gpu_bwd(g, out, M, single_pass=None, workspace=ws_small)]
+    torch.cuda.synchronize()
+    assert binding.bdlm_get_device_status() == 0
+    for a, b in zip(auto_small, two):
+        assert torch.equal(a, b)
+    for i in (1, 2, 4, 5):
+        assert torch.equal(auto_big[i], fused[i])
+    assert not all(torch.equal(two[i], fused[i]) for i in (1, 2, 4, 5))   # the two paths are told apart by their rounding
+    for i in (0, 3):
+        assert pu.rel_l2(synth.to_f64(auto_big[i]), synth.to_f64(two[i])) <= 1e-3
+    with pytest.raises(binding.BdlmError) as e:
+        pu.gpu_bwd(g, out, M, single_pass=True, workspace=ws_small)
+    assert e.value.status == -3
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_stays_usable():
+    """The library's self-test kernel lets one bounded wait run out (a barrier nothing completes, a limit of about a
+    millisecond of clock ticks): the device status reads BDLM_ERR_DEVICE_TIMEOUT exactly once, and the next
+    forward on the same context is correct."""
+    torch.cuda.synchronize()
+    assert binding.bdlm_get_device_status() == 0
+    binding.bdlm_selftest_wait_timeout(2_000_000)
+    assert binding.bdlm_get_device_status() == -5
+    assert binding.status_string(-5) == "BDLM_ERR_DEVICE_TIMEOUT"
+    assert binding.bdlm_get_device_status() == 0
+    with pytest.raises(binding.BdlmError):
+        binding.bdlm_selftest_wait_timeout(0)
+    pu.check_full(Workload("after_timeout", 1, 2, 1, 128, 256, 32), binding.IMPL_AUTO, check_bwd=False)

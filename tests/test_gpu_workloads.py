@@ -19,7 +19,7 @@ def test_sampled_rows_full_size(name):
     print(name, worst)
 
 
-@pytest.mark.parametrize("name", ["32k", "32k_w1024"])
+@pytest.mark.parametrize("name", ["32k", "32k_w1024", "32k_m512", "32k_m1024"])
 def test_sampled_rows_full_size_fused_backward(name):
     """The same check with the fused one-kernel backward, the configuration bench.py times."""
     w = WORKLOADS[name]

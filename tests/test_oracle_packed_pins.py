@@ -185,3 +185,81 @@ def test_partition_covers_everything_once_and_handles_odd_counts():
     assert seen == list(range(48))
     with pytest.raises(ValueError):
         schedule.zigzag_chunks(50, 3)
+
+
+@pytest.mark.parametrize("mode,window,row_chunk", [(0, 0, 3), (1, 0, 2), (0, 5, 3), (0, 0, 64)])
+def test_sampled_rows_packed_equal_full_packed_oracle(mode, window, row_chunk):
+    """`attn_rows_packed` (the checker of the full-size packed parity tests) against `attn_packed`, which the
+    brute-force and finite-difference pins above fix: same rows -> same O, LSE, dQ; and, because dK/dV are
+    linear in dO, its per-row K/V contributions equal the full backward with dO zeroed outside the sample.
+    The prefix table holds an empty prefix, a repeat, non-multiples of M and the full prefix (Eq.
+    dflash2-block-attention); the clean run starts at an offset; the sample is larger than a row chunk."""
+    rng = np.random.default_rng(41 + mode + window)
+    B, Lk, H, Hkv, d, M = 1, 40, 2, 1, 4, 4
+    prefix = [0, 6, 6, 17, 28, 40] if window == 0 else [0, 4, 9, 17, 28, 36]   # with a window blocks may not overlap
+    nb = len(prefix)
+    pos0, Lq = 9, 22
+    kc, vc = _rand(rng, B, Lk, Hkv, d), _rand(rng, B, Lk, Hkv, d)
+    qc, qn = _rand(rng, B, Lq, H, d), _rand(rng, B, nb * M, H, d)
+    kn, vn = _rand(rng, B, nb * M, Hkv, d), _rand(rng, B, nb * M, Hkv, d)
+    doc, don = _rand(rng, B, Lq, H, d), _rand(rng, B, nb * M, H, d)
+    rows_c = np.array([0, 1, 3, 4, 10, 11, 20, 21])
+    rows_n = np.array([0, 3, 4, 7, 9, 12, 15, 16, 22, 23])
+    kw = dict(block_prefix=prefix, clean_q_pos0=pos0, clean_mask_mode=mode, window=window)
+    full = orc.attn_packed(qc, kc, vc, qn, kn, vn, M, **kw)
+    for h in range(H):
+        doc_s, don_s = np.zeros_like(doc), np.zeros_like(don)
+        doc_s[0, rows_c, h] = doc[0, rows_c, h]
+        don_s[0, rows_n, h] = don[0, rows_n, h]
+        g = orc.attn_packed(qc, kc, vc, qn, kn, vn, M, do_clean=doc_s, do_noisy=don_s, **kw)
+        rc = orc.attn_rows_packed(orc.CLEAN, rows_c, qc[0, rows_c, h], kc[0, :, 0], vc[0, :, 0], kn[0, :, 0],
+                                  vn[0, :, 0], M, do_rows=doc[0, rows_c, h], row_chunk=row_chunk, **kw)
+        rn = orc.attn_rows_packed(orc.NOISY, rows_n, qn[0, rows_n, h], kc[0, :, 0], vc[0, :, 0], kn[0, :, 0],
+                                  vn[0, :, 0], M, do_rows=don[0, rows_n, h], row_chunk=row_chunk, **kw)
+        assert np.allclose(rc["o"], full["o_clean"][0, rows_c, h], atol=1e-13)
+        assert np.allclose(rc["lse"], full["lse_clean"][0, h, rows_c], atol=1e-13)
+        assert np.allclose(rn["o"], full["o_noisy"][0, rows_n, h], atol=1e-13)
+        assert np.allclose(rn["lse"], full["lse_noisy"][0, h, rows_n], atol=1e-13)
+        assert np.allclose(rc["dq"], g["dq_clean"][0, rows_c, h], atol=1e-13)
+        assert np.allclose(rn["dq"], g["dq_noisy"][0, rows_n, h], atol=1e-13)
+        assert np.allclose(rc["dk_clean"] + rn["dk_clean"], g["dk_clean"][0, :, 0], atol=1e-13)
+        assert np.allclose(rc["dv_clean"] + rn["dv_clean"], g["dv_clean"][0, :, 0], atol=1e-13)
+        assert np.allclose(rn["dk_noisy"], g["dk_noisy"][0, :, 0], atol=1e-13)
+        assert np.allclose(rn["dv_noisy"], g["dv_noisy"][0, :, 0], atol=1e-13)
+        assert np.abs(rc["dk_noisy"]).max() == 0 and np.abs(rc["dv_noisy"]).max() == 0
+        # unsorted, repeated-free sample order must not matter
+        perm = rng.permutation(len(rows_n))
+        rp = orc.attn_rows_packed(orc.NOISY, rows_n[perm], qn[0, rows_n[perm], h], kc[0, :, 0], vc[0, :, 0],
+                                  kn[0, :, 0], vn[0, :, 0], M, do_rows=don[0, rows_n[perm], h], row_chunk=row_chunk, **kw)
+        assert np.allclose(rp["o"], rn["o"][perm], atol=1e-13) and np.allclose(rp["dq"], rn["dq"][perm], atol=1e-13)
+
+
+def test_sampled_rows_packed_reduce_to_plain_sampled_rows():
+    """With the table b*M, no offset and every block present, the packed sampled-row oracle is the plain one."""
+    rng = np.random.default_rng(77)
+    L, d, M = 24, 4, 4
+    kc, vc, kn, vn = (_rand(rng, L, d) for _ in range(4))
+    rows = np.array([0, 3, 4, 9, 23])
+    q, do = _rand(rng, len(rows), d), _rand(rng, len(rows), d)
+    for stream in (orc.CLEAN, orc.NOISY):
+        a = orc.attn_rows(stream, rows, q, kc, vc, kn, vn, M, do_rows=do)
+        b = orc.attn_rows_packed(stream, rows, q, kc, vc, kn, vn, M, do_rows=do)
+        for key in a:
+            assert np.allclose(a[key], b[key], atol=1e-14), key
+
+
+def test_workload_pair_counts_equal_explicit_mask_counts():
+    """The FLOP denominators of the benchmark (`Workload.pairs_per_head`: closed forms of appendix B, the
+    windowed and the packed variants) against pairs counted from the oracle's explicit masks."""
+    from paper_2609_19242_b200 import synth
+    for L, M, W in [(64, 8, 0), (96, 4, 0), (64, 8, 20), (64, 8, 8), (48, 16, 5), (60, 6, 7), (64, 4, 1000), (32, 1, 3)]:
+        w = synth.Workload("t", 1, 2, 1, 8, L, M, window=W)
+        assert w.pairs_per_head() == orc.visible_pair_counts(L, M, window=W), (L, M, W)
+    for L, M, nb, seed in [(64, 4, 9, 0), (80, 8, 5, 3), (33, 3, 12, 5)]:
+        w = synth.Workload("p", 1, 2, 1, 8, L, M, n_blocks=nb, seed=seed)
+        vis = orc.visible_rows_packed(orc.NOISY, np.arange(nb * M), L, M, nb, w.anchors())
+        assert w.pairs_per_head() == (0, int(vis.sum()))
+    # appendix B totals (Eq. aligned-rank-work with P = 1) for the headline shapes, without building their masks
+    for name in ("32k", "csbp128k", "256k"):
+        w = synth.WORKLOADS[name]
+        assert w.pairs_per_head() == (w.L * (w.L + 1) // 2, w.L * (w.L + w.block_size) // 2)

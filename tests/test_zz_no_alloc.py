@@ -32,12 +32,19 @@ def test_static_scratch_backward_matches_regular_backward_twice(w):
     ref = [t.clone() for t in pu.gpu_bwd(g, fwd, M)]
     torch.cuda.synchronize()
     out = tuple(torch.empty_like(t) for t in ref)            # caller-owned outputs: the call allocates nothing
+    g2 = dict(g)
+    g2["do_clean"] = (g["do_clean"].float() * -2.0).to(torch.bfloat16)
+    g2["do_noisy"] = (g["do_noisy"].float() * 0.5).to(torch.bfloat16)
+    # first use on this device (the library looks up its scratch array's address), then the books are opened:
+    # from here on neither torch's allocator nor the driver may hand out a byte on behalf of these calls
+    binding.bdlm_attn_bwd_static_scratch(*[g[n] for n in pu.NAMES6], fwd[0], fwd[1], fwd[2], fwd[3],
+                                         g["do_clean"], g["do_noisy"], M, out=out)
+    torch.cuda.synchronize()
+    torch_before = (torch.cuda.memory_allocated(), torch.cuda.memory_reserved())
+    free_before = torch.cuda.mem_get_info()[0]
     for call in range(2):
         if call == 1:
             # second call with a different upstream gradient first, so stale scratch would show
-            g2 = dict(g)
-            g2["do_clean"] = (g["do_clean"].float() * -2.0).to(torch.bfloat16)
-            g2["do_noisy"] = (g["do_noisy"].float() * 0.5).to(torch.bfloat16)
             binding.bdlm_attn_bwd_static_scratch(*[g2[n] for n in pu.NAMES6], fwd[0], fwd[1], fwd[2], fwd[3],
                                                  g2["do_clean"], g2["do_noisy"], M, out=out)
         for t in out:
@@ -45,6 +52,8 @@ def test_static_scratch_backward_matches_regular_backward_twice(w):
         binding.bdlm_attn_bwd_static_scratch(*[g[n] for n in pu.NAMES6], fwd[0], fwd[1], fwd[2], fwd[3],
                                              g["do_clean"], g["do_noisy"], M, out=out)
         torch.cuda.synchronize()
+        assert (torch.cuda.memory_allocated(), torch.cuda.memory_reserved()) == torch_before
+        assert torch.cuda.mem_get_info()[0] == free_before
         assert binding.bdlm_get_device_status() == 0
         for got, want in zip(out, ref):
             assert torch.isfinite(got.float()).all()
@@ -65,3 +74,28 @@ def test_static_scratch_rejects_sizes_beyond_its_limit():
     # invalid parameters are still rejected as such
     bad = binding.make_params(1, 100, 16, 4, 2, 128)
     assert binding.lib().bdlm_attn_bwd_static_scratch(ctypes.byref(bad), *([fake] * 18), None) == -1
+
+
+def test_static_scratch_always_runs_the_two_pass_kernels_and_reports_errors_like_the_regular_call():
+    w = Workload("na_mode", 1, 4, 2, 128, 256, 32)
+    M = w.block_size
+    g = pu.to_cuda(synth.make_inputs(w, "cpu"))
+    fwd = pu.gpu_fwd(g, M)
+    ref = [t.clone() for t in pu.gpu_bwd(g, fwd, M, single_pass=False)]
+    out = tuple(torch.empty_like(t) for t in ref)
+    args = [binding._ptr(g[n]) for n in pu.NAMES6] + [binding._ptr(t) for t in (fwd[0], fwd[2], fwd[1], fwd[3])] + \
+           [binding._ptr(g["do_clean"]), binding._ptr(g["do_noisy"])] + [binding._ptr(t) for t in out]
+    for sp in (None, True, False):     # the field is ignored: the fused kernel's accumulators do not fit a fixed array
+        for t in out:
+            t.zero_()
+        p = binding.make_params(w.batch, w.L, M, w.H, w.H_kv, w.d, bwd_single_pass=sp)
+        rc = binding.lib().bdlm_attn_bwd_static_scratch(ctypes.byref(p), *args, binding._stream())
+        assert rc == 0
+        torch.cuda.synchronize()
+        for got, want in zip(out, ref):
+            assert torch.equal(got, want)
+    fake = ctypes.c_void_p(0x1000)
+    d96 = binding.make_params(1, 256, 16, 4, 2, 96)
+    assert binding.lib().bdlm_attn_bwd_static_scratch(ctypes.byref(d96), *([fake] * 18), None) == -2
+    d96.bwd_single_pass = 1
+    assert binding.lib().bdlm_attn_bwd_static_scratch(ctypes.byref(d96), *([fake] * 18), None) == -2
