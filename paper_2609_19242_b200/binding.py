@@ -22,7 +22,9 @@ BWD_AUTO, BWD_FUSED, BWD_TWO_PASS = 0, 1, 2
 EXPORTS = ("bdlm_workspace_bytes", "bdlm_attn_fwd", "bdlm_attn_bwd", "bdlm_lse_merge",
            "bdlm_status_string", "bdlm_get_device_status", "bdlm_set_trace_buffer",
            "bdlm_attn_bwd_static_scratch", "bdlm_workspace_bytes_packed", "bdlm_attn_fwd_packed",
-           "bdlm_attn_bwd_packed", "bdlm_selftest_wait_timeout")
+           "bdlm_attn_bwd_packed", "bdlm_selftest_wait_timeout", "bdlm_linear_ce_workspace_bytes",
+           "bdlm_linear_ce_fwd", "bdlm_linear_ce_bwd")
+LCE_WS_FWD, LCE_WS_BWD = 0, 1
 STATIC_SCRATCH_ROWS = 1 << 20
 TRACE_SLOTS = 256
 
@@ -47,6 +49,11 @@ class BdlmPackedGeometry(ctypes.Structure):
     _fields_ = [("Lq_clean", ctypes.c_int32), ("clean_q_pos0", ctypes.c_int32), ("n_blocks", ctypes.c_int32),
                 ("kv_chunk_len", ctypes.c_int32), ("block_prefix", ctypes.c_void_p),
                 ("kv_chunk_pos", ctypes.c_void_p), ("kv_pos_chunk", ctypes.c_void_p)]
+
+
+class BdlmLceParams(ctypes.Structure):
+    _fields_ = [("T", ctypes.c_int32), ("D", ctypes.c_int32), ("V", ctypes.c_int32), ("token_chunk", ctypes.c_int32),
+                ("grad_loss", ctypes.c_float), ("reserved", ctypes.c_int32 * 3)]
 
 
 _lib = None
@@ -85,6 +92,13 @@ def lib():
         L.bdlm_attn_fwd_packed.argtypes = [pp, gp] + [vp] * 10 + [vp]
         L.bdlm_attn_bwd_packed.restype = ctypes.c_int
         L.bdlm_attn_bwd_packed.argtypes = [pp, gp] + [vp] * 18 + [vp, ctypes.c_size_t, vp]
+        lp = ctypes.POINTER(BdlmLceParams)
+        L.bdlm_linear_ce_workspace_bytes.restype = ctypes.c_size_t
+        L.bdlm_linear_ce_workspace_bytes.argtypes = [lp, ctypes.c_int32]
+        L.bdlm_linear_ce_fwd.restype = ctypes.c_int
+        L.bdlm_linear_ce_fwd.argtypes = [lp] + [vp] * 7 + [vp, ctypes.c_size_t, vp]
+        L.bdlm_linear_ce_bwd.restype = ctypes.c_int
+        L.bdlm_linear_ce_bwd.argtypes = [lp] + [vp] * 7 + [vp, ctypes.c_size_t, vp]
         L.bdlm_selftest_wait_timeout.restype = ctypes.c_int
         L.bdlm_selftest_wait_timeout.argtypes = [ctypes.c_int64, vp]
         _lib = L
@@ -349,3 +363,53 @@ def bdlm_set_trace_buffer(counters) -> None:
         rc = lib().bdlm_set_trace_buffer(_ptr(counters), counters.numel() * 8)
     if rc != 0:
         raise BdlmError(rc, "bdlm_set_trace_buffer")
+
+
+# ------------------------------------------------------------------------------------------
+# token-chunked linear cross-entropy (include/bdlm_linear_ce.h)
+# ------------------------------------------------------------------------------------------
+def make_lce_params(T, D, V, token_chunk=0, grad_loss=1.0) -> BdlmLceParams:
+    p = BdlmLceParams()
+    p.T, p.D, p.V, p.token_chunk, p.grad_loss = int(T), int(D), int(V), int(token_chunk), float(grad_loss)
+    return p
+
+
+def bdlm_linear_ce_workspace_bytes(params: BdlmLceParams, which: int) -> int:
+    return int(lib().bdlm_linear_ce_workspace_bytes(ctypes.byref(params), which))
+
+
+def bdlm_linear_ce_fwd(h, w, labels, token_weight=None, *, out=None, workspace=None):
+    """Forward of the linear cross-entropy: h [T, D] bf16, w [V, D] bf16, labels [T] int32 (negative = ignored),
+    token_weight [T] fp32 or None.  Returns (loss [1] fp32, nll [T] fp32, lse [T] fp32), all on the device."""
+    T, D = h.shape
+    V = w.shape[0]
+    p = make_lce_params(T, D, V)
+    if out is None:
+        out = (torch.empty(1, dtype=torch.float32, device=h.device), torch.empty(T, dtype=torch.float32, device=h.device),
+               torch.empty(T, dtype=torch.float32, device=h.device))
+    if workspace is None:
+        workspace = torch.empty(max(bdlm_linear_ce_workspace_bytes(p, LCE_WS_FWD), 16), dtype=torch.uint8, device=h.device)
+    assert labels.dtype == torch.int32
+    rc = lib().bdlm_linear_ce_fwd(ctypes.byref(p), _ptr(h), _ptr(w), _ptr(labels), _ptr(token_weight), _ptr(out[0]),
+                                  _ptr(out[1]), _ptr(out[2]), _ptr(workspace), workspace.numel(), _stream())
+    if rc != 0:
+        raise BdlmError(rc, "bdlm_linear_ce_fwd")
+    return out
+
+
+def bdlm_linear_ce_bwd(h, w, labels, lse, token_weight=None, *, grad_loss=1.0, token_chunk=0, out=None, workspace=None):
+    """Backward of the linear cross-entropy for the upstream scalar gradient `grad_loss`.  Returns (dh [T, D] bf16,
+    dw [V, D] bf16).  `token_chunk` (a multiple of 128, 0 = default) bounds the dz scratch to token_chunk * V bf16."""
+    T, D = h.shape
+    V = w.shape[0]
+    p = make_lce_params(T, D, V, token_chunk=token_chunk, grad_loss=grad_loss)
+    if out is None:
+        out = (torch.empty_like(h), torch.empty_like(w))
+    if workspace is None:
+        workspace = torch.empty(max(bdlm_linear_ce_workspace_bytes(p, LCE_WS_BWD), 16), dtype=torch.uint8, device=h.device)
+    assert labels.dtype == torch.int32
+    rc = lib().bdlm_linear_ce_bwd(ctypes.byref(p), _ptr(h), _ptr(w), _ptr(labels), _ptr(token_weight), _ptr(lse),
+                                  _ptr(out[0]), _ptr(out[1]), _ptr(workspace), workspace.numel(), _stream())
+    if rc != 0:
+        raise BdlmError(rc, "bdlm_linear_ce_bwd")
+    return out

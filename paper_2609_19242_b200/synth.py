@@ -162,3 +162,47 @@ def sample_rows(w: Workload, n: int, seed: int, extra=()):
         more = rng.choice(pool, size=min(n, L) - len(rows), replace=False)
         rows = sorted(set(rows) | set(int(x) for x in more))
     return np.asarray(rows, dtype=np.int64)
+
+
+
+# ------------------------------------------------------------------------------------------
+# linear cross-entropy head (the step after the last layer)
+# ------------------------------------------------------------------------------------------
+@dataclass(frozen=True)
+class LceWorkload:
+    """Hidden states h ~ N(0,1), output embedding W ~ N(0,1) * logit_std / sqrt(D) (logits with a standard deviation
+    of `logit_std`), targets uniform over the vocabulary with a fraction `ignored` of positions set to -100 (clean
+    positions and unmasked tokens carry no loss), per-token weights uniform in [0.5, 2] (the w(t_b) of Eq.
+    bdlm-training-objective differ from block to block).  The paper gives neither the vocabulary nor the hidden size;
+    the named workload uses Llama-3-8B's (D = 4096, V = 128256)."""
+    name: str
+    T: int
+    D: int
+    V: int
+    logit_std: float = 2.0
+    ignored: float = 0.25
+    seed: int = 0
+
+    def flops(self):
+        """(forward, backward) FLOPs: the projection 2 T D V; backward = the dH and dW products, 4 T D V (the
+        recomputation of the logits is executed but not counted)."""
+        f = 2 * self.T * self.D * self.V
+        return f, 2 * f
+
+
+LCE_WORKLOADS = {
+    "lce_tiny": LceWorkload("lce_tiny", 200, 64, 1000),
+    "lce_8k": LceWorkload("lce_8k", 8192, 4096, 128256),
+}
+
+
+def make_lce_inputs(w: LceWorkload, device="cpu"):
+    g = torch.Generator(device=device)
+    g.manual_seed(w.seed)
+    h = torch.randn(w.T, w.D, generator=g, device=device, dtype=torch.float32).to(torch.bfloat16)
+    W = (torch.randn(w.V, w.D, generator=g, device=device, dtype=torch.float32) * (w.logit_std / w.D ** 0.5)).to(torch.bfloat16)
+    labels = torch.randint(0, w.V, (w.T,), generator=g, device=device, dtype=torch.int32)
+    drop = torch.rand(w.T, generator=g, device=device) < w.ignored
+    labels = torch.where(drop, torch.full_like(labels, -100), labels)
+    weight = 0.5 + 1.5 * torch.rand(w.T, generator=g, device=device, dtype=torch.float32)
+    return {"h": h, "w": W, "labels": labels, "weight": weight}

@@ -10,20 +10,25 @@ from paper_2609_19242_b200 import binding, synth
 TOL_O = 1e-2          # max |dO| elementwise on outputs
 TOL_LSE = 1e-3        # max |dLSE|
 TOL_GRAD = 2e-2       # relative L2 error of each of dQ, dK, dV per stream
-TOL_DQ_ROW = 5e-2     # sampled-row checks: relative L2 error of every single dQ row (Eq. correctness-query-gradient is
-                      # per row, so one wrong row must not hide in the pooled figure above); a row whose exact dQ is
-                      # (nearly) zero -- clean row 0 sees one key, so dS = 0 -- is measured against a tenth of the
-                      # sample's mean row norm instead of its own
+TOL_DQ_ROW = 5e-2     # sampled-row checks: every single dQ row (Eq. correctness-query-gradient is per row, so one wrong
+                      # row must not hide in the pooled figure above) must satisfy
+                      #     |dQ_i - ref_i| <= TOL_DQ_ROW * |ref_i| + 2^-8 * scale * |dO_i| * |O_i| * max_j |k_j|.
+                      # The second term is the error the kernels' arithmetic allows: they form dS = P * (dP - D) with
+                      # D_i = dO_i . O_i taken from the bf16 output, so D carries up to 2^-9 |dO_i| |O_i| of rounding
+                      # (twice that allowed here), which enters dQ_i as scale * dD_i * sum_j P_ij k_j.  Rows where dP - D
+                      # cancels (row 1 with its two keys) lose several per cent that way; for a typical late row the term
+                      # is a few per cent of |ref_i|, so a wrong row (error of the order of the row itself) still fails.
 
 
-def dq_row_error(got, ref):
-    """Worst per-row relative L2 error of dQ rows [n, d] (see TOL_DQ_ROW)."""
-    got = np.asarray(got, dtype=np.float64)
-    ref = np.asarray(ref, dtype=np.float64)
-    norms = np.linalg.norm(ref, axis=1)
-    floor = 0.1 * float(norms.mean()) if norms.size else 0.0
-    den = np.maximum(norms, max(floor, 1e-300))
-    return float((np.linalg.norm(got - ref, axis=1) / den).max()) if norms.size else 0.0
+def dq_row_excess(got, ref, o_ref, do_rows, scale, k_max_norm):
+    """Worst ratio of a dQ row's error to its allowance (see TOL_DQ_ROW); must be <= 1.  Rows are [n, d]."""
+    got, ref = np.asarray(got, dtype=np.float64), np.asarray(ref, dtype=np.float64)
+    if ref.shape[0] == 0:
+        return 0.0
+    allow = TOL_DQ_ROW * np.linalg.norm(ref, axis=1) + \
+        2.0 ** -8 * scale * np.linalg.norm(do_rows, axis=1) * np.linalg.norm(o_ref, axis=1) * k_max_norm
+    return float((np.linalg.norm(got - ref, axis=1) / np.maximum(allow, 1e-300)).max())
+
 
 NAMES6 = ["q_clean", "k_clean", "v_clean", "q_noisy", "k_noisy", "v_noisy"]
 
@@ -128,6 +133,7 @@ def check_sampled(w, impl, n_rows=256, g=None, fwd_out=None, check_bwd=True, rep
         for hk in range(w.H_kv):
             kv = {n: synth.to_f64(g[n][b, :, hk]) for n in ("k_clean", "v_clean", "k_noisy", "v_noisy")}
             acc = {n: np.zeros((w.L, w.d)) for n in ("dk_clean", "dv_clean", "dk_noisy", "dv_noisy")}
+            k_max = float(max(np.linalg.norm(kv["k_clean"], axis=1).max(), np.linalg.norm(kv["k_noisy"], axis=1).max()))
             dq_num = {sp: [0.0, 0.0] for sp in variants}
             dq_den = [0.0, 0.0]
             for h in range(hk * G, (hk + 1) * G):
@@ -146,7 +152,8 @@ def check_sampled(w, impl, n_rows=256, g=None, fwd_out=None, check_bwd=True, rep
                         for sp in variants:
                             dq_got = synth.to_f64(grads[sp][3 * s][b, rt, h])
                             dq_num[sp][s] += float(((dq_got - ref["dq"]) ** 2).sum())
-                            worst["dq_row"] = max(worst["dq_row"], dq_row_error(dq_got, ref["dq"]))
+                            worst["dq_row"] = max(worst["dq_row"], dq_row_excess(dq_got, ref["dq"], ref["o"], do_rows,
+                                                                                 1.0 / np.sqrt(w.d), k_max))
                         dq_den[s] += float((ref["dq"] ** 2).sum())
                         for n in acc:
                             acc[n] += ref[n]
@@ -165,7 +172,7 @@ def check_sampled(w, impl, n_rows=256, g=None, fwd_out=None, check_bwd=True, rep
     assert worst["lse"] <= TOL_LSE, worst
     if check_bwd:
         assert worst["dq"] <= TOL_GRAD and worst["dk"] <= TOL_GRAD and worst["dv"] <= TOL_GRAD, worst
-        assert worst["dq_row"] <= TOL_DQ_ROW, worst
+        assert worst["dq_row"] <= 1.0, worst
     return worst
 
 
@@ -204,6 +211,7 @@ def check_sampled_packed(w, impl, n_rows=256, single_pass=False):
             kv = {n: synth.to_f64(g[n][b, :, hk]) for n in ("k_clean", "v_clean", "k_noisy", "v_noisy")}
             acc = {"dk_clean": np.zeros((w.L, w.d)), "dv_clean": np.zeros((w.L, w.d)),
                    "dk_noisy": np.zeros((Ln, w.d)), "dv_noisy": np.zeros((Ln, w.d))}
+            k_max = float(max(np.linalg.norm(kv["k_clean"], axis=1).max(), np.linalg.norm(kv["k_noisy"], axis=1).max()))
             num = den = 0.0
             for h in range(hk * G, (hk + 1) * G):
                 rows = rows_of[(b, h)]
@@ -214,7 +222,8 @@ def check_sampled_packed(w, impl, n_rows=256, single_pass=False):
                 worst["o"] = max(worst["o"], float(np.abs(synth.to_f64(out[2][b, rt, h]) - ref["o"]).max()))
                 worst["lse"] = max(worst["lse"], float(np.abs(synth.to_f64(out[3][b, h, rt]) - ref["lse"]).max()))
                 num += float(((synth.to_f64(grads[3][b, rt, h]) - ref["dq"]) ** 2).sum())
-                worst["dq_row"] = max(worst["dq_row"], dq_row_error(synth.to_f64(grads[3][b, rt, h]), ref["dq"]))
+                worst["dq_row"] = max(worst["dq_row"], dq_row_excess(synth.to_f64(grads[3][b, rt, h]), ref["dq"], ref["o"],
+                                                                     synth.to_f64(g["do_noisy"][b, rt, h]), 1.0 / np.sqrt(w.d), k_max))
                 den += float((ref["dq"] ** 2).sum())
                 for n in acc:
                     acc[n] += ref[n]
@@ -226,5 +235,5 @@ def check_sampled_packed(w, impl, n_rows=256, single_pass=False):
                 worst[n[:2]] = max(worst[n[:2]], rel_l2(got, want))
     assert worst["o"] <= TOL_O and worst["lse"] <= TOL_LSE, worst
     assert worst["dq"] <= TOL_GRAD and worst["dk"] <= TOL_GRAD and worst["dv"] <= TOL_GRAD, worst
-    assert worst["dq_row"] <= TOL_DQ_ROW, worst
+    assert worst["dq_row"] <= 1.0, worst
     return worst

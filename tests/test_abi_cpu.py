@@ -124,3 +124,24 @@ def test_packed_geometry_is_checked_without_a_device():
     p2 = binding.make_params(1, 250, 16, 4, 2, 64)
     assert L.bdlm_workspace_bytes_packed(ctypes.byref(p2), ctypes.byref(g), binding.BDLM_WS_BWD) > 0
     assert binding.bdlm_workspace_bytes(p2, binding.BDLM_WS_BWD) == 0
+
+
+def test_linear_ce_arguments_are_checked_without_a_device():
+    L = binding.lib()
+    ok = ctypes.c_void_p(0x1000)
+    good = binding.make_lce_params(256, 64, 512)
+    assert binding.bdlm_linear_ce_workspace_bytes(good, binding.LCE_WS_FWD) >= 3 * 256 * 4
+    assert binding.bdlm_linear_ce_workspace_bytes(good, binding.LCE_WS_BWD) == 256 * 512 * 2          # one chunk: dz only
+    big = binding.make_lce_params(1000, 64, 512, token_chunk=256)
+    assert binding.bdlm_linear_ce_workspace_bytes(big, binding.LCE_WS_BWD) == 256 * 512 * 2 + 512 * 64 * 4   # + fp32 dW
+    for kw in (dict(T=0, D=64, V=512), dict(T=8, D=60, V=512), dict(T=8, D=64, V=500), dict(T=8, D=64, V=512, token_chunk=100),
+               dict(T=8, D=64, V=512, grad_loss=float("nan"))):
+        p = binding.make_lce_params(**kw)
+        assert binding.bdlm_linear_ce_workspace_bytes(p, binding.LCE_WS_FWD) == 0
+        assert L.bdlm_linear_ce_fwd(ctypes.byref(p), *([ok] * 7), ok, 1 << 30, None) == -1
+        assert L.bdlm_linear_ce_bwd(ctypes.byref(p), *([ok] * 7), ok, 1 << 30, None) == -1
+    assert L.bdlm_linear_ce_fwd(ctypes.byref(good), None, ok, ok, ok, ok, ok, ok, ok, 1 << 30, None) == -1     # null h
+    assert L.bdlm_linear_ce_fwd(ctypes.byref(good), ctypes.c_void_p(0x1008), ok, ok, ok, ok, ok, ok, ok, 1 << 30, None) == -1
+    assert L.bdlm_linear_ce_fwd(ctypes.byref(good), *([ok] * 7), ok, 64, None) == -3                             # workspace too small
+    assert L.bdlm_linear_ce_bwd(ctypes.byref(good), *([ok] * 7), ok, 64, None) == -3
+    assert L.bdlm_linear_ce_fwd(None, *([ok] * 7), ok, 1 << 30, None) == -1
