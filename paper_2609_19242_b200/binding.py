@@ -219,6 +219,9 @@ def bdlm_attn_bwd_static_scratch(q_clean, k_clean, v_clean, q_noisy, k_noisy, v_
     return out
 
 
+_checked_prefix_tables = set()
+
+
 def _packed_setup(q_clean, k_clean, q_noisy, block_size, block_prefix, clean_q_pos0, window, kv_chunks=None, **kw):
     """Parameters and geometry of a packed call.  `block_prefix` is an int32 CUDA tensor [n_blocks] (or None
     for b * block_size); its ordering rules are checked here on a host copy because the C library never reads
@@ -257,14 +260,21 @@ def _packed_setup(q_clean, k_clean, q_noisy, block_size, block_prefix, clean_q_p
             assert block_prefix.is_cuda and block_prefix.dtype == torch.int32 and block_prefix.is_contiguous()
             if block_prefix.numel() != g.n_blocks:
                 raise ValueError("block_prefix needs one entry per packed block")
-            host = block_prefix.cpu()
-            step = host[1:] - host[:-1]
-            if host.numel() and (int(host.min()) < 0 or int(host.max()) > L):
-                raise ValueError("block_prefix entries must lie in [0, L]")
-            if step.numel() and int(step.min()) < 0:
-                raise ValueError("block_prefix must be non-decreasing (sort the packed blocks)")
-            if window > 0 and step.numel() and int(step.min()) < block_size:
-                raise ValueError("with a sliding window the packed blocks must not overlap in position")
+            # the host copy synchronises the device: a table that was checked once (same storage, same version
+            # counter, same rules) is not copied again on the calls of later steps
+            key = (block_prefix.data_ptr(), block_prefix.numel(), block_prefix._version, L, block_size, window > 0)
+            if key not in _checked_prefix_tables:
+                host = block_prefix.cpu()
+                step = host[1:] - host[:-1]
+                if host.numel() and (int(host.min()) < 0 or int(host.max()) > L):
+                    raise ValueError("block_prefix entries must lie in [0, L]")
+                if step.numel() and int(step.min()) < 0:
+                    raise ValueError("block_prefix must be non-decreasing (sort the packed blocks)")
+                if window > 0 and step.numel() and int(step.min()) < block_size:
+                    raise ValueError("with a sliding window the packed blocks must not overlap in position")
+                if len(_checked_prefix_tables) >= 256:
+                    _checked_prefix_tables.clear()
+                _checked_prefix_tables.add(key)
             g.block_prefix = block_prefix.data_ptr()
     g._keep = keep
     return p, g

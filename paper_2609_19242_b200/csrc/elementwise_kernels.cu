@@ -145,6 +145,58 @@ __global__ void __launch_bounds__(256) dsum_kernel(const bf16* __restrict__ dout
   }
 }
 
+// The same sums for a tile of 32 consecutive rows x all H heads per block: dO and O are read as they lie
+// ([batch, L, H, d]: the tile is one contiguous piece), the sums go through shared memory and leave as 128-byte runs
+// along L of the [batch, H, L] result (written straight from the reading lanes they would be 4-byte stores H*4 apart).
+constexpr int DS_LB = 32;
+template <int D>
+__global__ void __launch_bounds__(256) dsum_tile_kernel(const bf16* __restrict__ dout, const bf16* __restrict__ o,
+                                                        float* __restrict__ dsum, int L, int H, int tiles_per_batch) {
+  extern __shared__ float sums[];          // [H][DS_LB + 1]
+  constexpr int LPR = D / 8;               // lanes per row
+  constexpr int RPP = 256 / LPR;           // rows per pass of the block
+  constexpr int UNROLL = 4;
+  const int b = blockIdx.x / tiles_per_batch, l0 = (blockIdx.x % tiles_per_batch) * DS_LB;
+  const int nl = min(DS_LB, L - l0);
+  const int nrows = nl * H;                // rows of the tile: r = li * H + h
+  const int64_t base = ((int64_t)b * L + l0) * H;
+  const int sub = threadIdx.x / LPR, c = threadIdx.x % LPR;
+  for (int r0 = 0; r0 < nrows; r0 += RPP * UNROLL) {
+    uint4 ua[UNROLL], ub[UNROLL];
+#pragma unroll
+    for (int j = 0; j < UNROLL; ++j) {
+      const int r = r0 + j * RPP + sub;
+      if (r < nrows) {
+        ua[j] = *reinterpret_cast<const uint4*>(dout + (base + r) * D + c * 8);
+        ub[j] = *reinterpret_cast<const uint4*>(o + (base + r) * D + c * 8);
+      } else {
+        ua[j] = make_uint4(0u, 0u, 0u, 0u); ub[j] = ua[j];
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < UNROLL; ++j) {
+      const uint32_t* pa = reinterpret_cast<const uint32_t*>(&ua[j]);
+      const uint32_t* pb = reinterpret_cast<const uint32_t*>(&ub[j]);
+      float acc = 0.f;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pa[e]));
+        const float2 y = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pb[e]));
+        acc = fmaf(x.x, y.x, fmaf(x.y, y.y, acc));
+      }
+#pragma unroll
+      for (int sft = LPR / 2; sft > 0; sft >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, sft);
+      const int r = r0 + j * RPP + sub;
+      if (c == 0 && r < nrows) sums[(r % H) * (DS_LB + 1) + r / H] = acc;
+    }
+  }
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < H * DS_LB; idx += 256) {
+    const int h = idx / DS_LB, li = idx % DS_LB;
+    if (li < nl) dsum[((int64_t)b * H + h) * L + l0 + li] = sums[h * (DS_LB + 1) + li];
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_merge(int n, int batch, int L, int H, int d, const void* const* o_parts,
@@ -178,6 +230,18 @@ cudaError_t launch_dsum(const KArgs& a, float* dsum_clean, float* dsum_noisy, cu
   for (int s = 0; s < 2; ++s) {
     if (a.q[s] == nullptr) continue;   // a stream without queries has no D rows
     const int rows = rows_q(a, s);
+    const size_t tile_smem = (size_t)a.H * (DS_LB + 1) * sizeof(float);
+    if (tile_smem <= 48 * 1024 && rows > 0) {   // the tiled form: coalesced on both sides
+      const int tpb = (rows + DS_LB - 1) / DS_LB;
+      const int64_t nblk = (int64_t)a.batch * tpb;
+      if (nblk <= 0x7fffffff) {
+        if (a.d == 128) dsum_tile_kernel<128><<<(int)nblk, 256, tile_smem, st>>>(a.dout[s], a.o[s], out[s], rows, a.H, tpb);
+        else dsum_tile_kernel<64><<<(int)nblk, 256, tile_smem, st>>>(a.dout[s], a.o[s], out[s], rows, a.H, tpb);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        continue;
+      }
+    }
     const int64_t nrows = (int64_t)a.batch * rows * a.H;
     const int rows_per_block = 8 * (32 / (a.d / 8)) * 4;   // 8 warps, 32 / (d / 8) rows per warp and pass, 4 passes
     const int blocks = (int)((nrows + rows_per_block - 1) / rows_per_block);
