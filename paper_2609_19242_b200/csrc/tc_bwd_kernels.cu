@@ -34,11 +34,14 @@ struct BwdMaps {
 constexpr int BWD_THREADS = 320;
 constexpr int TILE_BYTES = 2 * PANEL_BYTES;
 constexpr uint32_t IDESC_KK = make_idesc(128, 128, false, false);   // A, B both K-major
-constexpr uint32_t IDESC_KM = make_idesc(128, 128, false, true);    // B MN-major (a [k][n] tile as loaded)
+// B MN-major (a [k][n] tile as loaded) with N = the head dimension
+__host__ __device__ constexpr uint32_t idesc_km(int d) { return make_idesc(128, d, false, true); }
 
-__device__ __forceinline__ void tma_tile(uint32_t dst, const CUtensorMap* map, uint32_t bar, int col0, int row0, int b) {
-  tma_load_3d(dst, map, bar, col0, row0, b);
-  tma_load_3d(dst + PANEL_BYTES, map, bar, col0 + 64, row0, b);
+// One operand tile of head `head`: D / 64 panels of 64 columns (D = head dimension, 128 or 64).
+template <int D>
+__device__ __forceinline__ void tma_tile(uint32_t dst, const CUtensorMap* map, uint32_t bar, int head, int row0, int b) {
+  tma_load_3d(dst, map, bar, head * D, row0, b);
+  if (D == 128) tma_load_3d(dst + PANEL_BYTES, map, bar, head * D + 64, row0, b);
 }
 
 // Write a thread's 128 accumulator columns (4 x 32) as bf16 to a global row, scaled.
@@ -105,9 +108,11 @@ struct StepWalk {
   }
 };
 
-template <bool TR>
+template <bool TR, int D>
 __global__ void __launch_bounds__(DKDV_THREADS, 1)
 tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restrict__ status) {
+  constexpr uint32_t IDESC_KM = idesc_km(D);
+  constexpr int OPER_BYTES = TILE_BYTES * D / 128;   // bytes TMA delivers per operand tile (D = 64: one panel)
   extern __shared__ __align__(1024) uint8_t sm[];
   const uint32_t base = smem_u32(sm);
   const uint32_t sK = base, sV = base + TILE_BYTES, sQ0 = base + DKDV_Q0, sdO0 = base + DKDV_DO0, sP = base + DKDV_P;
@@ -178,9 +183,9 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
   } else if (warp == DKDV_PRODUCER) {
     // ------------------------------------------------------------------ producer
     if (lane == 0 && nsteps > 0) {   // a key tile no query sees writes zeros and waits for nothing: it must not leave a copy in flight
-      mbar_expect_tx(bar_kv, 2 * TILE_BYTES);
-      tma_tile(sK, &maps.k[ks], bar_kv, hk * 128, k0_row, b);
-      tma_tile(sV, &maps.v[ks], bar_kv, hk * 128, k0_row, b);
+      mbar_expect_tx(bar_kv, 2 * OPER_BYTES);
+      tma_tile<D>(sK, &maps.k[ks], bar_kv, hk, k0_row, b);
+      tma_tile<D>(sV, &maps.v[ks], bar_kv, hk, k0_row, b);
     }
     bool ok = true;
     long long w_empty = 0;
@@ -204,15 +209,15 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       if (lane == 0) {
-        mbar_expect_tx(bar_q_full + 8 * sd, TILE_BYTES);
-        tma_tile(sQ0 + sd * TILE_BYTES, &maps.q[st.qs], bar_q_full + 8 * sd, st.h * 128, st.q0, b);
+        mbar_expect_tx(bar_q_full + 8 * sd, OPER_BYTES);
+        tma_tile<D>(sQ0 + sd * TILE_BYTES, &maps.q[st.qs], bar_q_full + 8 * sd, st.h, st.q0, b);
       }
       if (i >= 2) ok = mbar_wait_timed<TR>(bar_do_empty + 8 * sd, ((i >> 1) - 1) & 1, abort_flag, w_empty);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       if (lane == 0) {
-        mbar_expect_tx(bar_do_full + 8 * sd, TILE_BYTES);   // one arrival of two; the LSE/D rows follow
-        tma_tile(sdO0 + sd * TILE_BYTES, &maps.dout[st.qs], bar_do_full + 8 * sd, st.h * 128, st.q0, b);
+        mbar_expect_tx(bar_do_full + 8 * sd, OPER_BYTES);   // one arrival of two; the LSE/D rows follow
+        tma_tile<D>(sdO0 + sd * TILE_BYTES, &maps.dout[st.qs], bar_do_full + 8 * sd, st.h, st.q0, b);
       }
       {
         float4 z2;
@@ -239,13 +244,13 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       ok = ok && mbar_wait_abortable(bar_q_full, 0, abort_flag);
       if (ok) {
         tc_fence_after();
-        gemm_ss_e(tmem, k_lo, qk_lo0, IDESC_KK, 0u, el);
+        gemm_ss_e<D / 16>(tmem, k_lo, qk_lo0, IDESC_KK, 0u, el);
         mma_commit_e(bar_st, el);
       }
       ok = ok && mbar_wait_abortable(bar_do_full, 0, abort_flag);
       if (ok) {
         tc_fence_after();
-        gemm_ss_e(tmem + 128, v_lo, dok_lo0, IDESC_KK, 0u, el);
+        gemm_ss_e<D / 16>(tmem + 128, v_lo, dok_lo0, IDESC_KK, 0u, el);
         mma_commit_e(bar_dpt, el);
       }
       for (int i = 0; i < nsteps && ok; ++i) {
@@ -257,7 +262,7 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
           ok = ok && mbar_wait_lean(bar_q_full + 8 * sn, ((i + 1) >> 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          gemm_ss_e(tmem, k_lo, qk_lo0 + sn * TILE_LO, IDESC_KK, 0u, el);
+          gemm_ss_e<D / 16>(tmem, k_lo, qk_lo0 + sn * TILE_LO, IDESC_KK, 0u, el);
           mma_commit_e(bar_st, el);
         }
         // dV += P^T dO_i   (P^T from shared memory, K-major: row = key, contraction = query)
@@ -278,7 +283,7 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
           ok = mbar_wait_lean(bar_do_full + 8 * sn, ((i + 1) >> 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          gemm_ss_e(tmem + 128, v_lo, dok_lo0 + sn * TILE_LO, IDESC_KK, 0u, el);
+          gemm_ss_e<D / 16>(tmem + 128, v_lo, dok_lo0 + sn * TILE_LO, IDESC_KK, 0u, el);
           mma_commit_e(bar_dpt, el);
         }
       }
@@ -446,10 +451,11 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       constexpr int EW = 256 / DKDV_NWG;                       // accumulator columns per thread
       const int acol = w * EW;                                 // first of them, in [0, 256)
       const bool is_dk = acol >= 128;
-      bf16* dst = (is_dk ? a.dk[ks] : a.dv[ks]) + (((int64_t)b * L + k0_row + r) * a.Hkv + hk) * 128 + (acol & 127);
+      bf16* dst = (is_dk ? a.dk[ks] : a.dv[ks]) + (((int64_t)b * L + k0_row + r) * a.Hkv + hk) * D + (acol & 127);
       const float sc = is_dk ? a.scale : 1.f;
+      static_assert(EW == 128, "one warpgroup per accumulator");
 #pragma unroll
-      for (int c = 0; c < EW / 32; ++c) {
+      for (int c = 0; c < D / 32; ++c) {
         uint32_t v[32];
         if (nsteps > 0) { tmem_ld32(tl + 256 + acol + c * 32, v); tmem_wait_ld(); }
         else {
@@ -479,9 +485,10 @@ constexpr int DQ_BARS = 7 * TILE_BYTES;
 constexpr int DQ_SMEM = DQ_BARS + 192;
 
 // Copy row `r` of a swizzled [128 x 128] bf16 tile into 64 TMEM columns (this thread's lane).
+template <int D>
 __device__ __forceinline__ void row_smem_to_tmem(const uint8_t* tile, int r, uint32_t taddr) {
 #pragma unroll
-  for (int half = 0; half < 2; ++half) {
+  for (int half = 0; half < D / 64; ++half) {
     uint32_t v[32];
 #pragma unroll
     for (int c = 0; c < 8; ++c) {
@@ -492,9 +499,11 @@ __device__ __forceinline__ void row_smem_to_tmem(const uint8_t* tile, int r, uin
   }
 }
 
-template <bool TR>
+template <bool TR, int D>
 __global__ void __launch_bounds__(BWD_THREADS, 1)
 tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restrict__ status) {
+  constexpr uint32_t IDESC_KM = idesc_km(D);
+  constexpr int OPER_BYTES = TILE_BYTES * D / 128;
   extern __shared__ __align__(1024) uint8_t sm[];
   const uint32_t base = smem_u32(sm);
   const uint32_t sQ = base, sdO = base + TILE_BYTES, sK0 = base + DQ_K0, sV0 = base + DQ_V0;
@@ -550,9 +559,9 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
     // fall through to the common exit
   } else if (warp == 8) {
     if (lane == 0 && nsteps > 0) {
-      mbar_expect_tx(bar_qdo, 2 * TILE_BYTES);
-      tma_tile(sQ, &maps.q[qs], bar_qdo, h * 128, q0, b);
-      tma_tile(sdO, &maps.dout[qs], bar_qdo, h * 128, q0, b);
+      mbar_expect_tx(bar_qdo, 2 * OPER_BYTES);
+      tma_tile<D>(sQ, &maps.q[qs], bar_qdo, h, q0, b);
+      tma_tile<D>(sdO, &maps.dout[qs], bar_qdo, h, q0, b);
       bool ok = true;
       long long w_empty = 0;
       const long long t_begin = tick<TR>();
@@ -561,13 +570,13 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
         const int ks = tile_ks(i), k0 = tile_k0(i);
         if (i >= 3) ok = mbar_wait_timed<TR>(bar_k_empty + 8 * sk, ((i / 3) - 1) & 1, abort_flag, w_empty);
         if (!ok) break;
-        mbar_expect_tx(bar_k_full + 8 * sk, TILE_BYTES);
+        mbar_expect_tx(bar_k_full + 8 * sk, OPER_BYTES);
         const int krow = ks == CLEAN ? clean_key_row(a, k0) : k0;   // where the tile's first key is stored
-        tma_tile(sK0 + sk * TILE_BYTES, &maps.k[ks], bar_k_full + 8 * sk, hk * 128, krow, b);
+        tma_tile<D>(sK0 + sk * TILE_BYTES, &maps.k[ks], bar_k_full + 8 * sk, hk, krow, b);
         if (i >= 2) ok = mbar_wait_timed<TR>(bar_v_empty + 8 * sv, ((i >> 1) - 1) & 1, abort_flag, w_empty);
         if (!ok) break;
-        mbar_expect_tx(bar_v_full + 8 * sv, TILE_BYTES);
-        tma_tile(sV0 + sv * TILE_BYTES, &maps.v[ks], bar_v_full + 8 * sv, hk * 128, krow, b);
+        mbar_expect_tx(bar_v_full + 8 * sv, OPER_BYTES);
+        tma_tile<D>(sV0 + sv * TILE_BYTES, &maps.v[ks], bar_v_full + 8 * sv, hk, krow, b);
       }
       trace_add(a.trace, 32 + 12, tick<TR>() - t_begin); trace_add(a.trace, 32 + 13, w_empty);
     }
@@ -583,13 +592,13 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
       ok = ok && mbar_wait_abortable(bar_k_full, 0, abort_flag);
       if (ok) {
         tc_fence_after();
-        gemm_ts_e(tmem + C_S, tmem + C_Q, kk_lo0, IDESC_KK, 0u, el);
+        gemm_ts_e<D / 16>(tmem + C_S, tmem + C_Q, kk_lo0, IDESC_KK, 0u, el);
         mma_commit_e(bar_s, el);
       }
       ok = ok && mbar_wait_abortable(bar_v_full, 0, abort_flag);
       if (ok) {
         tc_fence_after();
-        gemm_ts_e(tmem + C_DP, tmem + C_DO, vk_lo0, IDESC_KK, 0u, el);
+        gemm_ts_e<D / 16>(tmem + C_DP, tmem + C_DO, vk_lo0, IDESC_KK, 0u, el);
         mma_commit_e(bar_dp, el);
         mma_commit_e(bar_v_empty, el);
       }
@@ -602,7 +611,7 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
           if (!ok) break;
           tc_fence_after();
           const long long g0 = tick<TR>();
-          gemm_ts_e(tmem + C_S, tmem + C_Q, kk_lo0 + nk * TILE_LO, IDESC_KK, 0u, el);
+          gemm_ts_e<D / 16>(tmem + C_S, tmem + C_Q, kk_lo0 + nk * TILE_LO, IDESC_KK, 0u, el);
           mma_commit_e(bar_s, el);
           t_issue += tick<TR>() - g0;
         }
@@ -620,7 +629,7 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
           if (!ok) break;
           tc_fence_after();
           const long long g2 = tick<TR>();
-          gemm_ts_e(tmem + C_DP, tmem + C_DO, vk_lo0 + nv * TILE_LO, IDESC_KK, 0u, el);
+          gemm_ts_e<D / 16>(tmem + C_DP, tmem + C_DO, vk_lo0 + nv * TILE_LO, IDESC_KK, 0u, el);
           mma_commit_e(bar_dp, el);
           mma_commit_e(bar_v_empty + 8 * nv, el);
           t_issue += tick<TR>() - g2;
@@ -656,7 +665,7 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
       ok = mbar_wait_abortable(bar_qdo, 0, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       if (ok) {
-        row_smem_to_tmem(sm + (w == 0 ? 0 : TILE_BYTES), r, tl + (w == 0 ? C_Q : C_DO));
+        row_smem_to_tmem<D>(sm + (w == 0 ? 0 : TILE_BYTES), r, tl + (w == 0 ? C_Q : C_DO));
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(bar_aready);
@@ -736,11 +745,13 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
     }
     if (ok) {
       tc_fence_after();
-      bf16* dst = a.dq[qs] + (((int64_t)b * L + row) * a.H + h) * 128 + c0;
+      // each warpgroup writes half of the row's D gradient columns
+      constexpr int EC = D / 2;
+      bf16* dst = a.dq[qs] + (((int64_t)b * L + row) * a.H + h) * D + w * EC;
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
+      for (int c = 0; c < EC / 32; ++c) {
         uint32_t v[32];
-        if (nsteps > 0) { tmem_ld32(tl + C_DQ + c0 + c * 32, v); tmem_wait_ld(); }
+        if (nsteps > 0) { tmem_ld32(tl + C_DQ + w * EC + c * 32, v); tmem_wait_ld(); }
         else {
 #pragma unroll
           for (int e = 0; e < 32; ++e) v[e] = 0u;
@@ -800,9 +811,14 @@ constexpr uint32_t HPANEL_LO = HPANEL_BYTES >> 4, HT_LO = HT_BYTES >> 4;
 __host__ __device__ constexpr uint32_t koff_h(int kk) { return (kk >> 2) * HPANEL_LO + (kk & 3) * 2; }   // K-major slice of a 64-row tile
 __device__ __forceinline__ uint32_t desc_lo_mn_h(uint32_t addr) { return ((addr & 0x3FFFFu) >> 4) | (HPANEL_LO << 16); }
 
-template <bool TR>
+// D = head dimension.  With D = 64 the operand tiles are one panel wide, the contractions over the head dimension take
+// four k-slices and dV / dK have 64 columns; dQ^T keeps its 128 lanes (the upper 64 hold nothing of value and land in
+// the unused half of the 128-wide fp32 accumulator rows).
+template <bool TR, int D>
 __global__ void __launch_bounds__(BF_THREADS, 1)
 tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restrict__ status) {
+  constexpr uint32_t IDESC_KM = idesc_km(D);
+  constexpr int OPER_BYTES = TILE_BYTES * D / 128, HOPER_BYTES = HT_BYTES * D / 128;   // bytes TMA delivers per 128- / 64-row tile
   extern __shared__ __align__(1024) uint8_t sm[];
   const uint32_t base = smem_u32(sm);
   const uint32_t sK = base, sV = base + TILE_BYTES, sQ0 = base + BF_Q0, sdO0 = base + BF_DO0, sDS = base + BF_DS,
@@ -873,9 +889,9 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
   } else if (warp == 8) {
     // ------------------------------------------------------------------ producer
     if (lane == 0 && nsteps > 0) {   // a key tile no query sees writes zeros and waits for nothing: it must not leave a copy in flight
-      mbar_expect_tx(bar_kv, 2 * TILE_BYTES);
-      tma_tile(sK, &maps.k[ks], bar_kv, hk * 128, k0_row, b);
-      tma_tile(sV, &maps.v[ks], bar_kv, hk * 128, k0_row, b);
+      mbar_expect_tx(bar_kv, 2 * OPER_BYTES);
+      tma_tile<D>(sK, &maps.k[ks], bar_kv, hk, k0_row, b);
+      tma_tile<D>(sV, &maps.v[ks], bar_kv, hk, k0_row, b);
     }
     bool ok = true;
     long long w_empty = 0;
@@ -901,18 +917,18 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       if (!ok) break;
       if (lane == 0) {
         const uint32_t dst = sQ0 + sq * HT_BYTES, bar = bar_q_full + 8 * sq;
-        mbar_expect_tx(bar, HT_BYTES);
-        tma_load_3d(dst, &maps.q[st.qs], bar, st.h * 128, st.q0, b);
-        tma_load_3d(dst + HPANEL_BYTES, &maps.q[st.qs], bar, st.h * 128 + 64, st.q0, b);
+        mbar_expect_tx(bar, HOPER_BYTES);
+        tma_load_3d(dst, &maps.q[st.qs], bar, st.h * D, st.q0, b);
+        if (D == 128) tma_load_3d(dst + HPANEL_BYTES, &maps.q[st.qs], bar, st.h * D + 64, st.q0, b);
       }
       if (kd >= 1) ok = mbar_wait_timed<TR>(bar_do_empty + 8 * sd, (kd - 1) & 1, abort_flag, w_empty);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       if (lane == 0) {
         const uint32_t dst = sdO0 + sd * HT_BYTES, bar = bar_do_full + 8 * sd;
-        mbar_expect_tx(bar, HT_BYTES);
-        tma_load_3d(dst, &maps.dout[st.qs], bar, st.h * 128, st.q0, b);
-        tma_load_3d(dst + HPANEL_BYTES, &maps.dout[st.qs], bar, st.h * 128 + 64, st.q0, b);
+        mbar_expect_tx(bar, HOPER_BYTES);
+        tma_load_3d(dst, &maps.dout[st.qs], bar, st.h * D, st.q0, b);
+        if (D == 128) tma_load_3d(dst + HPANEL_BYTES, &maps.dout[st.qs], bar, st.h * D + 64, st.q0, b);
       }
       // the rows live in a ring of their own: the dO tile is free again as soon as dV has read it, the D rows
       // only when the compute warps have formed dS
@@ -947,13 +963,13 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       const uint32_t dsk_lo = desc_lo_k(sDS), dsm_lo = desc_lo_k(sDS);          // dS^T: K-major A (dK) / MN-major B with one 64-query group (dQ^T)
       auto issue_st = [&](int sq) {     // S^T = K Q^T, K from tensor memory
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk)
+        for (int kk = 0; kk < D / 16; ++kk)
           mma_ts_e(tmem, tmem + 64 + kk * 8, desc64(qk_lo0 + sq * HT_LO + koff_h(kk)), IDESC_N64, kk == 0 ? 0u : 1u, el);
         mma_commit_e(bar_st, el);
       };
       auto issue_dpt = [&](int sd) {             // dP^T = V dO^T
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk)
+        for (int kk = 0; kk < D / 16; ++kk)
           mma_ss_e(tmem + 128, desc64(v_lo + koff(kk)), desc64(dok_lo0 + sd * HT_LO + koff_h(kk)), IDESC_N64, kk == 0 ? 0u : 1u, el);
         mma_commit_e(bar_dpt, el);
       };
@@ -1116,7 +1132,7 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       ok = mbar_wait_abortable(bar_kv, 0, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       if (ok) {
-        row_smem_to_tmem(sm, r, tl + 64);
+        row_smem_to_tmem<D>(sm, r, tl + 64);
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(bar_kready);
@@ -1226,10 +1242,10 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
     }
     if (ok) {
       tc_fence_after();
-      bf16* dst = (w == 0 ? a.dv[ks] : a.dk[ks]) + (((int64_t)b * L + k0_row + r) * a.Hkv + hk) * 128;
+      bf16* dst = (w == 0 ? a.dv[ks] : a.dk[ks]) + (((int64_t)b * L + k0_row + r) * a.Hkv + hk) * D;
       const float sc = (w == 0) ? 1.f : a.scale;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < D / 32; ++c) {
         uint32_t v[32];
         if (nsteps > 0) { tmem_ld32(tl + 256 + w * 128 + c * 32, v); tmem_wait_ld(); }
         else {
@@ -1246,7 +1262,9 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
   if (warp == 8) tmem_dealloc(tmem, 512);
 }
 
-// fp32 dQ accumulator [batch, H, rows, 128] -> bf16 dQ [batch, rows, H, 128]; one warp per 128-element row
+// fp32 dQ accumulator [batch, H, rows, 128] -> bf16 dQ [batch, rows, H, D]; one warp per row (D = 64: the first 64
+// of the accumulator row's 128 floats)
+template <int D>
 __global__ void __launch_bounds__(256) dq_convert_kernel(const float* __restrict__ src, bf16* __restrict__ dst, int batch, int H, int rows) {
   const int lane = threadIdx.x & 31;
   const int64_t n = (int64_t)batch * rows * H;
@@ -1254,28 +1272,35 @@ __global__ void __launch_bounds__(256) dq_convert_kernel(const float* __restrict
     const int h = (int)(o % H);
     const int64_t bl = o / H;
     const int l = (int)(bl % rows), b = (int)(bl / rows);
-    const float4 u = reinterpret_cast<const float4*>(src + (((int64_t)b * H + h) * rows + l) * 128)[lane];
-    uint2 v;
-    v.x = pack_bf16(u.x, u.y); v.y = pack_bf16(u.z, u.w);
-    reinterpret_cast<uint2*>(dst + o * 128)[lane] = v;
+    const float* row = src + (((int64_t)b * H + h) * rows + l) * 128;
+    if (D == 128) {
+      const float4 u = reinterpret_cast<const float4*>(row)[lane];
+      uint2 v;
+      v.x = pack_bf16(u.x, u.y); v.y = pack_bf16(u.z, u.w);
+      reinterpret_cast<uint2*>(dst + o * D)[lane] = v;
+    } else {
+      const float2 u = reinterpret_cast<const float2*>(row)[lane];
+      reinterpret_cast<uint32_t*>(dst + o * D)[lane] = pack_bf16(u.x, u.y);
+    }
   }
 }
 
 }  // namespace
 
 bool tc_bwd_supported(const KArgs& a) {
-  return a.d == 128 && tc_rows_ok(a) && tc_encoder_available();
+  return (a.d == 128 || a.d == 64) && tc_rows_ok(a) && tc_encoder_available();
 }
 // fp32 dQ accumulators of the fused backward: one [batch, H, rows, 128] tensor per query stream
 size_t tc_bwd_fused_workspace(const bdlm_params* p, const bdlm_packed_geometry* g) {
-  if (p->d != 128 || p->impl == 1) return 0;
+  if ((p->d != 128 && p->d != 64) || p->impl == 1) return 0;
   const size_t rows_c = g != nullptr ? (size_t)g->Lq_clean : (size_t)p->L;
   const size_t rows_n = g != nullptr ? (size_t)g->n_blocks * p->block_size : (size_t)p->L;
   if (p->L % TILE != 0 || rows_c % TILE != 0 || rows_n % TILE != 0) return 0;   // such shapes take the mma.sync kernels
   return (rows_c + rows_n) * p->batch * p->H * 128 * sizeof(float);
 }
 
-cudaError_t launch_tc_bwd(const KArgs& a_in, void* extra_ws, int passes, cudaStream_t st) {
+template <int D>
+static cudaError_t launch_tc_bwd_d(const KArgs& a_in, void* extra_ws, int passes, cudaStream_t st) {
   KArgs a = a_in;
   const size_t dq32_elems[2] = {a.q[CLEAN] != nullptr ? (size_t)a.batch * a.H * a.Lqc * 128 : 0,
                                 a.q[NOISY] != nullptr ? (size_t)a.batch * a.H * a.Ln * 128 : 0};
@@ -1289,10 +1314,10 @@ cudaError_t launch_tc_bwd(const KArgs& a_in, void* extra_ws, int passes, cudaStr
     const int sq = a.q[s] != nullptr ? s : 1 - s;
     const int sk = a.k[s] != nullptr ? s : CLEAN;
     const int qbox = a.single_pass ? HT : TILE;   // the fused kernel loads 64 query rows per step
-    if (!tc_make_map(&maps.q[s], a.q[sq], a.H, rows_q(a, sq), a.batch, qbox)) return cudaErrorInvalidValue;
-    if (!tc_make_map(&maps.dout[s], a.dout[sq], a.H, rows_q(a, sq), a.batch, qbox)) return cudaErrorInvalidValue;
-    if (!tc_make_map(&maps.k[s], a.k[sk], a.Hkv, rows_k(a, sk), a.batch, TILE)) return cudaErrorInvalidValue;
-    if (!tc_make_map(&maps.v[s], a.v[sk], a.Hkv, rows_k(a, sk), a.batch, TILE)) return cudaErrorInvalidValue;
+    if (!tc_make_map(&maps.q[s], a.q[sq], a.H, rows_q(a, sq), a.batch, qbox, D)) return cudaErrorInvalidValue;
+    if (!tc_make_map(&maps.dout[s], a.dout[sq], a.H, rows_q(a, sq), a.batch, qbox, D)) return cudaErrorInvalidValue;
+    if (!tc_make_map(&maps.k[s], a.k[sk], a.Hkv, rows_k(a, sk), a.batch, TILE, D)) return cudaErrorInvalidValue;
+    if (!tc_make_map(&maps.v[s], a.v[sk], a.Hkv, rows_k(a, sk), a.batch, TILE, D)) return cudaErrorInvalidValue;
   }
   int* status = device_status_ptr();
   if (status == nullptr) return cudaErrorUnknown;
@@ -1301,34 +1326,38 @@ cudaError_t launch_tc_bwd(const KArgs& a_in, void* extra_ws, int passes, cudaStr
     // one kernel produces dK, dV and (through fp32 add-reductions) dQ; it runs for the DKDV pass bit, the DQ bit is a no-op
     if (passes & BDLM_BWD_PASS_DKDV) {
       if ((e = cudaMemsetAsync(a.dq32[0], 0, (dq32_elems[0] + dq32_elems[1]) * sizeof(float), st)) != cudaSuccess) return e;
-      auto kern = a.trace ? tc_bwdf_kernel<true> : tc_bwdf_kernel<false>;
+      auto kern = a.trace ? tc_bwdf_kernel<true, D> : tc_bwdf_kernel<false, D>;
       if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, BF_SMEM)) != cudaSuccess) return e;
       dim3 grid(max(a.L, a.k[NOISY] != nullptr ? a.Ln : 0) / TILE, a.Hkv, a.batch * 2);
       kern<<<grid, BF_THREADS, BF_SMEM, st>>>(maps, a, status);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
       for (int s2 = 0; s2 < 2; ++s2) {
         if (dq32_elems[s2] == 0) continue;
-        dq_convert_kernel<<<device_sm_count() * 8, 256, 0, st>>>(a.dq32[s2], a.dq[s2], a.batch, a.H, rows_q(a, s2));
+        dq_convert_kernel<D><<<device_sm_count() * 8, 256, 0, st>>>(a.dq32[s2], a.dq[s2], a.batch, a.H, rows_q(a, s2));
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
       }
     }
     return cudaSuccess;
   }
   if (passes & BDLM_BWD_PASS_DKDV) {
-    auto kern = a.trace ? tc_dkdv_kernel<true> : tc_dkdv_kernel<false>;
+    auto kern = a.trace ? tc_dkdv_kernel<true, D> : tc_dkdv_kernel<false, D>;
     if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, DKDV_SMEM)) != cudaSuccess) return e;
     dim3 grid(max(a.L, a.k[NOISY] != nullptr ? a.Ln : 0) / TILE, a.Hkv, a.batch * 2);
     kern<<<grid, DKDV_THREADS, DKDV_SMEM, st>>>(maps, a, status);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
   if (passes & BDLM_BWD_PASS_DQ) {
-    auto kern = a.trace ? tc_dq_kernel<true> : tc_dq_kernel<false>;
+    auto kern = a.trace ? tc_dq_kernel<true, D> : tc_dq_kernel<false, D>;
     if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, DQ_SMEM)) != cudaSuccess) return e;
     dim3 grid(max(a.q[CLEAN] != nullptr ? a.Lqc : 0, a.q[NOISY] != nullptr ? a.Ln : 0) / TILE, a.H, a.batch * 2);
     kern<<<grid, BWD_THREADS, DQ_SMEM, st>>>(maps, a, status);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
   return cudaSuccess;
+}
+
+cudaError_t launch_tc_bwd(const KArgs& a, void* extra_ws, int passes, cudaStream_t st) {
+  return a.d == 64 ? launch_tc_bwd_d<64>(a, extra_ws, passes, st) : launch_tc_bwd_d<128>(a, extra_ws, passes, st);
 }
 
 }  // namespace bdlm

@@ -240,13 +240,17 @@ constexpr uint32_t TILE_LO = (2 * PANEL_BYTES) >> 4;   // low-word stride betwee
 // GEMMs over a 128-deep contraction (8 k-slices of 16), issued by the elected lane of a converged warp (see
 // elect_one).  Suffixes: ss = both operands in shared memory, ts = A as bf16 pairs in tensor memory; operands
 // are K-major unless the name says mn/km/mm (B MN-major; A K-major and B MN-major; both MN-major).
+// KS = number of 16-deep slices of the contraction: 8 for a contraction over 128 keys / queries or a head dimension of
+// 128, 4 for a head dimension of 64 (the tile's second 64-column panel is then neither loaded nor read).
+template <int KS = 8>
 __device__ __forceinline__ void gemm_ss_e(uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t acc_first, uint32_t el) {
 #pragma unroll
-  for (int kk = 0; kk < 8; ++kk) mma_ss_e(d, desc64(a_lo + koff(kk)), desc64(b_lo + koff(kk)), idesc, kk == 0 ? acc_first : 1u, el);
+  for (int kk = 0; kk < KS; ++kk) mma_ss_e(d, desc64(a_lo + koff(kk)), desc64(b_lo + koff(kk)), idesc, kk == 0 ? acc_first : 1u, el);
 }
+template <int KS = 8>
 __device__ __forceinline__ void gemm_ts_e(uint32_t d, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc, uint32_t acc_first, uint32_t el) {
 #pragma unroll
-  for (int kk = 0; kk < 8; ++kk) mma_ts_e(d, a_tmem + kk * 8, desc64(b_lo + koff(kk)), idesc, kk == 0 ? acc_first : 1u, el);
+  for (int kk = 0; kk < KS; ++kk) mma_ts_e(d, a_tmem + kk * 8, desc64(b_lo + koff(kk)), idesc, kk == 0 ? acc_first : 1u, el);
 }
 template <int CW>
 __device__ __forceinline__ void gemm_ts_mn_cw_e(uint32_t d, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc, uint32_t acc_first, uint32_t el) {

@@ -39,12 +39,13 @@ EncodeTiledFn encode_fn() {
 
 bool tc_encoder_available() { return encode_fn() != nullptr; }
 
-// [batch, L, heads, 128] bf16 viewed as 3-D (heads*128, L, batch); box = 64 columns x `rows` rows.
+// [batch, L, heads, d] bf16 viewed as 3-D (heads*d, L, batch); box = 64 columns x `rows` rows.
 // Encoding a map costs the host a microsecond or two and a call needs six to eight of them, which shows at sizes
 // where a whole step takes a few milliseconds; a training loop passes the same tensors again and again, so each host
 // thread keeps the maps it encoded last in a small direct-mapped table keyed by (address, shape, box).  A map is a
 // plain 128-byte value that describes addresses and strides only, so a copy of it is as good as a fresh encode.
-bool tc_make_map(CUtensorMap* m, const void* ptr, int heads, int L, int batch, int rows) {
+bool tc_make_map(CUtensorMap* m, const void* ptr, int heads_in, int L, int batch, int rows, int d) {
+  const int heads = heads_in * (d / 64);   // in units of 64-column panels: the map only knows the row length
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr || ptr == nullptr) return false;
   struct Entry { const void* ptr; int heads, L, batch, rows; bool valid; CUtensorMap map; };
@@ -57,8 +58,8 @@ bool tc_make_map(CUtensorMap* m, const void* ptr, int heads, int L, int batch, i
     *m = e.map;
     return true;
   }
-  cuuint64_t gdim[3] = {(cuuint64_t)heads * 128, (cuuint64_t)L, (cuuint64_t)batch};
-  cuuint64_t gstride[2] = {(cuuint64_t)heads * 128 * 2, (cuuint64_t)L * heads * 128 * 2};
+  cuuint64_t gdim[3] = {(cuuint64_t)heads * 64, (cuuint64_t)L, (cuuint64_t)batch};
+  cuuint64_t gstride[2] = {(cuuint64_t)heads * 64 * 2, (cuuint64_t)L * heads * 64 * 2};
   cuuint32_t box[3] = {64, (cuuint32_t)rows, 1};
   cuuint32_t estr[3] = {1, 1, 1};
   CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), gdim, gstride, box, estr,
@@ -72,7 +73,6 @@ bool tc_make_map(CUtensorMap* m, const void* ptr, int heads, int L, int batch, i
 namespace {
 // ---------------------------------------------------------------- forward kernel
 constexpr uint32_t IDESC_QK = make_idesc(128, 128, false, false);
-constexpr uint32_t IDESC_PV = make_idesc(128, 128, false, true);
 constexpr int TILE_BYTES = 2 * PANEL_BYTES;   // 128 x 128 bf16
 
 // Key tiles visible from a run of query rows: a clean segment then a noisy segment, each a run
@@ -115,9 +115,13 @@ constexpr int FWDR_THREADS = 320;                            // 8 softmax warps,
 constexpr int FWDR_BARS = 6 * TILE_BYTES;                    // after Q (2 tiles) and the K/V ring (2 stages x 2 tiles)
 constexpr int FWDR_SMEM = FWDR_BARS + 256 + 1024;
 
-template <bool TR, bool PAIRQ>
+// D = head dimension (128 or 64).  With D = 64 a tile is one 64-column panel: the second panel of every shared-memory
+// tile stays unused, Q K^T contracts over four k-slices and P V produces 64 output columns.
+template <bool TR, bool PAIRQ, int D>
 __global__ void __launch_bounds__(FWDR_THREADS, 1)
 tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restrict__ status) {
+  constexpr uint32_t IDESC_PV = make_idesc(128, D, false, true);
+  constexpr int OPER_BYTES = TILE_BYTES * D / 128;   // bytes TMA delivers per operand tile
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
@@ -163,12 +167,12 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
 
   if (warp == 8) {
     if (lane == 0 && nt > 0) {
-      mbar_expect_tx(bar_q, 2 * TILE_BYTES);
-      tma_load_3d(sQ, &maps.q[qs], bar_q, h0 * 128, q0, b);
-      tma_load_3d(sQ + PANEL_BYTES, &maps.q[qs], bar_q, h0 * 128 + 64, q0, b);
+      mbar_expect_tx(bar_q, 2 * OPER_BYTES);
+      tma_load_3d(sQ, &maps.q[qs], bar_q, h0 * D, q0, b);
+      if (D == 128) tma_load_3d(sQ + PANEL_BYTES, &maps.q[qs], bar_q, h0 * D + 64, q0, b);
       // (rows past the end of the tensor are filled with zeros)
-      tma_load_3d(sQ + TILE_BYTES, &maps.q[qs], bar_q, (h0 + HSTEP) * 128, q0 + QSTEP, b);
-      tma_load_3d(sQ + TILE_BYTES + PANEL_BYTES, &maps.q[qs], bar_q, (h0 + HSTEP) * 128 + 64, q0 + QSTEP, b);
+      tma_load_3d(sQ + TILE_BYTES, &maps.q[qs], bar_q, (h0 + HSTEP) * D, q0 + QSTEP, b);
+      if (D == 128) tma_load_3d(sQ + TILE_BYTES + PANEL_BYTES, &maps.q[qs], bar_q, (h0 + HSTEP) * D + 64, q0 + QSTEP, b);
       bool ok = true;
       for (int t = 0; t < nt && ok; ++t) {
         const int s = t & 1;
@@ -176,13 +180,13 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
         if (!ok) break;
         const int ks = tile_ks(t), k0 = tile_k0(t);
         const uint32_t dK = sK0 + s * 2 * TILE_BYTES, dV = dK + TILE_BYTES;
-        mbar_expect_tx(bar_k_full + 8 * s, TILE_BYTES);
+        mbar_expect_tx(bar_k_full + 8 * s, OPER_BYTES);
         const int krow = ks == CLEAN ? clean_key_row(a, k0) : k0;   // where the tile's first key is stored
-        tma_load_3d(dK, &maps.k[ks], bar_k_full + 8 * s, hk * 128, krow, b);
-        tma_load_3d(dK + PANEL_BYTES, &maps.k[ks], bar_k_full + 8 * s, hk * 128 + 64, krow, b);
-        mbar_expect_tx(bar_v_full + 8 * s, TILE_BYTES);
-        tma_load_3d(dV, &maps.v[ks], bar_v_full + 8 * s, hk * 128, krow, b);
-        tma_load_3d(dV + PANEL_BYTES, &maps.v[ks], bar_v_full + 8 * s, hk * 128 + 64, krow, b);
+        tma_load_3d(dK, &maps.k[ks], bar_k_full + 8 * s, hk * D, krow, b);
+        if (D == 128) tma_load_3d(dK + PANEL_BYTES, &maps.k[ks], bar_k_full + 8 * s, hk * D + 64, krow, b);
+        mbar_expect_tx(bar_v_full + 8 * s, OPER_BYTES);
+        tma_load_3d(dV, &maps.v[ks], bar_v_full + 8 * s, hk * D, krow, b);
+        if (D == 128) tma_load_3d(dV + PANEL_BYTES, &maps.v[ks], bar_v_full + 8 * s, hk * D + 64, krow, b);
       }
     }
   } else if (warp == 9) {
@@ -195,9 +199,9 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
       ok = ok && mbar_wait_abortable(bar_k_full, 0, abort_flag);
       if (ok) {
         tc_fence_after();
-        gemm_ss_e(tmem, qa_lo, k_lo0, IDESC_QK, 0u, el);
+        gemm_ss_e<D / 16>(tmem, qa_lo, k_lo0, IDESC_QK, 0u, el);
         mma_commit_e(bar_s, el);
-        gemm_ss_e(tmem + 128, qb_lo, k_lo0, IDESC_QK, 0u, el);
+        gemm_ss_e<D / 16>(tmem + 128, qb_lo, k_lo0, IDESC_QK, 0u, el);
         mma_commit_e(bar_s + 8, el);
       }
       // O += P V over key half j of the tile: four k-slices of 16 keys
@@ -229,7 +233,7 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
           ok = mbar_wait_timed<TR>(bar_k_full + 8 * (s ^ 1), ((t + 1) >> 1) & 1, abort_flag, w_k);
           if (!ok) break;
           tc_fence_after();
-          gemm_ss_e(tmem, qa_lo, nk_lo, IDESC_QK, 0u, el);
+          gemm_ss_e<D / 16>(tmem, qa_lo, nk_lo, IDESC_QK, 0u, el);
           mma_commit_e(bar_s, el);
         }
         // head B
@@ -244,7 +248,7 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
         mma_commit_e(bar_o + 8, el);
         mma_commit_e(bar_kv_empty + 8 * s, el);
         if (t + 1 < nt) {
-          gemm_ss_e(tmem + 128, qb_lo, nk_lo, IDESC_QK, 0u, el);
+          gemm_ss_e<D / 16>(tmem + 128, qb_lo, nk_lo, IDESC_QK, 0u, el);
           mma_commit_e(bar_s + 8, el);
         }
       }
@@ -311,7 +315,7 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
           if (!ok) break;
           tc_fence_after();
 #pragma unroll 1
-          for (int c = 0; c < 4; ++c) {
+          for (int c = 0; c < D / 32; ++c) {
             uint32_t o[32];
             tmem_ld32(tO + c * 32, o);
             tmem_wait_ld();
@@ -361,9 +365,9 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
     if (ok) {
       tc_fence_after();
       const float inv = l > 0.f ? 1.f / l : 0.f;
-      bf16* orow = a.o[qs] + (((int64_t)b * Lq + row) * a.H + h) * 128;
+      bf16* orow = a.o[qs] + (((int64_t)b * Lq + row) * a.H + h) * D;
 #pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < D / 32; ++c) {
         uint32_t o[32];
         if (nt > 0) { tmem_ld32(tO + c * 32, o); tmem_wait_ld(); }
 #pragma unroll
@@ -399,25 +403,26 @@ bool tc_rows_ok(const KArgs& a) {
 }
 
 bool tc_fwd_supported(const KArgs& a) {
-  return a.d == 128 && tc_rows_ok(a) && encode_fn() != nullptr;
+  return (a.d == 128 || a.d == 64) && tc_rows_ok(a) && encode_fn() != nullptr;
 }
 
-cudaError_t launch_tc_fwd(const KArgs& a, cudaStream_t st) {
+template <int D>
+static cudaError_t launch_tc_fwd_d(const KArgs& a, cudaStream_t st) {
   FwdMaps maps;
   for (int s = 0; s < 2; ++s) {
     // a stream that is left out gets the other stream's tensors as placeholders: its maps are never used
     const int sq = a.q[s] ? s : 1 - s;
-    if (!tc_make_map(&maps.q[s], a.q[sq], a.H, rows_q(a, sq), a.batch, TILE)) return cudaErrorInvalidValue;
+    if (!tc_make_map(&maps.q[s], a.q[sq], a.H, rows_q(a, sq), a.batch, TILE, D)) return cudaErrorInvalidValue;
     const int sk = (s == NOISY && (a.q[NOISY] == nullptr || a.Ln == 0 || !a.diag)) ? CLEAN : s;
-    if (!tc_make_map(&maps.k[s], a.k[sk], a.Hkv, rows_k(a, sk), a.batch, TILE)) return cudaErrorInvalidValue;
-    if (!tc_make_map(&maps.v[s], a.v[sk], a.Hkv, rows_k(a, sk), a.batch, TILE)) return cudaErrorInvalidValue;
+    if (!tc_make_map(&maps.k[s], a.k[sk], a.Hkv, rows_k(a, sk), a.batch, TILE, D)) return cudaErrorInvalidValue;
+    if (!tc_make_map(&maps.v[s], a.v[sk], a.Hkv, rows_k(a, sk), a.batch, TILE, D)) return cudaErrorInvalidValue;
   }
   const int qrows = max(a.q[CLEAN] != nullptr ? a.Lqc : 0, a.q[NOISY] != nullptr ? a.Ln : 0);
   int* status = device_status_ptr();
   if (status == nullptr) return cudaErrorUnknown;
   cudaError_t e;
   if (a.G % 2 == 0) {   // two heads of one KV group per CTA, one softmax warpgroup per head
-    auto kern = a.trace ? tc_fwdr_kernel<true, false> : tc_fwdr_kernel<false, false>;
+    auto kern = a.trace ? tc_fwdr_kernel<true, false, D> : tc_fwdr_kernel<false, false, D>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, FWDR_SMEM);
     if (e != cudaSuccess) return e;
     dim3 grid(qrows / TILE, a.H / 2, a.batch * 2);
@@ -425,12 +430,16 @@ cudaError_t launch_tc_fwd(const KArgs& a, cudaStream_t st) {
     return cudaGetLastError();
   }
   // odd group size: two consecutive query tiles of one head per CTA
-  auto kern = a.trace ? tc_fwdr_kernel<true, true> : tc_fwdr_kernel<false, true>;
+  auto kern = a.trace ? tc_fwdr_kernel<true, true, D> : tc_fwdr_kernel<false, true, D>;
   e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, FWDR_SMEM);
   if (e != cudaSuccess) return e;
   dim3 grid((qrows / TILE + 1) / 2, a.H, a.batch * 2);
   kern<<<grid, FWDR_THREADS, FWDR_SMEM, st>>>(maps, a, status);
   return cudaGetLastError();
+}
+
+cudaError_t launch_tc_fwd(const KArgs& a, cudaStream_t st) {
+  return a.d == 64 ? launch_tc_fwd_d<64>(a, st) : launch_tc_fwd_d<128>(a, st);
 }
 
 }  // namespace bdlm

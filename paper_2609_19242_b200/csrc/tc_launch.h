@@ -10,8 +10,8 @@ namespace bdlm {
 int* device_status_ptr();
 
 bool tc_encoder_available();
-// Tensor map over a [batch, L, heads, 128] bf16 tensor, box = 64 columns x `rows` rows, 128-byte swizzle.
-bool tc_make_map(CUtensorMap* m, const void* ptr, int heads, int L, int batch, int rows);
+// Tensor map over a [batch, L, heads, d] bf16 tensor (d = 64 or 128), box = 64 columns x `rows` rows, 128-byte swizzle.
+bool tc_make_map(CUtensorMap* m, const void* ptr, int heads, int L, int batch, int rows, int d);
 
 bool tc_rows_ok(const KArgs& a);
 bool tc_fwd_supported(const KArgs& a);

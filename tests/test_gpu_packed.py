@@ -313,3 +313,11 @@ def test_clean_key_tiles_that_no_query_sees(single_pass):
                           do_noisy=x["do_noisy"], block_prefix=prefix)
     for i, n in ((1, "dk_clean"), (2, "dv_clean"), (3, "dq_noisy"), (4, "dk_noisy"), (5, "dv_noisy")):
         assert pu.rel_l2(synth.to_f64(g_full[i]), ref[n]) <= pu.TOL_GRAD, n
+
+
+def test_packed_form_with_head_dimension_64_on_the_tensor_core_kernels():
+    rng = np.random.default_rng(3)
+    t = _draw(31, 1, 512, 256, 256, 4, 2, 64)
+    _run_and_check(t, 32, binding.IMPL_TCGEN05, prefix=sorted(int(v) for v in rng.integers(0, 513, size=8)), pos0=128)
+    _run_and_check(t, 32, binding.IMPL_TCGEN05, prefix=sorted(int(v) for v in rng.integers(0, 513, size=8)), pos0=128,
+                   single_pass=True)

@@ -291,3 +291,34 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_stays_usable()
     with pytest.raises(binding.BdlmError):
         binding.bdlm_selftest_wait_timeout(0)
     pu.check_full(Workload("after_timeout", 1, 2, 1, 128, 256, 32), binding.IMPL_AUTO, check_bwd=False)
+
+
+@pytest.mark.parametrize("w,mode", [(synth.WORKLOADS["tiny"], 0),                                  # the BASELINE tiny configuration: MHA, M = 16
+                                    (Workload("d64_gqa", 2, 4, 2, 64, 384, 32), 0),
+                                    (Workload("d64_g4_m256", 1, 4, 1, 64, 512, 256), 1),
+                                    (Workload("d64_g3_window", 1, 3, 1, 64, 640, 64, window=200), 0)],
+                         ids=lambda x: x.name if hasattr(x, "name") else str(x))
+def test_head_dimension_64_on_the_tensor_core_kernels(w, mode):
+    """d = 64 on the tcgen05 kernels (one 64-column panel per operand tile, four k-slices over the head dimension):
+    forward, two-pass backward and fused backward, forced with impl = 2 so that a fallback would show as an error."""
+    pu.check_full(w, binding.IMPL_TCGEN05, mode=mode)
+    pu.check_full(w, binding.IMPL_TCGEN05, mode=mode, single_pass=True)
+    # the portable kernels on the same inputs stay available as the cross-check
+    pu.check_full(w, binding.IMPL_PORTABLE, mode=mode)
+
+
+def test_head_dimension_64_default_dispatch_is_the_tensor_core_path():
+    """impl = 0 takes the tensor-core kernels for d = 64 (bitwise the impl = 2 results), and the packed form does too."""
+    w = Workload("d64_auto", 1, 4, 2, 64, 256, 16)
+    g = pu.to_cuda(synth.make_inputs(w, "cpu"))
+    M = w.block_size
+    a = pu.gpu_fwd(g, M)
+    b = pu.gpu_fwd(g, M, impl=binding.IMPL_TCGEN05)
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
+    ga = pu.gpu_bwd(g, a, M)
+    gb = pu.gpu_bwd(g, a, M, impl=binding.IMPL_TCGEN05)
+    torch.cuda.synchronize()
+    for x, y in zip(ga, gb):
+        assert torch.equal(x, y)
+    assert binding.bdlm_get_device_status() == 0
