@@ -84,7 +84,7 @@ void fill(KArgs& a, const bdlm_params* p, const bdlm_packed_geometry* g) {
     const int dev = current_device();
     a.trace = dev >= 0 ? g_trace[dev] : nullptr;
   }
-  a.single_pass = 0; a.dq32[0] = a.dq32[1] = nullptr;
+  a.single_pass = 0; a.dq32[0] = a.dq32[1] = nullptr; a.dq32_rows[0] = a.dq32_rows[1] = 0;
 }
 
 bool is_sm100() {

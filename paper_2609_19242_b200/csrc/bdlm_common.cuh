@@ -50,7 +50,8 @@ struct KArgs {
   __nv_bfloat16* dv[2];
   unsigned long long* trace;   // optional cycle counters (bdlm_set_trace_buffer), else nullptr
   int single_pass;             // backward: the fused kernel forms dQ^T per step and adds it into dq32 by TMA bulk add-reductions
-  float* dq32[2];              // fp32 dQ accumulators [batch, H, rows, 128] (fused backward), else nullptr
+  float* dq32[2];              // fp32 dQ accumulators [batch, H, dq32_rows, 128] (fused backward), else nullptr
+  int dq32_rows[2];            // their row counts: the stream's query rows rounded up to the 64-row step of the fused kernel
 };
 
 __host__ __device__ __forceinline__ int rows_q(const KArgs& a, int qs) { return qs == CLEAN ? a.Lqc : a.Ln; }

@@ -193,9 +193,22 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
     // the LSE and D rows of a step are fetched one step ahead, so that the round trip to global memory lies under
     // the waits for the ring stages instead of in front of the stage's full barrier
     auto fetch_rows = [&](const QStep& s, float4& z, float4& dd) {
-      const int64_t row0 = ((int64_t)b * a.H + s.h) * rows_q(a, s.qs) + s.q0;
-      z = reinterpret_cast<const float4*>(a.lse[s.qs] + row0)[lane];
-      dd = reinterpret_cast<const float4*>(a.dsum[s.qs] + row0)[lane];
+      const int Lq = rows_q(a, s.qs);
+      const int64_t row0 = ((int64_t)b * a.H + s.h) * Lq + s.q0;
+      if ((Lq & 3) == 0 && s.q0 + TILE <= Lq) {
+        z = reinterpret_cast<const float4*>(a.lse[s.qs] + row0)[lane];
+        dd = reinterpret_cast<const float4*>(a.dsum[s.qs] + row0)[lane];
+      } else {   // a tile that runs past the end of the tensor (or rows that are not 16-byte aligned): P = 0 and D = 0 there
+        float zz[4], ds[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const bool in = s.q0 + 4 * lane + e < Lq;
+          zz[e] = in ? a.lse[s.qs][row0 + 4 * lane + e] : INFINITY;
+          ds[e] = in ? a.dsum[s.qs][row0 + 4 * lane + e] : 0.f;
+        }
+        z = make_float4(zz[0], zz[1], zz[2], zz[3]);
+        dd = make_float4(ds[0], ds[1], ds[2], ds[3]);
+      }
     };
     float4 z_next = make_float4(0.f, 0.f, 0.f, 0.f), d_next = z_next;
     if (nsteps > 0) fetch_rows(step_cur(), z_next, d_next);
@@ -462,7 +475,7 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
 #pragma unroll
           for (int e = 0; e < 32; ++e) v[e] = 0u;
         }
-        store_row_chunk(dst + c * 32, v, sc);
+        if (k0_row + r < L) store_row_chunk(dst + c * 32, v, sc);   // key rows past the end of the tensor are not written
       }
     }
   }
@@ -527,10 +540,11 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
   {
     int lo_f, hi_f, lo_l, hi_l;
     visible_interval(a, qs, 0, q0, lo_f, hi_f);
-    visible_interval(a, qs, 0, q0 + TILE - 1, lo_l, hi_l);
+    const int q_last = min(q0 + TILE, L) - 1;
+    visible_interval(a, qs, 0, q_last, lo_l, hi_l);
     lo0 = lo_f; lo_last0 = lo_l; hi_first0 = hi_f; nt0 = hi_l > lo_f ? (hi_l - lo_f + TILE - 1) / TILE : 0;
     visible_interval(a, qs, 1, q0, lo_f, hi_f);
-    visible_interval(a, qs, 1, q0 + TILE - 1, lo_l, hi_l);
+    visible_interval(a, qs, 1, q_last, lo_l, hi_l);
     lo1 = lo_f; lo_last1 = lo_l; hi_first1 = hi_f; nt1 = hi_l > lo_f ? (hi_l - lo_f + TILE - 1) / TILE : 0;
   }
   const int nsteps = nt0 + nt1;
@@ -648,15 +662,16 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
     const int row = q0 + r;
     const uint32_t tl = tmem + ((uint32_t)((warp & 3) * 32) << 16);
     const int c0 = w * 64;
+    const bool row_ok = row < L;   // a row past the end of the tensor: P = 0, nothing read or written
     float lse2 = INFINITY, dsum = 0.f;
-    {
+    int rlo0 = 0, rhi0 = 0, rlo1 = 0, rhi1 = 0;
+    if (row_ok) {
       const float z = a.lse[qs][((int64_t)b * a.H + h) * L + row];
       if (isfinite(z)) lse2 = z * LOG2E;
       dsum = a.dsum[qs][((int64_t)b * a.H + h) * L + row];
+      visible_interval(a, qs, 0, row, rlo0, rhi0);
+      visible_interval(a, qs, 1, row, rlo1, rhi1);
     }
-    int rlo0, rhi0, rlo1, rhi1;
-    visible_interval(a, qs, 0, row, rlo0, rhi0);
-    visible_interval(a, qs, 1, row, rlo1, rhi1);
     bool ok = true;
     long long w_s = 0, w_dp = 0, c_ld = 0, c_exp = 0, c_ds = 0;
     Stopwatch<TR> sw;
@@ -687,7 +702,8 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
       tc_fence_before();
       mbar_arrive(bar_sfree);
       sw.lap(c_ld);
-      const bool need_mask = ks == 0 ? (k0 < lo_last0 || k0 + TILE > hi_first0) : (k0 < lo_last1 || k0 + TILE > hi_first1);
+      const bool need_mask = (ks == 0 ? (k0 < lo_last0 || k0 + TILE > hi_first0) : (k0 < lo_last1 || k0 + TILE > hi_first1)) ||
+                             q0 + TILE > L;
       if (!need_mask) {
 #pragma unroll
         for (int c8 = 0; c8 < 8; ++c8) {
@@ -756,7 +772,7 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
 #pragma unroll
           for (int e = 0; e < 32; ++e) v[e] = 0u;
         }
-        store_row_chunk(dst + c * 32, v, a.scale);
+        if (row_ok) store_row_chunk(dst + c * 32, v, a.scale);
       }
     }
   }
@@ -900,9 +916,16 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
     // the LSE (lanes 0-15) and D (lanes 16-31) rows of a step are fetched one step ahead, so that the round trip
     // to global memory lies under the waits for the ring stages instead of in front of the stage's full barrier
     auto fetch_rows = [&](const QStep& s) {
-      const int64_t row0 = ((int64_t)b * a.H + s.h) * rows_q(a, s.qs) + s.q0;
+      const int Lq = rows_q(a, s.qs);
+      const int64_t row0 = ((int64_t)b * a.H + s.h) * Lq + s.q0;
       const float* src = (lane < 16 ? a.lse[s.qs] : a.dsum[s.qs]) + row0;
-      return reinterpret_cast<const float4*>(src)[lane & 15];
+      if ((Lq & 3) == 0 && s.q0 + HT <= Lq) return reinterpret_cast<const float4*>(src)[lane & 15];
+      // a step that runs past the end of the tensor (or rows that are not 16-byte aligned): P = 0 and D = 0 there
+      const float fill = lane < 16 ? INFINITY : 0.f;
+      float v[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) v[e] = (s.q0 + 4 * (lane & 15) + e < Lq) ? src[4 * (lane & 15) + e] : fill;
+      return make_float4(v[0], v[1], v[2], v[3]);
     };
     float4 rows_next = make_float4(0.f, 0.f, 0.f, 0.f);
     if (nsteps > 0) rows_next = fetch_rows(step_cur());
@@ -1057,7 +1080,7 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
       }
       const long long t0 = tick<TR>();
       if (ok) tc_fence_after();
-      float* dst = a.dq32[st.qs] + (((int64_t)b * a.H + st.h) * rows_q(a, st.qs) + st.q0) * 128;
+      float* dst = a.dq32[st.qs] + (((int64_t)b * a.H + st.h) * a.dq32_rows[st.qs] + st.q0) * 128;
       uint32_t v[64];
       if (ok) {   // the whole tile into registers first: the tensor core gets its columns back at once
         uint32_t (*c)[32] = reinterpret_cast<uint32_t (*)[32]>(v);
@@ -1252,7 +1275,7 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
 #pragma unroll
           for (int e = 0; e < 32; ++e) v[e] = 0u;
         }
-        store_row_chunk(dst + c * 32, v, sc);
+        if (k0_row + r < L) store_row_chunk(dst + c * 32, v, sc);   // key rows past the end of the tensor are not written
       }
     }
   }
@@ -1265,14 +1288,15 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
 // fp32 dQ accumulator [batch, H, rows, 128] -> bf16 dQ [batch, rows, H, D]; one warp per row (D = 64: the first 64
 // of the accumulator row's 128 floats)
 template <int D>
-__global__ void __launch_bounds__(256) dq_convert_kernel(const float* __restrict__ src, bf16* __restrict__ dst, int batch, int H, int rows) {
+__global__ void __launch_bounds__(256) dq_convert_kernel(const float* __restrict__ src, bf16* __restrict__ dst, int batch, int H, int rows,
+                                                         int src_rows) {
   const int lane = threadIdx.x & 31;
   const int64_t n = (int64_t)batch * rows * H;
   for (int64_t o = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5); o < n; o += (int64_t)gridDim.x * 8) {
     const int h = (int)(o % H);
     const int64_t bl = o / H;
     const int l = (int)(bl % rows), b = (int)(bl / rows);
-    const float* row = src + (((int64_t)b * H + h) * rows + l) * 128;
+    const float* row = src + (((int64_t)b * H + h) * src_rows + l) * 128;
     if (D == 128) {
       const float4 u = reinterpret_cast<const float4*>(row)[lane];
       uint2 v;
@@ -1287,6 +1311,8 @@ __global__ void __launch_bounds__(256) dq_convert_kernel(const float* __restrict
 
 }  // namespace
 
+static size_t pad64(size_t rows) { return (rows + 63) / 64 * 64; }
+
 bool tc_bwd_supported(const KArgs& a) {
   return (a.d == 128 || a.d == 64) && tc_rows_ok(a) && tc_encoder_available();
 }
@@ -1295,15 +1321,16 @@ size_t tc_bwd_fused_workspace(const bdlm_params* p, const bdlm_packed_geometry* 
   if ((p->d != 128 && p->d != 64) || p->impl == 1) return 0;
   const size_t rows_c = g != nullptr ? (size_t)g->Lq_clean : (size_t)p->L;
   const size_t rows_n = g != nullptr ? (size_t)g->n_blocks * p->block_size : (size_t)p->L;
-  if (p->L % TILE != 0 || rows_c % TILE != 0 || rows_n % TILE != 0) return 0;   // such shapes take the mma.sync kernels
-  return (rows_c + rows_n) * p->batch * p->H * 128 * sizeof(float);
+  // rows rounded up to the kernel's 64-row steps: a reduction always covers a whole step
+  return (pad64(rows_c) + pad64(rows_n)) * p->batch * p->H * 128 * sizeof(float);
 }
 
 template <int D>
 static cudaError_t launch_tc_bwd_d(const KArgs& a_in, void* extra_ws, int passes, cudaStream_t st) {
   KArgs a = a_in;
-  const size_t dq32_elems[2] = {a.q[CLEAN] != nullptr ? (size_t)a.batch * a.H * a.Lqc * 128 : 0,
-                                a.q[NOISY] != nullptr ? (size_t)a.batch * a.H * a.Ln * 128 : 0};
+  a.dq32_rows[CLEAN] = a.q[CLEAN] != nullptr ? (int)pad64(a.Lqc) : 0;
+  a.dq32_rows[NOISY] = a.q[NOISY] != nullptr ? (int)pad64(a.Ln) : 0;
+  const size_t dq32_elems[2] = {(size_t)a.batch * a.H * a.dq32_rows[CLEAN] * 128, (size_t)a.batch * a.H * a.dq32_rows[NOISY] * 128};
   if (a.single_pass) {
     a.dq32[0] = static_cast<float*>(extra_ws);
     a.dq32[1] = a.dq32[0] + dq32_elems[0];
@@ -1328,12 +1355,12 @@ static cudaError_t launch_tc_bwd_d(const KArgs& a_in, void* extra_ws, int passes
       if ((e = cudaMemsetAsync(a.dq32[0], 0, (dq32_elems[0] + dq32_elems[1]) * sizeof(float), st)) != cudaSuccess) return e;
       auto kern = a.trace ? tc_bwdf_kernel<true, D> : tc_bwdf_kernel<false, D>;
       if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, BF_SMEM)) != cudaSuccess) return e;
-      dim3 grid(max(a.L, a.k[NOISY] != nullptr ? a.Ln : 0) / TILE, a.Hkv, a.batch * 2);
+      dim3 grid((max(a.L, a.k[NOISY] != nullptr ? a.Ln : 0) + TILE - 1) / TILE, a.Hkv, a.batch * 2);
       kern<<<grid, BF_THREADS, BF_SMEM, st>>>(maps, a, status);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
       for (int s2 = 0; s2 < 2; ++s2) {
         if (dq32_elems[s2] == 0) continue;
-        dq_convert_kernel<D><<<device_sm_count() * 8, 256, 0, st>>>(a.dq32[s2], a.dq[s2], a.batch, a.H, rows_q(a, s2));
+        dq_convert_kernel<D><<<device_sm_count() * 8, 256, 0, st>>>(a.dq32[s2], a.dq[s2], a.batch, a.H, rows_q(a, s2), a.dq32_rows[s2]);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
       }
     }
@@ -1342,14 +1369,14 @@ static cudaError_t launch_tc_bwd_d(const KArgs& a_in, void* extra_ws, int passes
   if (passes & BDLM_BWD_PASS_DKDV) {
     auto kern = a.trace ? tc_dkdv_kernel<true, D> : tc_dkdv_kernel<false, D>;
     if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, DKDV_SMEM)) != cudaSuccess) return e;
-    dim3 grid(max(a.L, a.k[NOISY] != nullptr ? a.Ln : 0) / TILE, a.Hkv, a.batch * 2);
+    dim3 grid((max(a.L, a.k[NOISY] != nullptr ? a.Ln : 0) + TILE - 1) / TILE, a.Hkv, a.batch * 2);
     kern<<<grid, DKDV_THREADS, DKDV_SMEM, st>>>(maps, a, status);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
   if (passes & BDLM_BWD_PASS_DQ) {
     auto kern = a.trace ? tc_dq_kernel<true, D> : tc_dq_kernel<false, D>;
     if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, DQ_SMEM)) != cudaSuccess) return e;
-    dim3 grid(max(a.q[CLEAN] != nullptr ? a.Lqc : 0, a.q[NOISY] != nullptr ? a.Ln : 0) / TILE, a.H, a.batch * 2);
+    dim3 grid((max(a.q[CLEAN] != nullptr ? a.Lqc : 0, a.q[NOISY] != nullptr ? a.Ln : 0) + TILE - 1) / TILE, a.H, a.batch * 2);
     kern<<<grid, BWD_THREADS, DQ_SMEM, st>>>(maps, a, status);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }

@@ -280,7 +280,7 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const bool need_mask = sch.need_mask(ks, k0) || (PAIRQ && q0 + QROWS > Lq);
+      const bool need_mask = sch.need_mask(ks, k0) || q0 + QROWS > Lq;   // rows past the end of the tensor see nothing
       const int vlo = (ks == 0 ? rlo0 : rlo1) - k0, vhi = (ks == 0 ? rhi0 : rhi1) - k0;
       // the whole row of the tile in registers: one pass over S
       const long long tp0 = tick<TR>();
@@ -394,11 +394,13 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
 
 }  // namespace
 
-// every tensor a tensor-core kernel touches must have a multiple of 128 rows
+// Row counts need not be multiples of the 128-row tile: TMA fills the rows of a tile that lie past the end of a tensor
+// with zeros, the masks never show a key past the end, and rows past the end are neither read from the per-row arrays
+// nor written.  Only the gathered K/V order keeps its own rule (chunks of a multiple of 128 rows: checked at the boundary).
 bool tc_rows_ok(const KArgs& a) {
-  if (a.L % TILE != 0) return false;
-  if (a.q[CLEAN] != nullptr && (a.Lqc % TILE != 0 || a.Lqc == 0)) return false;
-  if (a.q[NOISY] != nullptr && (a.Ln % TILE != 0 || a.Ln == 0)) return false;
+  if (a.L <= 0) return false;
+  if (a.q[CLEAN] != nullptr && a.Lqc <= 0) return false;
+  if (a.q[NOISY] != nullptr && a.Ln <= 0) return false;
   return true;
 }
 
@@ -425,7 +427,7 @@ static cudaError_t launch_tc_fwd_d(const KArgs& a, cudaStream_t st) {
     auto kern = a.trace ? tc_fwdr_kernel<true, false, D> : tc_fwdr_kernel<false, false, D>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, FWDR_SMEM);
     if (e != cudaSuccess) return e;
-    dim3 grid(qrows / TILE, a.H / 2, a.batch * 2);
+    dim3 grid((qrows + TILE - 1) / TILE, a.H / 2, a.batch * 2);
     kern<<<grid, FWDR_THREADS, FWDR_SMEM, st>>>(maps, a, status);
     return cudaGetLastError();
   }
@@ -433,7 +435,7 @@ static cudaError_t launch_tc_fwd_d(const KArgs& a, cudaStream_t st) {
   auto kern = a.trace ? tc_fwdr_kernel<true, true, D> : tc_fwdr_kernel<false, true, D>;
   e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, FWDR_SMEM);
   if (e != cudaSuccess) return e;
-  dim3 grid((qrows / TILE + 1) / 2, a.H, a.batch * 2);
+  dim3 grid(((qrows + TILE - 1) / TILE + 1) / 2, a.H, a.batch * 2);
   kern<<<grid, FWDR_THREADS, FWDR_SMEM, st>>>(maps, a, status);
   return cudaGetLastError();
 }

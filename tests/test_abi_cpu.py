@@ -87,10 +87,12 @@ def test_workspace_size_formula():
     acc = 2 * 2 * 8 * 512 * 128 * 4
     assert mk(False) == d_rows and mk(True) == d_rows + acc and mk(None) == d_rows + acc
     assert mk(None, impl=binding.IMPL_PORTABLE) == d_rows
+    # a length that is no multiple of the fused kernel's 64-row steps: the accumulators are padded to whole steps
     ragged = binding.make_params(1, 160, 32, 4, 2, 128, bwd_single_pass=True)
-    assert binding.bdlm_workspace_bytes(ragged, binding.BDLM_WS_BWD) < 2 * 160 * 4 * 128 * 4
+    assert binding.bdlm_workspace_bytes(ragged, binding.BDLM_WS_BWD) == 2 * 160 * 4 * 4 + 2 * 192 * 4 * 128 * 4
+    # head dimension 64 takes the tensor-core kernels too; its accumulator rows keep 128 floats
     d64 = binding.make_params(1, 256, 16, 4, 2, 64, bwd_single_pass=None)
-    assert binding.bdlm_workspace_bytes(d64, binding.BDLM_WS_BWD) == 2 * 4 * 256 * 4
+    assert binding.bdlm_workspace_bytes(d64, binding.BDLM_WS_BWD) == 2 * 4 * 256 * 4 + 2 * 256 * 4 * 128 * 4
     # a forced fused backward refuses a workspace that holds only the D rows; the automatic mode accepts it
     ok = ctypes.c_void_p(0x1000)
     forced = binding.make_params(2, 512, 32, 8, 2, 128, bwd_single_pass=True)

@@ -41,12 +41,21 @@ def test_random_plain_configurations(case):
     pu.check_full(w, binding.IMPL_AUTO, mode=mode)
 
 
-@pytest.mark.parametrize("case", [c for c in _plain_cases(24, 2024) if c[0].d == 128 and c[0].L % 128 == 0],
-                         ids=lambda c: f"{c[0].name}-L{c[0].L}-M{c[0].block_size}-H{c[0].H}/{c[0].H_kv}-w{c[0].window}-m{c[1]}")
+@pytest.mark.parametrize("case", _plain_cases(24, 2024),
+                         ids=lambda c: f"{c[0].name}-L{c[0].L}-M{c[0].block_size}-H{c[0].H}/{c[0].H_kv}-d{c[0].d}-w{c[0].window}-m{c[1]}")
 def test_random_plain_configurations_fused_backward(case):
-    """The tensor-core shaped cases again through the fused one-kernel backward."""
+    """Every case again through the fused one-kernel backward, forced onto the tensor-core kernels (head dimension 64
+    and lengths that are no multiple of the 128-row tile included)."""
     w, mode = case
-    pu.check_full(w, binding.IMPL_AUTO, mode=mode, single_pass=True)
+    pu.check_full(w, binding.IMPL_TCGEN05, mode=mode, single_pass=True)
+
+
+@pytest.mark.parametrize("case", _plain_cases(24, 2024),
+                         ids=lambda c: f"{c[0].name}-L{c[0].L}-M{c[0].block_size}-H{c[0].H}/{c[0].H_kv}-d{c[0].d}-w{c[0].window}-m{c[1]}")
+def test_random_plain_configurations_portable_kernels(case):
+    """The mma.sync kernels stay the explicit cross-check (impl = 1) now that the default never reaches them."""
+    w, mode = case
+    pu.check_full(w, binding.IMPL_PORTABLE, mode=mode)
 
 
 def _larger_cases(n, seed):

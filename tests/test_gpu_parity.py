@@ -322,3 +322,47 @@ def test_head_dimension_64_default_dispatch_is_the_tensor_core_path():
     for x, y in zip(ga, gb):
         assert torch.equal(x, y)
     assert binding.bdlm_get_device_status() == 0
+
+
+@pytest.mark.parametrize("w,mode", [(Workload("ragged_tail_tc", 1, 2, 1, 64, 200, 8), 0),          # one full tile + 72 rows
+                                    (Workload("ragged_short_tc", 1, 4, 2, 128, 40, 8), 0),         # less than one tile
+                                    (Workload("ragged_w100_tc", 1, 4, 2, 128, 456, 8, window=100), 0),
+                                    (Workload("ragged_odd_tc", 2, 3, 1, 128, 322, 7), 1),          # rows not 16-byte aligned in LSE / D
+                                    (Workload("ragged_m1_tc", 1, 2, 2, 64, 130, 1), 0),
+                                    (Workload("ragged_bigblock_tc", 1, 4, 1, 128, 600, 300), 1)],
+                         ids=lambda x: x.name if hasattr(x, "name") else str(x))
+def test_lengths_that_are_no_multiple_of_the_tile_on_the_tensor_core_kernels(w, mode):
+    """TMA zero-fills the part of a tile past the end of a tensor; keys past the end are never visible, rows past the
+    end are neither read from LSE / D nor written.  Forced with impl = 2: forward, two-pass and fused backward."""
+    pu.check_full(w, binding.IMPL_TCGEN05, mode=mode)
+    pu.check_full(w, binding.IMPL_TCGEN05, mode=mode, single_pass=True)
+
+
+def test_ragged_outputs_do_not_touch_memory_past_the_tensors():
+    """Outputs and gradients sit inside larger buffers filled with a sentinel: nothing past the last real row moves."""
+    w = Workload("ragged_guard", 1, 4, 2, 128, 200, 8)
+    g = pu.to_cuda(synth.make_inputs(w, "cpu"))
+    M, L = w.block_size, w.L
+    pad = 64
+
+    def guarded(like, lse=False):
+        shape = (like.shape[0], like.shape[1], L + pad) if lse else (like.shape[0] * (L + pad),) + tuple(like.shape[2:])
+        return torch.full(shape, 7.0, dtype=like.dtype, device="cuda")
+
+    bufs_o = [guarded(g["q_clean"]), torch.full((w.batch * w.H * L + pad,), 7.0, device="cuda"),
+              guarded(g["q_noisy"]), torch.full((w.batch * w.H * L + pad,), 7.0, device="cuda")]
+    out = (bufs_o[0][:L].view(1, L, w.H, w.d), bufs_o[1][:w.H * L].view(1, w.H, L),
+           bufs_o[2][:L].view(1, L, w.H, w.d), bufs_o[3][:w.H * L].view(1, w.H, L))
+    binding.bdlm_attn_fwd(*[g[n] for n in pu.NAMES6], M, out=out, impl=binding.IMPL_TCGEN05)
+    gb = [guarded(g[n]) for n in pu.NAMES6]
+    grads = tuple(b[:L].view(1, L, g[n].shape[2], w.d) for b, n in zip(gb, pu.NAMES6))
+    for sp in (False, True):
+        binding.bdlm_attn_bwd(*[g[n] for n in pu.NAMES6], out[0], out[1], out[2], out[3], g["do_clean"], g["do_noisy"], M,
+                              out=grads, impl=binding.IMPL_TCGEN05, single_pass=sp)
+        torch.cuda.synchronize()
+        assert binding.bdlm_get_device_status() == 0
+        for b in (bufs_o[0], bufs_o[2]) + tuple(gb):
+            assert float((b[L:].float() - 7.0).abs().max()) == 0.0
+        for b in (bufs_o[1], bufs_o[3]):
+            assert float((b[w.H * L:] - 7.0).abs().max()) == 0.0
+        assert torch.isfinite(grads[0].float()).all()
