@@ -412,11 +412,11 @@ def sharded_forward_leg(run, peaks, steps, warmup):
             "max_abs_diff_vs_unsharded_forward": diff}
 
 
-def linear_ce_leg(binding, peaks, steps, warmup):
+def linear_ce_leg(binding, peaks, steps, warmup, name="lce_8k"):
     """The loss head after the last layer (token-chunked linear cross-entropy) on the Llama-3-8B-shaped workload:
     forward (projection with the log-sum-exp in the GEMM's epilogue) and backward (logits again + dz, dH, dW), timed
     separately with events.  Counted FLOPs: 2 T D V forward, 4 T D V backward (the recomputed logits are not counted)."""
-    w = synth.LCE_WORKLOADS["lce_8k"]
+    w = synth.LCE_WORKLOADS[name]
     g = synth.make_lce_inputs(w, "cuda")
     pf = binding.make_lce_params(w.T, w.D, w.V)
     ws_f = torch.empty(binding.bdlm_linear_ce_workspace_bytes(pf, binding.LCE_WS_FWD), dtype=torch.uint8, device="cuda")
@@ -666,6 +666,7 @@ def main():
                     help="backward: one fused kernel (dQ through fp32 add-reductions) or the bitwise reproducible two-pass path")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--linear-ce-only", action="store_true", help="run only the linear cross-entropy leg and print its JSON")
+    ap.add_argument("--lce-workload", default="lce_8k", choices=sorted(synth.LCE_WORKLOADS))
     ap.add_argument("--no-other-configs", dest="other_configs", action="store_false",
                     help="skip the csbp128k / 256k / block-size legs that the default 32k run appends")
     args = ap.parse_args()
@@ -678,7 +679,7 @@ def main():
         if args.linear_ce_only:
             from paper_2609_19242_b200 import binding
             torch.cuda.set_device(0)
-            print(json.dumps({"linear_ce": linear_ce_leg(binding, load_peaks(), args.steps, args.warmup)}), flush=True)
+            print(json.dumps({"linear_ce": linear_ce_leg(binding, load_peaks(), args.steps, args.warmup, args.lce_workload)}), flush=True)
             return
         run_ours(args, w)
 

@@ -130,13 +130,41 @@ __device__ __forceinline__ void visible_queries_of_clean_key(const KArgs& a, int
   }
 }
 
+// Number of SMs of the current device (cached per device ordinal; 1 if the query fails).
+int device_sm_count();
+
+// The tensor-core kernels run one CTA per (tile, head or head pair, batch element x stream) on a one-dimensional grid;
+// CTAs start in the order of their index.  The work of a tile grows linearly with its position (appendix B, Eq.
+// block-work-by-position), and x counts tiles from the heaviest down.  Two orders:
+//   tile_major = 0   x fastest: the CTAs running at one time are neighbouring tiles of one head, so they walk the same
+//                    Q / dO / K / V tiles (and, in the fused backward, the same dQ accumulator tiles) together;
+//   tile_major = 1   x slowest: the heaviest tiles of every head, batch element and stream start first -- longest job
+//                    first over the whole launch.  Chosen by the launchers when the heaviest tile is a sizeable part of
+//                    the ideal duration of the launch (short sequences), where the first order would start the heavy
+//                    tiles of the second and later batch elements too late.
+struct TileGrid { int nx, ny, nz, tile_major; };
+__device__ __forceinline__ void tile_grid_decode(const TileGrid& g, int& x, int& y, int& z) {
+  int i = blockIdx.x;
+  if (!g.tile_major) { x = i % g.nx; i /= g.nx; y = i % g.ny; z = i / g.ny; }
+  else { const int c = g.ny * g.nz; x = i / c; i -= x * c; y = i % g.ny; z = i / g.ny; }
+}
+inline TileGrid make_tile_grid(int nx, int ny, int nz) {
+  TileGrid g = {nx, ny, nz, 0};
+  // heaviest tile ~ nx units, whole launch ~ ny nz nx (nx + 1) / 2 units over the device's SMs: tile-major when the
+  // heaviest tile exceeds a fifth of the ideal duration
+  g.tile_major = (10LL * device_sm_count() > (long long)ny * nz * (nx + 1)) ? 1 : 0;
+  return g;
+}
+// Number of CTAs, or 0 if it does not fit a grid dimension.
+inline unsigned tile_grid_blocks(const TileGrid& g) {
+  const long long n = (long long)g.nx * g.ny * g.nz;
+  return n > 0x7fffffffLL ? 0u : (unsigned)n;
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
-
-// Number of SMs of the current device (cached per device ordinal; 1 if the query fails).
-int device_sm_count();
 
 // Launchers (host).  Each enqueues on `st` and returns the launch's cudaError_t.
 cudaError_t launch_portable_fwd(const KArgs& a, cudaStream_t st);

@@ -110,7 +110,7 @@ struct StepWalk {
 
 template <bool TR, int D>
 __global__ void __launch_bounds__(DKDV_THREADS, 1)
-tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restrict__ status) {
+tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, const TileGrid tg, int* __restrict__ status) {
   constexpr uint32_t IDESC_KM = idesc_km(D);
   constexpr int OPER_BYTES = TILE_BYTES * D / 128;   // bytes TMA delivers per operand tile (D = 64: one panel)
   extern __shared__ __align__(1024) uint8_t sm[];
@@ -126,8 +126,10 @@ tc_dkdv_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + DKDV_BARS + 128);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + DKDV_BARS + 136);
 
-  const int ks = blockIdx.z & 1, b = blockIdx.z >> 1, hk = blockIdx.y;
-  const int k0_row = blockIdx.x * TILE;   // the tile's first key in memory; key tile 0 has the most query tiles: scheduled first
+  int bx, by, bz;
+  tile_grid_decode(tg, bx, by, bz);
+  const int ks = bz & 1, b = bz >> 1, hk = by;
+  const int k0_row = bx * TILE;   // the tile's first key in memory; key tile 0 has the most query tiles: started first
   const int k0 = ks == CLEAN ? clean_key_pos(a, k0_row) : k0_row;   // and its position
   const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;   // warp index, provably uniform
   const int L = rows_k(a, ks), M = a.M;   // rows of this stream's K/V tensors
@@ -514,7 +516,7 @@ __device__ __forceinline__ void row_smem_to_tmem(const uint8_t* tile, int r, uin
 
 template <bool TR, int D>
 __global__ void __launch_bounds__(BWD_THREADS, 1)
-tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restrict__ status) {
+tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, const TileGrid tg, int* __restrict__ status) {
   constexpr uint32_t IDESC_KM = idesc_km(D);
   constexpr int OPER_BYTES = TILE_BYTES * D / 128;
   extern __shared__ __align__(1024) uint8_t sm[];
@@ -528,8 +530,10 @@ tc_dq_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restric
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + DQ_BARS + 144);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + DQ_BARS + 152);
 
-  const int qs = blockIdx.z & 1, b = blockIdx.z >> 1, h = blockIdx.y, hk = h / a.G;
-  const int q0 = (gridDim.x - 1 - blockIdx.x) * TILE;
+  int bx, by, bz;
+  tile_grid_decode(tg, bx, by, bz);
+  const int qs = bz & 1, b = bz >> 1, h = by, hk = h / a.G;
+  const int q0 = (tg.nx - 1 - bx) * TILE;
   const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;   // warp index, provably uniform
   if (a.q[qs] == nullptr) return;
   const int L = rows_q(a, qs);   // rows of this stream's query tensors
@@ -832,7 +836,7 @@ __device__ __forceinline__ uint32_t desc_lo_mn_h(uint32_t addr) { return ((addr 
 // the unused half of the 128-wide fp32 accumulator rows).
 template <bool TR, int D>
 __global__ void __launch_bounds__(BF_THREADS, 1)
-tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restrict__ status) {
+tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, const TileGrid tg, int* __restrict__ status) {
   constexpr uint32_t IDESC_KM = idesc_km(D);
   constexpr int OPER_BYTES = TILE_BYTES * D / 128, HOPER_BYTES = HT_BYTES * D / 128;   // bytes TMA delivers per 128- / 64-row tile
   extern __shared__ __align__(1024) uint8_t sm[];
@@ -850,8 +854,10 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, int* __restr
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + BF_BARS + 208);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + BF_BARS + 216);
 
-  const int ks = blockIdx.z & 1, b = blockIdx.z >> 1, hk = blockIdx.y;
-  const int k0_row = blockIdx.x * TILE;   // the tile's first key in memory; key tile 0 has the most query tiles: scheduled first
+  int bx, by, bz;
+  tile_grid_decode(tg, bx, by, bz);
+  const int ks = bz & 1, b = bz >> 1, hk = by;
+  const int k0_row = bx * TILE;   // the tile's first key in memory; key tile 0 has the most query tiles: started first
   const int k0 = ks == CLEAN ? clean_key_pos(a, k0_row) : k0_row;   // and its position
   const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;   // warp index, provably uniform
   const int L = rows_k(a, ks), M = a.M;
@@ -1355,8 +1361,9 @@ static cudaError_t launch_tc_bwd_d(const KArgs& a_in, void* extra_ws, int passes
       if ((e = cudaMemsetAsync(a.dq32[0], 0, (dq32_elems[0] + dq32_elems[1]) * sizeof(float), st)) != cudaSuccess) return e;
       auto kern = a.trace ? tc_bwdf_kernel<true, D> : tc_bwdf_kernel<false, D>;
       if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, BF_SMEM)) != cudaSuccess) return e;
-      dim3 grid((max(a.L, a.k[NOISY] != nullptr ? a.Ln : 0) + TILE - 1) / TILE, a.Hkv, a.batch * 2);
-      kern<<<grid, BF_THREADS, BF_SMEM, st>>>(maps, a, status);
+      const TileGrid tg = make_tile_grid((max(a.L, a.k[NOISY] != nullptr ? a.Ln : 0) + TILE - 1) / TILE, a.Hkv, a.batch * 2);
+      if (tile_grid_blocks(tg) == 0) return cudaErrorInvalidValue;
+      kern<<<tile_grid_blocks(tg), BF_THREADS, BF_SMEM, st>>>(maps, a, tg, status);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
       for (int s2 = 0; s2 < 2; ++s2) {
         if (dq32_elems[s2] == 0) continue;
@@ -1369,15 +1376,17 @@ static cudaError_t launch_tc_bwd_d(const KArgs& a_in, void* extra_ws, int passes
   if (passes & BDLM_BWD_PASS_DKDV) {
     auto kern = a.trace ? tc_dkdv_kernel<true, D> : tc_dkdv_kernel<false, D>;
     if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, DKDV_SMEM)) != cudaSuccess) return e;
-    dim3 grid((max(a.L, a.k[NOISY] != nullptr ? a.Ln : 0) + TILE - 1) / TILE, a.Hkv, a.batch * 2);
-    kern<<<grid, DKDV_THREADS, DKDV_SMEM, st>>>(maps, a, status);
+    const TileGrid tg = make_tile_grid((max(a.L, a.k[NOISY] != nullptr ? a.Ln : 0) + TILE - 1) / TILE, a.Hkv, a.batch * 2);
+    if (tile_grid_blocks(tg) == 0) return cudaErrorInvalidValue;
+    kern<<<tile_grid_blocks(tg), DKDV_THREADS, DKDV_SMEM, st>>>(maps, a, tg, status);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
   if (passes & BDLM_BWD_PASS_DQ) {
     auto kern = a.trace ? tc_dq_kernel<true, D> : tc_dq_kernel<false, D>;
     if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, DQ_SMEM)) != cudaSuccess) return e;
-    dim3 grid((max(a.q[CLEAN] != nullptr ? a.Lqc : 0, a.q[NOISY] != nullptr ? a.Ln : 0) + TILE - 1) / TILE, a.H, a.batch * 2);
-    kern<<<grid, BWD_THREADS, DQ_SMEM, st>>>(maps, a, status);
+    const TileGrid tg = make_tile_grid((max(a.q[CLEAN] != nullptr ? a.Lqc : 0, a.q[NOISY] != nullptr ? a.Ln : 0) + TILE - 1) / TILE, a.H, a.batch * 2);
+    if (tile_grid_blocks(tg) == 0) return cudaErrorInvalidValue;
+    kern<<<tile_grid_blocks(tg), BWD_THREADS, DQ_SMEM, st>>>(maps, a, tg, status);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
   return cudaSuccess;

@@ -119,7 +119,7 @@ constexpr int FWDR_SMEM = FWDR_BARS + 256 + 1024;
 // tile stays unused, Q K^T contracts over four k-slices and P V produces 64 output columns.
 template <bool TR, bool PAIRQ, int D>
 __global__ void __launch_bounds__(FWDR_THREADS, 1)
-tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restrict__ status) {
+tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, const TileGrid tg, int* __restrict__ status) {
   constexpr uint32_t IDESC_PV = make_idesc(128, D, false, true);
   constexpr int OPER_BYTES = TILE_BYTES * D / 128;   // bytes TMA delivers per operand tile
   extern __shared__ uint8_t smem_raw[];
@@ -132,12 +132,14 @@ tc_fwdr_kernel(const __grid_constant__ FwdMaps maps, const KArgs a, int* __restr
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + FWDR_BARS + 128);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + FWDR_BARS + 136);
 
-  const int qs = blockIdx.z & 1, b = blockIdx.z >> 1;
+  int bx, by, bz;
+  tile_grid_decode(tg, bx, by, bz);
+  const int qs = bz & 1, b = bz >> 1;
   if (a.q[qs] == nullptr) return;
   // warpgroup w works on head h0 + w * HSTEP, query rows q0 + w * QSTEP ...
   constexpr int HSTEP = PAIRQ ? 0 : 1, QSTEP = PAIRQ ? TILE : 0, QROWS = PAIRQ ? 2 * TILE : TILE;
-  const int h0 = PAIRQ ? blockIdx.y : blockIdx.y * 2, hk = h0 / a.G;
-  const int q0 = (gridDim.x - 1 - blockIdx.x) * QROWS;
+  const int h0 = PAIRQ ? by : by * 2, hk = h0 / a.G;
+  const int q0 = (tg.nx - 1 - bx) * QROWS;   // the last query tile sees the most keys: started first
   const int Lq = rows_q(a, qs);
   if (q0 >= Lq) return;
   const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;   // warp index, provably uniform
@@ -427,16 +429,18 @@ static cudaError_t launch_tc_fwd_d(const KArgs& a, cudaStream_t st) {
     auto kern = a.trace ? tc_fwdr_kernel<true, false, D> : tc_fwdr_kernel<false, false, D>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, FWDR_SMEM);
     if (e != cudaSuccess) return e;
-    dim3 grid((qrows + TILE - 1) / TILE, a.H / 2, a.batch * 2);
-    kern<<<grid, FWDR_THREADS, FWDR_SMEM, st>>>(maps, a, status);
+    const TileGrid tg = make_tile_grid((qrows + TILE - 1) / TILE, a.H / 2, a.batch * 2);
+    if (tile_grid_blocks(tg) == 0) return cudaErrorInvalidValue;
+    kern<<<tile_grid_blocks(tg), FWDR_THREADS, FWDR_SMEM, st>>>(maps, a, tg, status);
     return cudaGetLastError();
   }
   // odd group size: two consecutive query tiles of one head per CTA
   auto kern = a.trace ? tc_fwdr_kernel<true, true, D> : tc_fwdr_kernel<false, true, D>;
   e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, FWDR_SMEM);
   if (e != cudaSuccess) return e;
-  dim3 grid(((qrows + TILE - 1) / TILE + 1) / 2, a.H, a.batch * 2);
-  kern<<<grid, FWDR_THREADS, FWDR_SMEM, st>>>(maps, a, status);
+  const TileGrid tg = make_tile_grid(((qrows + TILE - 1) / TILE + 1) / 2, a.H, a.batch * 2);
+  if (tile_grid_blocks(tg) == 0) return cudaErrorInvalidValue;
+  kern<<<tile_grid_blocks(tg), FWDR_THREADS, FWDR_SMEM, st>>>(maps, a, tg, status);
   return cudaGetLastError();
 }
 

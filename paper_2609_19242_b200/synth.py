@@ -193,6 +193,8 @@ class LceWorkload:
 LCE_WORKLOADS = {
     "lce_tiny": LceWorkload("lce_tiny", 200, 64, 1000),
     "lce_8k": LceWorkload("lce_8k", 8192, 4096, 128256),
+    # small enough for a full profiler capture, operands still larger than L2
+    "lce_small": LceWorkload("lce_small", 4096, 2048, 32768),
 }
 
 
