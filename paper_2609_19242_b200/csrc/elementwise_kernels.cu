@@ -1,6 +1,8 @@
 // Bandwidth-bound kernels of the BDLM attention path: the LSE merge of partial outputs
 // (Eq. csbp-lse-merge over n partials, final division included) and the
 // backward preprocess D_i = sum_d dO_i,d * O_i,d.
+#include <type_traits>
+
 #include "bdlm_common.cuh"
 
 namespace bdlm {
@@ -22,8 +24,9 @@ struct MergeArgs {
 // partial (z_j = -inf) gets weight 0, a row whose partials are all empty gets O = 0 and z = -inf.  Then the
 // partial outputs are streamed through once, four partials' loads in flight at a time, and added up with their
 // weights -- no running rescale and nothing another thread could overwrite.
-template <bool F32IN, int EPT>
-__global__ void __launch_bounds__(256) merge_kernel(MergeArgs ma, int64_t total_chunks, int L, int H, int d,
+// NP = the number of partials rounded up to a multiple of four: the weights are a register array of that length.
+template <bool F32IN, int EPT, int NP>
+__global__ void __launch_bounds__(256, 3) merge_kernel(MergeArgs ma, int64_t total_chunks, int L, int H, int d,
                                                     bf16* __restrict__ o_out, float* __restrict__ lse_out) {
   constexpr int NV = F32IN ? EPT / 4 : EPT / 8;   // 16-byte vectors per thread and partial
   const int cpr = d / EPT;   // chunks per (row, head)
@@ -36,17 +39,32 @@ __global__ void __launch_bounds__(256) merge_kernel(MergeArgs ma, int64_t total_
     const int64_t bidx = row / L;
     const int i = (int)(row % L);
     const int64_t lidx = (bidx * H + h) * L + i;
-    float wgt[MAX_PARTIALS];
+    // The partial outputs do not depend on the weights: the first four partials' loads go out together with the
+    // LSE loads; each later group of four is requested once the group in hand has been added up.
+    uint4 cur[4][NV];
+    auto request = [&](int j0, uint4 (&buf)[4][NV]) {
+#pragma unroll
+      for (int jj = 0; jj < 4; ++jj) {
+        if (j0 + jj < ma.n) {
+          const uint4* p = F32IN ? reinterpret_cast<const uint4*>(static_cast<const float*>(ma.o[j0 + jj]) + idx * EPT)
+                                 : reinterpret_cast<const uint4*>(static_cast<const bf16*>(ma.o[j0 + jj]) + idx * EPT);
+#pragma unroll
+          for (int v = 0; v < NV; ++v) buf[jj][v] = p[v];
+        }
+      }
+    };
+    request(0, cur);
+    float wgt[NP];
     float m = -INFINITY;
 #pragma unroll
-    for (int j = 0; j < MAX_PARTIALS; ++j) {
+    for (int j = 0; j < NP; ++j) {
       wgt[j] = j < ma.n ? ma.lse[j][lidx] : -INFINITY;
       m = fmaxf(m, wgt[j]);
     }
     const float m_ref = (m == -INFINITY) ? 0.f : m;   // all empty: every weight becomes exp(-inf) = 0
     float wsum = 0.f;
 #pragma unroll
-    for (int j = 0; j < MAX_PARTIALS; ++j) {
+    for (int j = 0; j < NP; ++j) {
       wgt[j] = (wgt[j] == -INFINITY) ? 0.f : expf(wgt[j] - m_ref);
       wsum += wgt[j];
     }
@@ -55,28 +73,18 @@ __global__ void __launch_bounds__(256) merge_kernel(MergeArgs ma, int64_t total_
 #pragma unroll
     for (int e = 0; e < EPT; ++e) acc[e] = 0.f;
 #pragma unroll
-    for (int j0 = 0; j0 < MAX_PARTIALS; j0 += 4) {
+    for (int j0 = 0; j0 < NP; j0 += 4) {
       if (j0 >= ma.n) break;
-      uint4 u4[4][NV];
-#pragma unroll
-      for (int jj = 0; jj < 4; ++jj) {
-        if (j0 + jj < ma.n) {
-          const uint4* p = F32IN ? reinterpret_cast<const uint4*>(static_cast<const float*>(ma.o[j0 + jj]) + idx * EPT)
-                                 : reinterpret_cast<const uint4*>(static_cast<const bf16*>(ma.o[j0 + jj]) + idx * EPT);
-#pragma unroll
-          for (int v = 0; v < NV; ++v) u4[jj][v] = p[v];
-        }
-      }
 #pragma unroll
       for (int jj = 0; jj < 4; ++jj) {
         if (j0 + jj >= ma.n) break;
         const float wj = wgt[j0 + jj] * inv;
         if (F32IN) {
-          const float* pf = reinterpret_cast<const float*>(&u4[jj][0]);
+          const float* pf = reinterpret_cast<const float*>(&cur[jj][0]);
 #pragma unroll
           for (int e = 0; e < EPT; ++e) acc[e] = fmaf(wj, pf[e], acc[e]);
         } else {
-          const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&u4[jj][0]);
+          const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&cur[jj][0]);
 #pragma unroll
           for (int e = 0; e < EPT / 2; ++e) {
             const float2 f = __bfloat1622float2(p2[e]);
@@ -85,6 +93,7 @@ __global__ void __launch_bounds__(256) merge_kernel(MergeArgs ma, int64_t total_
           }
         }
       }
+      if (j0 + 4 < ma.n) request(j0 + 4, cur);
     }
 #pragma unroll
     for (int v = 0; v < EPT / 8; ++v) {
@@ -208,19 +217,30 @@ cudaError_t launch_merge(int n, int batch, int L, int H, int d, const void* cons
     ma.o[j] = j < n ? o_parts[j] : nullptr;
     ma.lse[j] = j < n ? lse_parts[j] : nullptr;
   }
-  // few partials: 16 elements per thread (more bytes in flight per thread); otherwise 8
+  // few partials: 16 elements per thread (more bytes in flight per thread); otherwise 8 (more warps per SM)
   const int ept = (d % 16 == 0 && n <= 3) ? 16 : 8;
   const int64_t total = (int64_t)batch * L * H * (d / ept);
   int64_t want = (total + 255) / 256;
   const int64_t cap = (int64_t)device_sm_count() * 16;
   int blocks = (int)(want < cap ? (want > 0 ? want : 1) : cap);
   bf16* oo = static_cast<bf16*>(o_out);
+  auto go = [&](auto f32in, auto ept_c, auto np_c) {
+    merge_kernel<decltype(f32in)::value, decltype(ept_c)::value, decltype(np_c)::value>
+        <<<blocks, 256, 0, st>>>(ma, total, L, H, d, oo, lse_out);
+  };
+  auto by_np = [&](auto f32in, auto ept_c) {
+    if (n <= 4) go(f32in, ept_c, std::integral_constant<int, 4>{});
+    else if (n <= 8) go(f32in, ept_c, std::integral_constant<int, 8>{});
+    else if (n <= 12) go(f32in, ept_c, std::integral_constant<int, 12>{});
+    else go(f32in, ept_c, std::integral_constant<int, 16>{});
+  };
+  // (16 elements per thread only go with up to three partials, i.e. with four weights)
   if (dtype == 1) {
-    if (ept == 16) merge_kernel<true, 16><<<blocks, 256, 0, st>>>(ma, total, L, H, d, oo, lse_out);
-    else merge_kernel<true, 8><<<blocks, 256, 0, st>>>(ma, total, L, H, d, oo, lse_out);
+    if (ept == 16) go(std::true_type{}, std::integral_constant<int, 16>{}, std::integral_constant<int, 4>{});
+    else by_np(std::true_type{}, std::integral_constant<int, 8>{});
   } else {
-    if (ept == 16) merge_kernel<false, 16><<<blocks, 256, 0, st>>>(ma, total, L, H, d, oo, lse_out);
-    else merge_kernel<false, 8><<<blocks, 256, 0, st>>>(ma, total, L, H, d, oo, lse_out);
+    if (ept == 16) go(std::false_type{}, std::integral_constant<int, 16>{}, std::integral_constant<int, 4>{});
+    else by_np(std::false_type{}, std::integral_constant<int, 8>{});
   }
   return cudaGetLastError();
 }
