@@ -113,3 +113,16 @@ def test_full_size_sampled_tokens():
     # the scalar loss against the per-token values the kernel itself wrote (the sum is the only new arithmetic here)
     want = float((g["weight"].double() * nll.double()).sum())
     assert abs(float(loss) - want) <= 1e-5 * abs(want)
+
+
+def test_all_positions_ignored_gives_zero_loss_and_zero_gradients():
+    w = LceWorkload("all_ignored", 130, 64, 520)
+    inp = {k: v.cuda() for k, v in synth.make_lce_inputs(w, "cpu").items()}
+    labels = torch.full_like(inp["labels"], -1)
+    loss, nll, lse = binding.bdlm_linear_ce_fwd(inp["h"], inp["w"], labels, None)
+    dh, dw = binding.bdlm_linear_ce_bwd(inp["h"], inp["w"], labels, lse, None)
+    torch.cuda.synchronize()
+    assert float(loss) == 0.0 and float(nll.abs().max()) == 0.0
+    assert float(dh.float().abs().max()) == 0.0 and float(dw.float().abs().max()) == 0.0
+    ref = lce.linear_ce_forward(synth.to_f64(inp["h"]), synth.to_f64(inp["w"]), labels.cpu().numpy())
+    assert np.abs(synth.to_f64(lse) - ref[2]).max() <= TOL_LSE

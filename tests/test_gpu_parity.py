@@ -366,3 +366,10 @@ def test_ragged_outputs_do_not_touch_memory_past_the_tensors():
         for b in (bufs_o[1], bufs_o[3]):
             assert float((b[w.H * L:] - 7.0).abs().max()) == 0.0
         assert torch.isfinite(grads[0].float()).all()
+
+
+def test_many_heads_take_the_row_wise_d_preprocess():
+    """With several hundred heads the tile of the D preprocess (32 rows x all heads) no longer fits shared memory and the
+    warp-per-row form runs instead; both forms feed the same backward."""
+    w = Workload("many_heads", 1, 384, 96, 64, 128, 16)
+    pu.check_full(w, binding.IMPL_AUTO)
