@@ -348,33 +348,6 @@ __global__ void __launch_bounds__(256) lce_sum_kernel(const float* __restrict__ 
 }
 
 // ------------------------------------------------------------------------------------------ host
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-EncodeTiledFn lce_encode_fn() {
-  static EncodeTiledFn fn = [] {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess) p = nullptr;
-    if (q != cudaDriverEntryPointSuccess) p = nullptr;
-    return reinterpret_cast<EncodeTiledFn>(p);
-  }();
-  return fn;
-}
-
-// Row-major bf16 matrix [rows, cols] with leading dimension ld (elements); box = 64 columns x box_rows rows.
-bool make_map_2d(CUtensorMap* m, const void* ptr, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
-  EncodeTiledFn fn = lce_encode_fn();
-  if (fn == nullptr || ptr == nullptr) return false;
-  cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  cuuint64_t gstride[1] = {(cuuint64_t)ld * 2};
-  cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), gdim, gstride, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 // Operand descriptions of one product: A is [M x K] (K-major) or [K x M] (MN-major) in memory, B likewise with N.
 struct Operand { const void* ptr; int64_t ld; int mn; };
 
@@ -382,8 +355,8 @@ template <int EPI>
 cudaError_t launch_gemm(GemmArgs a, const Operand& A, const Operand& B, cudaStream_t st) {
   GemmMaps maps;
   a.a_mn = A.mn; a.b_mn = B.mn;
-  const bool okA = A.mn ? make_map_2d(&maps.a, A.ptr, a.K, a.M, A.ld, 64) : make_map_2d(&maps.a, A.ptr, a.M, a.K, A.ld, BM);
-  const bool okB = B.mn ? make_map_2d(&maps.b, B.ptr, a.K, a.N, B.ld, 64) : make_map_2d(&maps.b, B.ptr, a.N, a.K, B.ld, BN);
+  const bool okA = A.mn ? tc_make_map_2d(&maps.a, A.ptr, a.K, a.M, A.ld, 64) : tc_make_map_2d(&maps.a, A.ptr, a.M, a.K, A.ld, BM);
+  const bool okB = B.mn ? tc_make_map_2d(&maps.b, B.ptr, a.K, a.N, B.ld, 64) : tc_make_map_2d(&maps.b, B.ptr, a.N, a.K, B.ld, BN);
   if (!okA || !okB) return cudaErrorInvalidValue;
   a.m_tiles = (a.M + BM - 1) / BM;
   a.n_tiles = (a.N + BN - 1) / BN;
@@ -459,7 +432,7 @@ int bdlm_linear_ce_fwd(const bdlm_lce_params* p, const void* h, const void* w, c
       (reinterpret_cast<uintptr_t>(nll) & 3u) || (reinterpret_cast<uintptr_t>(token_weight) & 3u))
     return BDLM_ERR_INVALID_ARG;
   if (workspace_bytes < bdlm_linear_ce_workspace_bytes(p, BDLM_LCE_WS_FWD)) return BDLM_ERR_WORKSPACE_TOO_SMALL;
-  if (!sm100() || lce_encode_fn() == nullptr) return BDLM_ERR_UNSUPPORTED;
+  if (!sm100() || !tc_encoder_available()) return BDLM_ERR_UNSUPPORTED;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const int runs = fwd_runs(p->V);
   const size_t per = align256((size_t)p->T * sizeof(float));
@@ -490,7 +463,7 @@ int bdlm_linear_ce_bwd(const bdlm_lce_params* p, const void* h, const void* w, c
       (reinterpret_cast<uintptr_t>(lse) & 3u) || (reinterpret_cast<uintptr_t>(token_weight) & 3u))
     return BDLM_ERR_INVALID_ARG;
   if (workspace_bytes < bdlm_linear_ce_workspace_bytes(p, BDLM_LCE_WS_BWD)) return BDLM_ERR_WORKSPACE_TOO_SMALL;
-  if (!sm100() || lce_encode_fn() == nullptr) return BDLM_ERR_UNSUPPORTED;
+  if (!sm100() || !tc_encoder_available()) return BDLM_ERR_UNSUPPORTED;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const int T = p->T, D = p->D, V = p->V;
   const int tc_ = default_chunk(p);

@@ -13,6 +13,10 @@ bool tc_encoder_available();
 // Tensor map over a [batch, L, heads, d] bf16 tensor (d = 64 or 128), box = 64 columns x `rows` rows, 128-byte swizzle.
 bool tc_make_map(CUtensorMap* m, const void* ptr, int heads, int L, int batch, int rows, int d);
 
+// Tensor map over a row-major bf16 matrix [rows, cols] with leading dimension ld (elements): box = 64 columns x
+// `box_rows` rows, 128-byte swizzle, zero fill outside the matrix.
+bool tc_make_map_2d(CUtensorMap* m, const void* ptr, int64_t rows, int64_t cols, int64_t ld, int box_rows);
+
 bool tc_rows_ok(const KArgs& a);
 bool tc_fwd_supported(const KArgs& a);
 bool tc_bwd_supported(const KArgs& a);
