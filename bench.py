@@ -36,12 +36,12 @@ NAMES6 = ["q_clean", "k_clean", "v_clean", "q_noisy", "k_noisy", "v_noisy"]
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of a kernel from a one-pass ncu capture of
 # this command, keyed by (workload, kernel), each with the digest of the kernel sources it was captured on
 # (kernel_source_digest): a figure is reported only for the build it belongs to.
-_CAPTURED_ON = "58cebb4f2442bf0e"
+_CAPTURED_ON = "754db68427b84cd2"
 NCU_TRAFFIC = {
-    ("32k", "fwd"): {"bytes": 966811392 + 528489472, "kernel_source": _CAPTURED_ON},
-    ("32k", "bwd_fused"): {"bytes": 5987548416 + 3462409216, "kernel_source": _CAPTURED_ON},
-    ("32k", "bwd_dkdv"): {"bytes": 2395995904 + 249831936, "kernel_source": _CAPTURED_ON},
-    ("32k", "bwd_dq"): {"bytes": 1539676928 + 518457344, "kernel_source": _CAPTURED_ON},
+    ("32k", "fwd"): {"bytes": 967984896 + 528709376, "kernel_source": _CAPTURED_ON},
+    ("32k", "bwd_fused"): {"bytes": 5990126592 + 3445277952, "kernel_source": _CAPTURED_ON},
+    ("32k", "bwd_dkdv"): {"bytes": 2380354048 + 250223104, "kernel_source": _CAPTURED_ON},
+    ("32k", "bwd_dq"): {"bytes": 1540890368 + 518644224, "kernel_source": _CAPTURED_ON},
 }
 TRAFFIC_NOTE = ("dram__bytes_read.sum + dram__bytes_write.sum per launch from a one-pass ncu capture of this command on "
                 "the 32k workload")
