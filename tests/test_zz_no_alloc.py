@@ -56,9 +56,9 @@ def test_static_scratch_backward_matches_regular_backward_twice(w):
                 assert pu.rel_l2(synth.to_f64(got), synth.to_f64(want)) <= pu.TOL_GRAD
                 assert _max_abs_diff(got, want) == 0.0
 
-    # A first round does everything once: the library looks up its scratch array's address on this device, and the
+    # A first pass does everything once: the library looks up its scratch array's address on this device, and the
     # driver loads the code of every kernel used below (the library's and those of the test's own torch calls), which
-    # takes device memory the first time.  Then the books are opened: in the second round neither torch's allocator
+    # takes device memory the first time.  Then the books are opened: in the second pass neither torch's allocator
     # nor the driver may hand out a byte at the points where the entry point has just run.
     two_calls(None)
     torch.cuda.synchronize()
