@@ -27,10 +27,8 @@ wait_timeout_selftest_kernel(long long limit_ticks, int* __restrict__ status) {
   }
   __syncthreads();
   const int warp = threadIdx.x >> 5;
-  bool ok;
-  if (warp == 0) ok = mbar_wait_abortable(bar, 0, abort_flag, limit_ticks);   // runs out, raises the flag
-  else ok = mbar_wait_abortable(bar, 0, abort_flag);                          // leaves when it sees the flag
-  (void)ok;
+  if (warp == 0) (void)mbar_wait_abortable(bar, 0, abort_flag, limit_ticks);   // runs out, raises the flag
+  else (void)mbar_wait_abortable(bar, 0, abort_flag);                          // leaves when it sees the flag
   __syncthreads();
   if (threadIdx.x == 0 && *abort_flag) atomicExch(status, (int)BDLM_ERR_DEVICE_TIMEOUT);
 }
