@@ -63,7 +63,8 @@ def test_csbp128k_shards_merge_and_oracle():
     for got, ref, tol in ((o_c, full[0], pu.TOL_O), (l_c, full[1], pu.TOL_LSE), (o_n, full[2], pu.TOL_O), (l_n, full[3], pu.TOL_LSE)):
         assert float((got.float() - ref.float()).abs().max()) <= tol
     # the merged result feeds the oracle comparison and the (unsharded) backward
-    pu.check_sampled(w, binding.IMPL_AUTO, g=g, fwd_out=(o_c, l_c, o_n, l_n))
+    # (both backward paths against one evaluation of the oracle: the fused one is what bench.py times at this size)
+    pu.check_sampled(w, binding.IMPL_AUTO, g=g, fwd_out=(o_c, l_c, o_n, l_n), single_pass=(False, True))
 
 
 def test_256k_sampled_rows():
