@@ -1296,21 +1296,37 @@ tc_bwdf_kernel(const __grid_constant__ BwdMaps maps, const KArgs a, const TileGr
 template <int D>
 __global__ void __launch_bounds__(256) dq_convert_kernel(const float* __restrict__ src, bf16* __restrict__ dst, int batch, int H, int rows,
                                                          int src_rows) {
+  constexpr int U = 4;   // rows per warp in flight: the kernel is a pure stream
   const int lane = threadIdx.x & 31;
   const int64_t n = (int64_t)batch * rows * H;
-  for (int64_t o = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5); o < n; o += (int64_t)gridDim.x * 8) {
-    const int h = (int)(o % H);
-    const int64_t bl = o / H;
-    const int l = (int)(bl % rows), b = (int)(bl / rows);
-    const float* row = src + (((int64_t)b * H + h) * src_rows + l) * 128;
-    if (D == 128) {
-      const float4 u = reinterpret_cast<const float4*>(row)[lane];
-      uint2 v;
-      v.x = pack_bf16(u.x, u.y); v.y = pack_bf16(u.z, u.w);
-      reinterpret_cast<uint2*>(dst + o * D)[lane] = v;
-    } else {
-      const float2 u = reinterpret_cast<const float2*>(row)[lane];
-      reinterpret_cast<uint32_t*>(dst + o * D)[lane] = pack_bf16(u.x, u.y);
+  const int64_t warps = (int64_t)gridDim.x * 8;
+  for (int64_t o0 = ((int64_t)blockIdx.x * 8 + (threadIdx.x >> 5)) * U; o0 < n; o0 += warps * U) {
+    float4 u4[U];
+    float2 u2[U];
+#pragma unroll
+    for (int j = 0; j < U; ++j) {
+      const int64_t o = o0 + j;
+      if (o < n) {
+        const int h = (int)(o % H);
+        const int64_t bl = o / H;
+        const int l = (int)(bl % rows), b = (int)(bl / rows);
+        const float* row = src + (((int64_t)b * H + h) * src_rows + l) * 128;
+        if (D == 128) u4[j] = reinterpret_cast<const float4*>(row)[lane];
+        else u2[j] = reinterpret_cast<const float2*>(row)[lane];
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < U; ++j) {
+      const int64_t o = o0 + j;
+      if (o < n) {
+        if (D == 128) {
+          uint2 v;
+          v.x = pack_bf16(u4[j].x, u4[j].y); v.y = pack_bf16(u4[j].z, u4[j].w);
+          reinterpret_cast<uint2*>(dst + o * D)[lane] = v;
+        } else {
+          reinterpret_cast<uint32_t*>(dst + o * D)[lane] = pack_bf16(u2[j].x, u2[j].y);
+        }
+      }
     }
   }
 }
@@ -1367,7 +1383,7 @@ static cudaError_t launch_tc_bwd_d(const KArgs& a_in, void* extra_ws, int passes
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
       for (int s2 = 0; s2 < 2; ++s2) {
         if (dq32_elems[s2] == 0) continue;
-        dq_convert_kernel<D><<<device_sm_count() * 8, 256, 0, st>>>(a.dq32[s2], a.dq[s2], a.batch, a.H, rows_q(a, s2), a.dq32_rows[s2]);
+        dq_convert_kernel<D><<<device_sm_count() * 16, 256, 0, st>>>(a.dq32[s2], a.dq[s2], a.batch, a.H, rows_q(a, s2), a.dq32_rows[s2]);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
       }
     }
