@@ -36,12 +36,12 @@ NAMES6 = ["q_clean", "k_clean", "v_clean", "q_noisy", "k_noisy", "v_noisy"]
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of a kernel from a one-pass ncu capture of
 # this command, keyed by (workload, kernel), each with the digest of the kernel sources it was captured on
 # (kernel_source_digest): a figure is reported only for the build it belongs to.
-_CAPTURED_ON = "754db68427b84cd2"
+_CAPTURED_ON = "4289fc252fec25f2"
 NCU_TRAFFIC = {
-    ("32k", "fwd"): {"bytes": 967984896 + 528709376, "kernel_source": _CAPTURED_ON},
-    ("32k", "bwd_fused"): {"bytes": 5990126592 + 3445277952, "kernel_source": _CAPTURED_ON},
-    ("32k", "bwd_dkdv"): {"bytes": 2380354048 + 250223104, "kernel_source": _CAPTURED_ON},
-    ("32k", "bwd_dq"): {"bytes": 1540890368 + 518644224, "kernel_source": _CAPTURED_ON},
+    ("32k", "fwd"): {"bytes": 967480576 + 528095488, "kernel_source": _CAPTURED_ON},
+    ("32k", "bwd_fused"): {"bytes": 5889652992 + 3375495168, "kernel_source": _CAPTURED_ON},
+    ("32k", "bwd_dkdv"): {"bytes": 2371290368 + 249625600, "kernel_source": _CAPTURED_ON},
+    ("32k", "bwd_dq"): {"bytes": 1543090432 + 519066880, "kernel_source": _CAPTURED_ON},
 }
 TRAFFIC_NOTE = ("dram__bytes_read.sum + dram__bytes_write.sum per launch from a one-pass ncu capture of this command on "
                 "the 32k workload")
