@@ -344,6 +344,14 @@ class LayerRun:
         return ms_total, per_step, per_kernel, clocks
 
 
+def clock_normalised(ms, clocks):
+    """ms x median SM MHz = clock cycles per step in units of 10^9: runs on power-capped boxes whose clocks settle at
+    different frequencies are compared on this figure."""
+    if not clocks or not clocks.get("sm_mhz"):
+        return None
+    return ms * clocks["sm_mhz"] * 1e-6
+
+
 def fractions(tflops, peaks):
     return {"frac_burst": tflops / peaks["bf16_tflops"], "frac_sustained": tflops / peaks["bf16_tflops_sustained"],
             "frac_nominal_2250": tflops / 2250.0}
@@ -478,6 +486,7 @@ def other_config_line(name, binding, peaks, impl, fused, steps, warmup, local):
            "value": tf, "unit": UNIT, "ms_per_step": ms_step, "ms_per_step_min": float(np.min(per_step)),
            "ms_per_step_median": float(np.median(per_step)), "per_kernel_ms": per_kernel, "clocks": clocks}
     out.update(fractions(tf, peaks))
+    out["gclk_per_step"] = clock_normalised(ms_step, clocks)
     if w.kv_shards > 1:
         out["sharded_fwd"] = sharded_forward_leg(run, peaks, steps, warmup)
     del run
@@ -646,7 +655,7 @@ def run_ours(args, w):
                        "backward": "fused (one kernel; dQ through fp32 add-reductions)" if fused else "two-pass (dK/dV, then dQ)"},
             "pct_of_bf16_peak": {"measured_burst": 100 * pct["frac_burst"], "measured_sustained": 100 * pct["frac_sustained"],
                                  "nominal_2250": 100 * pct["frac_nominal_2250"], "source": peaks["source"]},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": (6 if fused else 5) * K, "roofline": roofline, "cpu_baseline": cpu,
+            "clocks": clocks, "gclk_per_step": clock_normalised(ms_step, clocks), "e2e": e2e, "gpu_launches": (6 if fused else 5) * K, "roofline": roofline, "cpu_baseline": cpu,
             "other_configs": others}
     print(json.dumps(line), flush=True)
     if world > 1:
