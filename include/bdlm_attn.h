@@ -56,7 +56,8 @@ typedef struct {
                                   position 0 of the full [batch, L, H_kv, d] tensors. */
   int32_t kv_range_set;        /* 0: ignore kv_begin/kv_end (full range); 1: use them (may be empty) */
   int32_t include_noisy_diag;  /* 1: noisy queries also attend their own noisy block; 0: clean-shard partial only */
-  int32_t impl;                /* 0: automatic; 1: force the portable mma.sync kernels; 2: force the tcgen05 kernels */
+  int32_t impl;                /* 0: automatic (the tcgen05 kernels: head dimension 64 or 128, any length); 1: force the
+                                  portable mma.sync kernels (a slow cross-check); 2: force the tcgen05 kernels */
   int32_t bwd_passes;          /* backward only: 0 = all passes; otherwise a bit set of BDLM_BWD_PASS_* to run
                                   (lets a caller time the passes separately; each pass needs the earlier ones'
                                   results from a previous call with the same workspace) */
@@ -65,8 +66,8 @@ typedef struct {
                                   Each CTA adds its dQ tiles into an fp32 accumulator in the workspace (bulk add-reductions),
                                   so dQ is reproducible only up to fp32 summation order; dK and dV are bitwise reproducible
                                   (fixed order).  Needs the workspace bdlm_workspace_bytes[_packed] reports for this setting
-                                  (BDLM_ERR_WORKSPACE_TOO_SMALL otherwise); shapes the tensor-core kernels do not take
-                                  (d = 64, rows not a multiple of 128, impl = 1) run the two-pass path.
+                                  (BDLM_ERR_WORKSPACE_TOO_SMALL otherwise); with impl = 1 (the mma.sync kernels) the
+                                  two-pass path runs.
                                   BDLM_BWD_TWO_PASS (2): dK/dV pass + dQ pass, fixed summation order, every gradient
                                   bitwise reproducible; needs only the D rows in the workspace.
                                   BDLM_BWD_AUTO (0, the default of a zeroed struct): the fused kernel when the workspace
@@ -113,7 +114,7 @@ int bdlm_attn_fwd(const bdlm_params* p,
  * fp32 summation order when the fused kernel runs (see bdlm_params.bwd_single_pass for which one
  * does).  Requires the full clean key range.
  * The workspace holds D_i = sum_d dO_i,d * O_i,d and, for the fused kernel, an fp32 dQ accumulator
- * [batch, H, rows, 128] per query stream; nothing in it has to be initialised or kept between calls.
+ * [batch, H, rows rounded up to 64, 128] per query stream; nothing in it has to be initialised or kept between calls.
  * bdlm_workspace_bytes(p, BDLM_WS_BWD) reports the size for p->bwd_single_pass; with the default
  * (BDLM_BWD_AUTO) that is the fused kernel's size, and a call given less than that -- but at least
  * the BDLM_BWD_TWO_PASS size -- runs the two-pass kernels.
