@@ -92,7 +92,7 @@ def check_full(w, impl, mode=0, check_bwd=True, inp=None, single_pass=False):
     assert binding.bdlm_get_device_status() == 0
 
 
-def check_sampled(w, impl, n_rows=256, g=None, fwd_out=None, check_bwd=True, report=None, single_pass=False):
+def check_sampled(w, impl, n_rows=256, g=None, fwd_out=None, check_bwd=True, report=None, single_pass=False, mode=0):
     """Sampled-row parity for sizes the full oracle cannot do: per (batch, head, stream)
     `n_rows` stratified query rows are recomputed by the oracle.  O and LSE come from the
     full forward.  dQ at the sampled rows comes from the full backward (a row's dQ depends on
@@ -105,7 +105,7 @@ def check_sampled(w, impl, n_rows=256, g=None, fwd_out=None, check_bwd=True, rep
     if g is None:
         g = synth.make_inputs(w, "cuda")
     if fwd_out is None:
-        fwd_out = gpu_fwd(g, M, impl=impl, window=w.window)
+        fwd_out = gpu_fwd(g, M, impl=impl, window=w.window, clean_mask_mode=mode)
     torch.cuda.synchronize()
     G = w.H // w.H_kv
     rows_of = {}
@@ -121,9 +121,10 @@ def check_sampled(w, impl, n_rows=256, g=None, fwd_out=None, check_bwd=True, rep
             src = g["do_clean"] if s == 0 else g["do_noisy"]
             do_sp[s][b, r, h] = src[b, r, h]
         for sp in variants:
-            grads[sp] = [t.clone() for t in gpu_bwd(g, fwd_out, M, impl=impl, window=w.window, single_pass=sp)]
+            grads[sp] = [t.clone() for t in gpu_bwd(g, fwd_out, M, impl=impl, window=w.window, single_pass=sp,
+                                                    clean_mask_mode=mode)]
             grads_sp[sp] = [t.clone() for t in gpu_bwd(g, fwd_out, M, do_clean=do_sp[0], do_noisy=do_sp[1], impl=impl,
-                                                       window=w.window, single_pass=sp)]
+                                                       window=w.window, single_pass=sp, clean_mask_mode=mode)]
         torch.cuda.synchronize()
         assert binding.bdlm_get_device_status() == 0
     worst = {"o": 0.0, "lse": 0.0, "dq": 0.0, "dq_row": 0.0, "dk": 0.0, "dv": 0.0}
@@ -143,7 +144,7 @@ def check_sampled(w, impl, n_rows=256, g=None, fwd_out=None, check_bwd=True, rep
                     q_rows = synth.to_f64(g[qn[s]][b, rt, h])
                     do_rows = synth.to_f64(g[don[s]][b, rt, h]) if check_bwd else None
                     ref = orc.attn_rows(s, rows, q_rows, kv["k_clean"], kv["v_clean"], kv["k_noisy"],
-                                        kv["v_noisy"], M, do_rows=do_rows, window=w.window)
+                                        kv["v_noisy"], M, do_rows=do_rows, window=w.window, clean_mask_mode=mode)
                     o_got = synth.to_f64(fwd_out[2 * s][b, rt, h])
                     l_got = synth.to_f64(fwd_out[2 * s + 1][b, h, rt])
                     worst["o"] = max(worst["o"], float(np.abs(o_got - ref["o"]).max()))

@@ -72,3 +72,10 @@ def test_256k_sampled_rows():
     w = WORKLOADS["256k"]
     worst = pu.check_sampled(w, binding.IMPL_AUTO, single_pass=(False, True))
     print("256k", worst)
+
+
+def test_8k_sampled_rows_clean_mask_mode_1():
+    """The other reading of "block-causal" (a clean query sees its whole own clean block) at a full-size workload,
+    both backward paths."""
+    worst = pu.check_sampled(WORKLOADS["8k"], binding.IMPL_AUTO, single_pass=(False, True), mode=1)
+    print("8k mode 1", worst)
